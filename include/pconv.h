@@ -1,0 +1,190 @@
+/*
+ * pconv.h -- C ABI of the B200 pattern-sparse 3x3 convolution library (PCONV forward pass).
+ *
+ * The operation is the paper's Eq. 1 (cross-correlation, no kernel flip) applied per layer,
+ *
+ *     y[n,o,i,j] = act( b[o] + sum_c sum_{u,v<3} xpad[n,c,i*s+u-1,j*s+v-1] * W[o,c,u,v] ),
+ *
+ * for weights that carry the two sparsities of the paper's "Sparse Convolution Pattern" section:
+ * every surviving (filter o, input channel c) kernel has its non-zeros inside one 3x3 binary
+ * pattern of a small set (pattern pruning: 4 of 9 taps, the "2.25x" of the pattern-count tables),
+ * and whole kernels are removed (connectivity pruning).  The library skips every pruned kernel and
+ * every tap outside the pattern; the result equals the dense convolution up to summation order.
+ * Zero padding 1, stride 1 or 2, dilation 1, groups 1, optional bias and fused ReLU are fixed by
+ * this build (the paper does not state them).
+ *
+ * General rules
+ *  - Every call returns a pconv_status; nothing throws, aborts or prints.  Out-parameters are
+ *    written only on PCONV_OK unless stated otherwise.
+ *  - "host" pointers are ordinary CPU memory; "dev" pointers are CUDA device memory of the current
+ *    device.  `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *  - Tensors are dense and contiguous: activations NCHW, weights OIHW ([C_out][C_in][3][3]).
+ *  - Pattern masks are 9-bit integers: bit (3*u + v) set <=> tap (row u, column v) may be
+ *    non-zero; bit 4 is the centre.
+ *  - Storage type PCONV_F32: x, y and packed weights are fp32.  PCONV_F16: x, y and packed
+ *    weights are IEEE fp16 (weights rounded to nearest even at pack time); bias and every
+ *    accumulation stay fp32, and the output is rounded once at the store.
+ */
+#ifndef PCONV_H_
+#define PCONV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct pconv_handle pconv_handle; /* one packed layer; opaque, library-owned */
+typedef struct pconv_stack pconv_stack;   /* a chain of packed layers with its activations */
+
+typedef enum {
+  PCONV_OK = 0,
+  PCONV_ERR_NULL = 1,              /* a required pointer is NULL */
+  PCONV_ERR_SHAPE = 2,             /* non-positive or inconsistent sizes, bad stride */
+  PCONV_ERR_PATTERN_SET = 3,       /* a mask without exactly 4 of 9 bits, duplicates, bad count */
+  PCONV_ERR_KERNEL_NOT_IN_SET = 4, /* a kernel's non-zeros fit no pattern (or not 0/4 when strict) */
+  PCONV_ERR_RANGE = 5,             /* NaN/Inf weight, or overflow when rounding to fp16 */
+  PCONV_ERR_UNSUPPORTED = 6,       /* unknown storage type or flag */
+  PCONV_ERR_ALIGN = 7,             /* a device pointer is not aligned as required */
+  PCONV_ERR_ALLOC = 8,             /* host or device allocation failed */
+  PCONV_ERR_CUDA = 9,              /* a CUDA runtime call or a kernel launch failed */
+  PCONV_ERR_DEVICE_TIMEOUT = 10    /* a kernel's bounded wait ran out (see pconv_device_status) */
+} pconv_status;
+
+enum { PCONV_F32 = 0, PCONV_F16 = 1 };
+
+enum {
+  PCONV_RELU = 1u,    /* forward: y = max(0, .) after the bias */
+  PCONV_STRICT4 = 2u, /* pack: every kernel must have exactly 0 or 4 non-zeros */
+  /* Kernel selection (forward).  Default: the library picks per shape.  These bits exist so that
+   * tests and benchmarks can pin one implementation; they never change the result beyond
+   * summation order. */
+  PCONV_KERNEL_SIMPLE = 0x100u, /* one thread per output, walks the per-filter kernel list */
+  PCONV_KERNEL_TILED = 0x200u,  /* shared-memory halo tiles, register-blocked FFMA2 path */
+  PCONV_KERNEL_GENERIC_TAPS = 0x400u /* tiled path with run-time 9-bit masks (any pattern set) */
+};
+
+#define PCONV_MAX_PATTERNS 16
+
+typedef struct {
+  int c_out, c_in, stride, storage, n_patterns;
+  long long kept_kernels;                       /* surviving (o,c) kernels */
+  long long per_pattern[PCONV_MAX_PATTERNS];    /* kernels per pattern id; sums to kept_kernels */
+  int min_per_filter, max_per_filter;           /* surviving kernels per filter */
+  int n_groups, group_size;                     /* filter groups of the tiled layout */
+  long long max_group_kernels, min_group_kernels; /* load balance of the grouping */
+  long long packed_bytes;                       /* device bytes held by the handle */
+  int canonical_patterns;                       /* 1 if the set is served by the specialised code */
+} pconv_stats_t;
+
+/*
+ * pconv_pack -- host-side packer: layerwise information extraction, filter/kernel reorder and
+ * compressed weight storage (paper, "Compiler-assisted DNN Inference Framework": steps (i) and
+ * (ii), and the index-free storage that pattern regularity allows).
+ *
+ *  w_oihw_host  [c_out][c_in][3][3] fp32, HOST; read during the call only (caller keeps it).
+ *  patterns     n_patterns masks, HOST; each must have exactly 4 of 9 bits, all distinct,
+ *               1 <= n_patterns <= PCONV_MAX_PATTERNS.
+ *  stride       1 or 2.   storage  PCONV_F32 or PCONV_F16.   flags  0 or PCONV_STRICT4.
+ *  stream       stream used for the upload; the call synchronises it before returning.
+ *  out          receives the handle (owns its device buffers until pconv_free).
+ *  bad_o,bad_c  optional; on PCONV_ERR_KERNEL_NOT_IN_SET / PCONV_ERR_RANGE they receive the first
+ *               offending kernel (written on those errors only).
+ *
+ * A kernel's support is the set of its non-zero taps (-0.0 counts as zero).  Empty support =
+ * pruned.  Otherwise it is assigned the lowest pattern id whose mask contains the support; zeros
+ * inside the mask are stored as zeros.  A filter with no surviving kernel is legal.
+ * Filters are permuted into groups of 16 balanced by surviving-kernel count; outputs are always
+ * written at the original filter index.
+ */
+pconv_status pconv_pack(const float* w_oihw_host, int c_out, int c_in, const uint16_t* patterns,
+                        int n_patterns, int stride, int storage, unsigned flags, void* stream,
+                        pconv_handle** out, int* bad_o, int* bad_c);
+
+/*
+ * pconv_forward -- the hot path (Eq. 1 over surviving taps only: per-pattern 4-tap multiply-add,
+ * the paper's "load redundancy elimination" -- only inputs under non-zero taps are touched --
+ * with bias and ReLU fused).
+ *
+ *  x_dev     [n][c_in][h_in][w_in], DEVICE, storage type of the handle, 16-byte aligned.
+ *  bias_dev  [c_out] fp32, DEVICE, or NULL for no bias.
+ *  y_dev     [n][c_out][h_out][w_out], DEVICE, same storage type, 16-byte aligned, must not
+ *            overlap x.  h_out = (h_in - 1) / stride + 1, likewise w_out.
+ *  flags     PCONV_RELU and/or one PCONV_KERNEL_* bit.
+ *
+ * Asynchronous on `stream`; allocates nothing and never synchronises.  PCONV_ERR_CUDA reports
+ * launch-time errors only.  A handle is immutable: concurrent forwards on several streams are
+ * allowed.  n == 0 is a no-op.
+ */
+pconv_status pconv_forward(const pconv_handle* h, const void* x_dev, const float* bias_dev,
+                           void* y_dev, int n, int h_in, int w_in, unsigned flags, void* stream);
+
+/* Releases the handle and its device buffers.  NULL is allowed. */
+void pconv_free(pconv_handle* h);
+
+/*
+ * pconv_maxpool2x2 -- the plain 2x2 / stride-2 max-pool that separates the VGG blocks
+ * (y[n,c,i,j] = max of x[n,c,2i..2i+1,2j..2j+1]; odd trailing rows/columns are dropped).
+ * x_dev [n][c][h][w] and y_dev [n][c][h/2][w/2] are DEVICE pointers of `storage` type.
+ */
+pconv_status pconv_maxpool2x2(const void* x_dev, void* y_dev, int n, int c, int h, int w,
+                              int storage, void* stream);
+
+/* ---- test and inspection aids --------------------------------------------------------------- */
+
+/* Decodes the DEVICE copy of the packed layer back to dense OIHW fp32 on the HOST
+ * (w_out: c_out*c_in*9 floats).  fp16 handles return the rounded values.  Synchronous. */
+pconv_status pconv_unpack(const pconv_handle* h, float* w_oihw_host_out);
+
+/* Fills *out with the layer's structure counts. */
+pconv_status pconv_stats(const pconv_handle* h, pconv_stats_t* out);
+
+/* Copies the filter permutation to the HOST: perm_out[slot] = original filter index or -1 for a
+ * padding slot; perm_out has n_groups*group_size entries. */
+pconv_status pconv_filter_order(const pconv_handle* h, int* perm_out);
+
+/* Synchronises the device and returns PCONV_ERR_DEVICE_TIMEOUT if any forward on this handle
+ * abandoned a bounded wait since the handle was created (then *where, if given, receives the
+ * internal wait id), else PCONV_OK. */
+pconv_status pconv_device_status(const pconv_handle* h, int* where);
+
+/* Constant, NUL-terminated description of a status. */
+const char* pconv_status_str(pconv_status s);
+
+/* ---- layer stacks ---------------------------------------------------------------------------- */
+
+/*
+ * pconv_stack_create -- chains layers: x -> conv(layers[0]) [-> maxpool] -> conv(layers[1]) ...
+ * for a fixed input shape (n, h, w), as in the VGG-16 stacks of the evaluation.  The stack
+ * allocates its two ping-pong activation buffers on the device here (never during forward), and
+ * borrows the handles and bias pointers, which must outlive it.
+ *  layers      n_layers handles (HOST array), same storage type, c_in of layer k+1 = c_out of k.
+ *  bias_dev    n_layers DEVICE pointers (HOST array; entries may be NULL), or NULL.
+ *  pool_after  n_layers bytes (HOST), non-zero = a 2x2 max-pool follows that layer; or NULL.
+ *  flags       applied to every layer's forward (PCONV_RELU, kernel selection).
+ */
+pconv_status pconv_stack_create(const pconv_handle* const* layers, const float* const* bias_dev,
+                                const unsigned char* pool_after, int n_layers, int n, int h, int w,
+                                unsigned flags, pconv_stack** out);
+
+/* Shape of the stack's result: [n][c][h][w] (any pointer may be NULL). */
+pconv_status pconv_stack_out_shape(const pconv_stack* s, int* n, int* c, int* h, int* w);
+
+/* Runs the chain with DEVICE input and output; asynchronous on `stream`, allocates nothing.
+ * Two forwards of the same stack must not overlap (they share the activation buffers). */
+pconv_status pconv_stack_forward(pconv_stack* s, const void* x_dev, void* y_dev, void* stream);
+
+/* The same with HOST input and output: copies x to the device, runs the chain, copies the result
+ * back and synchronises `stream` before returning.  Pinned host memory makes the copies
+ * asynchronous; pageable memory also works.  Uses two extra device buffers owned by the stack. */
+pconv_status pconv_stack_forward_host(pconv_stack* s, const void* x_host, void* y_host,
+                                      void* stream);
+
+/* Releases the stack (not the handles).  NULL is allowed. */
+void pconv_stack_free(pconv_stack* s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PCONV_H_ */

@@ -1,0 +1,239 @@
+// C ABI entry points: argument checks, kernel selection, layer stacks.
+#include <cstring>
+#include <new>
+
+#include "pconv_internal.h"
+
+using namespace pconv;
+
+extern "C" const char* pconv_status_str(pconv_status s) {
+  switch (s) {
+    case PCONV_OK: return "ok";
+    case PCONV_ERR_NULL: return "required pointer is NULL";
+    case PCONV_ERR_SHAPE: return "bad shape or stride";
+    case PCONV_ERR_PATTERN_SET: return "bad pattern set";
+    case PCONV_ERR_KERNEL_NOT_IN_SET: return "a kernel fits no pattern of the set";
+    case PCONV_ERR_RANGE: return "non-finite weight or fp16 overflow";
+    case PCONV_ERR_UNSUPPORTED: return "unsupported storage type or flag";
+    case PCONV_ERR_ALIGN: return "misaligned device pointer";
+    case PCONV_ERR_ALLOC: return "allocation failed";
+    case PCONV_ERR_CUDA: return "CUDA error";
+    case PCONV_ERR_DEVICE_TIMEOUT: return "a kernel abandoned a bounded wait";
+  }
+  return "unknown status";
+}
+
+extern "C" pconv_status pconv_forward(const pconv_handle* h, const void* x, const float* bias,
+                                      void* y, int n, int h_in, int w_in, unsigned flags,
+                                      void* stream_v) {
+  if (!h || !x || !y) return PCONV_ERR_NULL;
+  if (n < 0 || h_in <= 0 || w_in <= 0) return PCONV_ERR_SHAPE;
+  const unsigned known =
+      PCONV_RELU | PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED | PCONV_KERNEL_GENERIC_TAPS;
+  if (flags & ~known) return PCONV_ERR_UNSUPPORTED;
+  const unsigned sel = flags & (PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED | PCONV_KERNEL_GENERIC_TAPS);
+  if (sel & (sel - 1)) return PCONV_ERR_UNSUPPORTED;  // at most one selection bit
+  if (((uintptr_t)x | (uintptr_t)y) & 15u) return PCONV_ERR_ALIGN;
+  if (bias && ((uintptr_t)bias & 3u)) return PCONV_ERR_ALIGN;
+  if (n == 0) return PCONV_OK;
+  const DeviceLayer& L = h->d;
+  {  // x and y must not overlap
+    const size_t es = (L.storage == PCONV_F16) ? 2 : 4;
+    const int ho = (h_in - 1) / L.stride + 1, wo = (w_in - 1) / L.stride + 1;
+    const char* xb = (const char*)x;
+    const char* yb = (const char*)y;
+    const size_t xs = (size_t)n * L.c_in * h_in * w_in * es, ys = (size_t)n * L.c_out * ho * wo * es;
+    if (xb < yb + ys && yb < xb + xs) return PCONV_ERR_SHAPE;
+  }
+  cudaStream_t stream = (cudaStream_t)stream_v;
+  const bool relu = flags & PCONV_RELU;
+  cudaError_t e;
+  if (sel == PCONV_KERNEL_SIMPLE) {
+    e = launch_simple(L, x, bias, y, n, h_in, w_in, relu, stream);
+  } else if (sel == PCONV_KERNEL_TILED || sel == PCONV_KERNEL_GENERIC_TAPS) {
+    if (!tiled_supported(L, n, h_in, w_in)) return PCONV_ERR_UNSUPPORTED;
+    const bool generic = (sel == PCONV_KERNEL_GENERIC_TAPS) || !h->canonical;
+    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, generic, stream);
+  } else if (tiled_supported(L, n, h_in, w_in)) {
+    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, !h->canonical, stream);
+  } else {
+    e = launch_simple(L, x, bias, y, n, h_in, w_in, relu, stream);
+  }
+  if (e != cudaSuccess) return PCONV_ERR_CUDA;
+  return PCONV_OK;
+}
+
+extern "C" pconv_status pconv_maxpool2x2(const void* x, void* y, int n, int c, int h, int w,
+                                         int storage, void* stream) {
+  if (!x || !y) return PCONV_ERR_NULL;
+  if (n < 0 || c <= 0 || h < 2 || w < 2) return PCONV_ERR_SHAPE;
+  if (storage != PCONV_F32 && storage != PCONV_F16) return PCONV_ERR_UNSUPPORTED;
+  if (launch_maxpool(x, y, n, c, h, w, storage, (cudaStream_t)stream) != cudaSuccess)
+    return PCONV_ERR_CUDA;
+  return PCONV_OK;
+}
+
+extern "C" pconv_status pconv_device_status(const pconv_handle* h, int* where) {
+  if (!h) return PCONV_ERR_NULL;
+  int v = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpy(&v, h->d.err, 4, cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    return PCONV_ERR_CUDA;
+  }
+  if (v) {
+    if (where) *where = v;
+    return PCONV_ERR_DEVICE_TIMEOUT;
+  }
+  return PCONV_OK;
+}
+
+// ---- stacks ---------------------------------------------------------------------------------------
+
+struct pconv_stack {
+  int n_layers, n, h, w, storage;
+  unsigned flags;
+  const pconv_handle** layers;
+  const float** bias;
+  unsigned char* pool;
+  int out_c, out_h, out_w;
+  size_t in_bytes, out_bytes, act_bytes;
+  void* act[2];   // ping-pong activations
+  void* io[2];    // device input / output used by the host entry point
+};
+
+extern "C" void pconv_stack_free(pconv_stack* s) {
+  if (!s) return;
+  for (int i = 0; i < 2; ++i) {
+    if (s->act[i]) cudaFree(s->act[i]);
+    if (s->io[i]) cudaFree(s->io[i]);
+  }
+  delete[] s->layers;
+  delete[] s->bias;
+  delete[] s->pool;
+  delete s;
+}
+
+extern "C" pconv_status pconv_stack_create(const pconv_handle* const* layers,
+                                           const float* const* bias_dev,
+                                           const unsigned char* pool_after, int n_layers, int n,
+                                           int h, int w, unsigned flags, pconv_stack** out) {
+  if (!layers || !out) return PCONV_ERR_NULL;
+  if (n_layers <= 0 || n <= 0 || h <= 0 || w <= 0) return PCONV_ERR_SHAPE;
+  for (int i = 0; i < n_layers; ++i)
+    if (!layers[i]) return PCONV_ERR_NULL;
+  pconv_stack* s = new (std::nothrow) pconv_stack();
+  if (!s) return PCONV_ERR_ALLOC;
+  std::memset(s, 0, sizeof(*s));
+  s->layers = new (std::nothrow) const pconv_handle*[n_layers];
+  s->bias = new (std::nothrow) const float*[n_layers];
+  s->pool = new (std::nothrow) unsigned char[n_layers];
+  if (!s->layers || !s->bias || !s->pool) {
+    pconv_stack_free(s);
+    return PCONV_ERR_ALLOC;
+  }
+  s->n_layers = n_layers;
+  s->n = n;
+  s->h = h;
+  s->w = w;
+  s->flags = flags;
+  s->storage = layers[0]->d.storage;
+  const size_t es = (s->storage == PCONV_F16) ? 2 : 4;
+  int ch = h, cw = w, cc = layers[0]->d.c_in;
+  size_t max_act = 0;
+  s->in_bytes = (size_t)n * cc * h * w * es;
+  for (int i = 0; i < n_layers; ++i) {
+    const pconv::DeviceLayer& L = layers[i]->d;
+    s->layers[i] = layers[i];
+    s->bias[i] = bias_dev ? bias_dev[i] : nullptr;
+    s->pool[i] = pool_after ? pool_after[i] : 0;
+    if (L.storage != s->storage || L.c_in != cc) {
+      pconv_stack_free(s);
+      return PCONV_ERR_SHAPE;
+    }
+    ch = (ch - 1) / L.stride + 1;
+    cw = (cw - 1) / L.stride + 1;
+    cc = L.c_out;
+    const size_t bytes = (size_t)n * cc * ch * cw * es;
+    if (bytes > max_act) max_act = bytes;
+    if (s->pool[i]) {
+      if (ch < 2 || cw < 2) {
+        pconv_stack_free(s);
+        return PCONV_ERR_SHAPE;
+      }
+      ch /= 2;
+      cw /= 2;
+    }
+  }
+  s->out_c = cc;
+  s->out_h = ch;
+  s->out_w = cw;
+  s->out_bytes = (size_t)n * cc * ch * cw * es;
+  s->act_bytes = max_act;
+  cudaError_t e = cudaMalloc(&s->act[0], max_act);
+  if (e == cudaSuccess) e = cudaMalloc(&s->act[1], max_act);
+  if (e == cudaSuccess) e = cudaMalloc(&s->io[0], s->in_bytes);
+  if (e == cudaSuccess) e = cudaMalloc(&s->io[1], s->out_bytes);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    pconv_stack_free(s);
+    return PCONV_ERR_ALLOC;
+  }
+  *out = s;
+  return PCONV_OK;
+}
+
+extern "C" pconv_status pconv_stack_out_shape(const pconv_stack* s, int* n, int* c, int* h,
+                                              int* w) {
+  if (!s) return PCONV_ERR_NULL;
+  if (n) *n = s->n;
+  if (c) *c = s->out_c;
+  if (h) *h = s->out_h;
+  if (w) *w = s->out_w;
+  return PCONV_OK;
+}
+
+extern "C" pconv_status pconv_stack_forward(pconv_stack* s, const void* x, void* y, void* stream) {
+  if (!s || !x || !y) return PCONV_ERR_NULL;
+  const void* cur = x;
+  int ch = s->h, cw = s->w, which = 0;
+  for (int i = 0; i < s->n_layers; ++i) {
+    const pconv::DeviceLayer& L = s->layers[i]->d;
+    const bool last_op = (i == s->n_layers - 1) && !s->pool[i];
+    void* dst = last_op ? y : s->act[which];
+    pconv_status st = pconv_forward(s->layers[i], cur, s->bias[i], dst, s->n, ch, cw, s->flags, stream);
+    if (st != PCONV_OK) return st;
+    ch = (ch - 1) / L.stride + 1;
+    cw = (cw - 1) / L.stride + 1;
+    cur = dst;
+    which ^= 1;
+    if (s->pool[i]) {
+      void* pd = (i == s->n_layers - 1) ? y : s->act[which];
+      st = pconv_maxpool2x2(cur, pd, s->n, L.c_out, ch, cw, s->storage, stream);
+      if (st != PCONV_OK) return st;
+      ch /= 2;
+      cw /= 2;
+      cur = pd;
+      which ^= 1;
+    }
+  }
+  return PCONV_OK;
+}
+
+extern "C" pconv_status pconv_stack_forward_host(pconv_stack* s, const void* x_host, void* y_host,
+                                                 void* stream_v) {
+  if (!s || !x_host || !y_host) return PCONV_ERR_NULL;
+  cudaStream_t stream = (cudaStream_t)stream_v;
+  if (cudaMemcpyAsync(s->io[0], x_host, s->in_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+    cudaGetLastError();
+    return PCONV_ERR_CUDA;
+  }
+  pconv_status st = pconv_stack_forward(s, s->io[0], s->io[1], stream_v);
+  if (st != PCONV_OK) return st;
+  if (cudaMemcpyAsync(y_host, s->io[1], s->out_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      cudaStreamSynchronize(stream) != cudaSuccess) {
+    cudaGetLastError();
+    return PCONV_ERR_CUDA;
+  }
+  return PCONV_OK;
+}

@@ -1,0 +1,81 @@
+// Internal declarations shared by the packer, the C ABI and the kernels (product code only).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "../../include/pconv.h"
+
+namespace pconv {
+
+constexpr int kGroup = 16;         // filters per group (accumulator rows of one consumer warp)
+constexpr int kChunk = 8;          // input channels per pipeline stage
+constexpr int kMaxBlockKernels = kGroup * kChunk;
+
+// Specialised code stream (one byte per entry) -- valid when the pattern set is a subset of the
+// eight masks the tiled kernel has straight-line bodies for.
+//   0..127        kernel: filter slot g = code >> 3, canonical pattern = code & 7
+//   128..135      advance (code - 127) channels inside the chunk and load that channel's window
+//   255           end of this (group, chunk) block
+constexpr int kCodeNext = 128;
+constexpr int kCodeEnd = 255;
+// Generic code stream (two bytes per entry) -- any 4-of-9 mask.
+//   (g << 9) | mask   kernel with run-time mask;   0x2000 | (adv-1)   advance;   0x4000   end
+constexpr int kGenNext = 0x2000;
+constexpr int kGenEnd = 0x4000;
+
+// The eight masks with specialised bodies, in canonical order (bit 3u+v).
+constexpr uint16_t kCanonMasks[8] = {0x03A, 0x09A, 0x0B8, 0x0B2, 0x01B, 0x036, 0x0D8, 0x1B0};
+
+struct BlockDesc {      // one per (group, chunk); 32 bytes
+  uint32_t w_off;       // first kernel record of the block in the value stream
+  uint32_t n_k;         // kernel records in the block (<= kMaxBlockKernels)
+  uint32_t cs_off;      // byte offset of the specialised codes (4-byte aligned)
+  uint32_t cs_len;      // specialised code bytes including the end code
+  uint32_t cg_off;      // byte offset of the generic codes (4-byte aligned)
+  uint32_t cg_len;      // generic code bytes including the end code
+  uint32_t pad0, pad1;
+};
+
+struct DeviceLayer {         // device pointers of one packed layer (passed to kernels by value)
+  // per-filter lists in original filter order (simple kernel)
+  const int* row_ptr;        // [c_out + 1]
+  const uint32_t* csr_idx;   // channel | mask << 16
+  const float* csr_val;      // 4 floats per kernel
+  // grouped / chunked streams (tiled kernel)
+  const BlockDesc* blocks;   // [n_groups][n_chunks]
+  const void* wvals;         // 4 values per kernel: fp32 (16 B) or fp16 (8 B)
+  const uint8_t* codes_s;    // specialised codes (may be null)
+  const uint8_t* codes_g;    // generic codes
+  const int* perm;           // [n_groups * kGroup] original filter index or -1
+  int* err;                  // device status word (0 = fine)
+  int c_out, c_in, stride, storage, n_groups, n_chunks;
+};
+
+}  // namespace pconv
+
+struct pconv_handle {
+  pconv::DeviceLayer d;
+  int device;
+  int n_patterns;
+  uint16_t patterns[PCONV_MAX_PATTERNS];
+  int canon_id[PCONV_MAX_PATTERNS];  // canonical index of each pattern or -1
+  bool canonical;
+  pconv_stats_t stats;
+  long long n_kept;
+  size_t wvals_bytes, codes_s_bytes, codes_g_bytes;
+  void* dev_block;                   // the single device allocation
+  size_t dev_bytes;
+};
+
+namespace pconv {
+// kernels (defined in the .cu files); all asynchronous on `stream`
+cudaError_t launch_simple(const DeviceLayer& L, const void* x, const float* bias, void* y, int n,
+                          int h, int w, bool relu, cudaStream_t stream);
+cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias, void* y, int n,
+                         int h, int w, bool relu, bool generic_taps, cudaStream_t stream);
+bool tiled_supported(const DeviceLayer& L, int n, int h, int w);
+cudaError_t launch_maxpool(const void* x, void* y, int n, int c, int h, int w, int storage,
+                           cudaStream_t stream);
+}  // namespace pconv

@@ -1,0 +1,203 @@
+"""GPU parity: the CUDA library, called through the C ABI, against the CPU oracle on the same
+seeded inputs -- element by element, at sizes that span several tiles and ragged tails."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1909_05073_b200 import binding as B
+from paper_1909_05073_b200 import build as pbuild
+from paper_1909_05073_b200 import synth
+from util import check_close
+
+pytestmark = pytest.mark.gpu
+
+KERNELS = {"simple": B.KERNEL_SIMPLE, "tiled": B.KERNEL_TILED, "generic": B.KERNEL_GENERIC_TAPS,
+           "auto": 0}
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    pbuild.build()
+    B.lib()
+
+
+def run_layer(w, bias, x, stride=1, storage="f32", relu=True, kernel="auto", patterns=None):
+    st = B.F16 if storage == "f16" else B.F32
+    layer = B.Layer(w, patterns or synth.PATTERNS8, stride, st, bias)
+    xt = torch.from_numpy(x).cuda()
+    if storage == "f16":
+        xt = xt.half()
+    y = layer.forward(xt, relu=relu, kernel=KERNELS[kernel])
+    torch.cuda.synchronize()
+    status, where = B.pconv_device_status(layer.handle)
+    assert status == 0, ("device status", status, where)
+    layer.close()
+    return y.float().cpu().numpy()
+
+
+def oracle_layer(w, bias, x, stride=1, storage="f32", relu=True):
+    return oracle.conv3x3(x, w, bias, stride, relu, storage)
+
+
+SMALL = [  # (c_in, c_out, h, w, n, stride, keep)
+    (1, 1, 1, 1, 1, 1, 1.0),
+    (3, 5, 5, 7, 2, 1, 0.7),
+    (5, 17, 9, 9, 3, 1, 0.5),
+    (9, 33, 6, 35, 2, 1, 0.4),      # one column past a 32-wide tile
+    (16, 16, 37, 33, 1, 1, 0.3),
+    (20, 40, 14, 14, 2, 1, 0.35),
+    (8, 24, 7, 7, 5, 1, 0.5),
+    (4, 16, 2, 2, 9, 1, 0.6),
+    (7, 19, 4, 4, 6, 1, 0.5),
+    (3, 5, 5, 7, 2, 2, 0.7),
+    (12, 20, 28, 28, 2, 2, 0.4),
+    (16, 32, 14, 14, 3, 2, 0.35),
+    (6, 16, 9, 11, 2, 2, 0.5),
+    (5, 8, 1, 9, 2, 2, 0.8),
+]
+
+
+@pytest.mark.parametrize("kernel", ["simple", "tiled", "generic", "auto"])
+@pytest.mark.parametrize("storage", ["f32", "f16"])
+@pytest.mark.parametrize("case", SMALL, ids=lambda c: "x".join(str(v) for v in c))
+def test_small_layers_match_the_oracle(case, storage, kernel):
+    c_in, c_out, h, w, n, stride, keep = case
+    spec = synth.LayerSpec("t", c_in, c_out, h, w, stride, keep)
+    seed = 1000 + c_in * 7 + c_out + h
+    wt, bias, _ = synth.gen_weights(spec, seed)
+    x = synth.gen_input(spec, n, seed)
+    for relu in (True, False):
+        got = run_layer(wt, bias, x, stride, storage, relu, kernel)
+        ref = oracle_layer(wt, bias, x, stride, storage, relu)
+        check_close(got, ref, storage, "%s relu=%s" % (case, relu))
+
+
+@pytest.mark.parametrize("kernel", ["simple", "tiled", "generic"])
+def test_config1_full_layer(kernel):
+    cfg = synth.config(1)
+    spec = cfg.layers[0]
+    wt, bias, _ = synth.gen_weights(spec, synth.layer_seed(1, 0))
+    x = synth.gen_input(spec, cfg.batch, synth.layer_seed(1, 0))
+    got = run_layer(wt, bias, x, kernel=kernel)
+    check_close(got, oracle_layer(wt, bias, x), "f32", "config 1")
+
+
+@pytest.mark.parametrize("kernel", ["simple", "tiled", "generic"])
+@pytest.mark.parametrize("stride", [1, 2])
+def test_single_tap_shift_through_the_gpu(kernel, stride):
+    """Each of the 9 taps alone is a sub-support of some pattern (non-strict packing), and the
+    output must be the shifted, zero-filled input exactly."""
+    rng = np.random.default_rng(4)
+    h, w = 9, 13
+    x = rng.normal(size=(1, 3, h, w)).astype(np.float32)
+    for t in range(9):
+        wt = np.zeros((2, 3, 3, 3), np.float32)
+        wt[1, 2, t // 3, t % 3] = 1.0
+        got = run_layer(wt, None, x, stride, "f32", False, kernel)
+        ref = oracle_layer(wt, None, x, stride, "f32", False)
+        assert np.array_equal(got, ref), t
+        assert not got[:, 0].any()
+
+
+@pytest.mark.parametrize("kernel", ["simple", "tiled", "generic"])
+def test_empty_filters_and_no_bias(kernel):
+    spec = synth.LayerSpec("t", 6, 20, 10, 10, 1, 0.5)
+    wt, bias, _ = synth.gen_weights(spec, 77)
+    wt[3] = 0
+    wt[17] = 0
+    x = synth.gen_input(spec, 2, 77)
+    got = run_layer(wt, bias, x, kernel=kernel)
+    check_close(got, oracle_layer(wt, bias, x), "f32", "empty filters")
+    assert np.allclose(got[:, 3], max(bias[3], 0.0))
+    allzero = np.zeros_like(wt)
+    got = run_layer(allzero, None, x, relu=False, kernel=kernel)
+    assert not got.any()
+
+
+@pytest.mark.parametrize("kernel", ["simple", "generic", "auto"])
+def test_twelve_patterns_and_noncanonical_sets(kernel):
+    spec = synth.LayerSpec("t", 24, 40, 18, 21, 1, 0.4, probs=(1 / 12,) * 12)
+    wt, bias, ids = synth.gen_weights(spec, 5, synth.PATTERNS12)
+    assert ids.max() == 11
+    x = synth.gen_input(spec, 2, 5)
+    got = run_layer(wt, bias, x, kernel=kernel, patterns=synth.PATTERNS12)
+    check_close(got, oracle_layer(wt, bias, x), "f32", "12 patterns")
+
+
+@pytest.mark.parametrize("storage", ["f32", "f16"])
+def test_pack_unpack_round_trip_and_stats(storage):
+    for cid in (1, 3, 5):
+        cfg = synth.config(cid)
+        spec = cfg.layers[-1]
+        wt, bias, ids = synth.gen_weights(spec, synth.layer_seed(cid, 0))
+        layer = B.Layer(wt, cfg.patterns, spec.stride, B.F16 if storage == "f16" else B.F32,
+                        strict4=True)
+        back = layer.unpack()
+        expect = wt if storage == "f32" else wt.astype(np.float16).astype(np.float32)
+        assert np.array_equal(back, expect)
+        s = layer.stats()
+        kept = ids >= 0
+        assert s.kept_kernels == kept.sum()
+        assert sum(s.per_pattern[:8]) == s.kept_kernels
+        assert [s.per_pattern[p] for p in range(8)] == [(ids == p).sum() for p in range(8)]
+        assert s.min_per_filter == kept.sum(1).min() and s.max_per_filter == kept.sum(1).max()
+        assert s.canonical_patterns == 1
+        perm = B.pconv_filter_order(layer.handle)
+        assert sorted(perm[perm >= 0]) == list(range(spec.c_out))
+        # reorder balances groups: heaviest group within a few kernels of the lightest
+        assert s.max_group_kernels - s.min_group_kernels <= max(16, 0.05 * s.max_group_kernels)
+        layer.close()
+
+
+def test_fp16_rounding_matches_ieee():
+    vals = np.concatenate([
+        np.random.default_rng(0).normal(0, 1, 2000), np.random.default_rng(1).normal(0, 1e-5, 2000),
+        np.array([65504.0, 65519.9, 6.1e-5, 5.96e-8, 2.98e-8, 2.9e-8, 3.1e-8, 1e-9, -0.0,
+                  1.0009765625, 1.00048828125, 1.00146484375])]).astype(np.float32)
+    n = (len(vals) + 3) // 4
+    wt = np.zeros((1, n, 3, 3), np.float32)
+    pos = [(0, 1), (1, 0), (1, 1), (1, 2)]       # pattern id 0
+    flat = np.resize(vals, 4 * n)
+    for c in range(n):
+        for s, (u, v) in enumerate(pos):
+            wt[0, c, u, v] = flat[4 * c + s]
+    layer = B.Layer(wt, synth.PATTERNS8, 1, B.F16)
+    assert np.array_equal(layer.unpack(), wt.astype(np.float16).astype(np.float32))
+    layer.close()
+
+
+def test_forward_argument_errors():
+    spec = synth.LayerSpec("t", 4, 4, 8, 8, 1, 0.5)
+    wt, bias, _ = synth.gen_weights(spec, 1)
+    layer = B.Layer(wt, synth.PATTERNS8)
+    x = torch.zeros(1, 4, 8, 8, device="cuda")
+    y = torch.zeros(1, 4, 8, 8, device="cuda")
+    with pytest.raises(B.PconvError) as e:
+        B.pconv_forward(layer.handle, x, None, y, flags=0x8000)
+    assert e.value.status == 6
+    with pytest.raises(B.PconvError) as e:
+        B.pconv_forward(layer.handle, x, None, y, flags=B.KERNEL_SIMPLE | B.KERNEL_TILED)
+    assert e.value.status == 6
+    with pytest.raises(B.PconvError) as e:
+        B.pconv_forward(layer.handle, x, None, x)                    # aliasing
+    assert e.value.status == 2
+    with pytest.raises(B.PconvError) as e:
+        B.pconv_forward(layer.handle, x.view(-1)[1:].view(-1)[:252].view(1, 4, 7, 9), None, y)
+    assert e.value.status == 7                                       # misaligned x
+    layer.close()
+
+
+@pytest.mark.parametrize("storage", ["f32", "f16"])
+def test_maxpool_matches_the_oracle(storage):
+    rng = np.random.default_rng(9)
+    for shape in [(2, 3, 8, 6), (1, 5, 7, 9), (3, 2, 2, 2)]:
+        x = rng.normal(size=shape).astype(np.float32)
+        xt = torch.from_numpy(x).cuda()
+        if storage == "f16":
+            xt = xt.half()
+            x = xt.float().cpu().numpy()
+        y = torch.empty(shape[0], shape[1], shape[2] // 2, shape[3] // 2, dtype=xt.dtype,
+                        device="cuda")
+        B.pconv_maxpool2x2(xt, y)
+        assert np.array_equal(y.float().cpu().numpy(), oracle.maxpool2x2(x))
