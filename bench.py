@@ -1,0 +1,312 @@
+#!/usr/bin/env python
+"""Benchmark of the PCONV forward path: the VGG-16 conv stack (13 pattern-sparse 3x3 layers and
+the four 2x2 max-pools between the blocks) on one 224x224 image per GPU, fp32.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A step is one pass of the whole stack over one image (per rank).  `value` is effective TFLOP/s
+(2 x surviving multiply-adds of all ranks / device time, inputs resident in HBM); `e2e` is the same
+figure through the host entry point (input copied from pinned host memory and the result copied
+back inside the timed region).  `--impl reference` times the CPU oracle on the same workload.
+Under torchrun every rank runs its own image (batch sharding, no collective on the data path).
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_1909_05073_b200 import synth  # noqa: E402
+
+CID = 2
+METRIC = "pattern-conv effective TFLOP/s (2 x surviving MACs / s), VGG-16 conv stack, batch 1 per GPU"
+# FP32 FMA peak of the part: SMs x 128 lanes x 2 flop x max SM clock
+ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+
+
+def build_workload():
+    cfg = synth.config(CID)
+    layers = []
+    for li, spec in enumerate(cfg.layers):
+        w, b, ids = synth.gen_weights(spec, synth.layer_seed(CID, li), cfg.patterns)
+        layers.append((spec, w, b, int((ids >= 0).sum())))
+    x = synth.gen_input(cfg.layers[0], 1, synth.layer_seed(CID, 0))
+    return cfg, layers, x
+
+
+def surviving_flops(layers):
+    return sum(2 * 4 * kept * s.h_out * s.w_out for s, _, _, kept in layers)
+
+
+def algorithmic_bytes(layers):
+    """Minimal HBM bytes of the conv layers: input once, output once, 4 values + 2 index bytes per
+    surviving kernel, bias."""
+    return sum(4 * (s.c_in * s.h * s.w + s.c_out * s.h_out * s.w_out) + kept * 18 + 4 * s.c_out
+               for s, _, _, kept in layers)
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        clocks, reasons, mx = [], set(), None
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 6:
+                continue
+            try:
+                clocks.append(float(r[0]))
+                mx = float(r[1])
+            except ValueError:
+                continue
+            for n, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(clocks) if clocks else None, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(clocks)}
+
+
+def run_reference(args):
+    """The CPU oracle, as it stands, on the same stack: one image per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    cfg, layers, x = build_workload()
+    flops = surviving_flops(layers)
+
+    def step():
+        a = x
+        for spec, w, b, _ in layers:
+            a = oracle.conv3x3(a, w, b, spec.stride, True)
+            if spec.pool_after:
+                a = oracle.maxpool2x2(a)
+        return a
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    ms = dt / args.steps * 1e3
+    val = flops / (ms * 1e-3) / 1e12
+    cores = oracle.num_threads()
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "config 2: VGG-16 conv stack, 224x224x3, batch 1, fp32, 8 patterns, "
+                               "keep 1.0 / 0.3", "images_per_step": 1},
+        "ms_per_image": ms,
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
+                         "sample": "whole stack (13 conv + 4 pool), 1 image per step, dense "
+                                   "direct convolution in fp64"},
+        "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_1909_05073_b200 import binding as B
+    from paper_1909_05073_b200 import build as pbuild
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA library is the only implementation")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if local == 0:
+        pbuild.build()
+    if world > 1:
+        dist.barrier()
+    B.lib()
+
+    cfg, layers, x_np = build_workload()
+    flops = surviving_flops(layers)
+    conv_layers = [B.Layer(w, cfg.patterns, s.stride, B.F32, b, strict4=True) for s, w, b, _ in layers]
+    pools = [s.pool_after for s, _, _, _ in layers]
+    spec0 = layers[0][0]
+    stack = B.Stack(conv_layers, pools, 1, spec0.h, spec0.w, B.RELU)
+    x = torch.from_numpy(x_np).cuda()
+    y = torch.empty(stack.out_shape, dtype=torch.float32, device="cuda")
+    x_host = torch.from_numpy(x_np).pin_memory()
+    y_host = torch.empty(stack.out_shape, dtype=torch.float32).pin_memory()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # > 126 MB of L2
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- device-resident timing -----------------------------------------------------------------
+    for _ in range(args.warmup):
+        stack.forward(x, y)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    sync_all()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+          for _ in range(args.steps)]
+    for e0, e1 in ev:
+        flush.zero_()
+        e0.record()
+        stack.forward(x, y)
+        e1.record()
+    sync_all()
+    ms_total = sum(e0.elapsed_time(e1) for e0, e1 in ev)
+
+    # ---- per-kernel pass: the dominant kernel's launches timed one by one ------------------------
+    acts = []
+    a = x
+    for layer, pool in zip(conv_layers, pools):
+        o = torch.empty(layer.out_shape(a.shape), dtype=torch.float32, device="cuda")
+        acts.append((a, o))
+        a = o
+        if pool:
+            p = torch.empty(o.shape[0], o.shape[1], o.shape[2] // 2, o.shape[3] // 2,
+                            dtype=torch.float32, device="cuda")
+            B.pconv_maxpool2x2(o, p)
+            a = p
+    conv_ms = [0.0] * len(conv_layers)
+    for _ in range(args.steps):
+        flush.zero_()
+        pairs = []
+        for layer, (xi, oi), pool in zip(conv_layers, acts, pools):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            layer.forward(xi, relu=True, out=oi)
+            e1.record()
+            pairs.append((e0, e1))
+        torch.cuda.synchronize()
+        for i, (e0, e1) in enumerate(pairs):
+            conv_ms[i] += e0.elapsed_time(e1) / args.steps
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- end to end through the host entry point -------------------------------------------------
+    for _ in range(min(args.warmup, 3)):
+        stack.forward_host(x_host, y_host)
+    sync_all()
+    e2e_total = 0.0
+    for _ in range(args.steps):
+        flush.zero_()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        stack.forward_host(x_host, y_host)      # synchronises its stream before returning
+        e2e_total += time.perf_counter() - t0
+    sync_all()
+
+    t = torch.tensor([ms_total, e2e_total * 1e3], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = float(t[0]) / args.steps
+    e2e_ms = float(t[1]) / args.steps
+    status, where = B.pconv_device_status(conv_layers[0].handle)
+    if status != 0:
+        raise SystemExit("device reported an abandoned wait (%d)" % where)
+
+    if rank == 0:
+        import oracle
+        t0 = time.perf_counter()
+        a_ref = x_np
+        for spec, w, b, _ in layers:
+            a_ref = oracle.conv3x3(a_ref, w, b, spec.stride, True)
+            if spec.pool_after:
+                a_ref = oracle.maxpool2x2(a_ref)
+        cpu_s = time.perf_counter() - t0
+        got = y_host.numpy()
+        err = np.abs(got - a_ref)
+        parity_ok = bool((err <= 1e-4 * (1 + np.abs(a_ref))).all())
+        conv_time_ms = sum(conv_ms)
+        achieved = flops / (conv_time_ms * 1e-3) / 1e12
+        value = world * flops / (ms_step * 1e-3) / 1e12
+        out = {
+            "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": {"workload": "config 2: VGG-16 conv stack, 224x224x3, batch 1 per GPU, fp32, "
+                                   "8 patterns, keep 1.0 (conv1) / 0.3", "images_per_step": world,
+                       "l2": "flushed between timed steps (256 MB write)", "parallelism": "batch sharding, no collective"},
+            "ms_per_image": ms_step,
+            "surviving_gflop_per_image": flops / 1e9,
+            "roofline_time_us_per_image": flops / (ALU_PEAK_TFLOPS * 1e12) * 1e6,
+            "clocks": clocks,
+            "e2e": {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                    "ms_per_step": e2e_ms, "h2d_bytes_per_step": int(x_host.numel() * 4),
+                    "d2h_bytes_per_step": int(y_host.numel() * 4)},
+            "gpu_launches": args.steps * (len(conv_layers) + sum(pools)),
+            "roofline": {"bound": "alu", "kernel": "tiled_kernel (13 conv launches per step)",
+                         "achieved": achieved, "peak": ALU_PEAK_TFLOPS, "unit": "TFLOP/s",
+                         "frac": achieved / ALU_PEAK_TFLOPS,
+                         "peak_source": "148 SMs x 128 FP32 lanes x 2 x 1.965 GHz (derived; "
+                                        "no FP32 figure in MEASURED_PEAKS.json)",
+                         "launch_ms_sum": conv_time_ms, "traffic": None,
+                         "algorithmic_bytes": algorithmic_bytes(layers),
+                         "per_layer_us": [round(m * 1e3, 2) for m in conv_ms]},
+            "cpu_baseline": {"value": flops / cpu_s / 1e12, "unit": "TFLOP/s",
+                             "cores": oracle.num_threads(), "kind": "oracle", "seconds": cpu_s,
+                             "sample": "whole stack, 1 image (dense direct convolution, fp64)"},
+            "parity": {"ok": parity_ok, "max_abs_err": float(err.max())},
+        }
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

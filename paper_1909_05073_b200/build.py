@@ -11,11 +11,21 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", 
               "-shared", "-Xcompiler", "-fPIC"]
 
 
+def generate():
+    """Writes the generated PTX dispatch text (csrc/dispatch_s*.inc) next to the sources."""
+    sys.path.insert(0, CSRC)
+    try:
+        import gen_dispatch
+        gen_dispatch.main(CSRC)
+    finally:
+        sys.path.remove(CSRC)
+
+
 def _stale():
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)]
+    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if not f.endswith(".inc")]
     deps.append(os.path.join(HERE, "..", "include", "pconv.h"))
     return any(os.path.getmtime(d) > t for d in deps)
 
@@ -24,6 +34,7 @@ def build(force=False, verbose=False):
     """Compile the CUDA library if it is missing or older than its sources; returns its path."""
     if not force and not _stale():
         return LIB
+    generate()
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = LIB + ".tmp%d" % os.getpid()
     cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + \

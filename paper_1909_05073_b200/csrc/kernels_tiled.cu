@@ -28,12 +28,12 @@ namespace {
 
 typedef unsigned long long u64;
 
-constexpr int kConsumerWarps = 8;
+constexpr int kConsumerWarps = 12;
 constexpr int kProducerWarps = 4;
 constexpr int kThreads = 32 * (kConsumerWarps + kProducerWarps);
 constexpr int kMaxStages = 4;
 constexpr int kWSlot = kMaxBlockKernels * 32;  // bytes per (group, stage): {w0,w0,w1,w1,w2,w2,w3,w3}
-constexpr int kCodeSlot = 288;                 // bytes per (group, stage)
+constexpr int kCodeSlot = 160;                 // bytes per (group, stage)
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr int kSmemLimit = 227 * 1024;
 
@@ -47,7 +47,7 @@ struct Geo {
   int wys, wy, ng;       // warp grid: warp -> (warp % wys, warp / wys); rows >= wy are idle
   int pairs;             // sub-tile pairs per CTA = wy * sw
   int rows, pitch, substride, chan_stride;  // float2 units
-  int stages, x_stage_bytes, stage_bytes, tab_off, stage_off;
+  int stages, x_stage_bytes, stage_bytes, tab_off, desc_off, stage_off;
   int relu, is_half;
 };
 
@@ -61,14 +61,6 @@ __device__ __forceinline__ void ffma2(u64& d, u64 a, u64 b) {
 __device__ __forceinline__ u64 lds64(uint32_t addr) {
   u64 v;
   asm volatile("ld.shared.b64 %0, [%1];" : "=l"(v) : "r"(addr));
-  return v;
-}
-__device__ __forceinline__ void lds128(u64& a, u64& b, uint32_t addr) {
-  asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "r"(addr));
-}
-__device__ __forceinline__ uint32_t lds_u8(uint32_t addr) {
-  uint32_t v;
-  asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(addr));
   return v;
 }
 __device__ __forceinline__ uint32_t lds_u16(uint32_t addr) {
@@ -85,6 +77,17 @@ __device__ __forceinline__ void sts128f(uint32_t addr, float a, float b, float c
 }
 __device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
   asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(src_bytes)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+// The mbarrier receives one arrival from this thread once all its earlier cp.async have landed.
+__device__ __forceinline__ void cp_async_arrive(uint32_t bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
@@ -111,41 +114,33 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* er
   return false;
 }
 
-// ---- compile-time tap tables ------------------------------------------------------------------------
-__host__ __device__ constexpr int nth_set_bit(unsigned mask, int n) {
-  int seen = 0;
-  for (int t = 0; t < 9; ++t)
-    if (mask >> t & 1) {
-      if (seen == n) return t;
-      ++seen;
-    }
-  return 0;
-}
-
 template <int S>
 struct Win {
   static constexpr int kRows = (S == 1) ? 6 : 9;
 };
 
-// One surviving kernel, specialised on its mask and filter slot: taps 0,1, refill their weight
-// registers with the next record, taps 2,3, refill (the refills complete under the other half's
-// FMAs and under the next dispatch).
-template <unsigned MASK, int S, int G>
-__device__ __forceinline__ void kernel_body(u64 (&acc)[kGroup][4], const u64 (&win)[Win<S>::kRows][3],
-                                            u64& w0, u64& w1, u64& w2, u64& w3, uint32_t& wp) {
-  constexpr int t0 = nth_set_bit(MASK, 0), t1 = nth_set_bit(MASK, 1);
-  constexpr int t2 = nth_set_bit(MASK, 2), t3 = nth_set_bit(MASK, 3);
-#pragma unroll
-  for (int k = 0; k < 4; ++k) ffma2(acc[G][k], win[S * k + t0 / 3][t0 % 3], w0);
-#pragma unroll
-  for (int k = 0; k < 4; ++k) ffma2(acc[G][k], win[S * k + t1 / 3][t1 % 3], w1);
-  lds128(w0, w1, wp);
-#pragma unroll
-  for (int k = 0; k < 4; ++k) ffma2(acc[G][k], win[S * k + t2 / 3][t2 % 3], w2);
-#pragma unroll
-  for (int k = 0; k < 4; ++k) ffma2(acc[G][k], win[S * k + t3 / 3][t3 % 3], w3);
-  lds128(w2, w3, wp + 16);
-  wp += 32;
+// The specialised dispatch loop of one (warp, chunk): generated PTX (see gen_dispatch.py) with an
+// indexed jump per byte code and one straight-line body per (filter slot, pattern).
+#define PC_ACC4(G) "+l"(acc[G][0]), "+l"(acc[G][1]), "+l"(acc[G][2]), "+l"(acc[G][3])
+#define PC_ACC_ALL \
+  PC_ACC4(0), PC_ACC4(1), PC_ACC4(2), PC_ACC4(3), PC_ACC4(4), PC_ACC4(5), PC_ACC4(6), PC_ACC4(7)
+template <int S>
+__device__ __forceinline__ void dispatch_chunk(u64 (&acc)[kGroup][4], uint32_t cp, uint32_t wp,
+                                               uint32_t xptr, uint32_t chan_b, uint32_t pitch_b,
+                                               uint32_t off_mid) {
+  if (S == 1) {
+    asm volatile(
+#include "dispatch_s1.inc"
+        : PC_ACC_ALL
+        : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(pitch_b), "r"(off_mid)
+        : "memory");
+  } else {
+    asm volatile(
+#include "dispatch_s2.inc"
+        : PC_ACC_ALL
+        : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(pitch_b), "r"(off_mid)
+        : "memory");
+  }
 }
 
 // Any 4-of-9 mask, taken at run time: nine warp-uniform tests, a weight load per taken tap.
@@ -176,29 +171,88 @@ __device__ __forceinline__ void load_window(u64 (&win)[Win<S>::kRows][3], uint32
   }
 }
 
-#define PC_CASE(G, P)                                                               \
-  case (G * 8 + P):                                                                  \
-    kernel_body<kCanonMasks[P], S, G>(acc, win, w0, w1, w2, w3, wp);                 \
-    break;
-#define PC_CASES(G) \
-  PC_CASE(G, 0) PC_CASE(G, 1) PC_CASE(G, 2) PC_CASE(G, 3) PC_CASE(G, 4) PC_CASE(G, 5) PC_CASE(G, 6) PC_CASE(G, 7)
 #define PG_CASE(G)                                          \
   case G:                                                   \
     kernel_body_generic<S, G>(acc, win, code & 0x1FFu, wp); \
     break;
 
-template <typename T>
-__device__ __forceinline__ float ldg_f(const T* p);
-template <>
-__device__ __forceinline__ float ldg_f<float>(const float* p) { return __ldg(p); }
-template <>
-__device__ __forceinline__ float ldg_f<__half>(const __half* p) { return __half2float(__ldg(p)); }
+__device__ __forceinline__ float ldg_f(const __half* p) { return __half2float(__ldg(p)); }
 
 // ---- producer: stage one chunk -----------------------------------------------------------------------
-template <int S, bool GENERIC, typename T>
-__device__ __forceinline__ void produce_chunk(const DeviceLayer& L, const Geo& g, const T* __restrict__ x,
-                                              const SubTile* tab, uint32_t stage_base, int k, int pw,
-                                              int lane) {
+// Input columns staged for row element i of a sub-tile, relative to its first output column
+// (stride 1: i-1; stride 2: the odd columns 2i-1 first, then the even columns).
+template <int S>
+__device__ __forceinline__ int staged_dx(int i, int tw) {
+  if (S == 1) return i - 1;
+  return (i <= tw) ? (2 * i - 1) : (2 * (i - tw - 1));
+}
+
+// fp32 storage: everything is fetched with cp.async (zero-fill outside the image), so the producer
+// never waits for data and several chunks are in flight; each thread's arrival on the stage's full
+// barrier fires when its own copies have landed.
+template <int S>
+__device__ __forceinline__ void produce_chunk_async(const DeviceLayer& L, const Geo& g,
+                                                    const float* __restrict__ x, const SubTile* tab,
+                                                    const uint4* desc, const uint8_t* codes,
+                                                    uint32_t stage_base, int k, int pw, int lane) {
+  const int c0 = k * kChunk;
+  const int nc = min(kChunk, L.c_in - c0);
+  const size_t hw = (size_t)g.h * g.w;
+  const int n_rows = g.pairs * g.rows;
+  const uint32_t chan_b = (uint32_t)g.chan_stride * 8u;
+  for (int row = pw; row < n_rows; row += kProducerWarps) {
+    const int p = row / g.rows, r = row - p * g.rows;
+    const SubTile A = tab[2 * p], B = tab[2 * p + 1];
+    const int iyA = A.y0 * S - 1 + r, iyB = B.y0 * S - 1 + r;
+    const bool vA = A.valid && iyA >= 0 && iyA < g.h;
+    const bool vB = B.valid && iyB >= 0 && iyB < g.h;
+    const float* pa = x + ((size_t)A.n * L.c_in + c0) * hw + (size_t)(vA ? iyA : 0) * g.w;
+    const float* pb = x + ((size_t)B.n * L.c_in + c0) * hw + (size_t)(vB ? iyB : 0) * g.w;
+    const uint32_t dst_row = stage_base + (uint32_t)((p * g.substride + r * g.pitch) * 8);
+    for (int i = lane; i < g.pitch; i += 32) {
+      const int dx = staged_dx<S>(i, g.tw);
+      const int ixA = A.x0 * S + dx, ixB = B.x0 * S + dx;
+      const bool okA = vA && ixA >= 0 && ixA < g.w;
+      const bool okB = vB && ixB >= 0 && ixB < g.w;
+      const float* sa = okA ? pa + ixA : x;
+      const float* sb = okB ? pb + ixB : x;
+      const size_t step_a = okA ? hw : 0, step_b = okB ? hw : 0;
+      const uint32_t na = okA ? 4u : 0u, nb = okB ? 4u : 0u;
+      uint32_t dst = dst_row + (uint32_t)i * 8;
+      for (int cc = 0; cc < nc; ++cc) {
+        cp_async4(dst, sa, na);
+        cp_async4(dst + 4, sb, nb);
+        sa += step_a;
+        sb += step_b;
+        dst += chan_b;
+      }
+    }
+  }
+  const int ptid = pw * 32 + lane;
+  const uint32_t wbase = stage_base + g.x_stage_bytes;
+  const uint32_t cbase = wbase + g.ng * kWSlot;
+  for (int j = 0; j < g.ng; ++j) {
+    const uint4 d = desc[j * L.n_chunks + k];  // {w_off, n_k, code_off, code_len}
+    if ((uint32_t)ptid < d.y) {
+      const float* src = reinterpret_cast<const float*>(L.wvals) + (size_t)(d.x + ptid) * 4;
+      const uint32_t wd = wbase + j * kWSlot + ptid * 32;
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        cp_async4(wd + 8 * t, src + t, 4);
+        cp_async4(wd + 8 * t + 4, src + t, 4);
+      }
+    }
+    if ((uint32_t)ptid * 16 < d.w) cp_async16(cbase + j * kCodeSlot + ptid * 16, codes + d.z + ptid * 16);
+  }
+}
+
+// fp16 storage: loads, converts to fp32 and stores (the interleaved fp32 layout cannot be produced
+// by an asynchronous copy of 2-byte elements).
+template <int S>
+__device__ __forceinline__ void produce_chunk_half(const DeviceLayer& L, const Geo& g,
+                                                   const __half* __restrict__ x, const SubTile* tab,
+                                                   const uint4* desc, const uint8_t* codes,
+                                                   uint32_t stage_base, int k, int pw, int lane) {
   const int c0 = k * kChunk;
   const int nc = min(kChunk, L.c_in - c0);
   const size_t hw = (size_t)g.h * g.w;
@@ -209,13 +263,11 @@ __device__ __forceinline__ void produce_chunk(const DeviceLayer& L, const Geo& g
     const int iyA = A.y0 * S - 1 + r, iyB = B.y0 * S - 1 + r;
     const bool vA = A.valid && iyA >= 0 && iyA < g.h;
     const bool vB = B.valid && iyB >= 0 && iyB < g.h;
-    const T* pa = x + ((size_t)A.n * L.c_in + c0) * hw + (size_t)(vA ? iyA : 0) * g.w;
-    const T* pb = x + ((size_t)B.n * L.c_in + c0) * hw + (size_t)(vB ? iyB : 0) * g.w;
+    const __half* pa = x + ((size_t)A.n * L.c_in + c0) * hw + (size_t)(vA ? iyA : 0) * g.w;
+    const __half* pb = x + ((size_t)B.n * L.c_in + c0) * hw + (size_t)(vB ? iyB : 0) * g.w;
     const uint32_t dst_row = stage_base + (uint32_t)((p * g.substride + r * g.pitch) * 8);
     for (int i = lane; i < g.pitch; i += 32) {
-      int dx;  // input column relative to the sub-tile's first output column (in input units)
-      if (S == 1) dx = i - 1;
-      else dx = (i <= g.tw) ? (2 * i - 1) : (2 * (i - g.tw - 1));
+      const int dx = staged_dx<S>(i, g.tw);
       const int ixA = A.x0 * S + dx, ixB = B.x0 * S + dx;
       const bool okA = vA && ixA >= 0 && ixA < g.w;
       const bool okB = vB && ixB >= 0 && ixB < g.w;
@@ -230,39 +282,25 @@ __device__ __forceinline__ void produce_chunk(const DeviceLayer& L, const Geo& g
       for (int cc = 0; cc < kChunk; ++cc) sts64f(dst + (uint32_t)(cc * g.chan_stride) * 8, va[cc], vb[cc]);
     }
   }
-  // weight records and codes of the CTA's groups
   const int ptid = pw * 32 + lane;
   const uint32_t wbase = stage_base + g.x_stage_bytes;
   const uint32_t cbase = wbase + g.ng * kWSlot;
   for (int j = 0; j < g.ng; ++j) {
-    const int gi = blockIdx.y * g.ng + j;
-    const uint32_t cdst = cbase + j * kCodeSlot;
-    if (gi >= L.n_groups) {
-      if (ptid == 0) sts32(cdst, GENERIC ? 0x40004000u : 0xFFFFFFFFu);
-      continue;
-    }
-    const uint4 b0 = __ldg(reinterpret_cast<const uint4*>(L.blocks + (size_t)gi * L.n_chunks + k));
-    const uint4 b1 = __ldg(reinterpret_cast<const uint4*>(L.blocks + (size_t)gi * L.n_chunks + k) + 1);
-    const uint32_t w_off = b0.x, n_k = b0.y;
-    const uint32_t c_off = GENERIC ? b1.x : b0.z, c_len = GENERIC ? b1.y : b0.w;
-    if ((uint32_t)ptid < n_k) {
-      float4 v;
-      if (sizeof(T) == 4) {
-        v = __ldg(reinterpret_cast<const float4*>(L.wvals) + w_off + ptid);
-      } else {
-        const uint2 raw = __ldg(reinterpret_cast<const uint2*>(L.wvals) + w_off + ptid);
-        const __half2 lo = *reinterpret_cast<const __half2*>(&raw.x);
-        const __half2 hi = *reinterpret_cast<const __half2*>(&raw.y);
-        v = make_float4(__low2float(lo), __high2float(lo), __low2float(hi), __high2float(hi));
-      }
+    const uint4 d = desc[j * L.n_chunks + k];
+    if ((uint32_t)ptid < d.y) {
+      const uint2 raw = __ldg(reinterpret_cast<const uint2*>(L.wvals) + d.x + ptid);
+      const __half2 lo = *reinterpret_cast<const __half2*>(&raw.x);
+      const __half2 hi = *reinterpret_cast<const __half2*>(&raw.y);
       const uint32_t wd = wbase + j * kWSlot + ptid * 32;
-      sts128f(wd, v.x, v.x, v.y, v.y);
-      sts128f(wd + 16, v.z, v.z, v.w, v.w);
+      sts128f(wd, __low2float(lo), __low2float(lo), __high2float(lo), __high2float(lo));
+      sts128f(wd + 16, __low2float(hi), __low2float(hi), __high2float(hi), __high2float(hi));
     }
-    const uint32_t n_words = (c_len + 3) >> 2;
-    const uint8_t* codes = GENERIC ? L.codes_g : L.codes_s;
-    if ((uint32_t)ptid < n_words)
-      sts32(cdst + ptid * 4, __ldg(reinterpret_cast<const uint32_t*>(codes + c_off) + ptid));
+    if ((uint32_t)ptid * 16 < d.w) {
+      const uint4 cv = __ldg(reinterpret_cast<const uint4*>(codes + d.z) + ptid);
+      asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(cbase + j * kCodeSlot + ptid * 16),
+                   "r"(cv.x), "r"(cv.y), "r"(cv.z), "r"(cv.w)
+                   : "memory");
+    }
   }
 }
 
@@ -277,7 +315,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
 
   if (tid == 0) {
     for (int s = 0; s < g.stages; ++s) {
-      mbar_init(sbase + 8 * s, kProducerWarps);
+      mbar_init(sbase + 8 * s, 32 * kProducerWarps);
       mbar_init(sbase + 8 * (kMaxStages + s), kConsumerWarps);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -295,28 +333,50 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
     t.x0 = (rem - tyi * g.tx) * g.tw;
     tab[i] = t;
   }
+  // block descriptors of the CTA's groups: {first record, records, code offset, code bytes}
+  uint4* desc = reinterpret_cast<uint4*>(smem + g.desc_off);
+  for (int i = tid; i < g.ng * L.n_chunks; i += kThreads) {
+    const int j = i / L.n_chunks, k = i - j * L.n_chunks;
+    const int gj = blockIdx.y * g.ng + j;
+    uint4 d = make_uint4(0u, 0u, 0u, 0u);
+    if (gj < L.n_groups) {
+      const uint4* src = reinterpret_cast<const uint4*>(L.blocks + (size_t)gj * L.n_chunks + k);
+      const uint4 b0 = __ldg(src), b1 = __ldg(src + 1);
+      d = GENERIC ? make_uint4(b0.x, b0.y, b1.x, b1.y) : make_uint4(b0.x, b0.y, b0.z, b0.w);
+    }
+    desc[i] = d;
+  }
+  // groups past the layer's last one never get codes staged: park an end code in every stage
+  for (int i = tid; i < g.ng * g.stages; i += kThreads) {
+    const int j = i % g.ng, s = i / g.ng;
+    if ((int)(blockIdx.y * g.ng + j) >= L.n_groups)
+      sts32(sbase + g.stage_off + s * g.stage_bytes + g.x_stage_bytes + g.ng * kWSlot + j * kCodeSlot,
+            GENERIC ? 0x40004000u : 0x48484848u);
+  }
   __syncthreads();
 
   if (warp >= kConsumerWarps) {
     // ===================================== producer warps =====================================
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
     const int pw = warp - kConsumerWarps;
+    const uint8_t* codes = GENERIC ? L.codes_g : L.codes_s;
     for (int k = 0; k < L.n_chunks; ++k) {
       const int s = k % g.stages, it = k / g.stages;
       if (it > 0 && !mbar_wait(sbase + 8 * (kMaxStages + s), (it - 1) & 1, L.err, 1)) return;
       const uint32_t stage_base = sbase + g.stage_off + s * g.stage_bytes;
-      if (g.is_half)
-        produce_chunk<S, GENERIC, __half>(L, g, (const __half*)x, tab, stage_base, k, pw, lane);
-      else
-        produce_chunk<S, GENERIC, float>(L, g, (const float*)x, tab, stage_base, k, pw, lane);
-      __syncwarp();
-      if (lane == 0) mbar_arrive(sbase + 8 * s);
+      if (g.is_half) {
+        produce_chunk_half<S>(L, g, (const __half*)x, tab, desc, codes, stage_base, k, pw, lane);
+        mbar_arrive(sbase + 8 * s);
+      } else {
+        produce_chunk_async<S>(L, g, (const float*)x, tab, desc, codes, stage_base, k, pw, lane);
+        cp_async_arrive(sbase + 8 * s);
+      }
     }
     return;
   }
 
   // ======================================= consumer warps =======================================
-  asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 144;");
   const int wyi = warp % g.wys, wgi = warp / g.wys;
   const int gi = blockIdx.y * g.ng + wgi;
   const bool active = (wyi < g.wy) && (gi < L.n_groups);
@@ -342,32 +402,12 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
       uint32_t xptr = stage_base + lane_off - chan_b;  // one channel before the chunk
       uint32_t wp = stage_base + g.x_stage_bytes + wgi * kWSlot;
       uint32_t cp = stage_base + g.x_stage_bytes + g.ng * kWSlot + wgi * kCodeSlot;
-      u64 win[Win<S>::kRows][3];
-#pragma unroll
-      for (int r = 0; r < Win<S>::kRows; ++r) win[r][0] = win[r][1] = win[r][2] = 0ull;
       if (!GENERIC) {
-        u64 w0, w1, w2, w3;
-        lds128(w0, w1, wp);
-        lds128(w2, w3, wp + 16);
-        wp += 32;
-        uint32_t code = lds_u8(cp);
-        ++cp;
-        for (;;) {
-          const uint32_t next = lds_u8(cp);
-          ++cp;
-          switch (code) {
-            PC_CASES(0) PC_CASES(1) PC_CASES(2) PC_CASES(3) PC_CASES(4) PC_CASES(5) PC_CASES(6) PC_CASES(7)
-            PC_CASES(8) PC_CASES(9) PC_CASES(10) PC_CASES(11) PC_CASES(12) PC_CASES(13) PC_CASES(14) PC_CASES(15)
-            case 128: case 129: case 130: case 131: case 132: case 133: case 134: case 135:
-              xptr += (code - 127u) * chan_b;
-              load_window<S>(win, xptr, pitch_b, off_mid, off_right);
-              break;
-            default:
-              goto chunk_done;
-          }
-          code = next;
-        }
+        dispatch_chunk<S>(acc, cp, wp, xptr, chan_b, pitch_b, off_mid);
       } else {
+        u64 win[Win<S>::kRows][3];
+#pragma unroll
+        for (int r = 0; r < Win<S>::kRows; ++r) win[r][0] = win[r][1] = win[r][2] = 0ull;
         for (;;) {
           const uint32_t code = lds_u16(cp);
           cp += 2;
@@ -379,13 +419,11 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
           }
           switch (code >> 9) {
             PG_CASE(0) PG_CASE(1) PG_CASE(2) PG_CASE(3) PG_CASE(4) PG_CASE(5) PG_CASE(6) PG_CASE(7)
-            PG_CASE(8) PG_CASE(9) PG_CASE(10) PG_CASE(11) PG_CASE(12) PG_CASE(13) PG_CASE(14) PG_CASE(15)
             default: break;
           }
         }
       }
     }
-  chunk_done:
     __syncwarp();
     if (lane == 0) mbar_arrive(sbase + 8 * (kMaxStages + s));
   }
@@ -440,7 +478,7 @@ bool make_geo(const DeviceLayer& L, int n, int h, int w, Geo* out) {
   const long long q = (long long)n * g.tx * g.ty;
   if (q > 0x7FFFFFFF) return false;
   g.q_total = (int)q;
-  g.ng = (L.n_groups >= 3) ? 4 : L.n_groups;
+  g.ng = (L.n_groups >= 6) ? 6 : (L.n_groups == 5 ? 6 : L.n_groups);
   g.wys = kConsumerWarps / g.ng;
   g.wy = g.wys;
   g.rows = (L.stride == 1) ? 6 : 9;
@@ -449,12 +487,14 @@ bool make_geo(const DeviceLayer& L, int n, int h, int w, Geo* out) {
   if (g.tw < 16)  // spread the sub-tiles of a half-warp over distinct banks
     while (g.substride % 16 != g.tw % 16) ++g.substride;
   g.tab_off = 8 * 2 * kMaxStages;
+  if (L.n_chunks > 512) return false;  // descriptor table budget (c_in <= 4096)
   for (;;) {
     g.pairs = g.wy * g.sw;
     g.chan_stride = g.pairs * g.substride;
     g.x_stage_bytes = kChunk * g.chan_stride * 8;
     g.stage_bytes = (g.x_stage_bytes + g.ng * (kWSlot + kCodeSlot) + 15) & ~15;
-    g.stage_off = (g.tab_off + 2 * g.pairs * (int)sizeof(SubTile) + 15) & ~15;
+    g.desc_off = (g.tab_off + 2 * g.pairs * (int)sizeof(SubTile) + 15) & ~15;
+    g.stage_off = g.desc_off + g.ng * L.n_chunks * 16;
     g.stages = (kSmemLimit - g.stage_off) / g.stage_bytes;
     if (g.stages > kMaxStages) g.stages = kMaxStages;
     if (g.stages >= 2 || g.wy == 1) break;
@@ -488,7 +528,7 @@ cudaError_t launch_one(const DeviceLayer& L, const Geo& g, const void* x, const 
 bool tiled_supported(const DeviceLayer& L, int n, int h, int w) {
   Geo g;
   if (n <= 0 || h <= 0 || w <= 0) return false;
-  if ((L.n_groups + 3) / 4 > 65535) return false;
+  if (L.n_groups > 65535) return false;
   return make_geo(L, n, h, w, &g);
 }
 

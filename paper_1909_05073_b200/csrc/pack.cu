@@ -237,8 +237,8 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
         std::memset(&bd, 0, sizeof(bd));
         bd.w_off = (uint32_t)((storage == PCONV_F16 ? wv16.size() : wv32.size()) / 4);
         bd.n_k = (uint32_t)items.size();
-        while (codes_s.size() % 4) codes_s.push_back(kCodeEnd);
-        while (codes_g.size() % 4) codes_g.push_back(0);
+        while (codes_s.size() % 16) codes_s.push_back(kCodeEnd);
+        while (codes_g.size() % 16) codes_g.push_back(0);
         bd.cs_off = (uint32_t)codes_s.size();
         bd.cg_off = (uint32_t)codes_g.size();
         int pos = c0 - 1;  // channel whose window is loaded

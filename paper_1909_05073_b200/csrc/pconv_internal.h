@@ -9,17 +9,17 @@
 
 namespace pconv {
 
-constexpr int kGroup = 16;         // filters per group (accumulator rows of one consumer warp)
+constexpr int kGroup = 8;          // filters per group (accumulator rows of one consumer warp)
 constexpr int kChunk = 8;          // input channels per pipeline stage
 constexpr int kMaxBlockKernels = kGroup * kChunk;
 
 // Specialised code stream (one byte per entry) -- valid when the pattern set is a subset of the
 // eight masks the tiled kernel has straight-line bodies for.
-//   0..127        kernel: filter slot g = code >> 3, canonical pattern = code & 7
-//   128..135      advance (code - 127) channels inside the chunk and load that channel's window
-//   255           end of this (group, chunk) block
-constexpr int kCodeNext = 128;
-constexpr int kCodeEnd = 255;
+//   0..63         kernel: filter slot g = code >> 3, canonical pattern = code & 7
+//   64..71        advance (code - 63) channels inside the chunk and load that channel's window
+//   72            end of this (group, chunk) block
+constexpr int kCodeNext = kGroup * 8;
+constexpr int kCodeEnd = kCodeNext + kChunk;
 // Generic code stream (two bytes per entry) -- any 4-of-9 mask.
 //   (g << 9) | mask   kernel with run-time mask;   0x2000 | (adv-1)   advance;   0x4000   end
 constexpr int kGenNext = 0x2000;
@@ -31,9 +31,9 @@ constexpr uint16_t kCanonMasks[8] = {0x03A, 0x09A, 0x0B8, 0x0B2, 0x01B, 0x036, 0
 struct BlockDesc {      // one per (group, chunk); 32 bytes
   uint32_t w_off;       // first kernel record of the block in the value stream
   uint32_t n_k;         // kernel records in the block (<= kMaxBlockKernels)
-  uint32_t cs_off;      // byte offset of the specialised codes (4-byte aligned)
+  uint32_t cs_off;      // byte offset of the specialised codes (16-byte aligned)
   uint32_t cs_len;      // specialised code bytes including the end code
-  uint32_t cg_off;      // byte offset of the generic codes (4-byte aligned)
+  uint32_t cg_off;      // byte offset of the generic codes (16-byte aligned)
   uint32_t cg_len;      // generic code bytes including the end code
   uint32_t pad0, pad1;
 };

@@ -1,0 +1,42 @@
+"""One synthetic layer, a warm-up launch and `reps` timed launches: the small case used for ncu
+captures (`python -m paper_1909_05073_b200.profile_case 64 64 56 32 1 0.35 [tiled|generic|simple] [f32|f16]`)."""
+import sys
+
+import numpy as np
+import torch
+
+from paper_1909_05073_b200 import binding as B
+from paper_1909_05073_b200 import synth
+
+
+def run(c_in, c_out, h, n, stride, keep, kernel="tiled", storage="f32", reps=3):
+    sel = {"tiled": B.KERNEL_TILED, "generic": B.KERNEL_GENERIC_TAPS, "simple": B.KERNEL_SIMPLE,
+           "auto": 0}[kernel]
+    st = B.F16 if storage == "f16" else B.F32
+    spec = synth.LayerSpec("p", c_in, c_out, h, h, stride, keep)
+    w, b, ids = synth.gen_weights(spec, 1)
+    layer = B.Layer(w, synth.PATTERNS8, stride, st, b)
+    x = torch.from_numpy(synth.gen_input(spec, n, 1)).cuda()
+    if st == B.F16:
+        x = x.half()
+    y = layer.forward(x, kernel=sel)
+    torch.cuda.synchronize()
+    us = []
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        layer.forward(x, kernel=sel, out=y)
+        e1.record()
+        torch.cuda.synchronize()
+        us.append(e0.elapsed_time(e1) * 1e3)
+    flops = 8 * int((ids >= 0).sum()) * n * spec.h_out * spec.w_out
+    t = float(np.median(us))
+    print("%.1f us  %.2f effective TFLOP/s  (%.1f%% of 74.45)" % (t, flops / t / 1e6,
+                                                                flops / t / 1e6 / 0.7445))
+    assert B.pconv_device_status(layer.handle)[0] == 0
+    return t
+
+
+if __name__ == "__main__":
+    a = sys.argv[1:]
+    run(int(a[0]), int(a[1]), int(a[2]), int(a[3]), int(a[4]), float(a[5]), *(a[6:8]))
