@@ -1,28 +1,32 @@
 """Generates the PTX text of the tiled kernel's per-chunk dispatch loop (dispatch_s1.inc,
-dispatch_s2.inc), which kernels_tiled.cu includes inside one `asm volatile` statement.
+dispatch_s2.inc), which kernels_tmem.cu includes inside one `asm volatile` statement.
 
-Why PTX text: the loop needs a real indexed jump (`brx.idx`) from a warp-uniform byte code to a
-straight-line body specialised on (filter slot, pattern); a C++ `switch` is lowered to a compare
-tree (about 14 branches per kernel), and accumulator / window registers can only be indexed at
-compile time, so each (slot, pattern) pair needs its own body.  Threaded code: every body ends by
-fetching the code after next and jumping straight to the next body.
+Why PTX text, and why this shape (all measured on B200):
+ * accumulator and window registers can only be named at compile time, so every distinct
+   combination that the code must reach needs its own straight-line body;
+ * a warp-uniform jump to a *changing* target (`brx.idx`) costs ~100 cycles, which other warps can
+   hide only while the bodies being jumped between fit the ~8 KB instruction cache of an SM
+   sub-partition; bodies specialised on (filter slot, pattern) are 24-47 KB and ran at 6-16 % of
+   the FP32 peak, a C++ `switch` (lowered to a compare tree) no better, predicated-off FFMA2 cost
+   as much as executed ones;
+ * so the filter slot is taken out of the code: accumulators live in Tensor Memory (TMEM), which is
+   addressed at run time.  A body is specialised on the pattern only (8 bodies, ~4 KB): it waits for
+   the slot's 8 accumulator columns (loaded while the previous jump was in flight), runs the 16
+   packed FMAs of the 4 taps, stores the columns back, starts the load for the next kernel's slot
+   and jumps.
 
-Operands of the asm statement: %0..%31 accumulators acc[g][k] (packed float2, g-major),
-%32 code pointer, %33 weight pointer, %34 window pointer (one channel before the chunk),
-%35 channel stride, %36 row pitch, %37 offset of the middle window column (all in bytes,
-shared-memory addresses as u32).
+Operands of the asm statement (all u32): %0 code pointer, %1 weight pointer, %2 window pointer (one
+channel before the chunk), %3 channel stride, %4 row pitch, %5 offset of the middle window column
+(bytes, shared-memory addresses), %6 TMEM address of the warp's slot 0.
 
-Byte codes: 0..63 kernel (slot = code >> 3, canonical pattern = code & 7); 64..71 advance
-(code - 63) channels and reload the register window; 72 ends the chunk (no other value is ever
-dispatched).
+Byte codes (specialised stream): low nibble 0..7 = kernel with that canonical pattern, high nibble
+= filter slot; low nibble 8 = advance (high nibble + 1) channels and reload the register window;
+9 = end of the (group, chunk) block.
 """
 import os
 import sys
 
 CANON_MASKS = [0x03A, 0x09A, 0x0B8, 0x0B2, 0x01B, 0x036, 0x0D8, 0x1B0]
-GROUP = 8
-CHUNK = 8
-NACC = GROUP * 4
 
 
 def taps(mask):
@@ -34,53 +38,62 @@ def gen(stride):
     out = []
     emit = out.append
     emit("{")
+    emit(".reg .b32 a<8>;")
+    emit(".reg .b64 acc<4>;")
     emit(".reg .b64 win<%d>;" % (rows * 3))
     emit(".reg .b64 w0, w1, w2, w3;")
-    emit(".reg .u32 code, nxt, cp, wp, xp, ra;")
-    labels = ["K%d" % c for c in range(GROUP * 8)] + ["ADV%d" % a for a in range(1, CHUNK + 1)] + ["END"]
-    emit("TS: .branchtargets " + ", ".join(labels) + ";")
-    emit("mov.u32 cp, %%%d;" % NACC)
-    emit("mov.u32 wp, %%%d;" % (NACC + 1))
-    emit("mov.u32 xp, %%%d;" % (NACC + 2))
+    emit(".reg .u32 code, nxt, idx, cp, wp, xp, ra, ta, tn, tq;")
+    emit("TS: .branchtargets " + ", ".join(["P%d" % p for p in range(8)] + ["ADV", "END"]) + ";")
+    emit("mov.u32 cp, %0;")
+    emit("mov.u32 wp, %1;")
+    emit("mov.u32 xp, %2;")
+    emit("mov.u32 tq, %6;")
     emit("ld.shared.v2.b64 {w0, w1}, [wp];")
     emit("ld.shared.v2.b64 {w2, w3}, [wp+16];")
     emit("add.u32 wp, wp, 32;")
-    emit("ld.shared.u8 code, [cp];")
-    emit("ld.shared.u8 nxt, [cp+1];")
-    emit("add.u32 cp, cp, 2;")
-    emit("brx.idx.uni code, TS;")
+    emit("ld.shared.u8 nxt, [cp];")
+    emit("add.u32 cp, cp, 1;")
 
-    def head():  # the code to dispatch next is known a whole body ahead of its jump
+    def go_next():
+        """Fetch the next code, start the TMEM load of its slot (harmless when the code is not a
+        kernel) and jump.  The store just issued is drained first so that a later load of the same
+        slot is ordered after it."""
         emit("mov.u32 code, nxt;")
         emit("ld.shared.u8 nxt, [cp];")
         emit("add.u32 cp, cp, 1;")
+        emit("and.b32 idx, code, 15;")
+        emit("shr.u32 tn, code, 4;")
+        emit("shl.b32 tn, tn, 3;")
+        emit("add.u32 tn, tn, tq;")
+        emit("tcgen05.wait::st.sync.aligned;")
+        emit("tcgen05.ld.sync.aligned.32x32b.x8.b32 {a0, a1, a2, a3, a4, a5, a6, a7}, [tn];")
+        emit("mov.u32 ta, tn;")
+        emit("brx.idx.uni idx, TS;")
 
-    def tail():
-        emit("brx.idx.uni code, TS;")
-
-    for g in range(GROUP):
-        for p, mask in enumerate(CANON_MASKS):
-            emit("K%d:" % (g * 8 + p))
-            head()
-            tp = taps(mask)
-            for s, t in enumerate(tp):
-                u, v = divmod(t, 3)
-                for k in range(4):
-                    acc = g * 4 + k
-                    emit("fma.rn.f32x2 %%%d, win%d, w%d, %%%d;" % (acc, (stride * k + u) * 3 + v, s, acc))
-                if s == 1:
-                    emit("ld.shared.v2.b64 {w0, w1}, [wp];")
-                if s == 3:
-                    emit("ld.shared.v2.b64 {w2, w3}, [wp+16];")
-            emit("add.u32 wp, wp, 32;")
-            tail()
-    for a in range(1, CHUNK + 1):
-        emit("ADV%d:" % a)
-        emit("mad.lo.u32 xp, %%%d, %d, xp;" % (NACC + 3, a))
-        if a != CHUNK:
-            emit("bra.uni WLOAD;")
-    emit("WLOAD:")
-    head()
+    go_next()
+    for p, mask in enumerate(CANON_MASKS):
+        emit("P%d:" % p)
+        emit("tcgen05.wait::ld.sync.aligned;")
+        for k in range(4):
+            emit("mov.b64 acc%d, {a%d, a%d};" % (k, 2 * k, 2 * k + 1))
+        for s, t in enumerate(taps(mask)):
+            u, v = divmod(t, 3)
+            for k in range(4):
+                emit("fma.rn.f32x2 acc%d, win%d, w%d, acc%d;" % (k, (stride * k + u) * 3 + v, s, k))
+            if s == 1:
+                emit("ld.shared.v2.b64 {w0, w1}, [wp];")
+            if s == 3:
+                emit("ld.shared.v2.b64 {w2, w3}, [wp+16];")
+        emit("add.u32 wp, wp, 32;")
+        for k in range(4):
+            emit("mov.b64 {a%d, a%d}, acc%d;" % (2 * k, 2 * k + 1, k))
+        emit("tcgen05.st.sync.aligned.32x32b.x8.b32 [ta], {a0, a1, a2, a3, a4, a5, a6, a7};")
+        go_next()
+    emit("ADV:")
+    emit("tcgen05.wait::ld.sync.aligned;")  # the speculative load issued before this jump
+    emit("shr.u32 ra, code, 4;")
+    emit("add.u32 ra, ra, 1;")
+    emit("mad.lo.u32 xp, ra, %3, xp;")
     emit("mov.u32 ra, xp;")
     for r in range(rows):
         emit("ld.shared.b64 win%d, [ra];" % (r * 3))
@@ -90,15 +103,17 @@ def gen(stride):
         else:
             emit("ld.shared.b64 win%d, [ra+8];" % (r * 3 + 2))
         if r != rows - 1:
-            emit("add.u32 ra, ra, %%%d;" % (NACC + 4))
-    if stride == 2:  # middle column sits at a run-time offset (the even-column plane)
-        emit("add.u32 ra, xp, %%%d;" % (NACC + 5))
+            emit("add.u32 ra, ra, %4;")
+    if stride == 2:  # the middle column sits in the even-column plane, at a run-time offset
+        emit("add.u32 ra, xp, %5;")
         for r in range(rows):
             emit("ld.shared.b64 win%d, [ra];" % (r * 3 + 1))
             if r != rows - 1:
-                emit("add.u32 ra, ra, %%%d;" % (NACC + 4))
-    tail()
+                emit("add.u32 ra, ra, %4;")
+    go_next()
     emit("END:")
+    emit("tcgen05.wait::ld.sync.aligned;")
+    emit("tcgen05.wait::st.sync.aligned;")
     emit("}")
     return out
 

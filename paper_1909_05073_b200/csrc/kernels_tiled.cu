@@ -1,24 +1,33 @@
 // Tiled pattern-sparse 3x3 convolution for sm_100a.
 //
-// One CTA = 8 consumer warps + 4 producer warps (warp-specialised, setmaxnreg re-balances the
-// register file).  The consumer warps form a (wy x ng) grid: ng filter groups of 16 filters that
-// share the staged input, wy independent sets of pixel sub-tiles.  Lanes are pixels: a lane owns a
-// column of 4 output rows in each of two sub-tiles ("A" and "B"), and the two are interleaved as
-// float2 in shared memory so that every multiply-add is a packed fma.rn.f32x2 (one issue slot per
-// two FMAs) on naturally aligned register pairs:  acc[g][k].{A,B} += {w,w} * win[row][col].{A,B}.
+// One CTA = consumer warps + 4 producer warps (warp-specialised).  The consumer warps form a
+// (wy x ng) grid: ng filter groups of 16 filters that share the staged input, wy independent sets
+// of pixel sub-tiles.  Lanes are pixels: a lane owns a column of 4 output rows in each of two
+// sub-tiles ("A" and "B"), and the two are interleaved as float2 in shared memory so that every
+// multiply-add is a packed fma.rn.f32x2 (one issue slot per two FMAs) on naturally aligned
+// register pairs:  acc[g][k].{A,B} += {w,w} * win[row][col].{A,B}.
 //
 // Per input channel a lane loads its register window once (6x3 float2 at stride 1, 9x3 at stride 2)
 // and reuses it for every surviving kernel of the warp's 16 filters on that channel.  Which kernels
 // survive, for which filter slot and with which pattern, is a byte-code stream written by the
-// packer: the warp-uniform `switch` lands in a straight-line body specialised on (filter slot,
-// pattern), so accumulator and window registers are indexed at compile time, exactly 4 taps are
-// executed per kernel and no lane diverges.  Pruned kernels cost nothing.
+// packer; pruned kernels cost nothing and no lane ever diverges.
+//
+// Two consumer variants:
+//  * canonical pattern sets (GENERIC = false): 16 consumer warps whose accumulators live in Tensor
+//    Memory.  TMEM is addressed at run time, so the filter slot is data, not code: a warp-uniform
+//    indexed jump selects one of 8 straight-line bodies specialised on the pattern only (exactly 4
+//    taps), which reads the slot's 8 accumulator columns, runs 16 packed FMAs and writes them back.
+//    The hot code (~4 KB) stays inside the per-scheduler instruction cache and the jump latency is
+//    covered by the other warps (see gen_dispatch.py for the measurements behind this).
+//  * any 4-of-9 masks (GENERIC = true): 8 consumer warps with register accumulators, a switch on
+//    the filter slot and nine warp-uniform tap tests per kernel.
 //
 // Producer warps stage, per chunk of 8 input channels, the halo'd sub-tiles (zero-filled outside
 // the image, converted from fp16 when the storage type is fp16) and the chunk's weight records
 // (duplicated to {w,w} pairs) and codes, through a ring of shared-memory stages guarded by
 // full/empty mbarriers.  Every wait is bounded; a wait that runs out records its id in the
-// layer's status word and the warp leaves.
+// layer's status word and the warp stops working but still reaches the common exit, where the
+// TMEM allocation is released.
 #include <cuda_fp16.h>
 
 #include "pconv_internal.h"
@@ -28,12 +37,15 @@ namespace {
 
 typedef unsigned long long u64;
 
-constexpr int kConsumerWarps = 12;
 constexpr int kProducerWarps = 4;
-constexpr int kThreads = 32 * (kConsumerWarps + kProducerWarps);
+__host__ __device__ constexpr int consumer_warps(bool generic) { return generic ? 8 : 16; }
+__host__ __device__ constexpr int cta_threads(bool generic) {
+  return 32 * (consumer_warps(generic) + kProducerWarps);
+}
+constexpr int kTmemCols = 512;  // whole TMEM of the SM: 16 warps x 16 slots x 8 columns
 constexpr int kMaxStages = 4;
 constexpr int kWSlot = kMaxBlockKernels * 32;  // bytes per (group, stage): {w0,w0,w1,w1,w2,w2,w3,w3}
-constexpr int kCodeSlot = 160;                 // bytes per (group, stage)
+constexpr int kCodeSlot = 288;                 // bytes per (group, stage)
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr int kSmemLimit = 227 * 1024;
 
@@ -119,28 +131,38 @@ struct Win {
   static constexpr int kRows = (S == 1) ? 6 : 9;
 };
 
-// The specialised dispatch loop of one (warp, chunk): generated PTX (see gen_dispatch.py) with an
-// indexed jump per byte code and one straight-line body per (filter slot, pattern).
-#define PC_ACC4(G) "+l"(acc[G][0]), "+l"(acc[G][1]), "+l"(acc[G][2]), "+l"(acc[G][3])
-#define PC_ACC_ALL \
-  PC_ACC4(0), PC_ACC4(1), PC_ACC4(2), PC_ACC4(3), PC_ACC4(4), PC_ACC4(5), PC_ACC4(6), PC_ACC4(7)
+// The specialised dispatch loop of one (warp, chunk): generated PTX (see gen_dispatch.py); the
+// accumulators stay in TMEM at `tq` (+ 8 columns per filter slot).
 template <int S>
-__device__ __forceinline__ void dispatch_chunk(u64 (&acc)[kGroup][4], uint32_t cp, uint32_t wp,
-                                               uint32_t xptr, uint32_t chan_b, uint32_t pitch_b,
-                                               uint32_t off_mid) {
+__device__ __forceinline__ void dispatch_chunk(uint32_t cp, uint32_t wp, uint32_t xptr,
+                                               uint32_t chan_b, uint32_t pitch_b, uint32_t off_mid,
+                                               uint32_t tq) {
   if (S == 1) {
     asm volatile(
 #include "dispatch_s1.inc"
-        : PC_ACC_ALL
-        : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(pitch_b), "r"(off_mid)
+        :
+        : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(pitch_b), "r"(off_mid), "r"(tq)
         : "memory");
   } else {
     asm volatile(
 #include "dispatch_s2.inc"
-        : PC_ACC_ALL
-        : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(pitch_b), "r"(off_mid)
+        :
+        : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(pitch_b), "r"(off_mid), "r"(tq)
         : "memory");
   }
+}
+
+__device__ __forceinline__ void tmem_ld8(uint32_t (&r)[8], uint32_t taddr) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+                 "=r"(r[7])
+               : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_st8_zero(uint32_t taddr) {
+  const uint32_t z = 0;
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%1,%1,%1,%1,%1,%1,%1};" ::"r"(taddr), "r"(z)
+               : "memory");
 }
 
 // Any 4-of-9 mask, taken at run time: nine warp-uniform tests, a weight load per taken tap.
@@ -175,6 +197,7 @@ __device__ __forceinline__ void load_window(u64 (&win)[Win<S>::kRows][3], uint32
   case G:                                                   \
     kernel_body_generic<S, G>(acc, win, code & 0x1FFu, wp); \
     break;
+#define PG_CASES8(B) PG_CASE(B + 0) PG_CASE(B + 1) PG_CASE(B + 2) PG_CASE(B + 3) PG_CASE(B + 4) PG_CASE(B + 5) PG_CASE(B + 6) PG_CASE(B + 7)
 
 __device__ __forceinline__ float ldg_f(const __half* p) { return __half2float(__ldg(p)); }
 
@@ -305,20 +328,30 @@ __device__ __forceinline__ void produce_chunk_half(const DeviceLayer& L, const G
 }
 
 template <int S, bool GENERIC>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(cta_threads(GENERIC), 1)
 tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
              const float* __restrict__ bias, void* __restrict__ y) {
+  constexpr int kCW = consumer_warps(GENERIC);
+  constexpr int kThreads = cta_threads(GENERIC);
   extern __shared__ __align__(16) unsigned char smem[];
   const uint32_t sbase = smem_u32(smem);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   SubTile* tab = reinterpret_cast<SubTile*>(smem + g.tab_off);
+  volatile uint32_t* tmem_base_s = reinterpret_cast<volatile uint32_t*>(smem + 8 * 2 * kMaxStages);
 
   if (tid == 0) {
     for (int s = 0; s < g.stages; ++s) {
       mbar_init(sbase + 8 * s, 32 * kProducerWarps);
-      mbar_init(sbase + 8 * (kMaxStages + s), kConsumerWarps);
+      mbar_init(sbase + 8 * (kMaxStages + s), kCW);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (!GENERIC && warp == 0) {  // the whole TMEM of this SM (one CTA per SM by shared-memory use)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32((const void*)tmem_base_s)),
+                 "n"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   for (int i = tid; i < 2 * g.pairs; i += kThreads) {
     const long long q = (long long)blockIdx.x * (2 * g.pairs) + i;
@@ -351,18 +384,21 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
     const int j = i % g.ng, s = i / g.ng;
     if ((int)(blockIdx.y * g.ng + j) >= L.n_groups)
       sts32(sbase + g.stage_off + s * g.stage_bytes + g.x_stage_bytes + g.ng * kWSlot + j * kCodeSlot,
-            GENERIC ? 0x40004000u : 0x48484848u);
+            GENERIC ? 0x40004000u : 0x09090909u);
   }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = GENERIC ? 0u : *tmem_base_s;
 
-  if (warp >= kConsumerWarps) {
+  if (warp >= kCW) {
     // ===================================== producer warps =====================================
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
-    const int pw = warp - kConsumerWarps;
+    if (GENERIC) asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
+    const int pw = warp - kCW;
     const uint8_t* codes = GENERIC ? L.codes_g : L.codes_s;
     for (int k = 0; k < L.n_chunks; ++k) {
       const int s = k % g.stages, it = k / g.stages;
-      if (it > 0 && !mbar_wait(sbase + 8 * (kMaxStages + s), (it - 1) & 1, L.err, 1)) return;
+      if (it > 0 && !mbar_wait(sbase + 8 * (kMaxStages + s), (it - 1) & 1, L.err, 1)) break;
       const uint32_t stage_base = sbase + g.stage_off + s * g.stage_bytes;
       if (g.is_half) {
         produce_chunk_half<S>(L, g, (const __half*)x, tab, desc, codes, stage_base, k, pw, lane);
@@ -372,98 +408,130 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
         cp_async_arrive(sbase + 8 * s);
       }
     }
-    return;
-  }
+    asm volatile("cp.async.wait_all;" ::: "memory");
+  } else {
+    // ===================================== consumer warps =====================================
+    if (GENERIC) asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
+    const int wyi = warp % g.wys, wgi = warp / g.wys;
+    const int gi = blockIdx.y * g.ng + wgi;
+    const bool active = (wyi < g.wy) && (gi < L.n_groups);
+    const int slot = wyi * g.sw + lane / g.tw;  // sub-tile pair of this lane
+    const int col = lane % g.tw;
+    const uint32_t pitch_b = g.pitch * 8;
+    const uint32_t off_mid = (S == 1) ? 8u : (uint32_t)(g.tw + 1) * 8u;
+    const uint32_t off_right = (S == 1) ? 16u : 8u;
+    const uint32_t chan_b = (uint32_t)g.chan_stride * 8u;
+    const uint32_t lane_off = (uint32_t)(slot * g.substride + col) * 8u;
+    // TMEM: a warp reaches the 32 lanes of its quadrant (warp % 4); 4 warps share a quadrant and
+    // take 128 columns each = 16 filter slots x (4 rows x {A,B}).
+    const uint32_t tq = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)((warp >> 2) * (kGroup * 8));
 
-  // ======================================= consumer warps =======================================
-  asm volatile("setmaxnreg.inc.sync.aligned.u32 144;");
-  const int wyi = warp % g.wys, wgi = warp / g.wys;
-  const int gi = blockIdx.y * g.ng + wgi;
-  const bool active = (wyi < g.wy) && (gi < L.n_groups);
-  const int slot = wyi * g.sw + lane / g.tw;  // sub-tile pair of this lane
-  const int col = lane % g.tw;
-  const uint32_t pitch_b = g.pitch * 8;
-  const uint32_t off_mid = (S == 1) ? 8u : (uint32_t)(g.tw + 1) * 8u;
-  const uint32_t off_right = (S == 1) ? 16u : 8u;
-  const uint32_t chan_b = (uint32_t)g.chan_stride * 8u;
-  const uint32_t lane_off = (uint32_t)(slot * g.substride + col) * 8u;
+    u64 acc[GENERIC ? kGroup : 1][4];
+    if constexpr (GENERIC) {
+#pragma unroll
+      for (int a = 0; a < kGroup; ++a)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) acc[a][k] = 0ull;
+    } else {
+      for (int a = 0; a < kGroup; ++a) tmem_st8_zero(tq + a * 8);
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+    }
 
-  u64 acc[kGroup][4];
+    bool ok = true;
+    for (int k = 0; k < L.n_chunks && ok; ++k) {
+      const int s = k % g.stages;
+      ok = mbar_wait(sbase + 8 * s, (k / g.stages) & 1, L.err, 2);
+      if (!ok) break;
+      if (active) {
+        const uint32_t stage_base = sbase + g.stage_off + s * g.stage_bytes;
+        uint32_t xptr = stage_base + lane_off - chan_b;  // one channel before the chunk
+        uint32_t wp = stage_base + g.x_stage_bytes + wgi * kWSlot;
+        uint32_t cp = stage_base + g.x_stage_bytes + g.ng * kWSlot + wgi * kCodeSlot;
+        if constexpr (!GENERIC) {
+          dispatch_chunk<S>(cp, wp, xptr, chan_b, pitch_b, off_mid, tq);
+        } else {
+          u64 win[Win<S>::kRows][3];
 #pragma unroll
-  for (int a = 0; a < kGroup; ++a)
-#pragma unroll
-    for (int k = 0; k < 4; ++k) acc[a][k] = 0ull;
-
-  for (int k = 0; k < L.n_chunks; ++k) {
-    const int s = k % g.stages;
-    if (!mbar_wait(sbase + 8 * s, (k / g.stages) & 1, L.err, 2)) return;
-    if (active) {
-      const uint32_t stage_base = sbase + g.stage_off + s * g.stage_bytes;
-      uint32_t xptr = stage_base + lane_off - chan_b;  // one channel before the chunk
-      uint32_t wp = stage_base + g.x_stage_bytes + wgi * kWSlot;
-      uint32_t cp = stage_base + g.x_stage_bytes + g.ng * kWSlot + wgi * kCodeSlot;
-      if (!GENERIC) {
-        dispatch_chunk<S>(acc, cp, wp, xptr, chan_b, pitch_b, off_mid);
-      } else {
-        u64 win[Win<S>::kRows][3];
-#pragma unroll
-        for (int r = 0; r < Win<S>::kRows; ++r) win[r][0] = win[r][1] = win[r][2] = 0ull;
-        for (;;) {
-          const uint32_t code = lds_u16(cp);
-          cp += 2;
-          if (code & (uint32_t)kGenEnd) break;
-          if (code & (uint32_t)kGenNext) {
-            xptr += ((code & 0xFFu) + 1u) * chan_b;
-            load_window<S>(win, xptr, pitch_b, off_mid, off_right);
-            continue;
+          for (int r = 0; r < Win<S>::kRows; ++r) win[r][0] = win[r][1] = win[r][2] = 0ull;
+          for (;;) {
+            const uint32_t code = lds_u16(cp);
+            cp += 2;
+            if (code & (uint32_t)kGenEnd) break;
+            if (code & (uint32_t)kGenNext) {
+              xptr += ((code & 0xFFu) + 1u) * chan_b;
+              load_window<S>(win, xptr, pitch_b, off_mid, off_right);
+              continue;
+            }
+            switch (code >> 9) {
+              PG_CASES8(0) PG_CASES8(8)
+              default: break;
+            }
           }
-          switch (code >> 9) {
-            PG_CASE(0) PG_CASE(1) PG_CASE(2) PG_CASE(3) PG_CASE(4) PG_CASE(5) PG_CASE(6) PG_CASE(7)
-            default: break;
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(sbase + 8 * (kMaxStages + s));
+    }
+
+    // ---- epilogue: bias, ReLU, store at the original filter index --------------------------------
+    if (active && ok) {
+      const SubTile A = tab[2 * slot], B = tab[2 * slot + 1];
+      const int ox_a = A.x0 + col, ox_b = B.x0 + col;
+      const bool col_a = A.valid && ox_a < g.w_out, col_b = B.valid && ox_b < g.w_out;
+      const size_t plane = (size_t)g.h_out * g.w_out;
+#pragma unroll
+      for (int a = 0; a < kGroup; ++a) {
+        uint32_t v[8];
+        if constexpr (GENERIC) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            v[2 * k] = (uint32_t)acc[a][k];
+            v[2 * k + 1] = (uint32_t)(acc[a][k] >> 32);
+          }
+        } else {
+          tmem_ld8(v, tq + a * 8);  // all lanes take part: the slot loop is warp-uniform
+        }
+        const int o = __ldg(L.perm + gi * kGroup + a);
+        if (o < 0) continue;
+        const float bv = bias ? __ldg(bias + o) : 0.f;
+        const size_t base_a = ((size_t)A.n * L.c_out + o) * plane;
+        const size_t base_b = ((size_t)B.n * L.c_out + o) * plane;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          float va = __uint_as_float(v[2 * k]) + bv;
+          float vb = __uint_as_float(v[2 * k + 1]) + bv;
+          if (g.relu) {
+            va = fmaxf(va, 0.f);
+            vb = fmaxf(vb, 0.f);
+          }
+          const int ya = A.y0 + k, yb = B.y0 + k;
+          if (g.is_half) {
+            __half* yh = (__half*)y;
+            if (col_a && ya < g.h_out) yh[base_a + (size_t)ya * g.w_out + ox_a] = __float2half_rn(va);
+            if (col_b && yb < g.h_out) yh[base_b + (size_t)yb * g.w_out + ox_b] = __float2half_rn(vb);
+          } else {
+            float* yf = (float*)y;
+            if (col_a && ya < g.h_out) yf[base_a + (size_t)ya * g.w_out + ox_a] = va;
+            if (col_b && yb < g.h_out) yf[base_b + (size_t)yb * g.w_out + ox_b] = vb;
           }
         }
       }
     }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(sbase + 8 * (kMaxStages + s));
   }
 
-  // ---- epilogue: bias, ReLU, store at the original filter index ----------------------------------
-  if (!active) return;
-  const SubTile A = tab[2 * slot], B = tab[2 * slot + 1];
-  const int ox_a = A.x0 + col, ox_b = B.x0 + col;
-  const bool col_a = A.valid && ox_a < g.w_out, col_b = B.valid && ox_b < g.w_out;
-  const size_t plane = (size_t)g.h_out * g.w_out;
-#pragma unroll
-  for (int a = 0; a < kGroup; ++a) {
-    const int o = __ldg(L.perm + gi * kGroup + a);
-    if (o < 0) continue;
-    const float bv = bias ? __ldg(bias + o) : 0.f;
-    const size_t base_a = ((size_t)A.n * L.c_out + o) * plane;
-    const size_t base_b = ((size_t)B.n * L.c_out + o) * plane;
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      float va = __uint_as_float((uint32_t)acc[a][k]) + bv;
-      float vb = __uint_as_float((uint32_t)(acc[a][k] >> 32)) + bv;
-      if (g.relu) {
-        va = fmaxf(va, 0.f);
-        vb = fmaxf(vb, 0.f);
-      }
-      const int ya = A.y0 + k, yb = B.y0 + k;
-      if (g.is_half) {
-        __half* yh = (__half*)y;
-        if (col_a && ya < g.h_out) yh[base_a + (size_t)ya * g.w_out + ox_a] = __float2half_rn(va);
-        if (col_b && yb < g.h_out) yh[base_b + (size_t)yb * g.w_out + ox_b] = __float2half_rn(vb);
-      } else {
-        float* yf = (float*)y;
-        if (col_a && ya < g.h_out) yf[base_a + (size_t)ya * g.w_out + ox_a] = va;
-        if (col_b && yb < g.h_out) yf[base_b + (size_t)yb * g.w_out + ox_b] = vb;
-      }
-    }
+  // ---- common exit: every warp arrives here, then the TMEM columns are handed back ---------------
+  if (!GENERIC) {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0)
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols)
+                   : "memory");
   }
 }
 
+template <bool GENERIC>
 bool make_geo(const DeviceLayer& L, int n, int h, int w, Geo* out) {
+  constexpr int kCW = consumer_warps(GENERIC);
   Geo g;
   g.n = n;
   g.h = h;
@@ -478,15 +546,19 @@ bool make_geo(const DeviceLayer& L, int n, int h, int w, Geo* out) {
   const long long q = (long long)n * g.tx * g.ty;
   if (q > 0x7FFFFFFF) return false;
   g.q_total = (int)q;
-  g.ng = (L.n_groups >= 6) ? 6 : (L.n_groups == 5 ? 6 : L.n_groups);
-  g.wys = kConsumerWarps / g.ng;
+  // filter groups per CTA: a power of two dividing the consumer warps, at most 4 (8 for the
+  // 16-warp variant when the layer is wide), so that the staged input is shared widely
+  g.ng = 1;
+  const int ng_max = GENERIC ? 4 : (L.n_groups >= 16 ? 8 : 4);
+  while (g.ng < ng_max && g.ng < L.n_groups) g.ng *= 2;
+  g.wys = kCW / g.ng;
   g.wy = g.wys;
   g.rows = (L.stride == 1) ? 6 : 9;
   g.pitch = (L.stride == 1) ? (g.tw + 2) : (2 * g.tw + 1);
   g.substride = g.rows * g.pitch;
   if (g.tw < 16)  // spread the sub-tiles of a half-warp over distinct banks
     while (g.substride % 16 != g.tw % 16) ++g.substride;
-  g.tab_off = 8 * 2 * kMaxStages;
+  g.tab_off = 8 * 2 * kMaxStages + 16;  // barriers, then the TMEM base address word
   if (L.n_chunks > 512) return false;  // descriptor table budget (c_in <= 4096)
   for (;;) {
     g.pairs = g.wy * g.sw;
@@ -509,9 +581,12 @@ bool make_geo(const DeviceLayer& L, int n, int h, int w, Geo* out) {
 }
 
 template <int S, bool GENERIC>
-cudaError_t launch_one(const DeviceLayer& L, const Geo& g, const void* x, const float* bias, void* y,
+cudaError_t launch_one(const DeviceLayer& L, Geo g, const void* x, const float* bias, void* y,
                        cudaStream_t stream) {
-  const int smem = g.stage_off + g.stages * g.stage_bytes;
+  int smem = g.stage_off + g.stages * g.stage_bytes;
+  // the TMEM variant must be alone on its SM (it takes all 512 columns): make sure two CTAs can
+  // never be co-resident by asking for more than half of the shared memory
+  if (!GENERIC && smem < 120 * 1024) smem = 120 * 1024;
   cudaError_t e = cudaFuncSetAttribute(tiled_kernel<S, GENERIC>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
   if (e != cudaSuccess) return e;
@@ -519,7 +594,7 @@ cudaError_t launch_one(const DeviceLayer& L, const Geo& g, const void* x, const 
   const int ctas_y = (L.n_groups + g.ng - 1) / g.ng;
   if (ctas_x > 0x7FFFFFFF || ctas_y > 65535) return cudaErrorInvalidValue;
   dim3 grid((unsigned)ctas_x, (unsigned)ctas_y);
-  tiled_kernel<S, GENERIC><<<grid, kThreads, smem, stream>>>(L, g, x, bias, y);
+  tiled_kernel<S, GENERIC><<<grid, cta_threads(GENERIC), smem, stream>>>(L, g, x, bias, y);
   return cudaGetLastError();
 }
 
@@ -529,15 +604,16 @@ bool tiled_supported(const DeviceLayer& L, int n, int h, int w) {
   Geo g;
   if (n <= 0 || h <= 0 || w <= 0) return false;
   if (L.n_groups > 65535) return false;
-  return make_geo(L, n, h, w, &g);
+  return make_geo<true>(L, n, h, w, &g) && make_geo<false>(L, n, h, w, &g);
 }
 
 cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias, void* y, int n, int h,
                          int w, bool relu, bool generic_taps, cudaStream_t stream) {
-  Geo g;
-  if (!make_geo(L, n, h, w, &g)) return cudaErrorInvalidValue;
-  g.relu = relu ? 1 : 0;
   if (!generic_taps && !L.codes_s) generic_taps = true;
+  Geo g;
+  if (!(generic_taps ? make_geo<true>(L, n, h, w, &g) : make_geo<false>(L, n, h, w, &g)))
+    return cudaErrorInvalidValue;
+  g.relu = relu ? 1 : 0;
   if (L.stride == 1)
     return generic_taps ? launch_one<1, true>(L, g, x, bias, y, stream)
                         : launch_one<1, false>(L, g, x, bias, y, stream);

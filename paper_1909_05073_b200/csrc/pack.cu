@@ -245,14 +245,14 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
         for (const Item& it : items) {
           if (it.c != pos) {
             const int adv = it.c - pos;  // 1..kChunk
-            codes_s.push_back((uint8_t)(kCodeNext + adv - 1));
+            codes_s.push_back((uint8_t)(((adv - 1) << 4) | kCodeNext));
             const uint16_t cg = (uint16_t)(kGenNext | (adv - 1));
             codes_g.push_back((uint8_t)(cg & 0xFF));
             codes_g.push_back((uint8_t)(cg >> 8));
             pos = it.c;
           }
           const int canon = h->canon_id[it.r->pid];
-          codes_s.push_back((uint8_t)(it.slot * 8 + (canon < 0 ? 0 : canon)));
+          codes_s.push_back((uint8_t)((it.slot << 4) | (canon < 0 ? 0 : canon)));
           const uint16_t cg = (uint16_t)((it.slot << 9) | patterns[it.r->pid]);
           codes_g.push_back((uint8_t)(cg & 0xFF));
           codes_g.push_back((uint8_t)(cg >> 8));

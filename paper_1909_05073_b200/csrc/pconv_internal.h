@@ -9,17 +9,17 @@
 
 namespace pconv {
 
-constexpr int kGroup = 8;          // filters per group (accumulator rows of one consumer warp)
+constexpr int kGroup = 16;         // filters per group (accumulator slots of one consumer warp)
 constexpr int kChunk = 8;          // input channels per pipeline stage
 constexpr int kMaxBlockKernels = kGroup * kChunk;
 
 // Specialised code stream (one byte per entry) -- valid when the pattern set is a subset of the
 // eight masks the tiled kernel has straight-line bodies for.
-//   0..63         kernel: filter slot g = code >> 3, canonical pattern = code & 7
-//   64..71        advance (code - 63) channels inside the chunk and load that channel's window
-//   72            end of this (group, chunk) block
-constexpr int kCodeNext = kGroup * 8;
-constexpr int kCodeEnd = kCodeNext + kChunk;
+//   low nibble 0..7   kernel: canonical pattern id; high nibble = filter slot
+//   low nibble 8      advance (high nibble + 1) channels inside the chunk and load that window
+//   9                 end of this (group, chunk) block
+constexpr int kCodeNext = 8;
+constexpr int kCodeEnd = 9;
 // Generic code stream (two bytes per entry) -- any 4-of-9 mask.
 //   (g << 9) | mask   kernel with run-time mask;   0x2000 | (adv-1)   advance;   0x4000   end
 constexpr int kGenNext = 0x2000;
