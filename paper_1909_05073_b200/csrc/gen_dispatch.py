@@ -11,9 +11,9 @@ Why PTX text, and why this shape (all measured on B200):
    as much as executed ones;
  * so the filter slot is taken out of the code: accumulators live in Tensor Memory (TMEM), which is
    addressed at run time.  A body is specialised on the pattern only (8 bodies, ~4 KB): it waits for
-   the slot's 8 accumulator columns (loaded while the previous jump was in flight), runs the 16
-   packed FMAs of the 4 taps, stores the columns back, starts the load for the next kernel's slot
-   and jumps.
+   the slot's 8 accumulator columns (requested by the previous body), runs the 16 packed FMAs of
+   the 4 taps, writes the columns back in two halves and refills each half's registers with the
+   next kernel's columns at once, then jumps.
 
 Operands of the asm statement (all u32): %0 code pointer, %1 weight pointer, %2 window pointer (one
 channel before the chunk), %3 channel stride, %4 row pitch, %5 offset of the middle window column
@@ -53,11 +53,14 @@ def gen(stride):
     emit("add.u32 wp, wp, 32;")
     emit("ld.shared.u8 nxt, [cp];")
     emit("add.u32 cp, cp, 1;")
+    emit("tcgen05.wait::st.sync.aligned;")
 
-    def go_next():
-        """Fetch the next code, start the TMEM load of its slot (harmless when the code is not a
-        kernel) and jump.  The store just issued is drained first so that a later load of the same
-        slot is ordered after it."""
+    LO = "{a0, a1, a2, a3}"
+    HI = "{a4, a5, a6, a7}"
+
+    def prep():
+        """Decode the next code as early as possible: its jump index (so that the jump-table
+        lookup is scheduled above the FMAs) and the TMEM address of its filter slot."""
         emit("mov.u32 code, nxt;")
         emit("ld.shared.u8 nxt, [cp];")
         emit("add.u32 cp, cp, 1;")
@@ -65,35 +68,69 @@ def gen(stride):
         emit("shr.u32 tn, code, 4;")
         emit("shl.b32 tn, tn, 3;")
         emit("add.u32 tn, tn, tq;")
-        emit("tcgen05.wait::st.sync.aligned;")
-        emit("tcgen05.ld.sync.aligned.32x32b.x8.b32 {a0, a1, a2, a3, a4, a5, a6, a7}, [tn];")
+
+    def load_lo():
+        emit("tcgen05.ld.sync.aligned.32x32b.x4.b32 %s, [tn];" % LO)
+
+    def load_hi():
+        emit("tcgen05.ld.sync.aligned.32x32b.x4.b32 %s, [tn+4];" % HI)
+
+    def jump():
         emit("mov.u32 ta, tn;")
         emit("brx.idx.uni idx, TS;")
 
-    go_next()
+    # prologue: first code of the chunk
+    prep()
+    load_lo()
+    load_hi()
+    jump()
+
+    # Kernel bodies.  The slot's 8 accumulator columns arrive as two halves (rows 0-1, rows 2-3 of
+    # the lane's pixel column); each half is written back as soon as its last FMA has issued and
+    # its registers are immediately refilled with the next kernel's half, so TMEM latency hides
+    # behind the remaining FMAs and the jump.  Inside a channel every kernel has a different slot,
+    # so such a load never follows a store to the same columns; stores are drained where the
+    # channel changes (ADV) and at the end.
     for p, mask in enumerate(CANON_MASKS):
+        tp = taps(mask)
+
+        def fma(s, ks):
+            u, v = divmod(tp[s], 3)
+            for k in ks:
+                emit("fma.rn.f32x2 acc%d, win%d, w%d, acc%d;" % (k, (stride * k + u) * 3 + v, s, k))
+
         emit("P%d:" % p)
         emit("tcgen05.wait::ld.sync.aligned;")
         for k in range(4):
             emit("mov.b64 acc%d, {a%d, a%d};" % (k, 2 * k, 2 * k + 1))
-        for s, t in enumerate(taps(mask)):
-            u, v = divmod(t, 3)
-            for k in range(4):
-                emit("fma.rn.f32x2 acc%d, win%d, w%d, acc%d;" % (k, (stride * k + u) * 3 + v, s, k))
-            if s == 1:
-                emit("ld.shared.v2.b64 {w0, w1}, [wp];")
-            if s == 3:
-                emit("ld.shared.v2.b64 {w2, w3}, [wp+16];")
+        prep()
+        fma(0, range(4))
+        fma(1, range(4))
+        emit("ld.shared.v2.b64 {w0, w1}, [wp];")
+        fma(2, (0, 1))
+        fma(3, (0, 1))
+        emit("mov.b64 {a0, a1}, acc0;")
+        emit("mov.b64 {a2, a3}, acc1;")
+        emit("tcgen05.st.sync.aligned.32x32b.x4.b32 [ta], %s;" % LO)
+        load_lo()
+        fma(2, (2, 3))
+        fma(3, (2, 3))
+        emit("ld.shared.v2.b64 {w2, w3}, [wp+16];")
         emit("add.u32 wp, wp, 32;")
-        for k in range(4):
-            emit("mov.b64 {a%d, a%d}, acc%d;" % (2 * k, 2 * k + 1, k))
-        emit("tcgen05.st.sync.aligned.32x32b.x8.b32 [ta], {a0, a1, a2, a3, a4, a5, a6, a7};")
-        go_next()
+        emit("mov.b64 {a4, a5}, acc2;")
+        emit("mov.b64 {a6, a7}, acc3;")
+        emit("tcgen05.st.sync.aligned.32x32b.x4.b32 [ta+4], %s;" % HI)
+        load_hi()
+        jump()
     emit("ADV:")
-    emit("tcgen05.wait::ld.sync.aligned;")  # the speculative load issued before this jump
+    emit("tcgen05.wait::ld.sync.aligned;")  # the speculative loads issued before this jump
+    emit("tcgen05.wait::st.sync.aligned;")  # a slot may come back in the next channel
     emit("shr.u32 ra, code, 4;")
     emit("add.u32 ra, ra, 1;")
     emit("mad.lo.u32 xp, ra, %3, xp;")
+    prep()
+    load_lo()
+    load_hi()
     emit("mov.u32 ra, xp;")
     for r in range(rows):
         emit("ld.shared.b64 win%d, [ra];" % (r * 3))
@@ -110,7 +147,7 @@ def gen(stride):
             emit("ld.shared.b64 win%d, [ra];" % (r * 3 + 1))
             if r != rows - 1:
                 emit("add.u32 ra, ra, %4;")
-    go_next()
+    jump()
     emit("END:")
     emit("tcgen05.wait::ld.sync.aligned;")
     emit("tcgen05.wait::st.sync.aligned;")

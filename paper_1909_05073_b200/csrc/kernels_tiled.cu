@@ -335,7 +335,9 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   constexpr int kThreads = cta_threads(GENERIC);
   extern __shared__ __align__(16) unsigned char smem[];
   const uint32_t sbase = smem_u32(smem);
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tid = threadIdx.x, lane = tid & 31;
+  // broadcast from lane 0: tells the compiler that everything derived from it is warp-uniform
+  const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
   SubTile* tab = reinterpret_cast<SubTile*>(smem + g.tab_off);
   volatile uint32_t* tmem_base_s = reinterpret_cast<volatile uint32_t*>(smem + 8 * 2 * kMaxStages);
 
