@@ -120,6 +120,25 @@ pconv_status pconv_pack(const float* w_oihw_host, int c_out, int c_in, const uin
 pconv_status pconv_forward(const pconv_handle* h, const void* x_dev, const float* bias_dev,
                            void* y_dev, int n, int h_in, int w_in, unsigned flags, void* stream);
 
+/*
+ * pconv_workspace_bytes / pconv_forward_ws -- the same operation as pconv_forward, with a
+ * caller-provided scratch buffer that lets the library split the input-channel range of a layer
+ * over several thread blocks when the batch offers too few output tiles to fill the GPU (batch-1
+ * layers).  Partial sums are accumulated in the workspace with fp32 atomics (so the summation
+ * order, not the result beyond rounding, varies from run to run) and the last block to finish an
+ * output tile applies bias / ReLU and writes y.  The paper has no counterpart; this is how the
+ * build recovers parallelism that the paper's one-image-at-a-time mobile setting never needed.
+ *
+ *  bytes       receives the workspace size for this handle and input shape (0 = never split).
+ *  ws_dev      DEVICE buffer of at least that size, 256-byte aligned, or NULL (= no split).
+ *              It must be all zero before its first use; every forward leaves it all zero again.
+ *              Forwards that share a workspace must not overlap in time.
+ */
+pconv_status pconv_workspace_bytes(const pconv_handle* h, int n, int h_in, int w_in, size_t* bytes);
+pconv_status pconv_forward_ws(const pconv_handle* h, const void* x_dev, const float* bias_dev,
+                              void* y_dev, int n, int h_in, int w_in, unsigned flags, void* ws_dev,
+                              size_t ws_bytes, void* stream);
+
 /* Releases the handle and its device buffers.  NULL is allowed. */
 void pconv_free(pconv_handle* h);
 
@@ -157,7 +176,8 @@ const char* pconv_status_str(pconv_status s);
 /*
  * pconv_stack_create -- chains layers: x -> conv(layers[0]) [-> maxpool] -> conv(layers[1]) ...
  * for a fixed input shape (n, h, w), as in the VGG-16 stacks of the evaluation.  The stack
- * allocates its two ping-pong activation buffers on the device here (never during forward), and
+ * allocates its two ping-pong activation buffers and the channel-split workspace of its layers on
+ * the device here (never during forward), and
  * borrows the handles and bias pointers, which must outlive it.
  *  layers      n_layers handles (HOST array), same storage type, c_in of layer k+1 = c_out of k.
  *  bias_dev    n_layers DEVICE pointers (HOST array; entries may be NULL), or NULL.

@@ -23,7 +23,7 @@ STATUS_NAMES = ["PCONV_OK", "PCONV_ERR_NULL", "PCONV_ERR_SHAPE", "PCONV_ERR_PATT
                 "PCONV_ERR_ALIGN", "PCONV_ERR_ALLOC", "PCONV_ERR_CUDA",
                 "PCONV_ERR_DEVICE_TIMEOUT"]
 
-EXPORTS = ["pconv_pack", "pconv_forward", "pconv_free", "pconv_maxpool2x2", "pconv_unpack",
+EXPORTS = ["pconv_pack", "pconv_forward", "pconv_forward_ws", "pconv_workspace_bytes", "pconv_free", "pconv_maxpool2x2", "pconv_unpack",
            "pconv_stats", "pconv_filter_order", "pconv_device_status", "pconv_status_str",
            "pconv_stack_create", "pconv_stack_out_shape", "pconv_stack_forward",
            "pconv_stack_forward_host", "pconv_stack_free"]
@@ -64,6 +64,8 @@ def lib():
         ip = ctypes.POINTER(ctypes.c_int)
         L.pconv_pack.argtypes = [vp, ci, ci, vp, ci, ci, ci, cu, vp, ctypes.POINTER(vp), ip, ip]
         L.pconv_forward.argtypes = [vp, vp, vp, vp, ci, ci, ci, cu, vp]
+        L.pconv_forward_ws.argtypes = [vp, vp, vp, vp, ci, ci, ci, cu, vp, ctypes.c_size_t, vp]
+        L.pconv_workspace_bytes.argtypes = [vp, ci, ci, ci, ctypes.POINTER(ctypes.c_size_t)]
         L.pconv_free.argtypes = [vp]
         L.pconv_free.restype = None
         L.pconv_maxpool2x2.argtypes = [vp, vp, ci, ci, ci, ci, ci, vp]
@@ -127,8 +129,15 @@ def pconv_free(handle):
     lib().pconv_free(handle)
 
 
-def pconv_forward(handle, x, bias, y, flags=0, stream=None):
-    """x, y: CUDA torch tensors (NCHW, contiguous); bias: CUDA fp32 tensor or None."""
+def pconv_workspace_bytes(handle, n, h, w):
+    b = ctypes.c_size_t(0)
+    _check(lib().pconv_workspace_bytes(handle, n, h, w, ctypes.byref(b)), "pconv_workspace_bytes")
+    return int(b.value)
+
+
+def pconv_forward(handle, x, bias, y, flags=0, stream=None, workspace=None):
+    """x, y: CUDA torch tensors (NCHW, contiguous); bias: CUDA fp32 tensor or None;
+    workspace: zeroed CUDA uint8 tensor from pconv_workspace_bytes, or None."""
     if not (x.is_cuda and y.is_cuda and x.is_contiguous() and y.is_contiguous()):
         raise ValueError("x and y must be contiguous CUDA tensors")
     n, _, h, w = x.shape
@@ -137,9 +146,15 @@ def pconv_forward(handle, x, bias, y, flags=0, stream=None):
         if not (bias.is_cuda and bias.is_contiguous()) or bias.dtype.itemsize != 4:
             raise ValueError("bias must be a contiguous CUDA float32 tensor")
         bp = ctypes.c_void_p(bias.data_ptr())
-    st = lib().pconv_forward(handle, ctypes.c_void_p(x.data_ptr()), bp,
-                             ctypes.c_void_p(y.data_ptr()), n, h, w, int(flags),
-                             _stream_ptr(stream))
+    if workspace is not None:
+        st = lib().pconv_forward_ws(handle, ctypes.c_void_p(x.data_ptr()), bp,
+                                    ctypes.c_void_p(y.data_ptr()), n, h, w, int(flags),
+                                    ctypes.c_void_p(workspace.data_ptr()), workspace.numel(),
+                                    _stream_ptr(stream))
+    else:
+        st = lib().pconv_forward(handle, ctypes.c_void_p(x.data_ptr()), bp,
+                                 ctypes.c_void_p(y.data_ptr()), n, h, w, int(flags),
+                                 _stream_ptr(stream))
     _check(st, "pconv_forward")
 
 
@@ -192,11 +207,24 @@ class Layer:
         n, _, h, w = x_shape
         return (n, self.c_out, (h - 1) // self.stride + 1, (w - 1) // self.stride + 1)
 
-    def forward(self, x, relu=True, kernel=0, out=None):
+    def workspace(self, x_shape):
+        """A zeroed workspace for inputs of this shape (cached), or None if never needed."""
+        import torch
+        n, _, h, w = x_shape
+        need = pconv_workspace_bytes(self.handle, n, h, w)
+        if need == 0:
+            return None
+        ws = getattr(self, "_ws", None)
+        if ws is None or ws.numel() < need:
+            ws = self._ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
+        return ws
+
+    def forward(self, x, relu=True, kernel=0, out=None, split=False):
         import torch
         if out is None:
             out = torch.empty(self.out_shape(x.shape), dtype=x.dtype, device=x.device)
-        pconv_forward(self.handle, x, self.bias, out, (RELU if relu else 0) | kernel)
+        ws = self.workspace(x.shape) if split else None
+        pconv_forward(self.handle, x, self.bias, out, (RELU if relu else 0) | kernel, workspace=ws)
         return out
 
     def stats(self):

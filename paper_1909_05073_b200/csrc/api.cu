@@ -23,9 +23,23 @@ extern "C" const char* pconv_status_str(pconv_status s) {
   return "unknown status";
 }
 
+extern "C" pconv_status pconv_workspace_bytes(const pconv_handle* h, int n, int h_in, int w_in,
+                                              size_t* bytes) {
+  if (!h || !bytes) return PCONV_ERR_NULL;
+  if (n < 0 || h_in <= 0 || w_in <= 0) return PCONV_ERR_SHAPE;
+  *bytes = (n == 0) ? 0 : tiled_workspace_bytes(h->d, n, h_in, w_in);
+  return PCONV_OK;
+}
+
 extern "C" pconv_status pconv_forward(const pconv_handle* h, const void* x, const float* bias,
                                       void* y, int n, int h_in, int w_in, unsigned flags,
                                       void* stream_v) {
+  return pconv_forward_ws(h, x, bias, y, n, h_in, w_in, flags, nullptr, 0, stream_v);
+}
+
+extern "C" pconv_status pconv_forward_ws(const pconv_handle* h, const void* x, const float* bias,
+                                         void* y, int n, int h_in, int w_in, unsigned flags,
+                                         void* ws, size_t ws_bytes, void* stream_v) {
   if (!h || !x || !y) return PCONV_ERR_NULL;
   if (n < 0 || h_in <= 0 || w_in <= 0) return PCONV_ERR_SHAPE;
   const unsigned known =
@@ -35,6 +49,7 @@ extern "C" pconv_status pconv_forward(const pconv_handle* h, const void* x, cons
   if (sel & (sel - 1)) return PCONV_ERR_UNSUPPORTED;  // at most one selection bit
   if (((uintptr_t)x | (uintptr_t)y) & 15u) return PCONV_ERR_ALIGN;
   if (bias && ((uintptr_t)bias & 3u)) return PCONV_ERR_ALIGN;
+  if (ws && ((uintptr_t)ws & 255u)) return PCONV_ERR_ALIGN;
   if (n == 0) return PCONV_OK;
   const DeviceLayer& L = h->d;
   {  // x and y must not overlap
@@ -53,9 +68,9 @@ extern "C" pconv_status pconv_forward(const pconv_handle* h, const void* x, cons
   } else if (sel == PCONV_KERNEL_TILED || sel == PCONV_KERNEL_GENERIC_TAPS) {
     if (!tiled_supported(L, n, h_in, w_in)) return PCONV_ERR_UNSUPPORTED;
     const bool generic = (sel == PCONV_KERNEL_GENERIC_TAPS) || !h->canonical;
-    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, generic, stream);
+    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, generic, ws, ws_bytes, stream);
   } else if (tiled_supported(L, n, h_in, w_in)) {
-    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, !h->canonical, stream);
+    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, !h->canonical, ws, ws_bytes, stream);
   } else {
     e = launch_simple(L, x, bias, y, n, h_in, w_in, relu, stream);
   }
@@ -100,6 +115,8 @@ struct pconv_stack {
   size_t in_bytes, out_bytes, act_bytes;
   void* act[2];   // ping-pong activations
   void* io[2];    // device input / output used by the host entry point
+  void* ws;       // channel-split workspace shared by the layers (kept zeroed between launches)
+  size_t ws_bytes;
 };
 
 extern "C" void pconv_stack_free(pconv_stack* s) {
@@ -108,6 +125,7 @@ extern "C" void pconv_stack_free(pconv_stack* s) {
     if (s->act[i]) cudaFree(s->act[i]);
     if (s->io[i]) cudaFree(s->io[i]);
   }
+  if (s->ws) cudaFree(s->ws);
   delete[] s->layers;
   delete[] s->bias;
   delete[] s->pool;
@@ -151,6 +169,8 @@ extern "C" pconv_status pconv_stack_create(const pconv_handle* const* layers,
       pconv_stack_free(s);
       return PCONV_ERR_SHAPE;
     }
+    const size_t wsb = tiled_workspace_bytes(L, n, ch, cw);
+    if (wsb > s->ws_bytes) s->ws_bytes = wsb;
     ch = (ch - 1) / L.stride + 1;
     cw = (cw - 1) / L.stride + 1;
     cc = L.c_out;
@@ -174,6 +194,10 @@ extern "C" pconv_status pconv_stack_create(const pconv_handle* const* layers,
   if (e == cudaSuccess) e = cudaMalloc(&s->act[1], max_act);
   if (e == cudaSuccess) e = cudaMalloc(&s->io[0], s->in_bytes);
   if (e == cudaSuccess) e = cudaMalloc(&s->io[1], s->out_bytes);
+  if (e == cudaSuccess && s->ws_bytes) {
+    e = cudaMalloc(&s->ws, s->ws_bytes);
+    if (e == cudaSuccess) e = cudaMemset(s->ws, 0, s->ws_bytes);
+  }
   if (e != cudaSuccess) {
     cudaGetLastError();
     pconv_stack_free(s);
@@ -201,7 +225,8 @@ extern "C" pconv_status pconv_stack_forward(pconv_stack* s, const void* x, void*
     const pconv::DeviceLayer& L = s->layers[i]->d;
     const bool last_op = (i == s->n_layers - 1) && !s->pool[i];
     void* dst = last_op ? y : s->act[which];
-    pconv_status st = pconv_forward(s->layers[i], cur, s->bias[i], dst, s->n, ch, cw, s->flags, stream);
+    pconv_status st = pconv_forward_ws(s->layers[i], cur, s->bias[i], dst, s->n, ch, cw, s->flags,
+                                       s->ws, s->ws_bytes, stream);
     if (st != PCONV_OK) return st;
     ch = (ch - 1) / L.stride + 1;
     cw = (cw - 1) / L.stride + 1;

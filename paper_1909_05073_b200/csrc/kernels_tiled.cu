@@ -29,6 +29,7 @@
 // layer's status word and the warp stops working but still reaches the common exit, where the
 // TMEM allocation is released.
 #include <cuda_fp16.h>
+#include <cstdlib>
 
 #include "pconv_internal.h"
 
@@ -48,6 +49,7 @@ constexpr int kWSlot = kMaxBlockKernels * 32;  // bytes per (group, stage): {w0,
 constexpr int kCodeSlot = 288;                 // bytes per (group, stage)
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr int kSmemLimit = 227 * 1024;
+constexpr int kNumSMs = 148;
 
 struct SubTile {
   int n, y0, x0, valid;  // image, first output row / column, inside the batch?
@@ -60,6 +62,7 @@ struct Geo {
   int pairs;             // sub-tile pairs per CTA = wy * sw
   int rows, pitch, substride, chan_stride;  // float2 units
   int stages, x_stage_bytes, stage_bytes, tab_off, desc_off, stage_off;
+  int ks, cps;           // channel splits (grid.z) and chunks per split
   int relu, is_half;
 };
 
@@ -327,10 +330,131 @@ __device__ __forceinline__ void produce_chunk_half(const DeviceLayer& L, const G
   }
 }
 
+// Outputs of one consumer warp (16 filter slots x 4 rows x {A,B} per lane).
+//   mode 0: y = act(accumulator + bias)               (no channel split)
+//   mode 1: workspace += accumulator                  (partial sum of a split)
+template <bool GENERIC>
+__device__ __forceinline__ void write_outputs(const DeviceLayer& L, const Geo& g, const SubTile* tab,
+                                              const float* __restrict__ bias, void* __restrict__ y,
+                                              float* __restrict__ ws,
+                                              const u64 (&acc)[GENERIC ? kGroup : 1][4], uint32_t tq,
+                                              int gi, int slot, int col, int mode) {
+  const SubTile A = tab[2 * slot], B = tab[2 * slot + 1];
+  const int ox_a = A.x0 + col, ox_b = B.x0 + col;
+  const bool col_a = A.valid && ox_a < g.w_out, col_b = B.valid && ox_b < g.w_out;
+  const size_t plane = (size_t)g.h_out * g.w_out;
+#pragma unroll
+  for (int a = 0; a < kGroup; ++a) {
+    uint32_t v[8];
+    if constexpr (GENERIC) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        v[2 * k] = (uint32_t)acc[a][k];
+        v[2 * k + 1] = (uint32_t)(acc[a][k] >> 32);
+      }
+    } else {
+      tmem_ld8(v, tq + a * 8);  // warp-uniform: all lanes take part
+    }
+    const int o = __ldg(L.perm + gi * kGroup + a);
+    if (o < 0) continue;
+    const float bv = bias ? __ldg(bias + o) : 0.f;
+    const size_t base_a = ((size_t)A.n * L.c_out + o) * plane;
+    const size_t base_b = ((size_t)B.n * L.c_out + o) * plane;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int ya = A.y0 + k, yb = B.y0 + k;
+      const bool in_a = col_a && ya < g.h_out, in_b = col_b && yb < g.h_out;
+      const size_t ia = base_a + (size_t)ya * g.w_out + ox_a;
+      const size_t ib = base_b + (size_t)yb * g.w_out + ox_b;
+      float va = __uint_as_float(v[2 * k]), vb = __uint_as_float(v[2 * k + 1]);
+      if (mode == 1) {
+        if (in_a) atomicAdd(ws + ia, va);
+        if (in_b) atomicAdd(ws + ib, vb);
+        continue;
+      }
+      va += bv;
+      vb += bv;
+      if (g.relu) {
+        va = fmaxf(va, 0.f);
+        vb = fmaxf(vb, 0.f);
+      }
+      if (g.is_half) {
+        __half* yh = (__half*)y;
+        if (in_a) yh[ia] = __float2half_rn(va);
+        if (in_b) yh[ib] = __float2half_rn(vb);
+      } else {
+        float* yf = (float*)y;
+        if (in_a) yf[ia] = va;
+        if (in_b) yf[ib] = vb;
+      }
+    }
+  }
+}
+
+// Mode 2 of the above for the last split of a tile, written so that many workspace loads are in
+// flight at once (4 filter slots = 32 independent loads per lane) instead of one per round trip.
+__device__ __forceinline__ void finalize_outputs(const DeviceLayer& L, const Geo& g, const SubTile* tab,
+                                                 const float* __restrict__ bias, void* __restrict__ y,
+                                                 float* __restrict__ ws, int gi, int slot, int col) {
+  const SubTile A = tab[2 * slot], B = tab[2 * slot + 1];
+  const int ox_a = A.x0 + col, ox_b = B.x0 + col;
+  const bool col_a = A.valid && ox_a < g.w_out, col_b = B.valid && ox_b < g.w_out;
+  const size_t plane = (size_t)g.h_out * g.w_out;
+  constexpr int kBatch = 4;
+  for (int a0 = 0; a0 < kGroup; a0 += kBatch) {
+    float v[kBatch][8];
+    size_t idx[kBatch][2];
+    int oo[kBatch];
+#pragma unroll
+    for (int b = 0; b < kBatch; ++b) {
+      const int o = __ldg(L.perm + gi * kGroup + a0 + b);
+      oo[b] = o;
+      idx[b][0] = ((size_t)A.n * L.c_out + (o < 0 ? 0 : o)) * plane + ox_a;
+      idx[b][1] = ((size_t)B.n * L.c_out + (o < 0 ? 0 : o)) * plane + ox_b;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const bool in_a = o >= 0 && col_a && A.y0 + k < g.h_out;
+        const bool in_b = o >= 0 && col_b && B.y0 + k < g.h_out;
+        v[b][2 * k] = in_a ? __ldcg(ws + idx[b][0] + (size_t)(A.y0 + k) * g.w_out) : 0.f;
+        v[b][2 * k + 1] = in_b ? __ldcg(ws + idx[b][1] + (size_t)(B.y0 + k) * g.w_out) : 0.f;
+      }
+    }
+#pragma unroll
+    for (int b = 0; b < kBatch; ++b) {
+      const int o = oo[b];
+      if (o < 0) continue;
+      const float bv = bias ? __ldg(bias + o) : 0.f;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const bool in_a = col_a && A.y0 + k < g.h_out, in_b = col_b && B.y0 + k < g.h_out;
+        const size_t ia = idx[b][0] + (size_t)(A.y0 + k) * g.w_out;
+        const size_t ib = idx[b][1] + (size_t)(B.y0 + k) * g.w_out;
+        float va = v[b][2 * k] + bv, vb = v[b][2 * k + 1] + bv;
+        if (g.relu) {
+          va = fmaxf(va, 0.f);
+          vb = fmaxf(vb, 0.f);
+        }
+        if (in_a) ws[ia] = 0.f;
+        if (in_b) ws[ib] = 0.f;
+        if (g.is_half) {
+          __half* yh = (__half*)y;
+          if (in_a) yh[ia] = __float2half_rn(va);
+          if (in_b) yh[ib] = __float2half_rn(vb);
+        } else {
+          float* yf = (float*)y;
+          if (in_a) yf[ia] = va;
+          if (in_b) yf[ib] = vb;
+        }
+      }
+    }
+  }
+}
+
 template <int S, bool GENERIC>
 __global__ void __launch_bounds__(cta_threads(GENERIC), 1)
 tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
-             const float* __restrict__ bias, void* __restrict__ y) {
+             const float* __restrict__ bias, void* __restrict__ y, float* __restrict__ ws,
+             int* __restrict__ counters) {
   constexpr int kCW = consumer_warps(GENERIC);
   constexpr int kThreads = cta_threads(GENERIC);
   extern __shared__ __align__(16) unsigned char smem[];
@@ -392,21 +516,41 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = GENERIC ? 0u : *tmem_base_s;
+  const int k0 = blockIdx.z * g.cps;                       // this CTA's chunk range
+  const int nk = min(L.n_chunks, k0 + g.cps) - k0;
+
+  // consumer-warp coordinates (meaningless for producer warps)
+  const int wyi = warp % g.wys, wgi = warp / g.wys;
+  const int gi = blockIdx.y * g.ng + wgi;
+  const bool active = (wyi < g.wy) && (gi < L.n_groups);
+  const int slot = wyi * g.sw + lane / g.tw;  // sub-tile pair of this lane
+  const int col = lane % g.tw;
+  const uint32_t pitch_b = g.pitch * 8;
+  const uint32_t off_mid = (S == 1) ? 8u : (uint32_t)(g.tw + 1) * 8u;
+  const uint32_t off_right = (S == 1) ? 16u : 8u;
+  const uint32_t chan_b = (uint32_t)g.chan_stride * 8u;
+  const uint32_t lane_off = (uint32_t)(slot * g.substride + col) * 8u;
+  // TMEM: a warp reaches the 32 lanes of its quadrant (warp % 4); 4 warps share a quadrant and
+  // take 128 columns each = 16 filter slots x (4 rows x {A,B}).
+  const uint32_t tq = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)((warp >> 2) * (kGroup * 8));
+
+  u64 acc[GENERIC ? kGroup : 1][4];
+  bool ok = true;
 
   if (warp >= kCW) {
     // ===================================== producer warps =====================================
     if (GENERIC) asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
     const int pw = warp - kCW;
     const uint8_t* codes = GENERIC ? L.codes_g : L.codes_s;
-    for (int k = 0; k < L.n_chunks; ++k) {
-      const int s = k % g.stages, it = k / g.stages;
+    for (int kk = 0; kk < nk; ++kk) {
+      const int s = kk % g.stages, it = kk / g.stages;
       if (it > 0 && !mbar_wait(sbase + 8 * (kMaxStages + s), (it - 1) & 1, L.err, 1)) break;
       const uint32_t stage_base = sbase + g.stage_off + s * g.stage_bytes;
       if (g.is_half) {
-        produce_chunk_half<S>(L, g, (const __half*)x, tab, desc, codes, stage_base, k, pw, lane);
+        produce_chunk_half<S>(L, g, (const __half*)x, tab, desc, codes, stage_base, k0 + kk, pw, lane);
         mbar_arrive(sbase + 8 * s);
       } else {
-        produce_chunk_async<S>(L, g, (const float*)x, tab, desc, codes, stage_base, k, pw, lane);
+        produce_chunk_async<S>(L, g, (const float*)x, tab, desc, codes, stage_base, k0 + kk, pw, lane);
         cp_async_arrive(sbase + 8 * s);
       }
     }
@@ -414,21 +558,6 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   } else {
     // ===================================== consumer warps =====================================
     if (GENERIC) asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
-    const int wyi = warp % g.wys, wgi = warp / g.wys;
-    const int gi = blockIdx.y * g.ng + wgi;
-    const bool active = (wyi < g.wy) && (gi < L.n_groups);
-    const int slot = wyi * g.sw + lane / g.tw;  // sub-tile pair of this lane
-    const int col = lane % g.tw;
-    const uint32_t pitch_b = g.pitch * 8;
-    const uint32_t off_mid = (S == 1) ? 8u : (uint32_t)(g.tw + 1) * 8u;
-    const uint32_t off_right = (S == 1) ? 16u : 8u;
-    const uint32_t chan_b = (uint32_t)g.chan_stride * 8u;
-    const uint32_t lane_off = (uint32_t)(slot * g.substride + col) * 8u;
-    // TMEM: a warp reaches the 32 lanes of its quadrant (warp % 4); 4 warps share a quadrant and
-    // take 128 columns each = 16 filter slots x (4 rows x {A,B}).
-    const uint32_t tq = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)((warp >> 2) * (kGroup * 8));
-
-    u64 acc[GENERIC ? kGroup : 1][4];
     if constexpr (GENERIC) {
 #pragma unroll
       for (int a = 0; a < kGroup; ++a)
@@ -439,10 +568,9 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
     }
 
-    bool ok = true;
-    for (int k = 0; k < L.n_chunks && ok; ++k) {
-      const int s = k % g.stages;
-      ok = mbar_wait(sbase + 8 * s, (k / g.stages) & 1, L.err, 2);
+    for (int kk = 0; kk < nk && ok; ++kk) {
+      const int s = kk % g.stages;
+      ok = mbar_wait(sbase + 8 * s, (kk / g.stages) & 1, L.err, 2);
       if (!ok) break;
       if (active) {
         const uint32_t stage_base = sbase + g.stage_off + s * g.stage_bytes;
@@ -475,64 +603,40 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
       if (lane == 0) mbar_arrive(sbase + 8 * (kMaxStages + s));
     }
 
-    // ---- epilogue: bias, ReLU, store at the original filter index --------------------------------
-    if (active && ok) {
-      const SubTile A = tab[2 * slot], B = tab[2 * slot + 1];
-      const int ox_a = A.x0 + col, ox_b = B.x0 + col;
-      const bool col_a = A.valid && ox_a < g.w_out, col_b = B.valid && ox_b < g.w_out;
-      const size_t plane = (size_t)g.h_out * g.w_out;
-#pragma unroll
-      for (int a = 0; a < kGroup; ++a) {
-        uint32_t v[8];
-        if constexpr (GENERIC) {
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            v[2 * k] = (uint32_t)acc[a][k];
-            v[2 * k + 1] = (uint32_t)(acc[a][k] >> 32);
-          }
-        } else {
-          tmem_ld8(v, tq + a * 8);  // all lanes take part: the slot loop is warp-uniform
-        }
-        const int o = __ldg(L.perm + gi * kGroup + a);
-        if (o < 0) continue;
-        const float bv = bias ? __ldg(bias + o) : 0.f;
-        const size_t base_a = ((size_t)A.n * L.c_out + o) * plane;
-        const size_t base_b = ((size_t)B.n * L.c_out + o) * plane;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          float va = __uint_as_float(v[2 * k]) + bv;
-          float vb = __uint_as_float(v[2 * k + 1]) + bv;
-          if (g.relu) {
-            va = fmaxf(va, 0.f);
-            vb = fmaxf(vb, 0.f);
-          }
-          const int ya = A.y0 + k, yb = B.y0 + k;
-          if (g.is_half) {
-            __half* yh = (__half*)y;
-            if (col_a && ya < g.h_out) yh[base_a + (size_t)ya * g.w_out + ox_a] = __float2half_rn(va);
-            if (col_b && yb < g.h_out) yh[base_b + (size_t)yb * g.w_out + ox_b] = __float2half_rn(vb);
-          } else {
-            float* yf = (float*)y;
-            if (col_a && ya < g.h_out) yf[base_a + (size_t)ya * g.w_out + ox_a] = va;
-            if (col_b && yb < g.h_out) yf[base_b + (size_t)yb * g.w_out + ox_b] = vb;
-          }
-        }
-      }
-    }
+    // ---- epilogue: final values straight to y, or partial sums into the workspace --------------
+    if (active && ok)
+      write_outputs<GENERIC>(L, g, tab, bias, y, ws, acc, tq, gi, slot, col, g.ks > 1 ? 1 : 0);
+    if (g.ks > 1) __threadfence();
   }
 
   // ---- common exit: every warp arrives here, then the TMEM columns are handed back ---------------
-  if (!GENERIC) {
+  if constexpr (!GENERIC) {
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 0)
       asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols)
                    : "memory");
+    if (g.ks > 1) {
+      // The split that arrives last at this output tile's ticket turns the summed partials into
+      // the layer's output and leaves workspace and ticket zeroed for the next launch.
+      volatile uint32_t* last = tmem_base_s + 1;
+      if (tid == 0) {
+        int* ticket = counters + blockIdx.y * gridDim.x + blockIdx.x;
+        const int t = atomicAdd(ticket, 1);
+        *last = (t == g.ks - 1) ? 1u : 0u;
+        if (t == g.ks - 1) *ticket = 0;
+      }
+      __syncthreads();
+      if (*last && warp < kCW && active && ok) {
+        __threadfence();
+        finalize_outputs(L, g, tab, bias, y, ws, gi, slot, col);
+      }
+    }
   }
 }
 
 template <bool GENERIC>
-bool make_geo(const DeviceLayer& L, int n, int h, int w, Geo* out) {
+bool make_geo(const DeviceLayer& L, int n, int h, int w, bool allow_split, Geo* out) {
   constexpr int kCW = consumer_warps(GENERIC);
   Geo g;
   g.n = n;
@@ -548,12 +652,17 @@ bool make_geo(const DeviceLayer& L, int n, int h, int w, Geo* out) {
   const long long q = (long long)n * g.tx * g.ty;
   if (q > 0x7FFFFFFF) return false;
   g.q_total = (int)q;
-  // filter groups per CTA: a power of two dividing the consumer warps, at most 4 (8 for the
-  // 16-warp variant when the layer is wide), so that the staged input is shared widely
-  g.ng = 1;
-  const int ng_max = GENERIC ? 4 : (L.n_groups >= 16 ? 8 : 4);
-  while (g.ng < ng_max && g.ng < L.n_groups) g.ng *= 2;
+  // Filter groups per CTA (ng) x pixel sets (wy) = consumer warps.  Wide ng shares the staged input
+  // among more filters; when the whole batch has few sub-tiles, pixel sets are traded for groups.
+  int ng_max = 1;
+  while (ng_max < kCW && ng_max < L.n_groups) ng_max *= 2;
+  g.ng = ng_max < (GENERIC ? 4 : 8) ? ng_max : (GENERIC ? 4 : 8);
   g.wys = kCW / g.ng;
+  const long long pairs_needed = (q + 1) / 2;
+  while (g.ng < ng_max && (long long)(g.wys / 2) * g.sw >= pairs_needed) {
+    g.ng *= 2;
+    g.wys /= 2;
+  }
   g.wy = g.wys;
   g.rows = (L.stride == 1) ? 6 : 9;
   g.pitch = (L.stride == 1) ? (g.tw + 2) : (2 * g.tw + 1);
@@ -571,11 +680,34 @@ bool make_geo(const DeviceLayer& L, int n, int h, int w, Geo* out) {
     g.stage_off = g.desc_off + g.ng * L.n_chunks * 16;
     g.stages = (kSmemLimit - g.stage_off) / g.stage_bytes;
     if (g.stages > kMaxStages) g.stages = kMaxStages;
-    if (g.stages >= 2 || g.wy == 1) break;
-    g.wy /= 2;
+    if (g.stages >= 2) break;
+    if (g.wy > 1) {
+      g.wy /= 2;          // fewer pixel sets (the other warp rows idle)
+    } else if (g.ng > 1) {
+      g.ng /= 2;          // fewer filter groups per CTA
+      g.wys = kCW / g.ng;
+    } else {
+      break;
+    }
   }
   if (g.stages < 2) return false;
-  if (g.stages > L.n_chunks) g.stages = (L.n_chunks < 1) ? 1 : L.n_chunks;
+  // Channel splits: when the output tiles do not fill the GPU, cut the channel range so that
+  // about one CTA per SM is launched (measured on 14x14 .. 56x56 batch-1 layers: the best split
+  // count is the one that fills a single wave; more splits only add reduction traffic).
+  g.ks = 1;
+  if (allow_split && !GENERIC) {
+    const long long ctas = ((q + 2 * g.pairs - 1) / (2 * g.pairs)) * ((L.n_groups + g.ng - 1) / g.ng);
+    long long ks = kNumSMs / ctas;
+    if (ks > L.n_chunks) ks = L.n_chunks;
+    if (ks > 1) g.ks = (int)ks;
+  }
+  if (allow_split && !GENERIC) {
+    const char* dbg = getenv("PCONV_DEBUG_KS");  // experiment hook
+    if (dbg) g.ks = atoi(dbg) < L.n_chunks ? (atoi(dbg) > 0 ? atoi(dbg) : 1) : L.n_chunks;
+  }
+  g.cps = (L.n_chunks + g.ks - 1) / g.ks;
+  g.ks = (L.n_chunks + g.cps - 1) / g.cps;
+  if (g.stages > g.cps) g.stages = g.cps;
   g.relu = 0;
   g.is_half = (L.storage == PCONV_F16);
   *out = g;
@@ -583,8 +715,8 @@ bool make_geo(const DeviceLayer& L, int n, int h, int w, Geo* out) {
 }
 
 template <int S, bool GENERIC>
-cudaError_t launch_one(const DeviceLayer& L, Geo g, const void* x, const float* bias, void* y,
-                       cudaStream_t stream) {
+cudaError_t launch_one(const DeviceLayer& L, Geo g, const void* x, const float* bias, void* y, float* ws,
+                       int* counters, cudaStream_t stream) {
   int smem = g.stage_off + g.stages * g.stage_bytes;
   // the TMEM variant must be alone on its SM (it takes all 512 columns): make sure two CTAs can
   // never be co-resident by asking for more than half of the shared memory
@@ -594,10 +726,14 @@ cudaError_t launch_one(const DeviceLayer& L, Geo g, const void* x, const float* 
   if (e != cudaSuccess) return e;
   const long long ctas_x = ((long long)g.q_total + 2 * g.pairs - 1) / (2 * g.pairs);
   const int ctas_y = (L.n_groups + g.ng - 1) / g.ng;
-  if (ctas_x > 0x7FFFFFFF || ctas_y > 65535) return cudaErrorInvalidValue;
-  dim3 grid((unsigned)ctas_x, (unsigned)ctas_y);
-  tiled_kernel<S, GENERIC><<<grid, cta_threads(GENERIC), smem, stream>>>(L, g, x, bias, y);
+  if (ctas_x > 0x7FFFFFFF || ctas_y > 65535 || g.ks > 65535) return cudaErrorInvalidValue;
+  dim3 grid((unsigned)ctas_x, (unsigned)ctas_y, (unsigned)g.ks);
+  tiled_kernel<S, GENERIC><<<grid, cta_threads(GENERIC), smem, stream>>>(L, g, x, bias, y, ws, counters);
   return cudaGetLastError();
+}
+
+size_t out_elems(const DeviceLayer& L, int n, int h, int w) {
+  return (size_t)n * L.c_out * ((h - 1) / L.stride + 1) * ((w - 1) / L.stride + 1);
 }
 
 }  // namespace
@@ -606,21 +742,40 @@ bool tiled_supported(const DeviceLayer& L, int n, int h, int w) {
   Geo g;
   if (n <= 0 || h <= 0 || w <= 0) return false;
   if (L.n_groups > 65535) return false;
-  return make_geo<true>(L, n, h, w, &g) && make_geo<false>(L, n, h, w, &g);
+  return make_geo<true>(L, n, h, w, false, &g) && make_geo<false>(L, n, h, w, false, &g);
+}
+
+// Workspace of the channel-split path: one fp32 partial sum per output element, then one ticket
+// per (pixel tile, filter-group set); 0 if this shape is never split.
+size_t tiled_workspace_bytes(const DeviceLayer& L, int n, int h, int w) {
+  Geo g;
+  if (!L.codes_s || !make_geo<false>(L, n, h, w, true, &g) || g.ks <= 1) return 0;
+  const size_t ctas = (((size_t)g.q_total + 2 * g.pairs - 1) / (2 * g.pairs)) *
+                      ((L.n_groups + g.ng - 1) / g.ng);
+  return ((out_elems(L, n, h, w) * 4 + 255) & ~(size_t)255) + ((ctas * 4 + 255) & ~(size_t)255);
 }
 
 cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias, void* y, int n, int h,
-                         int w, bool relu, bool generic_taps, cudaStream_t stream) {
+                         int w, bool relu, bool generic_taps, void* ws, size_t ws_bytes,
+                         cudaStream_t stream) {
   if (!generic_taps && !L.codes_s) generic_taps = true;
   Geo g;
-  if (!(generic_taps ? make_geo<true>(L, n, h, w, &g) : make_geo<false>(L, n, h, w, &g)))
+  const size_t need = generic_taps ? 0 : tiled_workspace_bytes(L, n, h, w);
+  const bool split = need > 0 && ws && ws_bytes >= need;
+  if (!(generic_taps ? make_geo<true>(L, n, h, w, false, &g) : make_geo<false>(L, n, h, w, split, &g)))
     return cudaErrorInvalidValue;
   g.relu = relu ? 1 : 0;
+  float* wsf = nullptr;
+  int* counters = nullptr;
+  if (g.ks > 1) {
+    wsf = (float*)ws;
+    counters = (int*)((char*)ws + ((out_elems(L, n, h, w) * 4 + 255) & ~(size_t)255));
+  }
   if (L.stride == 1)
-    return generic_taps ? launch_one<1, true>(L, g, x, bias, y, stream)
-                        : launch_one<1, false>(L, g, x, bias, y, stream);
-  return generic_taps ? launch_one<2, true>(L, g, x, bias, y, stream)
-                      : launch_one<2, false>(L, g, x, bias, y, stream);
+    return generic_taps ? launch_one<1, true>(L, g, x, bias, y, wsf, counters, stream)
+                        : launch_one<1, false>(L, g, x, bias, y, wsf, counters, stream);
+  return generic_taps ? launch_one<2, true>(L, g, x, bias, y, wsf, counters, stream)
+                      : launch_one<2, false>(L, g, x, bias, y, wsf, counters, stream);
 }
 
 }  // namespace pconv

@@ -335,6 +335,7 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
     d.storage = storage;
     d.n_groups = n_groups;
     d.n_chunks = n_chunks;
+    d.n_kept = n_kept;
 
     pconv_stats_t& st = h->stats;
     st.c_out = c_out;

@@ -51,6 +51,7 @@ struct DeviceLayer {         // device pointers of one packed layer (passed to k
   const int* perm;           // [n_groups * kGroup] original filter index or -1
   int* err;                  // device status word (0 = fine)
   int c_out, c_in, stride, storage, n_groups, n_chunks;
+  long long n_kept;          // surviving kernels of the layer
 };
 
 }  // namespace pconv
@@ -74,7 +75,9 @@ namespace pconv {
 cudaError_t launch_simple(const DeviceLayer& L, const void* x, const float* bias, void* y, int n,
                           int h, int w, bool relu, cudaStream_t stream);
 cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias, void* y, int n,
-                         int h, int w, bool relu, bool generic_taps, cudaStream_t stream);
+                         int h, int w, bool relu, bool generic_taps, void* ws, size_t ws_bytes,
+                         cudaStream_t stream);
+size_t tiled_workspace_bytes(const DeviceLayer& L, int n, int h, int w);
 bool tiled_supported(const DeviceLayer& L, int n, int h, int w);
 cudaError_t launch_maxpool(const void* x, void* y, int n, int c, int h, int w, int storage,
                            cudaStream_t stream);

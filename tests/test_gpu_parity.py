@@ -201,3 +201,73 @@ def test_maxpool_matches_the_oracle(storage):
                         device="cuda")
         B.pconv_maxpool2x2(xt, y)
         assert np.array_equal(y.float().cpu().numpy(), oracle.maxpool2x2(x))
+
+
+SPLIT_CASES = [  # batch-1 layers that the library splits over input channels when given a workspace
+    (64, 64, 14, 14, 1, 1, 0.4), (128, 96, 28, 28, 1, 1, 0.3), (96, 160, 7, 7, 2, 1, 0.35),
+    (72, 48, 28, 28, 1, 2, 0.4), (256, 64, 9, 11, 1, 1, 0.3),
+]
+
+
+@pytest.mark.parametrize("storage", ["f32", "f16"])
+@pytest.mark.parametrize("case", SPLIT_CASES, ids=lambda c: "x".join(str(v) for v in c))
+def test_channel_split_path_matches_the_oracle(case, storage):
+    c_in, c_out, h, w, n, stride, keep = case
+    spec = synth.LayerSpec("t", c_in, c_out, h, w, stride, keep)
+    wt, bias, _ = synth.gen_weights(spec, 4242 + c_in)
+    x = synth.gen_input(spec, n, 4242 + c_in)
+    layer = B.Layer(wt, synth.PATTERNS8, stride, B.F16 if storage == "f16" else B.F32, bias)
+    xt = torch.from_numpy(x).cuda()
+    if storage == "f16":
+        xt = xt.half()
+    assert B.pconv_workspace_bytes(layer.handle, n, h, w) > 0
+    ref = oracle_layer(wt, bias, x, stride, storage, True)
+    for _ in range(3):   # the workspace must come back zeroed: repeated calls stay correct
+        y = layer.forward(xt, relu=True, split=True)
+        torch.cuda.synchronize()
+        check_close(y.float().cpu().numpy(), ref, storage, "split %s" % (case,))
+    assert not layer._ws.any()
+    assert B.pconv_device_status(layer.handle)[0] == 0
+    layer.close()
+
+
+@pytest.mark.parametrize("storage", ["f32", "f16"])
+def test_stack_matches_the_chained_oracle(storage):
+    chans = [(3, 16), (16, 24), (24, 40), (40, 40)]
+    pools = [False, True, False, True]
+    h = 20
+    st = B.F16 if storage == "f16" else B.F32
+    layers, ws = [], []
+    hh = h
+    for i, (ci, co) in enumerate(chans):
+        spec = synth.LayerSpec("s%d" % i, ci, co, hh, hh, 1, 1.0 if i == 0 else 0.5, sigma=None,
+                               x_dist="uniform_01")
+        w, b, _ = synth.gen_weights(spec, 900 + i)
+        layers.append(B.Layer(w, synth.PATTERNS8, 1, st, b))
+        ws.append((w, b))
+        if pools[i]:
+            hh //= 2
+    x = synth.gen_input(synth.LayerSpec("in", 3, 16, h, h, 1, 1.0, x_dist="uniform_01"), 2, 901)
+    stack = B.Stack(layers, pools, 2, h, h, B.RELU)
+    xt = torch.from_numpy(x).cuda()
+    xh = x
+    if storage == "f16":
+        xt = xt.half()
+    y = torch.empty(stack.out_shape, dtype=xt.dtype, device="cuda")
+    stack.forward(xt, y)
+    torch.cuda.synchronize()
+    a = xh
+    for (w, b), pool in zip(ws, pools):
+        a = oracle.conv3x3(a, w, b, 1, True, storage)
+        if storage == "f16":        # activations are stored as fp16 between layers
+            a = a.astype(np.float16).astype(np.float32)
+        if pool:
+            a = oracle.maxpool2x2(a)
+    check_close(y.float().cpu().numpy(), a, storage, "stack")
+    # host entry point gives the same result
+    x_host = xt.cpu()
+    y_host = torch.empty(stack.out_shape, dtype=xt.dtype)
+    stack.forward_host(x_host, y_host)
+    assert torch.equal(y_host, y.cpu()) or storage == "f32" and np.allclose(
+        y_host.numpy(), y.cpu().numpy(), rtol=0, atol=1e-5)
+    stack.close()
