@@ -330,121 +330,114 @@ __device__ __forceinline__ void produce_chunk_half(const DeviceLayer& L, const G
   }
 }
 
-// Outputs of one consumer warp (16 filter slots x 4 rows x {A,B} per lane).
-//   mode 0: y = act(accumulator + bias)               (no channel split)
-//   mode 1: workspace += accumulator                  (partial sum of a split)
-template <bool GENERIC>
-__device__ __forceinline__ void write_outputs(const DeviceLayer& L, const Geo& g, const SubTile* tab,
-                                              const float* __restrict__ bias, void* __restrict__ y,
-                                              float* __restrict__ ws,
-                                              const u64 (&acc)[GENERIC ? kGroup : 1][4], uint32_t tq,
-                                              int gi, int slot, int col, int mode) {
+__device__ __forceinline__ void red_add_f32(float* p, float v) {
+  asm volatile("red.global.add.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
+}
+
+// Where a lane's outputs go: element offsets (inside one filter's plane stack) of the 4 rows of its
+// A and B pixels, or -1 where the pixel lies outside the image or the batch.
+struct LaneOut {
+  long long off[8];   // [2*k] = A row k, [2*k+1] = B row k
+};
+__device__ __forceinline__ LaneOut lane_outputs(const DeviceLayer& L, const Geo& g, const SubTile* tab,
+                                                int slot, int col) {
   const SubTile A = tab[2 * slot], B = tab[2 * slot + 1];
   const int ox_a = A.x0 + col, ox_b = B.x0 + col;
   const bool col_a = A.valid && ox_a < g.w_out, col_b = B.valid && ox_b < g.w_out;
-  const size_t plane = (size_t)g.h_out * g.w_out;
+  const long long plane = (long long)g.h_out * g.w_out;
+  LaneOut r;
 #pragma unroll
-  for (int a = 0; a < kGroup; ++a) {
-    uint32_t v[8];
-    if constexpr (GENERIC) {
+  for (int k = 0; k < 4; ++k) {
+    const int ya = A.y0 + k, yb = B.y0 + k;
+    r.off[2 * k] = (col_a && ya < g.h_out) ? ((long long)A.n * L.c_out * plane + (long long)ya * g.w_out + ox_a) : -1;
+    r.off[2 * k + 1] = (col_b && yb < g.h_out) ? ((long long)B.n * L.c_out * plane + (long long)yb * g.w_out + ox_b) : -1;
+  }
+  return r;
+}
+
+__device__ __forceinline__ void store_out(const Geo& g, void* __restrict__ y, long long i, float v) {
+  if (g.relu) v = fmaxf(v, 0.f);
+  if (g.is_half)
+    ((__half*)y)[i] = __float2half_rn(v);
+  else
+    ((float*)y)[i] = v;
+}
+
+// Outputs of one consumer warp (16 filter slots x 4 rows x {A,B} per lane).  `my_o` / `my_b` hold,
+// in lane a < 16, the original filter index and the bias of slot a (loaded at kernel start).
+//   mode 0: y = act(accumulator + bias)               (no channel split)
+//   mode 1: workspace += accumulator                  (partial sum of a split)
+template <bool GENERIC>
+__device__ __forceinline__ void write_outputs(const DeviceLayer& L, const Geo& g, const LaneOut& lo,
+                                              void* __restrict__ y, float* __restrict__ ws,
+                                              const u64 (&acc)[GENERIC ? kGroup : 1][4], uint32_t tq,
+                                              int my_o, float my_b, int mode) {
+  const long long plane = (long long)g.h_out * g.w_out;
+  auto emit = [&](int a, const uint32_t (&v)[8]) {
+    const int o = __shfl_sync(0xffffffffu, my_o, a);
+    const float bv = __shfl_sync(0xffffffffu, my_b, a);
+    if (o < 0) return;
+    const long long base = (long long)o * plane;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      if (lo.off[e] < 0) continue;
+      const float val = __uint_as_float(v[e]);
+      if (mode == 1)
+        red_add_f32(ws + base + lo.off[e], val);
+      else
+        store_out(g, y, base + lo.off[e], val + bv);
+    }
+  };
+  if constexpr (GENERIC) {
+#pragma unroll
+    for (int a = 0; a < kGroup; ++a) {
+      uint32_t v[8];
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         v[2 * k] = (uint32_t)acc[a][k];
         v[2 * k + 1] = (uint32_t)(acc[a][k] >> 32);
       }
-    } else {
-      tmem_ld8(v, tq + a * 8);  // warp-uniform: all lanes take part
+      emit(a, v);
     }
-    const int o = __ldg(L.perm + gi * kGroup + a);
-    if (o < 0) continue;
-    const float bv = bias ? __ldg(bias + o) : 0.f;
-    const size_t base_a = ((size_t)A.n * L.c_out + o) * plane;
-    const size_t base_b = ((size_t)B.n * L.c_out + o) * plane;
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const int ya = A.y0 + k, yb = B.y0 + k;
-      const bool in_a = col_a && ya < g.h_out, in_b = col_b && yb < g.h_out;
-      const size_t ia = base_a + (size_t)ya * g.w_out + ox_a;
-      const size_t ib = base_b + (size_t)yb * g.w_out + ox_b;
-      float va = __uint_as_float(v[2 * k]), vb = __uint_as_float(v[2 * k + 1]);
-      if (mode == 1) {
-        if (in_a) atomicAdd(ws + ia, va);
-        if (in_b) atomicAdd(ws + ib, vb);
-        continue;
-      }
-      va += bv;
-      vb += bv;
-      if (g.relu) {
-        va = fmaxf(va, 0.f);
-        vb = fmaxf(vb, 0.f);
-      }
-      if (g.is_half) {
-        __half* yh = (__half*)y;
-        if (in_a) yh[ia] = __float2half_rn(va);
-        if (in_b) yh[ib] = __float2half_rn(vb);
-      } else {
-        float* yf = (float*)y;
-        if (in_a) yf[ia] = va;
-        if (in_b) yf[ib] = vb;
-      }
+  } else {
+#pragma unroll 1
+    for (int a = 0; a < kGroup; ++a) {  // the slot is a run-time TMEM address: no unrolling needed
+      uint32_t v[8];
+      tmem_ld8(v, tq + a * 8);
+      emit(a, v);
     }
   }
 }
 
-// Mode 2 of the above for the last split of a tile, written so that many workspace loads are in
-// flight at once (4 filter slots = 32 independent loads per lane) instead of one per round trip.
-__device__ __forceinline__ void finalize_outputs(const DeviceLayer& L, const Geo& g, const SubTile* tab,
-                                                 const float* __restrict__ bias, void* __restrict__ y,
-                                                 float* __restrict__ ws, int gi, int slot, int col) {
-  const SubTile A = tab[2 * slot], B = tab[2 * slot + 1];
-  const int ox_a = A.x0 + col, ox_b = B.x0 + col;
-  const bool col_a = A.valid && ox_a < g.w_out, col_b = B.valid && ox_b < g.w_out;
-  const size_t plane = (size_t)g.h_out * g.w_out;
+// The last split of a tile: workspace -> y, leaving the workspace zeroed.  Four filter slots (32
+// independent loads per lane) are in flight at once.
+__device__ __forceinline__ void finalize_outputs(const DeviceLayer& L, const Geo& g, const LaneOut& lo,
+                                                 void* __restrict__ y, float* __restrict__ ws, int my_o,
+                                                 float my_b) {
+  const long long plane = (long long)g.h_out * g.w_out;
   constexpr int kBatch = 4;
+#pragma unroll 1
   for (int a0 = 0; a0 < kGroup; a0 += kBatch) {
     float v[kBatch][8];
-    size_t idx[kBatch][2];
-    int oo[kBatch];
+    long long base[kBatch];
+    float bv[kBatch];
 #pragma unroll
     for (int b = 0; b < kBatch; ++b) {
-      const int o = __ldg(L.perm + gi * kGroup + a0 + b);
-      oo[b] = o;
-      idx[b][0] = ((size_t)A.n * L.c_out + (o < 0 ? 0 : o)) * plane + ox_a;
-      idx[b][1] = ((size_t)B.n * L.c_out + (o < 0 ? 0 : o)) * plane + ox_b;
+      const int o = __shfl_sync(0xffffffffu, my_o, a0 + b);
+      bv[b] = __shfl_sync(0xffffffffu, my_b, a0 + b);
+      base[b] = (o < 0) ? -1 : (long long)o * plane;
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const bool in_a = o >= 0 && col_a && A.y0 + k < g.h_out;
-        const bool in_b = o >= 0 && col_b && B.y0 + k < g.h_out;
-        v[b][2 * k] = in_a ? __ldcg(ws + idx[b][0] + (size_t)(A.y0 + k) * g.w_out) : 0.f;
-        v[b][2 * k + 1] = in_b ? __ldcg(ws + idx[b][1] + (size_t)(B.y0 + k) * g.w_out) : 0.f;
-      }
+      for (int e = 0; e < 8; ++e)
+        v[b][e] = (base[b] >= 0 && lo.off[e] >= 0) ? __ldcg(ws + base[b] + lo.off[e]) : 0.f;
     }
 #pragma unroll
     for (int b = 0; b < kBatch; ++b) {
-      const int o = oo[b];
-      if (o < 0) continue;
-      const float bv = bias ? __ldg(bias + o) : 0.f;
+      if (base[b] < 0) continue;
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const bool in_a = col_a && A.y0 + k < g.h_out, in_b = col_b && B.y0 + k < g.h_out;
-        const size_t ia = idx[b][0] + (size_t)(A.y0 + k) * g.w_out;
-        const size_t ib = idx[b][1] + (size_t)(B.y0 + k) * g.w_out;
-        float va = v[b][2 * k] + bv, vb = v[b][2 * k + 1] + bv;
-        if (g.relu) {
-          va = fmaxf(va, 0.f);
-          vb = fmaxf(vb, 0.f);
-        }
-        if (in_a) ws[ia] = 0.f;
-        if (in_b) ws[ib] = 0.f;
-        if (g.is_half) {
-          __half* yh = (__half*)y;
-          if (in_a) yh[ia] = __float2half_rn(va);
-          if (in_b) yh[ib] = __float2half_rn(vb);
-        } else {
-          float* yf = (float*)y;
-          if (in_a) yf[ia] = va;
-          if (in_b) yf[ib] = vb;
-        }
+      for (int e = 0; e < 8; ++e) {
+        if (lo.off[e] < 0) continue;
+        ws[base[b] + lo.off[e]] = 0.f;
+        store_out(g, y, base[b] + lo.off[e], v[b][e] + bv[b]);
       }
     }
   }
@@ -534,6 +527,13 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   // take 128 columns each = 16 filter slots x (4 rows x {A,B}).
   const uint32_t tq = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)((warp >> 2) * (kGroup * 8));
 
+  // lane a < 16 keeps the original filter index and bias of slot a for the epilogue
+  int my_o = -1;
+  float my_b = 0.f;
+  if (warp < kCW && active && lane < kGroup) {
+    my_o = __ldg(L.perm + gi * kGroup + lane);
+    if (bias && my_o >= 0) my_b = __ldg(bias + my_o);
+  }
   u64 acc[GENERIC ? kGroup : 1][4];
   bool ok = true;
 
@@ -605,7 +605,8 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
 
     // ---- epilogue: final values straight to y, or partial sums into the workspace --------------
     if (active && ok)
-      write_outputs<GENERIC>(L, g, tab, bias, y, ws, acc, tq, gi, slot, col, g.ks > 1 ? 1 : 0);
+      write_outputs<GENERIC>(L, g, lane_outputs(L, g, tab, slot, col), y, ws, acc, tq, my_o, my_b,
+                             g.ks > 1 ? 1 : 0);
     if (g.ks > 1) __threadfence();
   }
 
@@ -629,7 +630,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
       __syncthreads();
       if (*last && warp < kCW && active && ok) {
         __threadfence();
-        finalize_outputs(L, g, tab, bias, y, ws, gi, slot, col);
+        finalize_outputs(L, g, lane_outputs(L, g, tab, slot, col), y, ws, my_o, my_b);
       }
     }
   }
