@@ -49,7 +49,8 @@ typedef enum {
   PCONV_ERR_ALIGN = 7,             /* a device pointer is not aligned as required */
   PCONV_ERR_ALLOC = 8,             /* host or device allocation failed */
   PCONV_ERR_CUDA = 9,              /* a CUDA runtime call or a kernel launch failed */
-  PCONV_ERR_DEVICE_TIMEOUT = 10    /* a kernel's bounded wait ran out (see pconv_device_status) */
+  PCONV_ERR_DEVICE_TIMEOUT = 10,   /* a kernel's bounded wait ran out (see pconv_device_status) */
+  PCONV_ERR_WORKSPACE = 11         /* the shape needs more scratch than the entry point can offer */
 } pconv_status;
 
 enum { PCONV_F32 = 0, PCONV_F16 = 1 };
@@ -138,6 +139,33 @@ pconv_status pconv_workspace_bytes(const pconv_handle* h, int n, int h_in, int w
 pconv_status pconv_forward_ws(const pconv_handle* h, const void* x_dev, const float* bias_dev,
                               void* y_dev, int n, int h_in, int w_in, unsigned flags, void* ws_dev,
                               size_t ws_bytes, void* stream);
+
+/*
+ * pconv_forward_static_ws -- pconv_forward_ws for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this entry point exists for integration, not for the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is forbidden or unavailable -- inside another
+ * framework's memory plan that hands out no scratch, in a process whose allocator is owned by
+ * someone else, or on a latency path that must never reach the driver's allocator.  Such callers
+ * still own x, y and the bias, but have nowhere to put the channel-split workspace.  Here the
+ * workspace is a fixed array inside the library's device image, PCONV_STATIC_WS_BYTES long; every
+ * GPU that loads the library holds that much memory until the process exits.
+ *
+ *  - Same arguments and result as pconv_forward_ws without the workspace pair.
+ *  - A shape whose workspace (pconv_workspace_bytes) exceeds PCONV_STATIC_WS_BYTES is refused
+ *    with PCONV_ERR_WORKSPACE and nothing is launched; shapes that need no workspace always pass.
+ *  - The call allocates nothing: no cudaMalloc / cudaFree, no allocating library routine.  The
+ *    first call on each device looks up the array's device address (cudaGetSymbolAddress) and
+ *    caches it; make that first call before starting any stream capture.
+ *  - Every call uses the same array.  It is cleared on `stream` (cudaMemsetAsync over the part the
+ *    shape needs) before the kernel runs, so an earlier call's leftovers never leak in -- but two
+ *    calls that overlap on the GPU (different streams, or concurrent handles) race on it and give
+ *    wrong results.  Serialise them, or use pconv_forward_ws with separate buffers.
+ */
+#define PCONV_STATIC_WS_BYTES (8u << 20)
+pconv_status pconv_forward_static_ws(const pconv_handle* h, const void* x_dev,
+                                     const float* bias_dev, void* y_dev, int n, int h_in, int w_in,
+                                     unsigned flags, void* stream);
 
 /* Releases the handle and its device buffers.  NULL is allowed. */
 void pconv_free(pconv_handle* h);

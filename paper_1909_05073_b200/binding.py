@@ -21,9 +21,10 @@ MAX_PATTERNS = 16
 STATUS_NAMES = ["PCONV_OK", "PCONV_ERR_NULL", "PCONV_ERR_SHAPE", "PCONV_ERR_PATTERN_SET",
                 "PCONV_ERR_KERNEL_NOT_IN_SET", "PCONV_ERR_RANGE", "PCONV_ERR_UNSUPPORTED",
                 "PCONV_ERR_ALIGN", "PCONV_ERR_ALLOC", "PCONV_ERR_CUDA",
-                "PCONV_ERR_DEVICE_TIMEOUT"]
+                "PCONV_ERR_DEVICE_TIMEOUT", "PCONV_ERR_WORKSPACE"]
 
-EXPORTS = ["pconv_pack", "pconv_forward", "pconv_forward_ws", "pconv_workspace_bytes", "pconv_free", "pconv_maxpool2x2", "pconv_unpack",
+EXPORTS = ["pconv_pack", "pconv_forward", "pconv_forward_ws", "pconv_forward_static_ws", "pconv_workspace_bytes",
+           "pconv_free", "pconv_maxpool2x2", "pconv_unpack",
            "pconv_stats", "pconv_filter_order", "pconv_device_status", "pconv_status_str",
            "pconv_stack_create", "pconv_stack_out_shape", "pconv_stack_forward",
            "pconv_stack_forward_host", "pconv_stack_free"]
@@ -65,6 +66,7 @@ def lib():
         L.pconv_pack.argtypes = [vp, ci, ci, vp, ci, ci, ci, cu, vp, ctypes.POINTER(vp), ip, ip]
         L.pconv_forward.argtypes = [vp, vp, vp, vp, ci, ci, ci, cu, vp]
         L.pconv_forward_ws.argtypes = [vp, vp, vp, vp, ci, ci, ci, cu, vp, ctypes.c_size_t, vp]
+        L.pconv_forward_static_ws.argtypes = [vp, vp, vp, vp, ci, ci, ci, cu, vp]
         L.pconv_workspace_bytes.argtypes = [vp, ci, ci, ci, ctypes.POINTER(ctypes.c_size_t)]
         L.pconv_free.argtypes = [vp]
         L.pconv_free.restype = None
@@ -156,6 +158,23 @@ def pconv_forward(handle, x, bias, y, flags=0, stream=None, workspace=None):
                                  ctypes.c_void_p(y.data_ptr()), n, h, w, int(flags),
                                  _stream_ptr(stream))
     _check(st, "pconv_forward")
+
+
+STATIC_WS_BYTES = 8 << 20
+
+
+def pconv_forward_static_ws(handle, x, bias, y, flags=0, stream=None):
+    """pconv_forward_ws on the library's built-in scratch array: for callers that must not
+    allocate device memory.  Raises PconvError(PCONV_ERR_WORKSPACE) if the shape needs more than
+    STATIC_WS_BYTES.  Calls that overlap on the GPU race on the shared array."""
+    if not (x.is_cuda and y.is_cuda and x.is_contiguous() and y.is_contiguous()):
+        raise ValueError("x and y must be contiguous CUDA tensors")
+    n, _, h, w = x.shape
+    bp = ctypes.c_void_p(bias.data_ptr()) if bias is not None else None
+    st = lib().pconv_forward_static_ws(handle, ctypes.c_void_p(x.data_ptr()), bp,
+                                       ctypes.c_void_p(y.data_ptr()), n, h, w, int(flags),
+                                       _stream_ptr(stream))
+    _check(st, "pconv_forward_static_ws")
 
 
 def pconv_maxpool2x2(x, y, stream=None):

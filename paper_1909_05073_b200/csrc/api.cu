@@ -1,5 +1,6 @@
 // C ABI entry points: argument checks, kernel selection, layer stacks.
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "pconv_internal.h"
@@ -19,6 +20,7 @@ extern "C" const char* pconv_status_str(pconv_status s) {
     case PCONV_ERR_ALLOC: return "allocation failed";
     case PCONV_ERR_CUDA: return "CUDA error";
     case PCONV_ERR_DEVICE_TIMEOUT: return "a kernel abandoned a bounded wait";
+    case PCONV_ERR_WORKSPACE: return "shape needs more scratch memory than this entry point has";
   }
   return "unknown status";
 }
@@ -76,6 +78,57 @@ extern "C" pconv_status pconv_forward_ws(const pconv_handle* h, const void* x, c
   }
   if (e != cudaSuccess) return PCONV_ERR_CUDA;
   return PCONV_OK;
+}
+
+// ---- the entry point that allocates nothing --------------------------------------------------------
+// Scratch for callers that cannot call cudaMalloc: a fixed array in this library's device image.
+// In host code the name below is only a handle for the runtime, not a device address; the address
+// every kernel needs is fetched per device with cudaGetSymbolAddress and cached.
+static __device__ __align__(256) unsigned char g_static_ws[PCONV_STATIC_WS_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_ws_mutex;
+void* g_static_ws_ptr[kMaxDevices] = {nullptr};
+
+// Device address of g_static_ws on the current device (looked up once per device), or nullptr.
+void* static_ws_address() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    cudaGetLastError();
+    return nullptr;
+  }
+  std::lock_guard<std::mutex> lock(g_static_ws_mutex);
+  if (!g_static_ws_ptr[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_ws) != cudaSuccess) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    g_static_ws_ptr[dev] = p;
+  }
+  return g_static_ws_ptr[dev];
+}
+}  // namespace
+
+extern "C" pconv_status pconv_forward_static_ws(const pconv_handle* h, const void* x,
+                                                const float* bias, void* y, int n, int h_in,
+                                                int w_in, unsigned flags, void* stream_v) {
+  if (!h || !x || !y) return PCONV_ERR_NULL;
+  if (n < 0 || h_in <= 0 || w_in <= 0) return PCONV_ERR_SHAPE;
+  if (n == 0) return PCONV_OK;
+  const size_t need = tiled_workspace_bytes(h->d, n, h_in, w_in);
+  if (need > (size_t)PCONV_STATIC_WS_BYTES) return PCONV_ERR_WORKSPACE;
+  if (need == 0)  // this shape is never split: no scratch involved
+    return pconv_forward_ws(h, x, bias, y, n, h_in, w_in, flags, nullptr, 0, stream_v);
+  void* ws = static_ws_address();
+  if (!ws) return PCONV_ERR_CUDA;
+  // the array keeps whatever the last call left (normally zeros, but not after an aborted launch)
+  if (cudaMemsetAsync(ws, 0, need, (cudaStream_t)stream_v) != cudaSuccess) {
+    cudaGetLastError();
+    return PCONV_ERR_CUDA;
+  }
+  return pconv_forward_ws(h, x, bias, y, n, h_in, w_in, flags, ws, need, stream_v);
 }
 
 extern "C" pconv_status pconv_maxpool2x2(const void* x, void* y, int n, int c, int h, int w,
