@@ -15,13 +15,21 @@ Why PTX text, and why this shape (all measured on B200):
    the 4 taps, writes the columns back in two halves and refills each half's registers with the
    next kernel's columns at once, then jumps.
 
-Operands of the asm statement (all u32): %0 code pointer, %1 weight pointer, %2 window pointer (one
-channel before the chunk), %3 channel stride, %4 row pitch, %5 offset of the middle window column
-(bytes, shared-memory addresses), %6 TMEM address of the warp's slot 0.
+Shared-memory loads, TMEM loads and TMEM stores all pass through one memory-instruction queue
+that retires roughly one instruction per 7-9 cycles per scheduler, whatever its width; with 16
+packed FMAs (32 pipe cycles) per kernel that queue is the next limit, so the loop is written to
+issue as few such instructions as it can: one 16-byte load for a kernel's four weights (pairs
+{w,w} are formed by register moves), one 16-byte load per record of up to 15 byte codes (shifted
+out of four registers), one TMEM load and one TMEM store of 8 columns, and nine 16-byte loads per
+channel window (the staged tile is stored column-major so that two rows come with one load).
 
-Byte codes (specialised stream): low nibble 0..7 = kernel with that canonical pattern, high nibble
-= filter slot; low nibble 8 = advance (high nibble + 1) channels and reload the register window;
-9 = end of the (group, chunk) block.
+Operands of the asm statement (all u32): %0 code pointer, %1 weight pointer, %2 window pointer (one
+channel before the chunk), %3 channel stride, %4 column stride of the staged tile, %5 offset of the
+middle window column (bytes, shared-memory addresses), %6 TMEM address of the warp's slot 0.
+
+Byte codes (specialised stream, 16-byte records): low nibble 0..7 = kernel with that canonical
+pattern, high nibble = filter slot; low nibble 8 = advance (high nibble) channels, reload the
+register window and fetch the next record; 9 = end of the (group, chunk) block.
 """
 import os
 import sys
@@ -39,114 +47,104 @@ def gen(stride):
     emit = out.append
     emit("{")
     emit(".reg .b32 a<8>;")
+    emit(".reg .b32 s<8>;")
     emit(".reg .b64 acc<4>;")
     emit(".reg .b64 win<%d>;" % (rows * 3))
     emit(".reg .b64 w0, w1, w2, w3;")
-    emit(".reg .u32 code, nxt, idx, cp, wp, xp, ra, ta, tn, tq;")
+    emit(".reg .b32 r0, r1, r2, r3;")          # raw weights of the next kernel
+    emit(".reg .b32 c0, c1, c2, c3;")          # the current record of byte codes
+    emit(".reg .u32 code, idx, cp, wp, xp, ra, ta, tn, tq;")
     emit("TS: .branchtargets " + ", ".join(["P%d" % p for p in range(8)] + ["ADV", "END"]) + ";")
     emit("mov.u32 cp, %0;")
     emit("mov.u32 wp, %1;")
     emit("mov.u32 xp, %2;")
     emit("mov.u32 tq, %6;")
-    emit("ld.shared.v2.b64 {w0, w1}, [wp];")
-    emit("ld.shared.v2.b64 {w2, w3}, [wp+16];")
-    emit("add.u32 wp, wp, 32;")
-    emit("ld.shared.u8 nxt, [cp];")
-    emit("add.u32 cp, cp, 1;")
+    emit("ld.shared.v4.b32 {r0, r1, r2, r3}, [wp];")
+    emit("add.u32 wp, wp, 16;")
+    emit("ld.shared.v4.b32 {c0, c1, c2, c3}, [cp];")
+    emit("add.u32 cp, cp, 16;")
     emit("tcgen05.wait::st.sync.aligned;")
 
-    LO = "{a0, a1, a2, a3}"
-    HI = "{a4, a5, a6, a7}"
+    A8 = "{a0, a1, a2, a3, a4, a5, a6, a7}"
+    S8 = "{s0, s1, s2, s3, s4, s5, s6, s7}"
 
     def prep():
-        """Decode the next code as early as possible: its jump index (so that the jump-table
-        lookup is scheduled above the FMAs) and the TMEM address of its filter slot."""
-        emit("mov.u32 code, nxt;")
-        emit("ld.shared.u8 nxt, [cp];")
-        emit("add.u32 cp, cp, 1;")
+        """Shift the next byte code out of the record registers; decode its jump index and the
+        TMEM address of its filter slot."""
+        emit("and.b32 code, c0, 255;")
+        emit("shf.r.wrap.b32 c0, c0, c1, 8;")
+        emit("shf.r.wrap.b32 c1, c1, c2, 8;")
+        emit("shf.r.wrap.b32 c2, c2, c3, 8;")
+        emit("shr.u32 c3, c3, 8;")
         emit("and.b32 idx, code, 15;")
         emit("shr.u32 tn, code, 4;")
         emit("shl.b32 tn, tn, 3;")
         emit("add.u32 tn, tn, tq;")
 
-    def load_lo():
-        emit("tcgen05.ld.sync.aligned.32x32b.x4.b32 %s, [tn];" % LO)
-
-    def load_hi():
-        emit("tcgen05.ld.sync.aligned.32x32b.x4.b32 %s, [tn+4];" % HI)
-
     def jump():
         emit("mov.u32 ta, tn;")
         emit("brx.idx.uni idx, TS;")
 
-    # prologue: first code of the chunk
+    # prologue: the first record holds only the terminator leading to the first channel
     prep()
-    load_lo()
-    load_hi()
+    emit("tcgen05.ld.sync.aligned.32x32b.x8.b32 %s, [tn];" % A8)
     jump()
 
-    # Kernel bodies.  The slot's 8 accumulator columns arrive as two halves (rows 0-1, rows 2-3 of
-    # the lane's pixel column); each half is written back as soon as its last FMA has issued and
-    # its registers are immediately refilled with the next kernel's half, so TMEM latency hides
-    # behind the remaining FMAs and the jump.  Inside a channel every kernel has a different slot,
-    # so such a load never follows a store to the same columns; stores are drained where the
-    # channel changes (ADV) and at the end.
+    # Kernel bodies.  On entry: the slot's 8 accumulator columns were requested by the previous
+    # body (`a`), the kernel's raw weights are in r0..r3.  The body forms the {w,w} pairs, requests
+    # the next kernel's weights, runs the 16 FMAs, stores the columns and only then requests the
+    # next slot's columns (inside a channel every kernel has a different slot, so that load never
+    # follows a store to the same columns; stores are drained where the channel changes).
     for p, mask in enumerate(CANON_MASKS):
         tp = taps(mask)
-
-        def fma(s, ks):
-            u, v = divmod(tp[s], 3)
-            for k in ks:
-                emit("fma.rn.f32x2 acc%d, win%d, w%d, acc%d;" % (k, (stride * k + u) * 3 + v, s, k))
-
         emit("P%d:" % p)
+        emit("mov.b64 w0, {r0, r0};")
+        emit("mov.b64 w1, {r1, r1};")
+        emit("mov.b64 w2, {r2, r2};")
+        emit("mov.b64 w3, {r3, r3};")
+        emit("ld.shared.v4.b32 {r0, r1, r2, r3}, [wp];")
+        emit("add.u32 wp, wp, 16;")
+        prep()
         emit("tcgen05.wait::ld.sync.aligned;")
         for k in range(4):
             emit("mov.b64 acc%d, {a%d, a%d};" % (k, 2 * k, 2 * k + 1))
-        prep()
-        fma(0, range(4))
-        fma(1, range(4))
-        emit("ld.shared.v2.b64 {w0, w1}, [wp];")
-        fma(2, (0, 1))
-        fma(3, (0, 1))
-        emit("mov.b64 {a0, a1}, acc0;")
-        emit("mov.b64 {a2, a3}, acc1;")
-        emit("tcgen05.st.sync.aligned.32x32b.x4.b32 [ta], %s;" % LO)
-        load_lo()
-        fma(2, (2, 3))
-        fma(3, (2, 3))
-        emit("ld.shared.v2.b64 {w2, w3}, [wp+16];")
-        emit("add.u32 wp, wp, 32;")
-        emit("mov.b64 {a4, a5}, acc2;")
-        emit("mov.b64 {a6, a7}, acc3;")
-        emit("tcgen05.st.sync.aligned.32x32b.x4.b32 [ta+4], %s;" % HI)
-        load_hi()
+        for s_, t in enumerate(tp):
+            u, v = divmod(t, 3)
+            for k in range(4):
+                emit("fma.rn.f32x2 acc%d, win%d, w%d, acc%d;" % (k, (stride * k + u) * 3 + v, s_, k))
+        for k in range(4):
+            emit("mov.b64 {s%d, s%d}, acc%d;" % (2 * k, 2 * k + 1, k))
+        emit("tcgen05.st.sync.aligned.32x32b.x8.b32 [ta], %s;" % S8)
+        emit("tcgen05.ld.sync.aligned.32x32b.x8.b32 %s, [tn];" % A8)
         jump()
+
+    # Advance: `code` >> 4 channels further, reload the window (column-major tile: two rows per
+    # 16-byte load) and fetch the next record of codes.
     emit("ADV:")
-    emit("tcgen05.wait::ld.sync.aligned;")  # the speculative loads issued before this jump
+    emit("tcgen05.wait::ld.sync.aligned;")  # the speculative load issued before this jump
     emit("tcgen05.wait::st.sync.aligned;")  # a slot may come back in the next channel
     emit("shr.u32 ra, code, 4;")
-    emit("add.u32 ra, ra, 1;")
     emit("mad.lo.u32 xp, ra, %3, xp;")
-    prep()
-    load_lo()
-    load_hi()
-    emit("mov.u32 ra, xp;")
-    for r in range(rows):
-        emit("ld.shared.b64 win%d, [ra];" % (r * 3))
+    emit("ld.shared.v4.b32 {c0, c1, c2, c3}, [cp];")
+    emit("add.u32 cp, cp, 16;")
+    cols = [("xp", 0), ("xp", 1), ("xp", 2)]
+    for v in range(3):
         if stride == 1:
-            emit("ld.shared.b64 win%d, [ra+8];" % (r * 3 + 1))
-            emit("ld.shared.b64 win%d, [ra+16];" % (r * 3 + 2))
+            emit("mad.lo.u32 ra, %%4, %d, xp;" % v) if v else emit("mov.u32 ra, xp;")
         else:
-            emit("ld.shared.b64 win%d, [ra+8];" % (r * 3 + 2))
-        if r != rows - 1:
-            emit("add.u32 ra, ra, %4;")
-    if stride == 2:  # the middle column sits in the even-column plane, at a run-time offset
-        emit("add.u32 ra, xp, %5;")
-        for r in range(rows):
-            emit("ld.shared.b64 win%d, [ra];" % (r * 3 + 1))
-            if r != rows - 1:
-                emit("add.u32 ra, ra, %4;")
+            # staged columns: odd plane first; the middle (even) column sits at a run-time offset
+            if v == 0:
+                emit("mov.u32 ra, xp;")
+            elif v == 1:
+                emit("add.u32 ra, xp, %5;")
+            else:
+                emit("add.u32 ra, xp, %4;")
+        for r in range(0, rows - 1, 2):
+            emit("ld.shared.v2.b64 {win%d, win%d}, [ra+%d];" % (r * 3 + v, (r + 1) * 3 + v, r * 8))
+        if rows % 2:
+            emit("ld.shared.b64 win%d, [ra+%d];" % ((rows - 1) * 3 + v, (rows - 1) * 8))
+    prep()
+    emit("tcgen05.ld.sync.aligned.32x32b.x8.b32 %s, [tn];" % A8)
     jump()
     emit("END:")
     emit("tcgen05.wait::ld.sync.aligned;")

@@ -45,7 +45,7 @@ __host__ __device__ constexpr int cta_threads(bool generic) {
 }
 constexpr int kTmemCols = 512;  // whole TMEM of the SM: 16 warps x 16 slots x 8 columns
 constexpr int kMaxStages = 4;
-constexpr int kWSlot = kMaxBlockKernels * 32;  // bytes per (group, stage): {w0,w0,w1,w1,w2,w2,w3,w3}
+constexpr int kWSlot = kMaxBlockKernels * 16 + 16;  // bytes per (group, stage): 4 fp32 per kernel
 constexpr int kCodeSlot = 288;                 // bytes per (group, stage)
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr int kSmemLimit = 227 * 1024;
@@ -60,7 +60,9 @@ struct Geo {
   int tw, sw, tx, ty, q_total;
   int wys, wy, ng;       // warp grid: warp -> (warp % wys, warp / wys); rows >= wy are idle
   int pairs;             // sub-tile pairs per CTA = wy * sw
-  int rows, pitch, substride, chan_stride;  // float2 units
+  int rows, pitch;       // staged rows and columns of one sub-tile
+  int colstride;         // bytes between staged columns (rows are contiguous float2)
+  int substride, chan_stride;  // bytes per (sub-tile pair, channel) and per channel
   int stages, x_stage_bytes, stage_bytes, tab_off, desc_off, stage_off;
   int ks, cps;           // channel splits (grid.z) and chunks per split
   int relu, is_half;
@@ -76,6 +78,11 @@ __device__ __forceinline__ void ffma2(u64& d, u64 a, u64 b) {
 __device__ __forceinline__ u64 lds64(uint32_t addr) {
   u64 v;
   asm volatile("ld.shared.b64 %0, [%1];" : "=l"(v) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr));
   return v;
 }
 __device__ __forceinline__ uint32_t lds_u16(uint32_t addr) {
@@ -138,19 +145,19 @@ struct Win {
 // accumulators stay in TMEM at `tq` (+ 8 columns per filter slot).
 template <int S>
 __device__ __forceinline__ void dispatch_chunk(uint32_t cp, uint32_t wp, uint32_t xptr,
-                                               uint32_t chan_b, uint32_t pitch_b, uint32_t off_mid,
+                                               uint32_t chan_b, uint32_t col_b, uint32_t off_mid,
                                                uint32_t tq) {
   if (S == 1) {
     asm volatile(
 #include "dispatch_s1.inc"
         :
-        : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(pitch_b), "r"(off_mid), "r"(tq)
+        : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(col_b), "r"(off_mid), "r"(tq)
         : "memory");
   } else {
     asm volatile(
 #include "dispatch_s2.inc"
         :
-        : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(pitch_b), "r"(off_mid), "r"(tq)
+        : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(col_b), "r"(off_mid), "r"(tq)
         : "memory");
   }
 }
@@ -176,8 +183,9 @@ __device__ __forceinline__ void kernel_body_generic(u64 (&acc)[kGroup][4],
 #pragma unroll
   for (int t = 0; t < 9; ++t) {
     if (mask >> t & 1) {
-      const u64 wv = lds64(wp);
-      wp += 8;
+      const uint32_t w1 = lds32(wp);
+      const u64 wv = ((u64)w1 << 32) | w1;
+      wp += 4;
 #pragma unroll
       for (int k = 0; k < 4; ++k) ffma2(acc[G][k], win[S * k + t / 3][t % 3], wv);
     }
@@ -186,13 +194,12 @@ __device__ __forceinline__ void kernel_body_generic(u64 (&acc)[kGroup][4],
 
 template <int S>
 __device__ __forceinline__ void load_window(u64 (&win)[Win<S>::kRows][3], uint32_t xptr,
-                                            uint32_t pitch_b, uint32_t off_mid, uint32_t off_right) {
+                                            uint32_t off_mid, uint32_t off_right) {
 #pragma unroll
   for (int r = 0; r < Win<S>::kRows; ++r) {
-    const uint32_t a = xptr + r * pitch_b;
-    win[r][0] = lds64(a);
-    win[r][1] = lds64(a + off_mid);
-    win[r][2] = lds64(a + off_right);
+    win[r][0] = lds64(xptr + r * 8);
+    win[r][1] = lds64(xptr + off_mid + r * 8);
+    win[r][2] = lds64(xptr + off_right + r * 8);
   }
 }
 
@@ -225,7 +232,7 @@ __device__ __forceinline__ void produce_chunk_async(const DeviceLayer& L, const 
   const int nc = min(kChunk, L.c_in - c0);
   const size_t hw = (size_t)g.h * g.w;
   const int n_rows = g.pairs * g.rows;
-  const uint32_t chan_b = (uint32_t)g.chan_stride * 8u;
+  const uint32_t chan_b = (uint32_t)g.chan_stride;
   for (int row = pw; row < n_rows; row += kProducerWarps) {
     const int p = row / g.rows, r = row - p * g.rows;
     const SubTile A = tab[2 * p], B = tab[2 * p + 1];
@@ -234,7 +241,7 @@ __device__ __forceinline__ void produce_chunk_async(const DeviceLayer& L, const 
     const bool vB = B.valid && iyB >= 0 && iyB < g.h;
     const float* pa = x + ((size_t)A.n * L.c_in + c0) * hw + (size_t)(vA ? iyA : 0) * g.w;
     const float* pb = x + ((size_t)B.n * L.c_in + c0) * hw + (size_t)(vB ? iyB : 0) * g.w;
-    const uint32_t dst_row = stage_base + (uint32_t)((p * g.substride + r * g.pitch) * 8);
+    const uint32_t dst_row = stage_base + (uint32_t)(p * g.substride + r * 8);
     for (int i = lane; i < g.pitch; i += 32) {
       const int dx = staged_dx<S>(i, g.tw);
       const int ixA = A.x0 * S + dx, ixB = B.x0 * S + dx;
@@ -244,7 +251,7 @@ __device__ __forceinline__ void produce_chunk_async(const DeviceLayer& L, const 
       const float* sb = okB ? pb + ixB : x;
       const size_t step_a = okA ? hw : 0, step_b = okB ? hw : 0;
       const uint32_t na = okA ? 4u : 0u, nb = okB ? 4u : 0u;
-      uint32_t dst = dst_row + (uint32_t)i * 8;
+      uint32_t dst = dst_row + (uint32_t)(i * g.colstride);
       for (int cc = 0; cc < nc; ++cc) {
         cp_async4(dst, sa, na);
         cp_async4(dst + 4, sb, nb);
@@ -259,15 +266,9 @@ __device__ __forceinline__ void produce_chunk_async(const DeviceLayer& L, const 
   const uint32_t cbase = wbase + g.ng * kWSlot;
   for (int j = 0; j < g.ng; ++j) {
     const uint4 d = desc[j * L.n_chunks + k];  // {w_off, n_k, code_off, code_len}
-    if ((uint32_t)ptid < d.y) {
-      const float* src = reinterpret_cast<const float*>(L.wvals) + (size_t)(d.x + ptid) * 4;
-      const uint32_t wd = wbase + j * kWSlot + ptid * 32;
-#pragma unroll
-      for (int t = 0; t < 4; ++t) {
-        cp_async4(wd + 8 * t, src + t, 4);
-        cp_async4(wd + 8 * t + 4, src + t, 4);
-      }
-    }
+    if ((uint32_t)ptid < d.y)
+      cp_async16(wbase + j * kWSlot + ptid * 16,
+                 reinterpret_cast<const float*>(L.wvals) + (size_t)(d.x + ptid) * 4);
     if ((uint32_t)ptid * 16 < d.w) cp_async16(cbase + j * kCodeSlot + ptid * 16, codes + d.z + ptid * 16);
   }
 }
@@ -291,7 +292,7 @@ __device__ __forceinline__ void produce_chunk_half(const DeviceLayer& L, const G
     const bool vB = B.valid && iyB >= 0 && iyB < g.h;
     const __half* pa = x + ((size_t)A.n * L.c_in + c0) * hw + (size_t)(vA ? iyA : 0) * g.w;
     const __half* pb = x + ((size_t)B.n * L.c_in + c0) * hw + (size_t)(vB ? iyB : 0) * g.w;
-    const uint32_t dst_row = stage_base + (uint32_t)((p * g.substride + r * g.pitch) * 8);
+    const uint32_t dst_row = stage_base + (uint32_t)(p * g.substride + r * 8);
     for (int i = lane; i < g.pitch; i += 32) {
       const int dx = staged_dx<S>(i, g.tw);
       const int ixA = A.x0 * S + dx, ixB = B.x0 * S + dx;
@@ -303,9 +304,9 @@ __device__ __forceinline__ void produce_chunk_half(const DeviceLayer& L, const G
         va[cc] = (okA && cc < nc) ? ldg_f(pa + cc * hw + ixA) : 0.f;
         vb[cc] = (okB && cc < nc) ? ldg_f(pb + cc * hw + ixB) : 0.f;
       }
-      const uint32_t dst = dst_row + (uint32_t)i * 8;
+      const uint32_t dst = dst_row + (uint32_t)(i * g.colstride);
 #pragma unroll
-      for (int cc = 0; cc < kChunk; ++cc) sts64f(dst + (uint32_t)(cc * g.chan_stride) * 8, va[cc], vb[cc]);
+      for (int cc = 0; cc < kChunk; ++cc) sts64f(dst + (uint32_t)(cc * g.chan_stride), va[cc], vb[cc]);
     }
   }
   const int ptid = pw * 32 + lane;
@@ -317,9 +318,8 @@ __device__ __forceinline__ void produce_chunk_half(const DeviceLayer& L, const G
       const uint2 raw = __ldg(reinterpret_cast<const uint2*>(L.wvals) + d.x + ptid);
       const __half2 lo = *reinterpret_cast<const __half2*>(&raw.x);
       const __half2 hi = *reinterpret_cast<const __half2*>(&raw.y);
-      const uint32_t wd = wbase + j * kWSlot + ptid * 32;
-      sts128f(wd, __low2float(lo), __low2float(lo), __high2float(lo), __high2float(lo));
-      sts128f(wd + 16, __low2float(hi), __low2float(hi), __high2float(hi), __high2float(hi));
+      sts128f(wbase + j * kWSlot + ptid * 16, __low2float(lo), __high2float(lo), __low2float(hi),
+              __high2float(hi));
     }
     if ((uint32_t)ptid * 16 < d.w) {
       const uint4 cv = __ldg(reinterpret_cast<const uint4*>(codes + d.z) + ptid);
@@ -518,11 +518,11 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   const bool active = (wyi < g.wy) && (gi < L.n_groups);
   const int slot = wyi * g.sw + lane / g.tw;  // sub-tile pair of this lane
   const int col = lane % g.tw;
-  const uint32_t pitch_b = g.pitch * 8;
-  const uint32_t off_mid = (S == 1) ? 8u : (uint32_t)(g.tw + 1) * 8u;
-  const uint32_t off_right = (S == 1) ? 16u : 8u;
-  const uint32_t chan_b = (uint32_t)g.chan_stride * 8u;
-  const uint32_t lane_off = (uint32_t)(slot * g.substride + col) * 8u;
+  const uint32_t col_b = (uint32_t)g.colstride;
+  const uint32_t off_mid = (S == 1) ? col_b : (uint32_t)(g.tw + 1) * col_b;  // window column 1
+  const uint32_t off_right = (S == 1) ? 2 * col_b : col_b;                   // window column 2
+  const uint32_t chan_b = (uint32_t)g.chan_stride;
+  const uint32_t lane_off = (uint32_t)(slot * g.substride) + (uint32_t)col * col_b;
   // TMEM: a warp reaches the 32 lanes of its quadrant (warp % 4); 4 warps share a quadrant and
   // take 128 columns each = 16 filter slots x (4 rows x {A,B}).
   const uint32_t tq = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)((warp >> 2) * (kGroup * 8));
@@ -578,7 +578,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
         uint32_t wp = stage_base + g.x_stage_bytes + wgi * kWSlot;
         uint32_t cp = stage_base + g.x_stage_bytes + g.ng * kWSlot + wgi * kCodeSlot;
         if constexpr (!GENERIC) {
-          dispatch_chunk<S>(cp, wp, xptr, chan_b, pitch_b, off_mid, tq);
+          dispatch_chunk<S>(cp, wp, xptr, chan_b, col_b, off_mid, tq);
         } else {
           u64 win[Win<S>::kRows][3];
 #pragma unroll
@@ -589,7 +589,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
             if (code & (uint32_t)kGenEnd) break;
             if (code & (uint32_t)kGenNext) {
               xptr += ((code & 0xFFu) + 1u) * chan_b;
-              load_window<S>(win, xptr, pitch_b, off_mid, off_right);
+              load_window<S>(win, xptr, off_mid, off_right);
               continue;
             }
             switch (code >> 9) {
@@ -667,15 +667,20 @@ bool make_geo(const DeviceLayer& L, int n, int h, int w, bool allow_split, Geo* 
   g.wy = g.wys;
   g.rows = (L.stride == 1) ? 6 : 9;
   g.pitch = (L.stride == 1) ? (g.tw + 2) : (2 * g.tw + 1);
-  g.substride = g.rows * g.pitch;
-  if (g.tw < 16)  // spread the sub-tiles of a half-warp over distinct banks
-    while (g.substride % 16 != g.tw % 16) ++g.substride;
+  // The staged tile is column-major: the rows of a column are contiguous float2, so a lane's
+  // window column comes in 16-byte loads.  48 B (80 B at stride 2) between columns keeps the 8
+  // lanes of a quarter-warp on distinct 16-byte bank groups; narrower sub-tiles are offset so that
+  // the sub-tiles sharing a quarter-warp do not collide.
+  g.colstride = (L.stride == 1) ? 48 : 80;
+  g.substride = g.pitch * g.colstride;
+  if (g.tw == 4) while (g.substride % 128 != 64) g.substride += 16;
+  if (g.tw == 2) while (g.substride % 128 != 32) g.substride += 16;
   g.tab_off = 8 * 2 * kMaxStages + 16;  // barriers, then the TMEM base address word
   if (L.n_chunks > 512) return false;  // descriptor table budget (c_in <= 4096)
   for (;;) {
     g.pairs = g.wy * g.sw;
     g.chan_stride = g.pairs * g.substride;
-    g.x_stage_bytes = kChunk * g.chan_stride * 8;
+    g.x_stage_bytes = kChunk * g.chan_stride;
     g.stage_bytes = (g.x_stage_bytes + g.ng * (kWSlot + kCodeSlot) + 15) & ~15;
     g.desc_off = (g.tab_off + 2 * g.pairs * (int)sizeof(SubTile) + 15) & ~15;
     g.stage_off = g.desc_off + g.ng * L.n_chunks * 16;

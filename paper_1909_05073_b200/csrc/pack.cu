@@ -241,18 +241,28 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
         while (codes_g.size() % 16) codes_g.push_back(0);
         bd.cs_off = (uint32_t)codes_s.size();
         bd.cg_off = (uint32_t)codes_g.size();
+        // Specialised stream: 16-byte records, each a run of kernel codes closed by a terminator
+        // (advance to another channel's window, or end); the kernel reads a record with one load.
+        std::vector<uint8_t> rec;
+        auto close_record = [&](uint8_t terminator) {
+          rec.push_back(terminator);
+          while (rec.size() < 16) rec.push_back((uint8_t)kCodeEnd);
+          codes_s.insert(codes_s.end(), rec.begin(), rec.end());
+          rec.clear();
+        };
         int pos = c0 - 1;  // channel whose window is loaded
         for (const Item& it : items) {
           if (it.c != pos) {
             const int adv = it.c - pos;  // 1..kChunk
-            codes_s.push_back((uint8_t)(((adv - 1) << 4) | kCodeNext));
+            close_record((uint8_t)((adv << 4) | kCodeNext));
             const uint16_t cg = (uint16_t)(kGenNext | (adv - 1));
             codes_g.push_back((uint8_t)(cg & 0xFF));
             codes_g.push_back((uint8_t)(cg >> 8));
             pos = it.c;
           }
+          if (rec.size() == 15) close_record((uint8_t)kCodeNext);  // same channel, next record
           const int canon = h->canon_id[it.r->pid];
-          codes_s.push_back((uint8_t)((it.slot << 4) | (canon < 0 ? 0 : canon)));
+          rec.push_back((uint8_t)((it.slot << 4) | (canon < 0 ? 0 : canon)));
           const uint16_t cg = (uint16_t)((it.slot << 9) | patterns[it.r->pid]);
           codes_g.push_back((uint8_t)(cg & 0xFF));
           codes_g.push_back((uint8_t)(cg >> 8));
@@ -261,7 +271,7 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
           else
             wv32.insert(wv32.end(), it.r->v, it.r->v + 4);
         }
-        codes_s.push_back((uint8_t)kCodeEnd);
+        close_record((uint8_t)kCodeEnd);
         codes_g.push_back((uint8_t)(kGenEnd & 0xFF));
         codes_g.push_back((uint8_t)(kGenEnd >> 8));
         bd.cs_len = (uint32_t)codes_s.size() - bd.cs_off;

@@ -13,11 +13,14 @@ constexpr int kGroup = 16;         // filters per group (accumulator slots of on
 constexpr int kChunk = 8;          // input channels per pipeline stage
 constexpr int kMaxBlockKernels = kGroup * kChunk;
 
-// Specialised code stream (one byte per entry) -- valid when the pattern set is a subset of the
-// eight masks the tiled kernel has straight-line bodies for.
+// Specialised code stream -- valid when the pattern set is a subset of the eight masks the tiled
+// kernel has straight-line bodies for.  A (group, chunk) block is a sequence of 16-byte records;
+// a record is a run of kernel codes closed by one terminator (unused bytes repeat the end code):
 //   low nibble 0..7   kernel: canonical pattern id; high nibble = filter slot
-//   low nibble 8      advance (high nibble + 1) channels inside the chunk and load that window
-//   9                 end of this (group, chunk) block
+//   low nibble 8      terminator: advance (high nibble, 0..8) channels inside the chunk, load that
+//                     channel's window and continue with the next record
+//   9                 terminator: end of the block
+// The first record of a block holds only the terminator that leads to its first channel.
 constexpr int kCodeNext = 8;
 constexpr int kCodeEnd = 9;
 // Generic code stream (two bytes per entry) -- any 4-of-9 mask.
