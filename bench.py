@@ -210,13 +210,14 @@ def run_ours(args):
             B.pconv_maxpool2x2(o, p)
             a = p
     conv_ms = [0.0] * len(conv_layers)
+    wss = [layer.workspace(xi.shape) for layer, (xi, _) in zip(conv_layers, acts)]
     for _ in range(args.steps):
         flush.zero_()
         pairs = []
-        for layer, (xi, oi), pool in zip(conv_layers, acts, pools):
+        for layer, (xi, oi), ws in zip(conv_layers, acts, wss):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            layer.forward(xi, relu=True, out=oi)
+            B.pconv_forward(layer.handle, xi, layer.bias, oi, B.RELU, workspace=ws)
             e1.record()
             pairs.append((e0, e1))
         torch.cuda.synchronize()
