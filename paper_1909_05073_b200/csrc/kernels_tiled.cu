@@ -136,6 +136,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* er
   return false;
 }
 
+#ifdef PCONV_TRACE
+#define PCONV_MARK(i)                                                         \
+  if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) { \
+    unsigned long long t_;                                                    \
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                    \
+    ((unsigned long long*)(L.err + 2))[i] = t_;                               \
+  }
+#else
+#define PCONV_MARK(i)
+#endif
+
 template <int S>
 struct Win {
   static constexpr int kRows = (S == 1) ? 6 : 9;
@@ -168,6 +179,12 @@ __device__ __forceinline__ void tmem_ld8(uint32_t (&r)[8], uint32_t taddr) {
                  "=r"(r[7])
                : "r"(taddr));
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_ld8_nowait(uint32_t (&r)[8], uint32_t taddr) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+                 "=r"(r[7])
+               : "r"(taddr));
 }
 __device__ __forceinline__ void tmem_st8_zero(uint32_t taddr) {
   const uint32_t z = 0;
@@ -401,10 +418,13 @@ __device__ __forceinline__ void write_outputs(const DeviceLayer& L, const Geo& g
     }
   } else {
 #pragma unroll 1
-    for (int a = 0; a < kGroup; ++a) {  // the slot is a run-time TMEM address: no unrolling needed
-      uint32_t v[8];
-      tmem_ld8(v, tq + a * 8);
-      emit(a, v);
+    for (int a0 = 0; a0 < kGroup; a0 += 4) {  // run-time TMEM addresses: four slots per round trip
+      uint32_t v[4][8];
+#pragma unroll
+      for (int b = 0; b < 4; ++b) tmem_ld8_nowait(v[b], tq + (a0 + b) * 8);
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+      for (int b = 0; b < 4; ++b) emit(a0 + b, v[b]);
     }
   }
 }
@@ -458,6 +478,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   SubTile* tab = reinterpret_cast<SubTile*>(smem + g.tab_off);
   volatile uint32_t* tmem_base_s = reinterpret_cast<volatile uint32_t*>(smem + 8 * 2 * kMaxStages);
 
+  PCONV_MARK(0)
   if (tid == 0) {
     for (int s = 0; s < g.stages; ++s) {
       mbar_init(sbase + 8 * s, 32 * kProducerWarps);
@@ -508,6 +529,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  PCONV_MARK(1)
   const uint32_t tmem_base = GENERIC ? 0u : *tmem_base_s;
   const int k0 = blockIdx.z * g.cps;                       // this CTA's chunk range
   const int nk = min(L.n_chunks, k0 + g.cps) - k0;
@@ -572,6 +594,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
       const int s = kk % g.stages;
       ok = mbar_wait(sbase + 8 * s, (kk / g.stages) & 1, L.err, 2);
       if (!ok) break;
+      if (kk == 0) { PCONV_MARK(2) }
       if (active) {
         const uint32_t stage_base = sbase + g.stage_off + s * g.stage_bytes;
         uint32_t xptr = stage_base + lane_off - chan_b;  // one channel before the chunk
@@ -603,17 +626,20 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
       if (lane == 0) mbar_arrive(sbase + 8 * (kMaxStages + s));
     }
 
+    PCONV_MARK(3)
     // ---- epilogue: final values straight to y, or partial sums into the workspace --------------
     if (active && ok)
       write_outputs<GENERIC>(L, g, lane_outputs(L, g, tab, slot, col), y, ws, acc, tq, my_o, my_b,
                              g.ks > 1 ? 1 : 0);
     if (g.ks > 1) __threadfence();
+    PCONV_MARK(4)
   }
 
   // ---- common exit: every warp arrives here, then the TMEM columns are handed back ---------------
   if constexpr (!GENERIC) {
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    PCONV_MARK(5)
     if (warp == 0)
       asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols)
                    : "memory");
@@ -632,6 +658,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
         __threadfence();
         finalize_outputs(L, g, lane_outputs(L, g, tab, slot, col), y, ws, my_o, my_b);
       }
+      PCONV_MARK(6)
     }
   }
 }
@@ -665,6 +692,10 @@ bool make_geo(const DeviceLayer& L, int n, int h, int w, bool allow_split, Geo* 
     g.wys /= 2;
   }
   g.wy = g.wys;
+  {  // warp rows beyond the batch's sub-tiles stay idle and are not staged
+    const long long need = (pairs_needed + g.sw - 1) / g.sw;
+    if (need < g.wy) g.wy = need < 1 ? 1 : (int)need;
+  }
   g.rows = (L.stride == 1) ? 6 : 9;
   g.pitch = (L.stride == 1) ? (g.tw + 2) : (2 * g.tw + 1);
   // The staged tile is column-major: the rows of a column are contiguous float2, so a lane's
