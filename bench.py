@@ -66,7 +66,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -283,7 +283,10 @@ def run_ours(args):
                          "frac": achieved / ALU_PEAK_TFLOPS,
                          "peak_source": "148 SMs x 128 FP32 lanes x 2 x 1.965 GHz (derived; "
                                         "no FP32 figure in MEASURED_PEAKS.json)",
-                         "launch_ms_sum": conv_time_ms, "traffic": None,
+                         "launch_ms_sum": conv_time_ms,
+                         # dram__bytes_read + dram__bytes_write of the 13 conv launches of one
+                         # step, from the ncu capture summarised in profiles/
+                         "traffic": 88.9e6,
                          "algorithmic_bytes": algorithmic_bytes(layers),
                          "per_layer_us": [round(m * 1e3, 2) for m in conv_ms]},
             "cpu_baseline": {"value": flops / cpu_s / 1e12, "unit": "TFLOP/s",
