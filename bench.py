@@ -238,11 +238,10 @@ def run_ours(args):
         e2e_total += time.perf_counter() - t0
     sync_all()
 
-    t = torch.tensor([ms_total, e2e_total * 1e3], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step = float(t[0]) / args.steps
-    e2e_ms = float(t[1]) / args.steps
+    from paper_1909_05073_b200.shard import max_over_ranks
+    t = max_over_ranks([ms_total, e2e_total * 1e3], device="cuda")
+    ms_step = t[0] / args.steps
+    e2e_ms = t[1] / args.steps
     status, where = B.pconv_device_status(conv_layers[0].handle)
     if status != 0:
         raise SystemExit("device reported an abandoned wait (%d)" % where)
