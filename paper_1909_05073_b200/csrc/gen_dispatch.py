@@ -1,5 +1,5 @@
 """Generates the PTX text of the tiled kernel's per-chunk dispatch loop (dispatch_s1.inc,
-dispatch_s2.inc), which kernels_tmem.cu includes inside one `asm volatile` statement.
+dispatch_s2.inc), which kernels_tiled.cu includes inside one `asm volatile` statement.
 
 Why PTX text, and why this shape (all measured on B200):
  * accumulator and window registers can only be named at compile time, so every distinct

@@ -29,7 +29,6 @@
 // layer's status word and the warp stops working but still reaches the common exit, where the
 // TMEM allocation is released.
 #include <cuda_fp16.h>
-#include <cstdlib>
 
 #include "pconv_internal.h"
 
@@ -237,6 +236,33 @@ __device__ __forceinline__ int staged_dx(int i, int tw) {
   return (i <= tw) ? (2 * i - 1) : (2 * (i - tw - 1));
 }
 
+// One staged element = one (sub-tile pair, row, column) position of the halo'd tile, holding the
+// A and the B pixel.  Elements are dealt to the 128 producer threads in flat order, so narrow
+// sub-tiles keep all lanes busy.
+struct StagedElem {
+  long long off_a, off_b;   // element offsets into x for channel c0 of the chunk, or -1
+  uint32_t dst;             // byte offset inside the channel's staged block
+};
+template <int S>
+__device__ __forceinline__ StagedElem staged_elem(const DeviceLayer& L, const Geo& g,
+                                                  const SubTile* tab, int e, int c0) {
+  constexpr int kRows = (S == 1) ? 6 : 9;
+  const int q = e / g.pitch, i = e - q * g.pitch;   // q = pair * rows + row
+  const int p = q / kRows, r = q - p * kRows;
+  const SubTile A = tab[2 * p], B = tab[2 * p + 1];
+  const int dx = staged_dx<S>(i, g.tw);
+  const int iyA = A.y0 * S - 1 + r, iyB = B.y0 * S - 1 + r;
+  const int ixA = A.x0 * S + dx, ixB = B.x0 * S + dx;
+  const long long hw = (long long)g.h * g.w;
+  StagedElem se;
+  se.off_a = (A.valid && iyA >= 0 && iyA < g.h && ixA >= 0 && ixA < g.w)
+                 ? ((long long)A.n * L.c_in + c0) * hw + (long long)iyA * g.w + ixA : -1;
+  se.off_b = (B.valid && iyB >= 0 && iyB < g.h && ixB >= 0 && ixB < g.w)
+                 ? ((long long)B.n * L.c_in + c0) * hw + (long long)iyB * g.w + ixB : -1;
+  se.dst = (uint32_t)(p * g.substride + i * g.colstride + r * 8);
+  return se;
+}
+
 // fp32 storage: everything is fetched with cp.async (zero-fill outside the image), so the producer
 // never waits for data and several chunks are in flight; each thread's arrival on the stage's full
 // barrier fires when its own copies have landed.
@@ -248,37 +274,24 @@ __device__ __forceinline__ void produce_chunk_async(const DeviceLayer& L, const 
   const int c0 = k * kChunk;
   const int nc = min(kChunk, L.c_in - c0);
   const size_t hw = (size_t)g.h * g.w;
-  const int n_rows = g.pairs * g.rows;
+  const int n_elem = g.pairs * g.rows * g.pitch;
   const uint32_t chan_b = (uint32_t)g.chan_stride;
-  for (int row = pw; row < n_rows; row += kProducerWarps) {
-    const int p = row / g.rows, r = row - p * g.rows;
-    const SubTile A = tab[2 * p], B = tab[2 * p + 1];
-    const int iyA = A.y0 * S - 1 + r, iyB = B.y0 * S - 1 + r;
-    const bool vA = A.valid && iyA >= 0 && iyA < g.h;
-    const bool vB = B.valid && iyB >= 0 && iyB < g.h;
-    const float* pa = x + ((size_t)A.n * L.c_in + c0) * hw + (size_t)(vA ? iyA : 0) * g.w;
-    const float* pb = x + ((size_t)B.n * L.c_in + c0) * hw + (size_t)(vB ? iyB : 0) * g.w;
-    const uint32_t dst_row = stage_base + (uint32_t)(p * g.substride + r * 8);
-    for (int i = lane; i < g.pitch; i += 32) {
-      const int dx = staged_dx<S>(i, g.tw);
-      const int ixA = A.x0 * S + dx, ixB = B.x0 * S + dx;
-      const bool okA = vA && ixA >= 0 && ixA < g.w;
-      const bool okB = vB && ixB >= 0 && ixB < g.w;
-      const float* sa = okA ? pa + ixA : x;
-      const float* sb = okB ? pb + ixB : x;
-      const size_t step_a = okA ? hw : 0, step_b = okB ? hw : 0;
-      const uint32_t na = okA ? 4u : 0u, nb = okB ? 4u : 0u;
-      uint32_t dst = dst_row + (uint32_t)(i * g.colstride);
-      for (int cc = 0; cc < nc; ++cc) {
-        cp_async4(dst, sa, na);
-        cp_async4(dst + 4, sb, nb);
-        sa += step_a;
-        sb += step_b;
-        dst += chan_b;
-      }
+  const int ptid = pw * 32 + lane;
+  for (int e = ptid; e < n_elem; e += 32 * kProducerWarps) {
+    const StagedElem se = staged_elem<S>(L, g, tab, e, c0);
+    const float* sa = se.off_a >= 0 ? x + se.off_a : x;
+    const float* sb = se.off_b >= 0 ? x + se.off_b : x;
+    const size_t step_a = se.off_a >= 0 ? hw : 0, step_b = se.off_b >= 0 ? hw : 0;
+    const uint32_t na = se.off_a >= 0 ? 4u : 0u, nb = se.off_b >= 0 ? 4u : 0u;
+    uint32_t dst = stage_base + se.dst;
+    for (int cc = 0; cc < nc; ++cc) {
+      cp_async4(dst, sa, na);
+      cp_async4(dst + 4, sb, nb);
+      sa += step_a;
+      sb += step_b;
+      dst += chan_b;
     }
   }
-  const int ptid = pw * 32 + lane;
   const uint32_t wbase = stage_base + g.x_stage_bytes;
   const uint32_t cbase = wbase + g.ng * kWSlot;
   for (int j = 0; j < g.ng; ++j) {
@@ -291,7 +304,8 @@ __device__ __forceinline__ void produce_chunk_async(const DeviceLayer& L, const 
 }
 
 // fp16 storage: loads, converts to fp32 and stores (the interleaved fp32 layout cannot be produced
-// by an asynchronous copy of 2-byte elements).
+// by an asynchronous copy of 2-byte elements).  Two staged elements (32 loads) are in flight per
+// thread at a time.
 template <int S>
 __device__ __forceinline__ void produce_chunk_half(const DeviceLayer& L, const Geo& g,
                                                    const __half* __restrict__ x, const SubTile* tab,
@@ -300,33 +314,30 @@ __device__ __forceinline__ void produce_chunk_half(const DeviceLayer& L, const G
   const int c0 = k * kChunk;
   const int nc = min(kChunk, L.c_in - c0);
   const size_t hw = (size_t)g.h * g.w;
-  const int n_rows = g.pairs * g.rows;
-  for (int row = pw; row < n_rows; row += kProducerWarps) {
-    const int p = row / g.rows, r = row - p * g.rows;
-    const SubTile A = tab[2 * p], B = tab[2 * p + 1];
-    const int iyA = A.y0 * S - 1 + r, iyB = B.y0 * S - 1 + r;
-    const bool vA = A.valid && iyA >= 0 && iyA < g.h;
-    const bool vB = B.valid && iyB >= 0 && iyB < g.h;
-    const __half* pa = x + ((size_t)A.n * L.c_in + c0) * hw + (size_t)(vA ? iyA : 0) * g.w;
-    const __half* pb = x + ((size_t)B.n * L.c_in + c0) * hw + (size_t)(vB ? iyB : 0) * g.w;
-    const uint32_t dst_row = stage_base + (uint32_t)(p * g.substride + r * 8);
-    for (int i = lane; i < g.pitch; i += 32) {
-      const int dx = staged_dx<S>(i, g.tw);
-      const int ixA = A.x0 * S + dx, ixB = B.x0 * S + dx;
-      const bool okA = vA && ixA >= 0 && ixA < g.w;
-      const bool okB = vB && ixB >= 0 && ixB < g.w;
-      float va[kChunk], vb[kChunk];
+  const int n_elem = g.pairs * g.rows * g.pitch;
+  const int ptid = pw * 32 + lane;
+  constexpr int kStep = 32 * kProducerWarps;
+  for (int e = ptid; e < n_elem; e += 2 * kStep) {
+    StagedElem se[2];
+    se[0] = staged_elem<S>(L, g, tab, e, c0);
+    const bool two = e + kStep < n_elem;
+    se[1] = two ? staged_elem<S>(L, g, tab, e + kStep, c0) : se[0];
+    float va[2][kChunk], vb[2][kChunk];
+#pragma unroll
+    for (int u = 0; u < 2; ++u)
 #pragma unroll
       for (int cc = 0; cc < kChunk; ++cc) {
-        va[cc] = (okA && cc < nc) ? ldg_f(pa + cc * hw + ixA) : 0.f;
-        vb[cc] = (okB && cc < nc) ? ldg_f(pb + cc * hw + ixB) : 0.f;
+        va[u][cc] = (se[u].off_a >= 0 && cc < nc) ? ldg_f(x + se[u].off_a + cc * hw) : 0.f;
+        vb[u][cc] = (se[u].off_b >= 0 && cc < nc) ? ldg_f(x + se[u].off_b + cc * hw) : 0.f;
       }
-      const uint32_t dst = dst_row + (uint32_t)(i * g.colstride);
 #pragma unroll
-      for (int cc = 0; cc < kChunk; ++cc) sts64f(dst + (uint32_t)(cc * g.chan_stride), va[cc], vb[cc]);
+    for (int u = 0; u < 2; ++u) {
+      if (u == 1 && !two) break;
+#pragma unroll
+      for (int cc = 0; cc < kChunk; ++cc)
+        sts64f(stage_base + se[u].dst + (uint32_t)(cc * g.chan_stride), va[u][cc], vb[u][cc]);
     }
   }
-  const int ptid = pw * 32 + lane;
   const uint32_t wbase = stage_base + g.x_stage_bytes;
   const uint32_t cbase = wbase + g.ng * kWSlot;
   for (int j = 0; j < g.ng; ++j) {
@@ -737,10 +748,6 @@ bool make_geo(const DeviceLayer& L, int n, int h, int w, bool allow_split, Geo* 
     long long ks = kNumSMs / ctas;
     if (ks > L.n_chunks) ks = L.n_chunks;
     if (ks > 1) g.ks = (int)ks;
-  }
-  if (allow_split && !GENERIC) {
-    const char* dbg = getenv("PCONV_DEBUG_KS");  // experiment hook
-    if (dbg) g.ks = atoi(dbg) < L.n_chunks ? (atoi(dbg) > 0 ? atoi(dbg) : 1) : L.n_chunks;
   }
   g.cps = (L.n_chunks + g.ks - 1) / g.ks;
   g.ks = (L.n_chunks + g.cps - 1) / g.cps;
