@@ -184,6 +184,28 @@ pconv_status pconv_maxpool2x2(const void* x_dev, void* y_dev, int n, int c, int 
  * (w_out: c_out*c_in*9 floats).  fp16 handles return the rounded values.  Synchronous. */
 pconv_status pconv_unpack(const pconv_handle* h, float* w_oihw_host_out);
 
+/* How the tiled kernel would run one forward (the paper has no counterpart: its tuning step picks
+ * tile sizes off line; here the library picks them per call from the shape). */
+typedef struct pconv_plan_t {
+  int generic_taps;      /* 1 = run-time masks (the pattern set is not the canonical eight, or asked) */
+  int warps_per_unit;    /* consumer warps that share one (pixels, filter group) and split each chunk's
+                            channels among themselves: 1, 2 or 4 */
+  int channel_splits;    /* CTAs that share one output tile through the workspace (1 = none) */
+  int groups_per_cta;    /* filter groups (of 16) per CTA */
+  int pixel_sets;        /* independent sets of 256 pixels per CTA */
+  int tile_width;        /* output columns of a sub-tile (2..32) */
+  int stages;            /* depth of the staging ring */
+  int smem_bytes;        /* dynamic shared memory the geometry needs */
+  long long ctas;        /* CTAs launched */
+} pconv_plan_t;
+
+/* Test / tuning aid: fills *plan with the geometry a tiled forward of this shape would use;
+ * with_workspace != 0 asks for the plan of pconv_forward_ws with a large enough workspace.
+ * flags: 0 or PCONV_KERNEL_GENERIC_TAPS.  Launches nothing.  PCONV_ERR_UNSUPPORTED if the tiled
+ * kernel cannot take the shape. */
+pconv_status pconv_plan(const pconv_handle* h, int n, int h_in, int w_in, unsigned flags,
+                        int with_workspace, pconv_plan_t* plan);
+
 /* Fills *out with the layer's structure counts. */
 pconv_status pconv_stats(const pconv_handle* h, pconv_stats_t* out);
 

@@ -23,7 +23,7 @@ STATUS_NAMES = ["PCONV_OK", "PCONV_ERR_NULL", "PCONV_ERR_SHAPE", "PCONV_ERR_PATT
                 "PCONV_ERR_ALIGN", "PCONV_ERR_ALLOC", "PCONV_ERR_CUDA",
                 "PCONV_ERR_DEVICE_TIMEOUT", "PCONV_ERR_WORKSPACE"]
 
-EXPORTS = ["pconv_pack", "pconv_forward", "pconv_forward_ws", "pconv_forward_static_ws", "pconv_workspace_bytes",
+EXPORTS = ["pconv_pack", "pconv_forward", "pconv_forward_ws", "pconv_forward_static_ws", "pconv_workspace_bytes", "pconv_plan",
            "pconv_free", "pconv_maxpool2x2", "pconv_unpack",
            "pconv_stats", "pconv_filter_order", "pconv_device_status", "pconv_status_str",
            "pconv_stack_create", "pconv_stack_out_shape", "pconv_stack_forward",
@@ -50,6 +50,13 @@ class Stats(ctypes.Structure):
                 ("packed_bytes", ctypes.c_longlong), ("canonical_patterns", ctypes.c_int)]
 
 
+class Plan(ctypes.Structure):
+    _fields_ = [("generic_taps", ctypes.c_int), ("warps_per_unit", ctypes.c_int),
+                ("channel_splits", ctypes.c_int), ("groups_per_cta", ctypes.c_int),
+                ("pixel_sets", ctypes.c_int), ("tile_width", ctypes.c_int), ("stages", ctypes.c_int),
+                ("smem_bytes", ctypes.c_int), ("ctas", ctypes.c_longlong)]
+
+
 _lib = None
 
 
@@ -68,6 +75,7 @@ def lib():
         L.pconv_forward_ws.argtypes = [vp, vp, vp, vp, ci, ci, ci, cu, vp, ctypes.c_size_t, vp]
         L.pconv_forward_static_ws.argtypes = [vp, vp, vp, vp, ci, ci, ci, cu, vp]
         L.pconv_workspace_bytes.argtypes = [vp, ci, ci, ci, ctypes.POINTER(ctypes.c_size_t)]
+        L.pconv_plan.argtypes = [vp, ci, ci, ci, cu, ci, ctypes.POINTER(Plan)]
         L.pconv_free.argtypes = [vp]
         L.pconv_free.restype = None
         L.pconv_maxpool2x2.argtypes = [vp, vp, ci, ci, ci, ci, ci, vp]
@@ -129,6 +137,14 @@ def pconv_pack(w_oihw, patterns, stride=1, storage=F32, flags=0, stream=None):
 
 def pconv_free(handle):
     lib().pconv_free(handle)
+
+
+def pconv_plan(handle, n, h, w, flags=0, with_workspace=False):
+    """The launch geometry of a tiled forward of this shape, as a dict."""
+    p = Plan()
+    _check(lib().pconv_plan(handle, n, h, w, int(flags), int(bool(with_workspace)), ctypes.byref(p)),
+           "pconv_plan")
+    return {k: int(getattr(p, k)) for k, _ in Plan._fields_}
 
 
 def pconv_workspace_bytes(handle, n, h, w):

@@ -33,6 +33,16 @@ extern "C" pconv_status pconv_workspace_bytes(const pconv_handle* h, int n, int 
   return PCONV_OK;
 }
 
+extern "C" pconv_status pconv_plan(const pconv_handle* h, int n, int h_in, int w_in, unsigned flags,
+                                   int with_workspace, pconv_plan_t* plan) {
+  if (!h || !plan) return PCONV_ERR_NULL;
+  if (n <= 0 || h_in <= 0 || w_in <= 0) return PCONV_ERR_SHAPE;
+  std::memset(plan, 0, sizeof(*plan));
+  if (!tiled_plan(h->d, n, h_in, w_in, (flags & PCONV_KERNEL_GENERIC_TAPS) != 0, with_workspace != 0, plan))
+    return PCONV_ERR_UNSUPPORTED;
+  return PCONV_OK;
+}
+
 extern "C" pconv_status pconv_forward(const pconv_handle* h, const void* x, const float* bias,
                                       void* y, int n, int h_in, int w_in, unsigned flags,
                                       void* stream_v) {

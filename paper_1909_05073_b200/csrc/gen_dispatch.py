@@ -23,13 +23,18 @@ issue as few such instructions as it can: one 16-byte load for a kernel's four w
 out of four registers), one TMEM load and one TMEM store of 8 columns, and nine 16-byte loads per
 channel window (the staged tile is stored column-major so that two rows come with one load).
 
-Operands of the asm statement (all u32): %0 code pointer, %1 weight pointer, %2 window pointer (one
-channel before the chunk), %3 channel stride, %4 column stride of the staged tile, %5 offset of the
-middle window column (bytes, shared-memory addresses), %6 TMEM address of the warp's slot 0.
+Operands of the asm statement (all u32): %0 code pointer (first record of the warp's channel
+range), %1 weight pointer (its first kernel), %2 window pointer (one channel before the chunk),
+%3 channel stride, %4 column stride of the staged tile, %5 offset of the middle window column
+(bytes, shared-memory addresses), %6 TMEM address of the warp's slot 0, %7 the entry code
+((first channel + 1) << 4: the advance that leads to the range's first channel), %8 window pointer
+of the first channel past the warp's range (all ones when the warp runs the block to its end).
 
 Byte codes (specialised stream, 16-byte records): low nibble 0..7 = kernel with that canonical
 pattern, high nibble = filter slot; low nibble 8 = advance (high nibble) channels, reload the
-register window and fetch the next record; 9 = end of the (group, chunk) block.
+register window and fetch the next record; 10 = the same, and the next channel lies in another
+quarter of the chunk (a warp that shares the chunk with others stops here when the quarter is not
+its own); 9 = end of the (group, chunk) block.
 """
 import os
 import sys
@@ -53,17 +58,19 @@ def gen(stride):
     emit(".reg .b64 w0, w1, w2, w3;")
     emit(".reg .b32 r0, r1, r2, r3;")          # raw weights of the next kernel
     emit(".reg .b32 c0, c1, c2, c3;")          # the current record of byte codes
-    emit(".reg .u32 code, idx, cp, wp, xp, ra, ta, tn, tq;")
-    emit("TS: .branchtargets " + ", ".join(["P%d" % p for p in range(8)] + ["ADV", "END"]) + ";")
+    emit(".reg .u32 code, idx, cp, wp, xp, ra, ta, tn, tq, xe;")
+    emit(".reg .pred pe;")
+    emit("TS: .branchtargets " + ", ".join(["P%d" % p for p in range(8)] + ["ADV", "END", "SUB"]) + ";")
     emit("mov.u32 cp, %0;")
     emit("mov.u32 wp, %1;")
     emit("mov.u32 xp, %2;")
     emit("mov.u32 tq, %6;")
+    emit("mov.u32 code, %7;")
+    emit("mov.u32 xe, %8;")
     emit("ld.shared.v4.b32 {r0, r1, r2, r3}, [wp];")
     emit("add.u32 wp, wp, 16;")
-    emit("ld.shared.v4.b32 {c0, c1, c2, c3}, [cp];")
-    emit("add.u32 cp, cp, 16;")
     emit("tcgen05.wait::st.sync.aligned;")
+    emit("bra.uni ADV;")                      # the entry code leads to the range's first channel
 
     A8 = "{a0, a1, a2, a3, a4, a5, a6, a7}"
     S8 = "{s0, s1, s2, s3, s4, s5, s6, s7}"
@@ -84,11 +91,6 @@ def gen(stride):
     def jump():
         emit("mov.u32 ta, tn;")
         emit("brx.idx.uni idx, TS;")
-
-    # prologue: the first record holds only the terminator leading to the first channel
-    prep()
-    emit("tcgen05.ld.sync.aligned.32x32b.x8.b32 %s, [tn];" % A8)
-    jump()
 
     # Kernel bodies.  On entry: the slot's 8 accumulator columns were requested by the previous
     # body (`a`), the kernel's raw weights are in r0..r3.  The body forms the {w,w} pairs, requests
@@ -120,6 +122,12 @@ def gen(stride):
 
     # Advance: `code` >> 4 channels further, reload the window (column-major tile: two rows per
     # 16-byte load) and fetch the next record of codes.
+    # Quarter boundary: stop if the next channel is past this warp's range, else advance.
+    emit("SUB:")
+    emit("shr.u32 ra, code, 4;")
+    emit("mad.lo.u32 ra, ra, %3, xp;")
+    emit("setp.ge.u32 pe, ra, xe;")
+    emit("@pe bra.uni END;")
     emit("ADV:")
     emit("tcgen05.wait::ld.sync.aligned;")  # the speculative load issued before this jump
     emit("tcgen05.wait::st.sync.aligned;")  # a slot may come back in the next channel

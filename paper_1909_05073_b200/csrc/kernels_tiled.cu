@@ -30,6 +30,11 @@
 // TMEM allocation is released.
 #include <cuda_fp16.h>
 
+#include <type_traits>
+#ifdef PCONV_TRACE
+#include <cstdlib>
+#endif
+
 #include "pconv_internal.h"
 
 namespace pconv {
@@ -57,7 +62,8 @@ struct SubTile {
 struct Geo {
   int n, h, w, h_out, w_out;
   int tw, sw, tx, ty, q_total;
-  int wys, wy, ng;       // warp grid: warp -> (warp % wys, warp / wys); rows >= wy are idle
+  int zs;                // consumer warps that share one (pixel set, filter group) and split its channels
+  int wys, wy, ng;       // warp grid: unit -> (unit % wys, unit / wys); rows >= wy are idle
   int pairs;             // sub-tile pairs per CTA = wy * sw
   int rows, pitch;       // staged rows and columns of one sub-tile
   int colstride;         // bytes between staged columns (rows are contiguous float2)
@@ -142,8 +148,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* er
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                    \
     ((unsigned long long*)(L.err + 2))[i] = t_;                               \
   }
+// latest time at which any CTA passed this point (slot i of the trace words)
+#define PCONV_MARK_MAX(i)                                                     \
+  if (threadIdx.x == 0) {                                                     \
+    unsigned long long t_;                                                    \
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                    \
+    atomicMax((unsigned long long*)(L.err + 2) + i, t_);                      \
+  }
 #else
 #define PCONV_MARK(i)
+#define PCONV_MARK_MAX(i)
 #endif
 
 template <int S>
@@ -156,18 +170,20 @@ struct Win {
 template <int S>
 __device__ __forceinline__ void dispatch_chunk(uint32_t cp, uint32_t wp, uint32_t xptr,
                                                uint32_t chan_b, uint32_t col_b, uint32_t off_mid,
-                                               uint32_t tq) {
+                                               uint32_t tq, uint32_t entry_code, uint32_t xend) {
   if (S == 1) {
     asm volatile(
 #include "dispatch_s1.inc"
         :
-        : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(col_b), "r"(off_mid), "r"(tq)
+        : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(col_b), "r"(off_mid), "r"(tq), "r"(entry_code),
+          "r"(xend)
         : "memory");
   } else {
     asm volatile(
 #include "dispatch_s2.inc"
         :
-        : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(col_b), "r"(off_mid), "r"(tq)
+        : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(col_b), "r"(off_mid), "r"(tq), "r"(entry_code),
+          "r"(xend)
         : "memory");
   }
 }
@@ -270,7 +286,7 @@ template <int S>
 __device__ __forceinline__ void produce_chunk_async(const DeviceLayer& L, const Geo& g,
                                                     const float* __restrict__ x, const SubTile* tab,
                                                     const uint4* desc, const uint8_t* codes,
-                                                    uint32_t stage_base, int k, int pw, int lane) {
+                                                    uint32_t stage_base, int k, int kk, int pw, int lane) {
   const int c0 = k * kChunk;
   const int nc = min(kChunk, L.c_in - c0);
   const size_t hw = (size_t)g.h * g.w;
@@ -295,7 +311,7 @@ __device__ __forceinline__ void produce_chunk_async(const DeviceLayer& L, const 
   const uint32_t wbase = stage_base + g.x_stage_bytes;
   const uint32_t cbase = wbase + g.ng * kWSlot;
   for (int j = 0; j < g.ng; ++j) {
-    const uint4 d = desc[j * L.n_chunks + k];  // {w_off, n_k, code_off, code_len}
+    const uint4 d = desc[2 * (j * g.cps + kk)];  // {w_off, n_k, code_off, code_len}
     if ((uint32_t)ptid < d.y)
       cp_async16(wbase + j * kWSlot + ptid * 16,
                  reinterpret_cast<const float*>(L.wvals) + (size_t)(d.x + ptid) * 4);
@@ -310,7 +326,7 @@ template <int S>
 __device__ __forceinline__ void produce_chunk_half(const DeviceLayer& L, const Geo& g,
                                                    const __half* __restrict__ x, const SubTile* tab,
                                                    const uint4* desc, const uint8_t* codes,
-                                                   uint32_t stage_base, int k, int pw, int lane) {
+                                                   uint32_t stage_base, int k, int kk, int pw, int lane) {
   const int c0 = k * kChunk;
   const int nc = min(kChunk, L.c_in - c0);
   const size_t hw = (size_t)g.h * g.w;
@@ -341,7 +357,7 @@ __device__ __forceinline__ void produce_chunk_half(const DeviceLayer& L, const G
   const uint32_t wbase = stage_base + g.x_stage_bytes;
   const uint32_t cbase = wbase + g.ng * kWSlot;
   for (int j = 0; j < g.ng; ++j) {
-    const uint4 d = desc[j * L.n_chunks + k];
+    const uint4 d = desc[2 * (j * g.cps + kk)];
     if ((uint32_t)ptid < d.y) {
       const uint2 raw = __ldg(reinterpret_cast<const uint2*>(L.wvals) + d.x + ptid);
       const __half2 lo = *reinterpret_cast<const __half2*>(&raw.x);
@@ -362,10 +378,12 @@ __device__ __forceinline__ void red_add_f32(float* p, float v) {
   asm volatile("red.global.add.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
 }
 
-// Where a lane's outputs go: element offsets (inside one filter's plane stack) of the 4 rows of its
-// A and B pixels, or -1 where the pixel lies outside the image or the batch.
+// Where a lane's outputs go: the element offsets (inside filter 0's plane of the A / B image) of
+// row 0 of its two pixels, and which of the 8 outputs lie inside the image and the batch
+// (bit 2k = A row k, bit 2k+1 = B row k).  Rows are w_out elements apart.
 struct LaneOut {
-  long long off[8];   // [2*k] = A row k, [2*k+1] = B row k
+  long long base_a, base_b;
+  uint32_t mask;
 };
 __device__ __forceinline__ LaneOut lane_outputs(const DeviceLayer& L, const Geo& g, const SubTile* tab,
                                                 int slot, int col) {
@@ -374,48 +392,90 @@ __device__ __forceinline__ LaneOut lane_outputs(const DeviceLayer& L, const Geo&
   const bool col_a = A.valid && ox_a < g.w_out, col_b = B.valid && ox_b < g.w_out;
   const long long plane = (long long)g.h_out * g.w_out;
   LaneOut r;
+  r.base_a = (long long)A.n * L.c_out * plane + (long long)A.y0 * g.w_out + ox_a;
+  r.base_b = (long long)B.n * L.c_out * plane + (long long)B.y0 * g.w_out + ox_b;
+  r.mask = 0;
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
-    const int ya = A.y0 + k, yb = B.y0 + k;
-    r.off[2 * k] = (col_a && ya < g.h_out) ? ((long long)A.n * L.c_out * plane + (long long)ya * g.w_out + ox_a) : -1;
-    r.off[2 * k + 1] = (col_b && yb < g.h_out) ? ((long long)B.n * L.c_out * plane + (long long)yb * g.w_out + ox_b) : -1;
+    if (col_a && A.y0 + k < g.h_out) r.mask |= 1u << (2 * k);
+    if (col_b && B.y0 + k < g.h_out) r.mask |= 2u << (2 * k);
   }
   return r;
 }
 
-__device__ __forceinline__ void store_out(const Geo& g, void* __restrict__ y, long long i, float v) {
-  if (g.relu) v = fmaxf(v, 0.f);
-  if (g.is_half)
+template <bool HALF, bool RELU>
+__device__ __forceinline__ void store_out(void* __restrict__ y, long long i, float v) {
+  if (RELU) v = fmaxf(v, 0.f);
+  if (HALF)
     ((__half*)y)[i] = __float2half_rn(v);
   else
     ((float*)y)[i] = v;
 }
 
-// Outputs of one consumer warp (16 filter slots x 4 rows x {A,B} per lane).  `my_o` / `my_b` hold,
-// in lane a < 16, the original filter index and the bias of slot a (loaded at kernel start).
-//   mode 0: y = act(accumulator + bias)               (no channel split)
-//   mode 1: workspace += accumulator                  (partial sum of a split)
-template <bool GENERIC>
-__device__ __forceinline__ void write_outputs(const DeviceLayer& L, const Geo& g, const LaneOut& lo,
-                                              void* __restrict__ y, float* __restrict__ ws,
-                                              const u64 (&acc)[GENERIC ? kGroup : 1][4], uint32_t tq,
-                                              int my_o, float my_b, int mode) {
-  const long long plane = (long long)g.h_out * g.w_out;
-  auto emit = [&](int a, const uint32_t (&v)[8]) {
-    const int o = __shfl_sync(0xffffffffu, my_o, a);
-    const float bv = __shfl_sync(0xffffffffu, my_b, a);
-    if (o < 0) return;
-    const long long base = (long long)o * plane;
+// Calls f with the storage type and the activation as compile-time flags.
+template <class F>
+__device__ __forceinline__ void with_flags(const Geo& g, F f) {
+  if (g.is_half) {
+    if (g.relu) f(std::true_type(), std::true_type()); else f(std::true_type(), std::false_type());
+  } else {
+    if (g.relu) f(std::false_type(), std::true_type()); else f(std::false_type(), std::false_type());
+  }
+}
+
+// The 8 outputs of one filter slot.  MODE 0: y = act(v + bias); MODE 1: workspace += v.
+template <int MODE, bool HALF, bool RELU>
+__device__ __forceinline__ void emit_slot(const Geo& g, const LaneOut& lo, void* __restrict__ y,
+                                          float* __restrict__ ws, long long fbase, float bv,
+                                          const uint32_t (&v)[8]) {
+  const long long ia = fbase + lo.base_a, ib = fbase + lo.base_b;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      if (lo.off[e] < 0) continue;
-      const float val = __uint_as_float(v[e]);
-      if (mode == 1)
-        red_add_f32(ws + base + lo.off[e], val);
-      else
-        store_out(g, y, base + lo.off[e], val + bv);
+  for (int k = 0; k < 4; ++k) {
+    const int row = k * g.w_out;
+    if (lo.mask >> (2 * k) & 1u) {
+      if (MODE == 1) red_add_f32(ws + ia + row, __uint_as_float(v[2 * k]));
+      else store_out<HALF, RELU>(y, ia + row, __uint_as_float(v[2 * k]) + bv);
     }
-  };
+    if (lo.mask >> (2 * k + 1) & 1u) {
+      if (MODE == 1) red_add_f32(ws + ib + row, __uint_as_float(v[2 * k + 1]));
+      else store_out<HALF, RELU>(y, ib + row, __uint_as_float(v[2 * k + 1]) + bv);
+    }
+  }
+}
+
+// Which accumulators a consumer warp writes out: filter slots [a0, a1) of the `zs` column sets
+// that start at TMEM address `t0` (128 columns apart), summed.  zs = 1: the warp's own 16 slots.
+struct OutRange {
+  uint32_t t0;
+  int zs, a0, a1;
+};
+
+// Four filter slots of a lane's accumulators, summed over the warps that split the channels.
+__device__ __forceinline__ void tmem_sum4(uint32_t (&v)[4][8], const OutRange& r, int a) {
+#pragma unroll
+  for (int b = 0; b < 4; ++b) tmem_ld8_nowait(v[b], r.t0 + (a + b) * 8);
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll 1
+  for (int j = 1; j < r.zs; ++j) {
+    uint32_t t[4][8];
+#pragma unroll
+    for (int b = 0; b < 4; ++b) tmem_ld8_nowait(t[b], r.t0 + j * (kGroup * 8) + (a + b) * 8);
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int b = 0; b < 4; ++b)
+#pragma unroll
+      for (int e = 0; e < 8; ++e)
+        v[b][e] = __float_as_uint(__uint_as_float(v[b][e]) + __uint_as_float(t[b][e]));
+  }
+}
+
+// Outputs of one consumer warp (filter slots x 4 rows x {A,B} per lane).  `my_o` / `my_b` hold, in
+// lane a < 16, the original filter index and the bias of slot a (loaded at kernel start).
+template <bool GENERIC, int MODE, bool HALF, bool RELU>
+__device__ __forceinline__ void write_outputs(const Geo& g, const LaneOut& lo, void* __restrict__ y,
+                                              float* __restrict__ ws,
+                                              const u64 (&acc)[GENERIC ? kGroup : 1][4],
+                                              const OutRange& r, int my_o, float my_b) {
+  const long long plane = (long long)g.h_out * g.w_out;
   if constexpr (GENERIC) {
 #pragma unroll
     for (int a = 0; a < kGroup; ++a) {
@@ -425,50 +485,67 @@ __device__ __forceinline__ void write_outputs(const DeviceLayer& L, const Geo& g
         v[2 * k] = (uint32_t)acc[a][k];
         v[2 * k + 1] = (uint32_t)(acc[a][k] >> 32);
       }
-      emit(a, v);
+      const int o = __shfl_sync(0xffffffffu, my_o, a);
+      const float bv = __shfl_sync(0xffffffffu, my_b, a);
+      if (o >= 0) emit_slot<MODE, HALF, RELU>(g, lo, y, ws, (long long)o * plane, bv, v);
     }
   } else {
 #pragma unroll 1
-    for (int a0 = 0; a0 < kGroup; a0 += 4) {  // run-time TMEM addresses: four slots per round trip
+    for (int a = r.a0; a < r.a1; a += 4) {  // run-time TMEM addresses: four slots per round trip
       uint32_t v[4][8];
+      tmem_sum4(v, r, a);
 #pragma unroll
-      for (int b = 0; b < 4; ++b) tmem_ld8_nowait(v[b], tq + (a0 + b) * 8);
-      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-      for (int b = 0; b < 4; ++b) emit(a0 + b, v[b]);
+      for (int b = 0; b < 4; ++b) {
+        const int o = __shfl_sync(0xffffffffu, my_o, a + b);
+        const float bv = __shfl_sync(0xffffffffu, my_b, a + b);
+        if (o >= 0) emit_slot<MODE, HALF, RELU>(g, lo, y, ws, (long long)o * plane, bv, v[b]);
+      }
     }
   }
 }
 
-// The last split of a tile: workspace -> y, leaving the workspace zeroed.  Four filter slots (32
-// independent loads per lane) are in flight at once.
-__device__ __forceinline__ void finalize_outputs(const DeviceLayer& L, const Geo& g, const LaneOut& lo,
-                                                 void* __restrict__ y, float* __restrict__ ws, int my_o,
-                                                 float my_b) {
+// The last split to finish a warp's part of an output tile: workspace -> y, leaving the workspace
+// zeroed.  Four filter slots (32 independent loads per lane) are in flight at once.
+template <bool HALF, bool RELU>
+__device__ __forceinline__ void finalize_outputs(const Geo& g, const LaneOut& lo, void* __restrict__ y,
+                                                 float* __restrict__ ws, int a_begin, int a_end,
+                                                 int my_o, float my_b) {
   const long long plane = (long long)g.h_out * g.w_out;
   constexpr int kBatch = 4;
 #pragma unroll 1
-  for (int a0 = 0; a0 < kGroup; a0 += kBatch) {
+  for (int a0 = a_begin; a0 < a_end; a0 += kBatch) {
     float v[kBatch][8];
-    long long base[kBatch];
+    long long fb[kBatch];
     float bv[kBatch];
 #pragma unroll
     for (int b = 0; b < kBatch; ++b) {
       const int o = __shfl_sync(0xffffffffu, my_o, a0 + b);
       bv[b] = __shfl_sync(0xffffffffu, my_b, a0 + b);
-      base[b] = (o < 0) ? -1 : (long long)o * plane;
+      fb[b] = (o < 0) ? -1 : (long long)o * plane;
+      const long long ia = fb[b] + lo.base_a, ib = fb[b] + lo.base_b;
+      const uint32_t m = (o < 0) ? 0u : lo.mask;
 #pragma unroll
-      for (int e = 0; e < 8; ++e)
-        v[b][e] = (base[b] >= 0 && lo.off[e] >= 0) ? __ldcg(ws + base[b] + lo.off[e]) : 0.f;
+      for (int k = 0; k < 4; ++k) {
+        const int row = k * g.w_out;
+        v[b][2 * k] = (m >> (2 * k) & 1u) ? __ldcg(ws + ia + row) : 0.f;
+        v[b][2 * k + 1] = (m >> (2 * k + 1) & 1u) ? __ldcg(ws + ib + row) : 0.f;
+      }
     }
 #pragma unroll
     for (int b = 0; b < kBatch; ++b) {
-      if (base[b] < 0) continue;
+      if (fb[b] < 0) continue;
+      const long long ia = fb[b] + lo.base_a, ib = fb[b] + lo.base_b;
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        if (lo.off[e] < 0) continue;
-        ws[base[b] + lo.off[e]] = 0.f;
-        store_out(g, y, base[b] + lo.off[e], v[b][e] + bv[b]);
+      for (int k = 0; k < 4; ++k) {
+        const int row = k * g.w_out;
+        if (lo.mask >> (2 * k) & 1u) {
+          ws[ia + row] = 0.f;
+          store_out<HALF, RELU>(y, ia + row, v[b][2 * k] + bv[b]);
+        }
+        if (lo.mask >> (2 * k + 1) & 1u) {
+          ws[ib + row] = 0.f;
+          store_out<HALF, RELU>(y, ib + row, v[b][2 * k + 1] + bv[b]);
+        }
       }
     }
   }
@@ -490,6 +567,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   volatile uint32_t* tmem_base_s = reinterpret_cast<volatile uint32_t*>(smem + 8 * 2 * kMaxStages);
 
   PCONV_MARK(0)
+  PCONV_MARK_MAX(8)
   if (tid == 0) {
     for (int s = 0; s < g.stages; ++s) {
       mbar_init(sbase + 8 * s, 32 * kProducerWarps);
@@ -517,36 +595,43 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
     t.x0 = (rem - tyi * g.tx) * g.tw;
     tab[i] = t;
   }
-  // block descriptors of the CTA's groups: {first record, records, code offset, code bytes}
+  const int k0 = blockIdx.z * g.cps;                       // this CTA's chunk range
+  const int nk = min(L.n_chunks, k0 + g.cps) - k0;
+  // Block descriptors of the CTA's groups and chunks, two 16-byte words each:
+  // {first kernel record, records, code offset, code bytes}, {-, -, quarter entries}.
   uint4* desc = reinterpret_cast<uint4*>(smem + g.desc_off);
-  for (int i = tid; i < g.ng * L.n_chunks; i += kThreads) {
-    const int j = i / L.n_chunks, k = i - j * L.n_chunks;
+  for (int i = tid; i < g.ng * g.cps; i += kThreads) {
+    const int j = i / g.cps, kk = i - j * g.cps;
     const int gj = blockIdx.y * g.ng + j;
-    uint4 d = make_uint4(0u, 0u, 0u, 0u);
-    if (gj < L.n_groups) {
-      const uint4* src = reinterpret_cast<const uint4*>(L.blocks + (size_t)gj * L.n_chunks + k);
+    uint4 d0 = make_uint4(0u, 0u, 0u, 0u), d1 = d0;
+    if (gj < L.n_groups && kk < nk) {
+      const uint4* src = reinterpret_cast<const uint4*>(L.blocks + (size_t)gj * L.n_chunks + k0 + kk);
       const uint4 b0 = __ldg(src), b1 = __ldg(src + 1);
-      d = GENERIC ? make_uint4(b0.x, b0.y, b1.x, b1.y) : make_uint4(b0.x, b0.y, b0.z, b0.w);
+      d0 = GENERIC ? make_uint4(b0.x, b0.y, b1.x, b1.y) : b0;
+      d1 = b1;
     }
-    desc[i] = d;
-  }
-  // groups past the layer's last one never get codes staged: park an end code in every stage
-  for (int i = tid; i < g.ng * g.stages; i += kThreads) {
-    const int j = i % g.ng, s = i / g.ng;
-    if ((int)(blockIdx.y * g.ng + j) >= L.n_groups)
-      sts32(sbase + g.stage_off + s * g.stage_bytes + g.x_stage_bytes + g.ng * kWSlot + j * kCodeSlot,
-            GENERIC ? 0x40004000u : 0x09090909u);
+    desc[2 * i] = d0;
+    desc[2 * i + 1] = d1;
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   PCONV_MARK(1)
   const uint32_t tmem_base = GENERIC ? 0u : *tmem_base_s;
-  const int k0 = blockIdx.z * g.cps;                       // this CTA's chunk range
-  const int nk = min(L.n_chunks, k0 + g.cps) - k0;
 
-  // consumer-warp coordinates (meaningless for producer warps)
-  const int wyi = warp % g.wys, wgi = warp / g.wys;
+  // Consumer-warp coordinates (meaningless for producer warps).  zs warps of one TMEM lane
+  // quadrant form a unit: they work on the same pixels and filter group, each on its own quarters
+  // of every chunk, with accumulators in its own 128 TMEM columns.
+  const int zs = GENERIC ? 1 : g.zs;
+  int unit = warp, z = 0;
+  if (zs == 2) {
+    unit = (warp & 3) + 4 * (warp >> 3);
+    z = (warp >> 2) & 1;
+  } else if (zs == 4) {
+    unit = warp & 3;
+    z = warp >> 2;
+  }
+  const int wyi = unit % g.wys, wgi = unit / g.wys;
   const int gi = blockIdx.y * g.ng + wgi;
   const bool active = (wyi < g.wy) && (gi < L.n_groups);
   const int slot = wyi * g.sw + lane / g.tw;  // sub-tile pair of this lane
@@ -558,7 +643,9 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   const uint32_t lane_off = (uint32_t)(slot * g.substride) + (uint32_t)col * col_b;
   // TMEM: a warp reaches the 32 lanes of its quadrant (warp % 4); 4 warps share a quadrant and
   // take 128 columns each = 16 filter slots x (4 rows x {A,B}).
-  const uint32_t tq = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)((warp >> 2) * (kGroup * 8));
+  const uint32_t tquad = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);
+  const uint32_t tq = tquad + (uint32_t)((warp >> 2) * (kGroup * 8));
+  const int q_per_warp = kQuarters / zs, q0 = z * q_per_warp;
 
   // lane a < 16 keeps the original filter index and bias of slot a for the epilogue
   int my_o = -1;
@@ -580,10 +667,10 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
       if (it > 0 && !mbar_wait(sbase + 8 * (kMaxStages + s), (it - 1) & 1, L.err, 1)) break;
       const uint32_t stage_base = sbase + g.stage_off + s * g.stage_bytes;
       if (g.is_half) {
-        produce_chunk_half<S>(L, g, (const __half*)x, tab, desc, codes, stage_base, k0 + kk, pw, lane);
+        produce_chunk_half<S>(L, g, (const __half*)x, tab, desc, codes, stage_base, k0 + kk, kk, pw, lane);
         mbar_arrive(sbase + 8 * s);
       } else {
-        produce_chunk_async<S>(L, g, (const float*)x, tab, desc, codes, stage_base, k0 + kk, pw, lane);
+        produce_chunk_async<S>(L, g, (const float*)x, tab, desc, codes, stage_base, k0 + kk, kk, pw, lane);
         cp_async_arrive(sbase + 8 * s);
       }
     }
@@ -612,7 +699,21 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
         uint32_t wp = stage_base + g.x_stage_bytes + wgi * kWSlot;
         uint32_t cp = stage_base + g.x_stage_bytes + g.ng * kWSlot + wgi * kCodeSlot;
         if constexpr (!GENERIC) {
-          dispatch_chunk<S>(cp, wp, xptr, chan_b, col_b, off_mid, tq);
+          // enter at the first of this warp's quarters that has a kernel; run to the range's end
+          const uint4 d1 = desc[2 * (wgi * g.cps + kk) + 1];
+          const u64 quarters = ((u64)d1.w << 32) | d1.z;
+          uint32_t ent = kQuarterEmpty;
+          for (int q = q0 + q_per_warp - 1; q >= q0; --q) {
+            const uint32_t e = (uint32_t)(quarters >> (16 * q)) & 0xFFFFu;
+            if (!(e & kQuarterEmpty)) ent = e;
+          }
+          if (!(ent & kQuarterEmpty)) {
+            const uint32_t xend = (q0 + q_per_warp == kQuarters)
+                                      ? 0xFFFFFFFFu
+                                      : xptr + (uint32_t)((q0 + q_per_warp) * kQuarterChannels + 1) * chan_b;
+            dispatch_chunk<S>(cp + (ent & 31u) * 16u, wp + ((ent >> 5) & 127u) * 16u, xptr, chan_b, col_b,
+                              off_mid, tq, (((ent >> 12) & 7u) + 1u) << 4, xend);
+          }
         } else {
           u64 win[Win<S>::kRows][3];
 #pragma unroll
@@ -638,49 +739,86 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
     }
 
     PCONV_MARK(3)
+    PCONV_MARK_MAX(9)
     // ---- epilogue: final values straight to y, or partial sums into the workspace --------------
-    if (active && ok)
-      write_outputs<GENERIC>(L, g, lane_outputs(L, g, tab, slot, col), y, ws, acc, tq, my_o, my_b,
-                             g.ks > 1 ? 1 : 0);
-    if (g.ks > 1) __threadfence();
-    PCONV_MARK(4)
+    OutRange orng;
+    orng.t0 = tq;
+    orng.zs = 1;
+    orng.a0 = 0;
+    orng.a1 = kGroup;
+    if constexpr (!GENERIC) {
+      if (zs > 1) {
+        // The warps of a unit hold partial sums over their own quarters in their own TMEM columns
+        // of the same lanes; once all have finished, each adds up and writes 16 / zs filter slots.
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(32 * kCW) : "memory");
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        orng.t0 = tquad + (uint32_t)(((warp >> 2) - z) * (kGroup * 8));
+        orng.zs = zs;
+        orng.a0 = z * (kGroup / zs);
+        orng.a1 = orng.a0 + kGroup / zs;
+      }
+    }
+    if (active && ok) {
+      const LaneOut lo = lane_outputs(L, g, tab, slot, col);
+      bool split = false;
+      if constexpr (!GENERIC) split = g.ks > 1;
+      if (!split) {
+        with_flags(g, [&](auto half, auto relu) {
+          write_outputs<GENERIC, 0, decltype(half)::value, decltype(relu)::value>(g, lo, y, ws, acc, orng,
+                                                                                   my_o, my_b);
+        });
+      } else {
+        write_outputs<GENERIC, 1, false, false>(g, lo, y, ws, acc, orng, my_o, my_b);
+        PCONV_MARK(4)
+        PCONV_MARK_MAX(10)
+        // Every warp owns the same part of the output tile in each of the ks splits, and takes a
+        // ticket for that part once its partial sums are visible.  The warp that draws the last
+        // ticket turns the summed partials into the layer's output and leaves workspace and
+        // ticket zeroed for the next launch; nobody waits for anybody, and the finishing work of a
+        // tile spreads over the CTAs that share it.
+        __threadfence();
+        __syncwarp();
+        int* ticket = counters + ((size_t)blockIdx.y * gridDim.x + blockIdx.x) * kCW + warp;
+        int t = 0;
+        if (lane == 0) {
+          t = atomicAdd(ticket, 1);
+          if (t == g.ks - 1) *ticket = 0;
+        }
+        t = __shfl_sync(0xffffffffu, t, 0);
+        if (t == g.ks - 1) {
+          __threadfence();
+          with_flags(g, [&](auto half, auto relu) {
+            finalize_outputs<decltype(half)::value, decltype(relu)::value>(g, lo, y, ws, orng.a0, orng.a1,
+                                                                          my_o, my_b);
+          });
+        }
+      }
+    }
+    PCONV_MARK(5)
   }
 
   // ---- common exit: every warp arrives here, then the TMEM columns are handed back ---------------
   if constexpr (!GENERIC) {
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    PCONV_MARK(5)
+    PCONV_MARK(6)
     if (warp == 0)
       asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols)
                    : "memory");
-    if (g.ks > 1) {
-      // The split that arrives last at this output tile's ticket turns the summed partials into
-      // the layer's output and leaves workspace and ticket zeroed for the next launch.
-      volatile uint32_t* last = tmem_base_s + 1;
-      if (tid == 0) {
-        int* ticket = counters + blockIdx.y * gridDim.x + blockIdx.x;
-        const int t = atomicAdd(ticket, 1);
-        *last = (t == g.ks - 1) ? 1u : 0u;
-        if (t == g.ks - 1) *ticket = 0;
-      }
-      __syncthreads();
-      if (*last && warp < kCW && active && ok) {
-        __threadfence();
-        finalize_outputs(L, g, lane_outputs(L, g, tab, slot, col), y, ws, my_o, my_b);
-      }
-      PCONV_MARK(6)
-    }
   }
+  PCONV_MARK_MAX(7)
 }
 
+// Geometry for `zs` consumer warps per unit and no channel split across CTAs.
 template <bool GENERIC>
-bool make_geo(const DeviceLayer& L, int n, int h, int w, bool allow_split, Geo* out) {
-  constexpr int kCW = consumer_warps(GENERIC);
+bool geo_for(const DeviceLayer& L, int n, int h, int w, int zs, Geo* out) {
+  const int units = consumer_warps(GENERIC) / zs;
   Geo g;
   g.n = n;
   g.h = h;
   g.w = w;
+  g.zs = zs;
   g.h_out = (h - 1) / L.stride + 1;
   g.w_out = (w - 1) / L.stride + 1;
   g.tw = 32;
@@ -691,12 +829,13 @@ bool make_geo(const DeviceLayer& L, int n, int h, int w, bool allow_split, Geo* 
   const long long q = (long long)n * g.tx * g.ty;
   if (q > 0x7FFFFFFF) return false;
   g.q_total = (int)q;
-  // Filter groups per CTA (ng) x pixel sets (wy) = consumer warps.  Wide ng shares the staged input
-  // among more filters; when the whole batch has few sub-tiles, pixel sets are traded for groups.
+  // Filter groups per CTA (ng) x pixel sets (wy) = units.  Wide ng shares the staged input among
+  // more filters; when the whole batch has few sub-tiles, pixel sets are traded for groups.
   int ng_max = 1;
-  while (ng_max < kCW && ng_max < L.n_groups) ng_max *= 2;
-  g.ng = ng_max < (GENERIC ? 4 : 8) ? ng_max : (GENERIC ? 4 : 8);
-  g.wys = kCW / g.ng;
+  while (ng_max < units && ng_max < L.n_groups) ng_max *= 2;
+  const int ng_pref = GENERIC ? 4 : 8;
+  g.ng = ng_max < ng_pref ? ng_max : ng_pref;
+  g.wys = units / g.ng;
   const long long pairs_needed = (q + 1) / 2;
   while (g.ng < ng_max && (long long)(g.wys / 2) * g.sw >= pairs_needed) {
     g.ng *= 2;
@@ -718,14 +857,16 @@ bool make_geo(const DeviceLayer& L, int n, int h, int w, bool allow_split, Geo* 
   if (g.tw == 4) while (g.substride % 128 != 64) g.substride += 16;
   if (g.tw == 2) while (g.substride % 128 != 32) g.substride += 16;
   g.tab_off = 8 * 2 * kMaxStages + 16;  // barriers, then the TMEM base address word
-  if (L.n_chunks > 512) return false;  // descriptor table budget (c_in <= 4096)
+  if (L.n_chunks > 512) return false;   // descriptor table budget (c_in <= 4096)
+  g.ks = 1;
+  g.cps = L.n_chunks;
   for (;;) {
     g.pairs = g.wy * g.sw;
     g.chan_stride = g.pairs * g.substride;
     g.x_stage_bytes = kChunk * g.chan_stride;
     g.stage_bytes = (g.x_stage_bytes + g.ng * (kWSlot + kCodeSlot) + 15) & ~15;
     g.desc_off = (g.tab_off + 2 * g.pairs * (int)sizeof(SubTile) + 15) & ~15;
-    g.stage_off = g.desc_off + g.ng * L.n_chunks * 16;
+    g.stage_off = g.desc_off + g.ng * L.n_chunks * 32;
     g.stages = (kSmemLimit - g.stage_off) / g.stage_bytes;
     if (g.stages > kMaxStages) g.stages = kMaxStages;
     if (g.stages >= 2) break;
@@ -733,29 +874,94 @@ bool make_geo(const DeviceLayer& L, int n, int h, int w, bool allow_split, Geo* 
       g.wy /= 2;          // fewer pixel sets (the other warp rows idle)
     } else if (g.ng > 1) {
       g.ng /= 2;          // fewer filter groups per CTA
-      g.wys = kCW / g.ng;
+      g.wys = units / g.ng;
     } else {
       break;
     }
   }
   if (g.stages < 2) return false;
-  // Channel splits: when the output tiles do not fill the GPU, cut the channel range so that
-  // about one CTA per SM is launched (measured on 14x14 .. 56x56 batch-1 layers: the best split
-  // count is the one that fills a single wave; more splits only add reduction traffic).
-  g.ks = 1;
-  if (allow_split && !GENERIC) {
-    const long long ctas = ((q + 2 * g.pairs - 1) / (2 * g.pairs)) * ((L.n_groups + g.ng - 1) / g.ng);
-    long long ks = kNumSMs / ctas;
-    if (ks > L.n_chunks) ks = L.n_chunks;
-    if (ks > 1) g.ks = (int)ks;
-  }
-  g.cps = (L.n_chunks + g.ks - 1) / g.ks;
-  g.ks = (L.n_chunks + g.cps - 1) / g.cps;
   if (g.stages > g.cps) g.stages = g.cps;
   g.relu = 0;
   g.is_half = (L.storage == PCONV_F16);
   *out = g;
   return true;
+}
+
+long long geo_tiles(const DeviceLayer& L, const Geo& g) {
+  return (((long long)g.q_total + 2 * g.pairs - 1) / (2 * g.pairs)) * ((L.n_groups + g.ng - 1) / g.ng);
+}
+
+// Cuts the chunk range of a geometry in ks parts (grid.z).
+void set_split(const DeviceLayer& L, Geo* g, int ks) {
+  if (ks < 1) ks = 1;
+  if (ks > L.n_chunks) ks = L.n_chunks;
+  g->cps = (L.n_chunks + ks - 1) / ks;
+  g->ks = (L.n_chunks + g->cps - 1) / g->cps;
+  g->stage_off = g->desc_off + g->ng * g->cps * 32;
+  int stages = (kSmemLimit - g->stage_off) / g->stage_bytes;
+  if (stages > kMaxStages) stages = kMaxStages;
+  if (stages > g->cps) stages = g->cps;
+  g->stages = stages;
+}
+
+// Estimated duration of a launch in units of one kernel (4 taps on a warp's 256 pixels, about
+// 0.18 us), from measurements of batch-1 layers: a CTA pays a fixed start (first chunk in flight)
+// and an epilogue that shrinks with the warps sharing a unit; CTAs run in waves of one per SM; a
+// channel split across CTAs adds the atomic traffic of every CTA's whole tile and its draining.
+double geo_cost(const DeviceLayer& L, const Geo& g) {
+  const double k_unit = (double)L.n_kept / (L.n_groups > 0 ? L.n_groups : 1);  // kernels of one group
+  const double per_chunk = 1.5;                                                // barrier, entry, exit
+  const double loop = k_unit / (g.zs * g.ks) + per_chunk * g.cps;
+  const double fixed = 28.0 + 17.0 / g.zs;
+  const long long ctas = geo_tiles(L, g) * g.ks;
+  const double waves = (double)((ctas + kNumSMs - 1) / kNumSMs);
+  return waves * (fixed + loop) + (g.ks > 1 ? 100.0 / g.zs : 0.0);
+}
+
+// The geometry of a launch.  Canonical pattern sets choose how the 16 consumer warps are used
+// (zs = 1, 2 or 4 warps per unit) and, when a workspace is available, whether the channel range
+// is also split across CTAs, by the estimate above.
+template <bool GENERIC>
+bool make_geo(const DeviceLayer& L, int n, int h, int w, bool allow_split, Geo* out) {
+  if (GENERIC) return geo_for<true>(L, n, h, w, 1, out);
+  bool found = false;
+  double best = 0.0;
+#ifdef PCONV_TRACE
+  const char* force_zs = getenv("PCONV_FORCE_ZS");
+  const char* force_ks = getenv("PCONV_FORCE_KS");
+#endif
+  for (int zs = 1; zs <= 4; zs *= 2) {
+    Geo g;
+#ifdef PCONV_TRACE
+    if (force_zs && atoi(force_zs) != zs) continue;
+#endif
+    if (!geo_for<false>(L, n, h, w, zs, &g)) continue;
+#ifdef PCONV_TRACE
+    if (force_ks && allow_split) {
+      set_split(L, &g, atoi(force_ks));
+      *out = g;
+      return true;
+    }
+#endif
+    for (int pass = 0; pass < 2; ++pass) {
+      Geo c = g;
+      if (pass == 1) {
+        if (!allow_split) break;
+        const long long tiles = geo_tiles(L, g);
+        const long long ks = kNumSMs / tiles;   // fill one wave
+        if (ks < 2) break;
+        set_split(L, &c, (int)ks);
+        if (c.ks < 2 || c.stages < 1) break;
+      }
+      const double cost = geo_cost(L, c);
+      if (!found || cost < best) {
+        found = true;
+        best = cost;
+        *out = c;
+      }
+    }
+  }
+  return found;
 }
 
 template <int S, bool GENERIC>
@@ -790,13 +996,32 @@ bool tiled_supported(const DeviceLayer& L, int n, int h, int w) {
 }
 
 // Workspace of the channel-split path: one fp32 partial sum per output element, then one ticket
-// per (pixel tile, filter-group set); 0 if this shape is never split.
+// per (pixel tile, filter-group set, consumer warp); 0 if this shape is never split.
 size_t tiled_workspace_bytes(const DeviceLayer& L, int n, int h, int w) {
   Geo g;
   if (!L.codes_s || !make_geo<false>(L, n, h, w, true, &g) || g.ks <= 1) return 0;
-  const size_t ctas = (((size_t)g.q_total + 2 * g.pairs - 1) / (2 * g.pairs)) *
-                      ((L.n_groups + g.ng - 1) / g.ng);
-  return ((out_elems(L, n, h, w) * 4 + 255) & ~(size_t)255) + ((ctas * 4 + 255) & ~(size_t)255);
+  const size_t ctas = (size_t)geo_tiles(L, g);
+  return ((out_elems(L, n, h, w) * 4 + 255) & ~(size_t)255) +
+         ((ctas * consumer_warps(false) * 4 + 255) & ~(size_t)255);
+}
+
+// The launch geometry launch_tiled would use (see pconv_plan_t).
+bool tiled_plan(const DeviceLayer& L, int n, int h, int w, bool generic_taps, bool with_workspace,
+                pconv_plan_t* out) {
+  if (!generic_taps && !L.codes_s) generic_taps = true;
+  Geo g;
+  if (!(generic_taps ? make_geo<true>(L, n, h, w, false, &g) : make_geo<false>(L, n, h, w, with_workspace, &g)))
+    return false;
+  out->generic_taps = generic_taps ? 1 : 0;
+  out->warps_per_unit = g.zs;
+  out->channel_splits = g.ks;
+  out->groups_per_cta = g.ng;
+  out->pixel_sets = g.wy;
+  out->tile_width = g.tw;
+  out->stages = g.stages;
+  out->ctas = geo_tiles(L, g) * g.ks;
+  out->smem_bytes = g.stage_off + g.stages * g.stage_bytes;
+  return true;
 }
 
 cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias, void* y, int n, int h,

@@ -243,22 +243,37 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
         bd.cg_off = (uint32_t)codes_g.size();
         // Specialised stream: 16-byte records, each a run of kernel codes closed by a terminator
         // (advance to another channel's window, or end); the kernel reads a record with one load.
+        // A quarter (kChunk / kQuarters channels) begins on a record boundary and its entry point
+        // is kept in the descriptor, so that several warps can share one block.
         std::vector<uint8_t> rec;
+        int n_rec = 0;
         auto close_record = [&](uint8_t terminator) {
           rec.push_back(terminator);
           while (rec.size() < 16) rec.push_back((uint8_t)kCodeEnd);
           codes_s.insert(codes_s.end(), rec.begin(), rec.end());
           rec.clear();
+          ++n_rec;
         };
-        int pos = c0 - 1;  // channel whose window is loaded
+        for (int q = 0; q < kQuarters; ++q) bd.quarter[q] = kQuarterEmpty;
+        int pos_s = -1;      // channel whose window the specialised stream has loaded (-1: none yet)
+        int pos_g = c0 - 1;  // the same for the generic stream
+        int n_item = 0;
         for (const Item& it : items) {
-          if (it.c != pos) {
-            const int adv = it.c - pos;  // 1..kChunk
-            close_record((uint8_t)((adv << 4) | kCodeNext));
+          if (it.c != pos_g) {
+            const int adv = it.c - pos_g;  // 1..kChunk
             const uint16_t cg = (uint16_t)(kGenNext | (adv - 1));
             codes_g.push_back((uint8_t)(cg & 0xFF));
             codes_g.push_back((uint8_t)(cg >> 8));
-            pos = it.c;
+            pos_g = it.c;
+          }
+          if (it.c != pos_s) {
+            const int qn = (it.c - c0) / kQuarterChannels;
+            const bool new_quarter = pos_s < 0 || qn != (pos_s - c0) / kQuarterChannels;
+            if (pos_s >= 0)
+              close_record((uint8_t)(((it.c - pos_s) << 4) | (new_quarter ? kCodeSub : kCodeNext)));
+            if (new_quarter)
+              bd.quarter[qn] = (uint16_t)(n_rec | (n_item << 5) | ((it.c - c0) << 12));
+            pos_s = it.c;
           }
           if (rec.size() == 15) close_record((uint8_t)kCodeNext);  // same channel, next record
           const int canon = h->canon_id[it.r->pid];
@@ -270,6 +285,7 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
             wv16.insert(wv16.end(), it.r->hv, it.r->hv + 4);
           else
             wv32.insert(wv32.end(), it.r->v, it.r->v + 4);
+          ++n_item;
         }
         close_record((uint8_t)kCodeEnd);
         codes_g.push_back((uint8_t)(kGenEnd & 0xFF));

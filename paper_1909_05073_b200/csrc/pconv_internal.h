@@ -20,9 +20,20 @@ constexpr int kMaxBlockKernels = kGroup * kChunk;
 //   low nibble 8      terminator: advance (high nibble, 0..8) channels inside the chunk, load that
 //                     channel's window and continue with the next record
 //   9                 terminator: end of the block
-// The first record of a block holds only the terminator that leads to its first channel.
+//   low nibble 10     the same as 8, and the next channel lies in another quarter of the chunk
+// A chunk is cut in kQuarters runs of kQuarterChannels channels.  A quarter's first kernel opens a
+// record, and the block descriptor keeps the quarter's entry point, so the consumer warps that share
+// a block can each take some of its quarters (a warp stops at the first code-10 terminator that
+// leads out of its range).  Nothing precedes a quarter's first kernel: whoever enters there loads
+// the window of the entry's channel first.
 constexpr int kCodeNext = 8;
 constexpr int kCodeEnd = 9;
+constexpr int kCodeSub = 10;
+constexpr int kQuarters = 4;
+constexpr int kQuarterChannels = kChunk / kQuarters;
+// Quarter entry: record index in the block (bits 0-4), kernel index in the block (bits 5-11),
+// channel inside the chunk (bits 12-14); bit 15 = the quarter has no kernel.
+constexpr uint16_t kQuarterEmpty = 0x8000;
 // Generic code stream (two bytes per entry) -- any 4-of-9 mask.
 //   (g << 9) | mask   kernel with run-time mask;   0x2000 | (adv-1)   advance;   0x4000   end
 constexpr int kGenNext = 0x2000;
@@ -38,7 +49,7 @@ struct BlockDesc {      // one per (group, chunk); 32 bytes
   uint32_t cs_len;      // specialised code bytes including the end code
   uint32_t cg_off;      // byte offset of the generic codes (16-byte aligned)
   uint32_t cg_len;      // generic code bytes including the end code
-  uint32_t pad0, pad1;
+  uint16_t quarter[kQuarters];  // entry points into the specialised stream
 };
 
 struct DeviceLayer {         // device pointers of one packed layer (passed to kernels by value)
@@ -82,6 +93,8 @@ cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias,
                          cudaStream_t stream);
 size_t tiled_workspace_bytes(const DeviceLayer& L, int n, int h, int w);
 bool tiled_supported(const DeviceLayer& L, int n, int h, int w);
+bool tiled_plan(const DeviceLayer& L, int n, int h, int w, bool generic_taps, bool with_workspace,
+                pconv_plan_t* out);
 cudaError_t launch_maxpool(const void* x, void* y, int n, int c, int h, int w, int storage,
                            cudaStream_t stream);
 }  // namespace pconv

@@ -52,13 +52,22 @@ def test_static_workspace_entry_point_matches_the_workspace_entry_point():
 
 def test_static_workspace_rejects_shapes_beyond_its_size():
     pbuild.build()
-    # 128 filters on one 640x32 image: 40 output tiles, so the channel range is split, and the
-    # partial sums (128*640*32*4 B = 10.5 MB) do not fit the 8 MiB array
-    spec = synth.LayerSpec("t", 32, 128, 640, 32, 1, 0.3)
-    w, b, _ = synth.gen_weights(spec, 5)
-    layer = B.Layer(w, synth.PATTERNS8, 1, B.F32, b)
-    assert B.pconv_workspace_bytes(layer.handle, 1, 640, 32) > B.STATIC_WS_BYTES
-    x = torch.zeros(1, 32, 640, 32, device="cuda")
+    # 128 filters on one 640x32 image: too few output tiles to fill the GPU, so a deep enough
+    # layer has its channel range split across CTAs, and the partial sums (128*640*32*4 B =
+    # 10.5 MB) do not fit the 8 MiB array.  The split is the library's choice: take the first depth
+    # for which it is made.
+    layer = None
+    for c_in in (512, 1024, 2048):
+        spec = synth.LayerSpec("t", c_in, 128, 640, 32, 1, 0.3)
+        w, b, _ = synth.gen_weights(spec, 5)
+        cand = B.Layer(w, synth.PATTERNS8, 1, B.F32, b)
+        if B.pconv_workspace_bytes(cand.handle, 1, 640, 32) > B.STATIC_WS_BYTES:
+            layer = cand
+            break
+        cand.close()
+    assert layer is not None, "no tested depth makes the library split this shape"
+    assert B.pconv_plan(layer.handle, 1, 640, 32, 0, True)["channel_splits"] > 1
+    x = torch.zeros(1, c_in, 640, 32, device="cuda")
     y = torch.full((1, 128, 640, 32), 7.0, device="cuda")
     with pytest.raises(B.PconvError) as e:
         B.pconv_forward_static_ws(layer.handle, x, layer.bias, y, B.RELU)
