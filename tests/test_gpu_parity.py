@@ -231,6 +231,41 @@ def test_channel_split_path_matches_the_oracle(case, storage):
     layer.close()
 
 
+PLAN_CASES = [  # shapes that make the library use each way of sharing the consumer warps
+    (16, 128, 32, 32, 74, 1, 0.5),    # as many tiles as SMs: one warp per unit
+    (64, 64, 224, 224, 1, 1, 0.3),    # one large image
+    (64, 128, 112, 112, 1, 1, 0.3),
+    (256, 256, 14, 14, 1, 1, 0.3),    # deep and small: warps share units and CTAs share tiles
+    (128, 128, 56, 56, 1, 2, 0.3),
+]
+
+
+def test_every_warp_sharing_plan_matches_the_oracle():
+    seen = set()
+    for case in PLAN_CASES:
+        c_in, c_out, h, w, n, stride, keep = case
+        spec = synth.LayerSpec("t", c_in, c_out, h, w, stride, keep)
+        wt, bias, _ = synth.gen_weights(spec, 777 + c_in)
+        x = synth.gen_input(spec, n, 777 + c_in)
+        layer = B.Layer(wt, synth.PATTERNS8, stride, B.F32, bias)
+        xt = torch.from_numpy(x).cuda()
+        ref = oracle_layer(wt, bias, x, stride, "f32", True)
+        for with_ws in (False, True):
+            plan = B.pconv_plan(layer.handle, n, h, w, 0, with_ws)
+            assert plan["generic_taps"] == 0 and plan["warps_per_unit"] in (1, 2, 4)
+            assert plan["smem_bytes"] <= 227 * 1024 and plan["stages"] >= 1
+            assert (plan["channel_splits"] > 1) == (with_ws and B.pconv_workspace_bytes(layer.handle, n, h, w) > 0)
+            seen.add((plan["warps_per_unit"], plan["channel_splits"] > 1))
+            for _ in range(2):
+                y = layer.forward(xt, relu=True, split=with_ws)
+                torch.cuda.synchronize()
+                check_close(y.float().cpu().numpy(), ref, "f32", "plan %s of %s" % (plan, case))
+        assert B.pconv_device_status(layer.handle)[0] == 0
+        layer.close()
+    assert {z for z, _ in seen} == {1, 2, 4}, seen
+    assert (4, True) in seen and (4, False) in seen, seen
+
+
 @pytest.mark.parametrize("storage", ["f32", "f16"])
 def test_stack_matches_the_chained_oracle(storage):
     chans = [(3, 16), (16, 24), (24, 40), (40, 40)]
