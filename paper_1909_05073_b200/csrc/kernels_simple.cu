@@ -57,6 +57,10 @@ template <typename T>
 __global__ void __launch_bounds__(256) maxpool_kernel(const T* __restrict__ x, T* __restrict__ y,
                                                       long long total, int h, int w, int h_out,
                                                       int w_out) {
+  // started early under programmatic stream serialisation: let the next kernel do the same, and
+  // wait for the producer of x
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < total;
        e += (long long)gridDim.x * blockDim.x) {
     const int j = (int)(e % w_out);
@@ -100,13 +104,20 @@ cudaError_t launch_maxpool(const void* x, void* y, int n, int c, int h, int w, i
   if (total == 0) return cudaSuccess;
   long long blocks = (total + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)blocks, 1, 1);
+  cfg.blockDim = dim3(256, 1, 1);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   if (storage == PCONV_F16)
-    maxpool_kernel<__half><<<(int)blocks, 256, 0, stream>>>((const __half*)x, (__half*)y, total, h,
-                                                            w, h_out, w_out);
-  else
-    maxpool_kernel<float><<<(int)blocks, 256, 0, stream>>>((const float*)x, (float*)y, total, h, w,
-                                                          h_out, w_out);
-  return cudaGetLastError();
+    return cudaLaunchKernelEx(&cfg, maxpool_kernel<__half>, (const __half*)x, (__half*)y, total, h, w,
+                              h_out, w_out);
+  return cudaLaunchKernelEx(&cfg, maxpool_kernel<float>, (const float*)x, (float*)y, total, h, w, h_out,
+                            w_out);
 }
 
 }  // namespace pconv

@@ -568,6 +568,9 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
 
   PCONV_MARK(0)
   PCONV_MARK_MAX(8)
+  // The next kernel of the stream may start its own set-up while this one runs (it waits for this
+  // grid to finish before it touches activations, see below).
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (tid == 0) {
     for (int s = 0; s < g.stages; ++s) {
       mbar_init(sbase + 8 * s, 32 * kProducerWarps);
@@ -616,6 +619,10 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  // Everything above reads only the packed layer.  When launched with programmatic stream
+  // serialisation the kernel has started before the previous one in the stream finished: wait
+  // for it here, before x is read and before y, workspace or tickets are written.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   PCONV_MARK(1)
   const uint32_t tmem_base = GENERIC ? 0u : *tmem_base_s;
 
@@ -977,9 +984,17 @@ cudaError_t launch_one(const DeviceLayer& L, Geo g, const void* x, const float* 
   const long long ctas_x = ((long long)g.q_total + 2 * g.pairs - 1) / (2 * g.pairs);
   const int ctas_y = (L.n_groups + g.ng - 1) / g.ng;
   if (ctas_x > 0x7FFFFFFF || ctas_y > 65535 || g.ks > 65535) return cudaErrorInvalidValue;
-  dim3 grid((unsigned)ctas_x, (unsigned)ctas_y, (unsigned)g.ks);
-  tiled_kernel<S, GENERIC><<<grid, cta_threads(GENERIC), smem, stream>>>(L, g, x, bias, y, ws, counters);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)ctas_x, (unsigned)ctas_y, (unsigned)g.ks);
+  cfg.blockDim = dim3(cta_threads(GENERIC), 1, 1);
+  cfg.dynamicSmemBytes = (size_t)smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, tiled_kernel<S, GENERIC>, L, g, x, bias, y, ws, counters);
 }
 
 size_t out_elems(const DeviceLayer& L, int n, int h, int w) {
