@@ -27,14 +27,14 @@ Operands of the asm statement (all u32): %0 code pointer (first record of the wa
 range), %1 weight pointer (its first kernel), %2 window pointer (one channel before the chunk),
 %3 channel stride, %4 column stride of the staged tile, %5 offset of the middle window column
 (bytes, shared-memory addresses), %6 TMEM address of the warp's slot 0, %7 the entry code
-((first channel + 1) << 4: the advance that leads to the range's first channel), %8 window pointer
-of the first channel past the warp's range (all ones when the warp runs the block to its end).
+((first channel + 1) << 4: the advance that leads to the range's first channel), %8 the number
+of quarter ends (code 10) after which the warp stops.
 
 Byte codes (specialised stream, 16-byte records): low nibble 0..7 = kernel with that canonical
-pattern, high nibble = filter slot; low nibble 8 = advance (high nibble) channels, reload the
-register window and fetch the next record; 10 = the same, and the next channel lies in another
-quarter of the chunk (a warp that shares the chunk with others stops here when the quarter is not
-its own); 9 = end of the (group, chunk) block.
+pattern, high nibble = filter slot; low nibble 8 = advance (high nibble, may be 0) channels, reload
+the register window and fetch the next record; 10 = the same, and a quarter of the block's kernels
+ends here (a warp that shares the block with others stops at the end of its last quarter); 9 = end
+of the (group, chunk) block.
 """
 import os
 import sys
@@ -122,11 +122,10 @@ def gen(stride):
 
     # Advance: `code` >> 4 channels further, reload the window (column-major tile: two rows per
     # 16-byte load) and fetch the next record of codes.
-    # Quarter boundary: stop if the next channel is past this warp's range, else advance.
+    # Quarter end: stop after the last of this warp's quarters, else advance.
     emit("SUB:")
-    emit("shr.u32 ra, code, 4;")
-    emit("mad.lo.u32 ra, ra, %3, xp;")
-    emit("setp.ge.u32 pe, ra, xe;")
+    emit("sub.u32 xe, xe, 1;")
+    emit("setp.eq.u32 pe, xe, 0;")
     emit("@pe bra.uni END;")
     emit("ADV:")
     emit("tcgen05.wait::ld.sync.aligned;")  # the speculative load issued before this jump

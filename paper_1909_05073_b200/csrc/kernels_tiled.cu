@@ -50,7 +50,7 @@ __host__ __device__ constexpr int cta_threads(bool generic) {
 constexpr int kTmemCols = 512;  // whole TMEM of the SM: 16 warps x 16 slots x 8 columns
 constexpr int kMaxStages = 4;
 constexpr int kWSlot = kMaxBlockKernels * 16 + 16;  // bytes per (group, stage): 4 fp32 per kernel
-constexpr int kCodeSlot = 288;                 // bytes per (group, stage)
+constexpr int kCodeSlot = 320;                 // bytes per (group, stage)
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr int kSmemLimit = 227 * 1024;
 constexpr int kNumSMs = 148;
@@ -170,20 +170,20 @@ struct Win {
 template <int S>
 __device__ __forceinline__ void dispatch_chunk(uint32_t cp, uint32_t wp, uint32_t xptr,
                                                uint32_t chan_b, uint32_t col_b, uint32_t off_mid,
-                                               uint32_t tq, uint32_t entry_code, uint32_t xend) {
+                                               uint32_t tq, uint32_t entry_code, uint32_t n_quarters) {
   if (S == 1) {
     asm volatile(
 #include "dispatch_s1.inc"
         :
         : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(col_b), "r"(off_mid), "r"(tq), "r"(entry_code),
-          "r"(xend)
+          "r"(n_quarters)
         : "memory");
   } else {
     asm volatile(
 #include "dispatch_s2.inc"
         :
         : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(col_b), "r"(off_mid), "r"(tq), "r"(entry_code),
-          "r"(xend)
+          "r"(n_quarters)
         : "memory");
   }
 }
@@ -695,10 +695,19 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
     }
 
+#ifdef PCONV_TRACE
+    long long t_wait = 0, t_work = 0;
+#endif
     for (int kk = 0; kk < nk && ok; ++kk) {
       const int s = kk % g.stages;
+#ifdef PCONV_TRACE
+      const long long tc0 = clock64();
+#endif
       ok = mbar_wait(sbase + 8 * s, (kk / g.stages) & 1, L.err, 2);
       if (!ok) break;
+#ifdef PCONV_TRACE
+      const long long tc1 = clock64();
+#endif
       if (kk == 0) { PCONV_MARK(2) }
       if (active) {
         const uint32_t stage_base = sbase + g.stage_off + s * g.stage_bytes;
@@ -706,21 +715,20 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
         uint32_t wp = stage_base + g.x_stage_bytes + wgi * kWSlot;
         uint32_t cp = stage_base + g.x_stage_bytes + g.ng * kWSlot + wgi * kCodeSlot;
         if constexpr (!GENERIC) {
-          // enter at the first of this warp's quarters that has a kernel; run to the range's end
+          // enter at the first of this warp's quarters that has a kernel; run through the others
           const uint4 d1 = desc[2 * (wgi * g.cps + kk) + 1];
           const u64 quarters = ((u64)d1.w << 32) | d1.z;
-          uint32_t ent = kQuarterEmpty;
+          uint32_t ent = kQuarterEmpty, n_q = 0;
           for (int q = q0 + q_per_warp - 1; q >= q0; --q) {
             const uint32_t e = (uint32_t)(quarters >> (16 * q)) & 0xFFFFu;
-            if (!(e & kQuarterEmpty)) ent = e;
+            if (!(e & kQuarterEmpty)) {
+              ent = e;
+              ++n_q;
+            }
           }
-          if (!(ent & kQuarterEmpty)) {
-            const uint32_t xend = (q0 + q_per_warp == kQuarters)
-                                      ? 0xFFFFFFFFu
-                                      : xptr + (uint32_t)((q0 + q_per_warp) * kQuarterChannels + 1) * chan_b;
+          if (n_q)
             dispatch_chunk<S>(cp + (ent & 31u) * 16u, wp + ((ent >> 5) & 127u) * 16u, xptr, chan_b, col_b,
-                              off_mid, tq, (((ent >> 12) & 7u) + 1u) << 4, xend);
-          }
+                              off_mid, tq, (((ent >> 12) & 7u) + 1u) << 4, n_q);
         } else {
           u64 win[Win<S>::kRows][3];
 #pragma unroll
@@ -743,7 +751,18 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(sbase + 8 * (kMaxStages + s));
+#ifdef PCONV_TRACE
+      t_wait += tc1 - tc0;
+      t_work += clock64() - tc1;
+#endif
     }
+#ifdef PCONV_TRACE
+    if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {
+      ((unsigned long long*)(L.err + 2))[11] = (unsigned long long)t_wait;
+      ((unsigned long long*)(L.err + 2))[12] = (unsigned long long)t_work;
+      ((unsigned long long*)(L.err + 2))[13] = (unsigned long long)nk;
+    }
+#endif
 
     PCONV_MARK(3)
     PCONV_MARK_MAX(9)

@@ -243,8 +243,9 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
         bd.cg_off = (uint32_t)codes_g.size();
         // Specialised stream: 16-byte records, each a run of kernel codes closed by a terminator
         // (advance to another channel's window, or end); the kernel reads a record with one load.
-        // A quarter (kChunk / kQuarters channels) begins on a record boundary and its entry point
-        // is kept in the descriptor, so that several warps can share one block.
+        // The block's kernels are cut in kQuarters runs of equal length (in stream order, so a cut
+        // may fall inside a channel); a run begins on a record boundary and its entry point is kept
+        // in the descriptor, so that several warps can share one block with equal work.
         std::vector<uint8_t> rec;
         int n_rec = 0;
         auto close_record = [&](uint8_t terminator) {
@@ -257,7 +258,8 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
         for (int q = 0; q < kQuarters; ++q) bd.quarter[q] = kQuarterEmpty;
         int pos_s = -1;      // channel whose window the specialised stream has loaded (-1: none yet)
         int pos_g = c0 - 1;  // the same for the generic stream
-        int n_item = 0;
+        int n_item = 0, q_prev = -1;
+        const int n_total = (int)items.size();
         for (const Item& it : items) {
           if (it.c != pos_g) {
             const int adv = it.c - pos_g;  // 1..kChunk
@@ -266,14 +268,15 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
             codes_g.push_back((uint8_t)(cg >> 8));
             pos_g = it.c;
           }
-          if (it.c != pos_s) {
-            const int qn = (it.c - c0) / kQuarterChannels;
-            const bool new_quarter = pos_s < 0 || qn != (pos_s - c0) / kQuarterChannels;
+          const int qn = (int)((long long)(n_item + 1) * kQuarters - 1) / n_total;  // run of item n_item
+          const bool new_quarter = n_item == 0 || qn != q_prev;
+          if (it.c != pos_s || new_quarter) {
             if (pos_s >= 0)
               close_record((uint8_t)(((it.c - pos_s) << 4) | (new_quarter ? kCodeSub : kCodeNext)));
             if (new_quarter)
               bd.quarter[qn] = (uint16_t)(n_rec | (n_item << 5) | ((it.c - c0) << 12));
             pos_s = it.c;
+            q_prev = qn;
           }
           if (rec.size() == 15) close_record((uint8_t)kCodeNext);  // same channel, next record
           const int canon = h->canon_id[it.r->pid];

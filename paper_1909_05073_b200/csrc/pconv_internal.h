@@ -20,17 +20,16 @@ constexpr int kMaxBlockKernels = kGroup * kChunk;
 //   low nibble 8      terminator: advance (high nibble, 0..8) channels inside the chunk, load that
 //                     channel's window and continue with the next record
 //   9                 terminator: end of the block
-//   low nibble 10     the same as 8, and the next channel lies in another quarter of the chunk
-// A chunk is cut in kQuarters runs of kQuarterChannels channels.  A quarter's first kernel opens a
-// record, and the block descriptor keeps the quarter's entry point, so the consumer warps that share
-// a block can each take some of its quarters (a warp stops at the first code-10 terminator that
-// leads out of its range).  Nothing precedes a quarter's first kernel: whoever enters there loads
-// the window of the entry's channel first.
+//   low nibble 10     the same as 8 (the advance may be 0), and a quarter of the block ends here
+// A block's kernels are cut, in stream order, in kQuarters runs of equal length.  A run's first
+// kernel opens a record, and the block descriptor keeps the run's entry point, so the consumer
+// warps that share a block can each take some of its quarters (a warp stops at the code-10
+// terminator that closes its last quarter).  Nothing precedes a quarter's first kernel: whoever
+// enters there loads the window of the entry's channel first.
 constexpr int kCodeNext = 8;
 constexpr int kCodeEnd = 9;
 constexpr int kCodeSub = 10;
 constexpr int kQuarters = 4;
-constexpr int kQuarterChannels = kChunk / kQuarters;
 // Quarter entry: record index in the block (bits 0-4), kernel index in the block (bits 5-11),
 // channel inside the chunk (bits 12-14); bit 15 = the quarter has no kernel.
 constexpr uint16_t kQuarterEmpty = 0x8000;
