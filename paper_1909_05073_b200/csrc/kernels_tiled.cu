@@ -48,7 +48,7 @@ __host__ __device__ constexpr int cta_threads(bool generic) {
   return 32 * (consumer_warps(generic) + kProducerWarps);
 }
 constexpr int kTmemCols = 512;  // whole TMEM of the SM: 16 warps x 16 slots x 8 columns
-constexpr int kMaxStages = 4;
+constexpr int kMaxStages = 8;
 constexpr int kWSlot = kMaxBlockKernels * 16 + 16;  // bytes per (group, stage): 4 fp32 per kernel
 constexpr int kCodeSlot = 320;                 // bytes per (group, stage)
 constexpr uint32_t kSpinLimit = 1u << 22;
@@ -279,35 +279,33 @@ __device__ __forceinline__ StagedElem staged_elem(const DeviceLayer& L, const Ge
   return se;
 }
 
-// fp32 storage: everything is fetched with cp.async (zero-fill outside the image), so the producer
-// never waits for data and several chunks are in flight; each thread's arrival on the stage's full
-// barrier fires when its own copies have landed.
+// A producer thread's staged elements are the same in every chunk (only the channel moves), so up
+// to kPreElems of them are worked out once, for channel 0, and kept in registers; threads of wider
+// tiles work the rest out per chunk.  dst == kSkipElem marks a slot past the tile's last element.
+constexpr int kPreElems = 4;
+constexpr uint32_t kSkipElem = 0xFFFFFFFFu;
+constexpr int kProducerThreads = 32 * kProducerWarps;
+
 template <int S>
-__device__ __forceinline__ void produce_chunk_async(const DeviceLayer& L, const Geo& g,
-                                                    const float* __restrict__ x, const SubTile* tab,
-                                                    const uint4* desc, const uint8_t* codes,
-                                                    uint32_t stage_base, int k, int kk, int pw, int lane) {
-  const int c0 = k * kChunk;
-  const int nc = min(kChunk, L.c_in - c0);
-  const size_t hw = (size_t)g.h * g.w;
+__device__ __forceinline__ void precompute_elems(StagedElem (&pre)[kPreElems], const DeviceLayer& L,
+                                                 const Geo& g, const SubTile* tab, int ptid) {
   const int n_elem = g.pairs * g.rows * g.pitch;
-  const uint32_t chan_b = (uint32_t)g.chan_stride;
-  const int ptid = pw * 32 + lane;
-  for (int e = ptid; e < n_elem; e += 32 * kProducerWarps) {
-    const StagedElem se = staged_elem<S>(L, g, tab, e, c0);
-    const float* sa = se.off_a >= 0 ? x + se.off_a : x;
-    const float* sb = se.off_b >= 0 ? x + se.off_b : x;
-    const size_t step_a = se.off_a >= 0 ? hw : 0, step_b = se.off_b >= 0 ? hw : 0;
-    const uint32_t na = se.off_a >= 0 ? 4u : 0u, nb = se.off_b >= 0 ? 4u : 0u;
-    uint32_t dst = stage_base + se.dst;
-    for (int cc = 0; cc < nc; ++cc) {
-      cp_async4(dst, sa, na);
-      cp_async4(dst + 4, sb, nb);
-      sa += step_a;
-      sb += step_b;
-      dst += chan_b;
+#pragma unroll
+  for (int i = 0; i < kPreElems; ++i) {
+    const int e = ptid + i * kProducerThreads;
+    if (e < n_elem) {
+      pre[i] = staged_elem<S>(L, g, tab, e, 0);
+    } else {
+      pre[i].off_a = pre[i].off_b = -1;
+      pre[i].dst = kSkipElem;
     }
   }
+}
+
+// The weight records and codes of the CTA's groups for chunk kk of its range.
+__device__ __forceinline__ void stage_blocks_async(const DeviceLayer& L, const Geo& g, const uint4* desc,
+                                                   const uint8_t* codes, uint32_t stage_base, int kk,
+                                                   int ptid) {
   const uint32_t wbase = stage_base + g.x_stage_bytes;
   const uint32_t cbase = wbase + g.ng * kWSlot;
   for (int j = 0; j < g.ng; ++j) {
@@ -319,40 +317,79 @@ __device__ __forceinline__ void produce_chunk_async(const DeviceLayer& L, const 
   }
 }
 
+// fp32 storage: everything is fetched with cp.async (zero-fill outside the image), so the producer
+// never waits for data and several chunks are in flight; each thread's arrival on the stage's full
+// barrier fires when its own copies have landed.
+template <int S>
+__device__ __forceinline__ void produce_chunk_async(const DeviceLayer& L, const Geo& g,
+                                                    const float* __restrict__ x, const SubTile* tab,
+                                                    const StagedElem (&pre)[kPreElems], const uint4* desc,
+                                                    const uint8_t* codes, uint32_t stage_base, int k, int kk,
+                                                    int ptid) {
+  const int c0 = k * kChunk;
+  const int nc = min(kChunk, L.c_in - c0);
+  const size_t hw = (size_t)g.h * g.w;
+  const int n_elem = g.pairs * g.rows * g.pitch;
+  const uint32_t chan_b = (uint32_t)g.chan_stride;
+  auto copy_elem = [&](const StagedElem& se, size_t chan_off) {
+    const float* sa = se.off_a >= 0 ? x + se.off_a + chan_off : x;
+    const float* sb = se.off_b >= 0 ? x + se.off_b + chan_off : x;
+    const size_t step_a = se.off_a >= 0 ? hw : 0, step_b = se.off_b >= 0 ? hw : 0;
+    const uint32_t na = se.off_a >= 0 ? 4u : 0u, nb = se.off_b >= 0 ? 4u : 0u;
+    uint32_t dst = stage_base + se.dst;
+    for (int cc = 0; cc < nc; ++cc) {
+      cp_async4(dst, sa, na);
+      cp_async4(dst + 4, sb, nb);
+      sa += step_a;
+      sb += step_b;
+      dst += chan_b;
+    }
+  };
+#pragma unroll
+  for (int i = 0; i < kPreElems; ++i)
+    if (pre[i].dst != kSkipElem) copy_elem(pre[i], (size_t)c0 * hw);
+  for (int e = ptid + kPreElems * kProducerThreads; e < n_elem; e += kProducerThreads)
+    copy_elem(staged_elem<S>(L, g, tab, e, c0), 0);
+  stage_blocks_async(L, g, desc, codes, stage_base, kk, ptid);
+}
+
 // fp16 storage: loads, converts to fp32 and stores (the interleaved fp32 layout cannot be produced
 // by an asynchronous copy of 2-byte elements).  Two staged elements (32 loads) are in flight per
 // thread at a time.
 template <int S>
 __device__ __forceinline__ void produce_chunk_half(const DeviceLayer& L, const Geo& g,
                                                    const __half* __restrict__ x, const SubTile* tab,
-                                                   const uint4* desc, const uint8_t* codes,
-                                                   uint32_t stage_base, int k, int kk, int pw, int lane) {
+                                                   const StagedElem (&pre)[kPreElems], const uint4* desc,
+                                                   const uint8_t* codes, uint32_t stage_base, int k, int kk,
+                                                   int ptid) {
   const int c0 = k * kChunk;
   const int nc = min(kChunk, L.c_in - c0);
   const size_t hw = (size_t)g.h * g.w;
   const int n_elem = g.pairs * g.rows * g.pitch;
-  const int ptid = pw * 32 + lane;
-  constexpr int kStep = 32 * kProducerWarps;
-  for (int e = ptid; e < n_elem; e += 2 * kStep) {
-    StagedElem se[2];
-    se[0] = staged_elem<S>(L, g, tab, e, c0);
-    const bool two = e + kStep < n_elem;
-    se[1] = two ? staged_elem<S>(L, g, tab, e + kStep, c0) : se[0];
+  const size_t chan_off = (size_t)c0 * hw;
+  auto copy_two = [&](const StagedElem& s0, const StagedElem& s1, bool two) {
     float va[2][kChunk], vb[2][kChunk];
 #pragma unroll
-    for (int u = 0; u < 2; ++u)
-#pragma unroll
-      for (int cc = 0; cc < kChunk; ++cc) {
-        va[u][cc] = (se[u].off_a >= 0 && cc < nc) ? ldg_f(x + se[u].off_a + cc * hw) : 0.f;
-        vb[u][cc] = (se[u].off_b >= 0 && cc < nc) ? ldg_f(x + se[u].off_b + cc * hw) : 0.f;
-      }
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      if (u == 1 && !two) break;
-#pragma unroll
-      for (int cc = 0; cc < kChunk; ++cc)
-        sts64f(stage_base + se[u].dst + (uint32_t)(cc * g.chan_stride), va[u][cc], vb[u][cc]);
+    for (int cc = 0; cc < kChunk; ++cc) {
+      va[0][cc] = (s0.off_a >= 0 && cc < nc) ? ldg_f(x + s0.off_a + chan_off + cc * hw) : 0.f;
+      vb[0][cc] = (s0.off_b >= 0 && cc < nc) ? ldg_f(x + s0.off_b + chan_off + cc * hw) : 0.f;
+      va[1][cc] = (two && s1.off_a >= 0 && cc < nc) ? ldg_f(x + s1.off_a + chan_off + cc * hw) : 0.f;
+      vb[1][cc] = (two && s1.off_b >= 0 && cc < nc) ? ldg_f(x + s1.off_b + chan_off + cc * hw) : 0.f;
     }
+#pragma unroll
+    for (int cc = 0; cc < kChunk; ++cc) {
+      sts64f(stage_base + s0.dst + (uint32_t)(cc * g.chan_stride), va[0][cc], vb[0][cc]);
+      if (two) sts64f(stage_base + s1.dst + (uint32_t)(cc * g.chan_stride), va[1][cc], vb[1][cc]);
+    }
+  };
+#pragma unroll
+  for (int i = 0; i < kPreElems; i += 2)
+    if (pre[i].dst != kSkipElem) copy_two(pre[i], pre[i + 1], pre[i + 1].dst != kSkipElem);
+  for (int e = ptid + kPreElems * kProducerThreads; e < n_elem; e += 2 * kProducerThreads) {
+    const StagedElem s0 = staged_elem<S>(L, g, tab, e, 0);
+    const bool two = e + kProducerThreads < n_elem;
+    const StagedElem s1 = two ? staged_elem<S>(L, g, tab, e + kProducerThreads, 0) : s0;
+    copy_two(s0, s1, two);
   }
   const uint32_t wbase = stage_base + g.x_stage_bytes;
   const uint32_t cbase = wbase + g.ng * kWSlot;
@@ -565,16 +602,18 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
   SubTile* tab = reinterpret_cast<SubTile*>(smem + g.tab_off);
   volatile uint32_t* tmem_base_s = reinterpret_cast<volatile uint32_t*>(smem + 8 * 2 * kMaxStages);
+  int* unit_ctr = reinterpret_cast<int*>(smem + 8 * 2 * kMaxStages + 16);  // next chunk of each unit
 
   PCONV_MARK(0)
   PCONV_MARK_MAX(8)
   // The next kernel of the stream may start its own set-up while this one runs (it waits for this
   // grid to finish before it touches activations, see below).
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (tid < kCW) unit_ctr[tid] = 0;
   if (tid == 0) {
     for (int s = 0; s < g.stages; ++s) {
       mbar_init(sbase + 8 * s, 32 * kProducerWarps);
-      mbar_init(sbase + 8 * (kMaxStages + s), kCW);
+      mbar_init(sbase + 8 * (kMaxStages + s), kCW / (GENERIC ? 1 : g.zs));
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -627,8 +666,8 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   const uint32_t tmem_base = GENERIC ? 0u : *tmem_base_s;
 
   // Consumer-warp coordinates (meaningless for producer warps).  zs warps of one TMEM lane
-  // quadrant form a unit: they work on the same pixels and filter group, each on its own quarters
-  // of every chunk, with accumulators in its own 128 TMEM columns.
+  // quadrant form a unit: they work on the same pixels and filter group and take the chunks in
+  // turn, each with accumulators in its own 128 TMEM columns.
   const int zs = GENERIC ? 1 : g.zs;
   int unit = warp, z = 0;
   if (zs == 2) {
@@ -652,7 +691,6 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   // take 128 columns each = 16 filter slots x (4 rows x {A,B}).
   const uint32_t tquad = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);
   const uint32_t tq = tquad + (uint32_t)((warp >> 2) * (kGroup * 8));
-  const int q_per_warp = kQuarters / zs, q0 = z * q_per_warp;
 
   // lane a < 16 keeps the original filter index and bias of slot a for the epilogue
   int my_o = -1;
@@ -667,17 +705,19 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   if (warp >= kCW) {
     // ===================================== producer warps =====================================
     if (GENERIC) asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
-    const int pw = warp - kCW;
+    const int ptid = (warp - kCW) * 32 + lane;
     const uint8_t* codes = GENERIC ? L.codes_g : L.codes_s;
+    StagedElem pre[kPreElems];
+    if (S == 1) precompute_elems<1>(pre, L, g, tab, ptid); else precompute_elems<2>(pre, L, g, tab, ptid);
     for (int kk = 0; kk < nk; ++kk) {
       const int s = kk % g.stages, it = kk / g.stages;
       if (it > 0 && !mbar_wait(sbase + 8 * (kMaxStages + s), (it - 1) & 1, L.err, 1)) break;
       const uint32_t stage_base = sbase + g.stage_off + s * g.stage_bytes;
       if (g.is_half) {
-        produce_chunk_half<S>(L, g, (const __half*)x, tab, desc, codes, stage_base, k0 + kk, kk, pw, lane);
+        produce_chunk_half<S>(L, g, (const __half*)x, tab, pre, desc, codes, stage_base, k0 + kk, kk, ptid);
         mbar_arrive(sbase + 8 * s);
       } else {
-        produce_chunk_async<S>(L, g, (const float*)x, tab, desc, codes, stage_base, k0 + kk, kk, pw, lane);
+        produce_chunk_async<S>(L, g, (const float*)x, tab, pre, desc, codes, stage_base, k0 + kk, kk, ptid);
         cp_async_arrive(sbase + 8 * s);
       }
     }
@@ -698,7 +738,16 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
 #ifdef PCONV_TRACE
     long long t_wait = 0, t_work = 0;
 #endif
-    for (int kk = 0; kk < nk && ok; ++kk) {
+    // The warps of a unit draw the chunks from the unit's counter, so a warp that got a heavier
+    // chunk (or started later) simply takes fewer.
+    int next_kk = 0;
+    while (ok) {
+      int kk = next_kk++;
+      if (zs > 1) {
+        if (lane == 0) kk = atomicAdd(unit_ctr + unit, 1);
+        kk = __shfl_sync(0xffffffffu, kk, 0);
+      }
+      if (kk >= nk) break;
       const int s = kk % g.stages;
 #ifdef PCONV_TRACE
       const long long tc0 = clock64();
@@ -715,11 +764,11 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
         uint32_t wp = stage_base + g.x_stage_bytes + wgi * kWSlot;
         uint32_t cp = stage_base + g.x_stage_bytes + g.ng * kWSlot + wgi * kCodeSlot;
         if constexpr (!GENERIC) {
-          // enter at the first of this warp's quarters that has a kernel; run through the others
+          // enter at the first quarter that has a kernel; run through the others
           const uint4 d1 = desc[2 * (wgi * g.cps + kk) + 1];
           const u64 quarters = ((u64)d1.w << 32) | d1.z;
           uint32_t ent = kQuarterEmpty, n_q = 0;
-          for (int q = q0 + q_per_warp - 1; q >= q0; --q) {
+          for (int q = kQuarters - 1; q >= 0; --q) {
             const uint32_t e = (uint32_t)(quarters >> (16 * q)) & 0xFFFFu;
             if (!(e & kQuarterEmpty)) {
               ent = e;
@@ -751,6 +800,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(sbase + 8 * (kMaxStages + s));
+      __syncwarp();
 #ifdef PCONV_TRACE
       t_wait += tc1 - tc0;
       t_work += clock64() - tc1;
@@ -836,6 +886,18 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   PCONV_MARK_MAX(7)
 }
 
+// Depth of the staging ring when `fit` stages fit in shared memory (0 = the geometry is not
+// usable).  The zs warps of a unit work on different chunks at the same time, so the ring holds at
+// least zs (then a warp that draws chunk k knows that chunk k - stages has been consumed, which
+// makes waiting on a slot's barrier by phase parity safe), and twice zs when it fits: one set of
+// chunks being worked on, one in flight.
+int pick_stages(int fit, int zs, int cps) {
+  int s = fit < 4 * (zs > 1 ? zs / 2 : 1) ? fit : 4 * (zs > 1 ? zs / 2 : 1);  // 4, 4, 8 for zs = 1, 2, 4
+  if (s > cps) s = cps;
+  if (s == cps) return s;
+  return s >= (zs == 1 ? 2 : zs) ? s : 0;
+}
+
 // Geometry for `zs` consumer warps per unit and no channel split across CTAs.
 template <bool GENERIC>
 bool geo_for(const DeviceLayer& L, int n, int h, int w, int zs, Geo* out) {
@@ -882,7 +944,7 @@ bool geo_for(const DeviceLayer& L, int n, int h, int w, int zs, Geo* out) {
   g.substride = g.pitch * g.colstride;
   if (g.tw == 4) while (g.substride % 128 != 64) g.substride += 16;
   if (g.tw == 2) while (g.substride % 128 != 32) g.substride += 16;
-  g.tab_off = 8 * 2 * kMaxStages + 16;  // barriers, then the TMEM base address word
+  g.tab_off = 8 * 2 * kMaxStages + 16 + 64;  // barriers, the TMEM base address word, unit counters
   if (L.n_chunks > 512) return false;   // descriptor table budget (c_in <= 4096)
   g.ks = 1;
   g.cps = L.n_chunks;
@@ -893,9 +955,8 @@ bool geo_for(const DeviceLayer& L, int n, int h, int w, int zs, Geo* out) {
     g.stage_bytes = (g.x_stage_bytes + g.ng * (kWSlot + kCodeSlot) + 15) & ~15;
     g.desc_off = (g.tab_off + 2 * g.pairs * (int)sizeof(SubTile) + 15) & ~15;
     g.stage_off = g.desc_off + g.ng * L.n_chunks * 32;
-    g.stages = (kSmemLimit - g.stage_off) / g.stage_bytes;
-    if (g.stages > kMaxStages) g.stages = kMaxStages;
-    if (g.stages >= 2) break;
+    g.stages = pick_stages((kSmemLimit - g.stage_off) / g.stage_bytes, zs, g.cps);
+    if (g.stages > 0) break;
     if (g.wy > 1) {
       g.wy /= 2;          // fewer pixel sets (the other warp rows idle)
     } else if (g.ng > 1) {
@@ -905,8 +966,7 @@ bool geo_for(const DeviceLayer& L, int n, int h, int w, int zs, Geo* out) {
       break;
     }
   }
-  if (g.stages < 2) return false;
-  if (g.stages > g.cps) g.stages = g.cps;
+  if (g.stages < 1) return false;
   g.relu = 0;
   g.is_half = (L.storage == PCONV_F16);
   *out = g;
@@ -924,9 +984,7 @@ void set_split(const DeviceLayer& L, Geo* g, int ks) {
   g->cps = (L.n_chunks + ks - 1) / ks;
   g->ks = (L.n_chunks + g->cps - 1) / g->cps;
   g->stage_off = g->desc_off + g->ng * g->cps * 32;
-  int stages = (kSmemLimit - g->stage_off) / g->stage_bytes;
-  if (stages > kMaxStages) stages = kMaxStages;
-  if (stages > g->cps) stages = g->cps;
+  const int stages = pick_stages((kSmemLimit - g->stage_off) / g->stage_bytes, g->zs, g->cps);
   g->stages = stages;
 }
 
@@ -937,7 +995,8 @@ void set_split(const DeviceLayer& L, Geo* g, int ks) {
 double geo_cost(const DeviceLayer& L, const Geo& g) {
   const double k_unit = (double)L.n_kept / (L.n_groups > 0 ? L.n_groups : 1);  // kernels of one group
   const double per_chunk = 1.5;                                                // barrier, entry, exit
-  const double loop = k_unit / (g.zs * g.ks) + per_chunk * g.cps;
+  const int turns = (g.cps + g.zs - 1) / g.zs;                                 // chunks per warp
+  const double loop = turns * (k_unit / L.n_chunks + per_chunk);
   const double fixed = 28.0 + 17.0 / g.zs;
   const long long ctas = geo_tiles(L, g) * g.ks;
   const double waves = (double)((ctas + kNumSMs - 1) / kNumSMs);
@@ -965,6 +1024,7 @@ bool make_geo(const DeviceLayer& L, int n, int h, int w, bool allow_split, Geo* 
 #ifdef PCONV_TRACE
     if (force_ks && allow_split) {
       set_split(L, &g, atoi(force_ks));
+      if (g.stages < 1) continue;
       *out = g;
       return true;
     }
