@@ -117,6 +117,9 @@ pconv_status pconv_pack(const float* w_oihw_host, int c_out, int c_in, const uin
  * Asynchronous on `stream`; allocates nothing and never synchronises.  PCONV_ERR_CUDA reports
  * launch-time errors only.  A handle is immutable: concurrent forwards on several streams are
  * allowed.  n == 0 is a no-op.
+ * The tiled kernels are launched with programmatic stream serialisation: a launch may begin its
+ * own set-up while the previous kernel of the stream is still running, and waits for that kernel
+ * to finish before it reads x or writes y, so stream order holds for every buffer named here.
  */
 pconv_status pconv_forward(const pconv_handle* h, const void* x_dev, const float* bias_dev,
                            void* y_dev, int n, int h_in, int w_in, unsigned flags, void* stream);
@@ -126,8 +129,10 @@ pconv_status pconv_forward(const pconv_handle* h, const void* x_dev, const float
  * caller-provided scratch buffer that lets the library split the input-channel range of a layer
  * over several thread blocks when the batch offers too few output tiles to fill the GPU (batch-1
  * layers).  Partial sums are accumulated in the workspace with fp32 atomics (so the summation
- * order, not the result beyond rounding, varies from run to run) and the last block to finish an
- * output tile applies bias / ReLU and writes y.  The paper has no counterpart; this is how the
+ * order, not the result beyond rounding, varies from run to run) and the last warp to finish a
+ * part of an output tile applies bias / ReLU and writes that part of y.  A forward that ends with
+ * PCONV_ERR_DEVICE_TIMEOUT (pconv_device_status) may leave the workspace non-zero: clear it before
+ * it is used again.  The paper has no counterpart; this is how the
  * build recovers parallelism that the paper's one-image-at-a-time mobile setting never needed.
  *
  *  bytes       receives the workspace size for this handle and input shape (0 = never split).
