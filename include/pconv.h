@@ -58,6 +58,9 @@ enum { PCONV_F32 = 0, PCONV_F16 = 1 };
 enum {
   PCONV_RELU = 1u,    /* forward: y = max(0, .) after the bias */
   PCONV_STRICT4 = 2u, /* pack: every kernel must have exactly 0 or 4 non-zeros */
+  PCONV_POOL2X2 = 4u, /* forward: a 2x2 / stride-2 max-pool is applied to the activated output in
+                         the same kernel (tiled kernels only); y then holds
+                         [n][c_out][h_out/2][w_out/2] */
   /* Kernel selection (forward).  Default: the library picks per shape.  These bits exist so that
    * tests and benchmarks can pin one implementation; they never change the result beyond
    * summation order. */
@@ -112,7 +115,12 @@ pconv_status pconv_pack(const float* w_oihw_host, int c_out, int c_in, const uin
  *  bias_dev  [c_out] fp32, DEVICE, or NULL for no bias.
  *  y_dev     [n][c_out][h_out][w_out], DEVICE, same storage type, 16-byte aligned, must not
  *            overlap x.  h_out = (h_in - 1) / stride + 1, likewise w_out.
- *  flags     PCONV_RELU and/or one PCONV_KERNEL_* bit.
+ *  flags     PCONV_RELU, PCONV_POOL2X2 and/or one PCONV_KERNEL_* bit.  With PCONV_POOL2X2 the
+ *            layer's output is max-pooled before it is stored (the VGG stacks of the evaluation
+ *            pool after conv2/4/7/10): y_dev is [n][c_out][h_out/2][w_out/2] (odd trailing row
+ *            and column dropped, as pconv_maxpool2x2 does), h_out and w_out must be >= 2, and the
+ *            call is refused with PCONV_ERR_UNSUPPORTED when no tiled kernel takes the shape or
+ *            PCONV_KERNEL_SIMPLE is asked for.
  *
  * Asynchronous on `stream`; allocates nothing and never synchronises.  PCONV_ERR_CUDA reports
  * launch-time errors only.  A handle is immutable: concurrent forwards on several streams are

@@ -14,7 +14,7 @@ LIB_PATH = os.path.join(HERE, "libpconv.so")
 
 OK = 0
 F32, F16 = 0, 1
-RELU, STRICT4 = 1, 2
+RELU, STRICT4, POOL2X2 = 1, 2, 4
 KERNEL_SIMPLE, KERNEL_TILED, KERNEL_GENERIC_TAPS = 0x100, 0x200, 0x400
 MAX_PATTERNS = 16
 
@@ -254,12 +254,15 @@ class Layer:
             ws = self._ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
         return ws
 
-    def forward(self, x, relu=True, kernel=0, out=None, split=False):
+    def forward(self, x, relu=True, kernel=0, out=None, split=False, pool=False):
         import torch
         if out is None:
-            out = torch.empty(self.out_shape(x.shape), dtype=x.dtype, device=x.device)
+            n, c, h, w = self.out_shape(x.shape)
+            shape = (n, c, h // 2, w // 2) if pool else (n, c, h, w)
+            out = torch.empty(shape, dtype=x.dtype, device=x.device)
         ws = self.workspace(x.shape) if split else None
-        pconv_forward(self.handle, x, self.bias, out, (RELU if relu else 0) | kernel, workspace=ws)
+        pconv_forward(self.handle, x, self.bias, out,
+                      (RELU if relu else 0) | (POOL2X2 if pool else 0) | kernel, workspace=ws)
         return out
 
     def stats(self):

@@ -55,7 +55,7 @@ extern "C" pconv_status pconv_forward_ws(const pconv_handle* h, const void* x, c
   if (!h || !x || !y) return PCONV_ERR_NULL;
   if (n < 0 || h_in <= 0 || w_in <= 0) return PCONV_ERR_SHAPE;
   const unsigned known =
-      PCONV_RELU | PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED | PCONV_KERNEL_GENERIC_TAPS;
+      PCONV_RELU | PCONV_POOL2X2 | PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED | PCONV_KERNEL_GENERIC_TAPS;
   if (flags & ~known) return PCONV_ERR_UNSUPPORTED;
   const unsigned sel = flags & (PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED | PCONV_KERNEL_GENERIC_TAPS);
   if (sel & (sel - 1)) return PCONV_ERR_UNSUPPORTED;  // at most one selection bit
@@ -69,20 +69,26 @@ extern "C" pconv_status pconv_forward_ws(const pconv_handle* h, const void* x, c
     const int ho = (h_in - 1) / L.stride + 1, wo = (w_in - 1) / L.stride + 1;
     const char* xb = (const char*)x;
     const char* yb = (const char*)y;
-    const size_t xs = (size_t)n * L.c_in * h_in * w_in * es, ys = (size_t)n * L.c_out * ho * wo * es;
+    const bool pooled = flags & PCONV_POOL2X2;
+    if (pooled && (ho < 2 || wo < 2)) return PCONV_ERR_SHAPE;
+    const size_t xs = (size_t)n * L.c_in * h_in * w_in * es;
+    const size_t ys = (size_t)n * L.c_out * (pooled ? ho / 2 : ho) * (pooled ? wo / 2 : wo) * es;
     if (xb < yb + ys && yb < xb + xs) return PCONV_ERR_SHAPE;
   }
   cudaStream_t stream = (cudaStream_t)stream_v;
   const bool relu = flags & PCONV_RELU;
+  const bool pool = flags & PCONV_POOL2X2;
   cudaError_t e;
+  if (pool && (sel == PCONV_KERNEL_SIMPLE || !tiled_supported(L, n, h_in, w_in)))
+    return PCONV_ERR_UNSUPPORTED;  // only the tiled kernels fuse the pool
   if (sel == PCONV_KERNEL_SIMPLE) {
     e = launch_simple(L, x, bias, y, n, h_in, w_in, relu, stream);
   } else if (sel == PCONV_KERNEL_TILED || sel == PCONV_KERNEL_GENERIC_TAPS) {
     if (!tiled_supported(L, n, h_in, w_in)) return PCONV_ERR_UNSUPPORTED;
     const bool generic = (sel == PCONV_KERNEL_GENERIC_TAPS) || !h->canonical;
-    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, generic, ws, ws_bytes, stream);
+    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, pool, generic, ws, ws_bytes, stream);
   } else if (tiled_supported(L, n, h_in, w_in)) {
-    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, !h->canonical, ws, ws_bytes, stream);
+    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, pool, !h->canonical, ws, ws_bytes, stream);
   } else {
     e = launch_simple(L, x, bias, y, n, h_in, w_in, relu, stream);
   }
@@ -286,16 +292,22 @@ extern "C" pconv_status pconv_stack_forward(pconv_stack* s, const void* x, void*
   int ch = s->h, cw = s->w, which = 0;
   for (int i = 0; i < s->n_layers; ++i) {
     const pconv::DeviceLayer& L = s->layers[i]->d;
-    const bool last_op = (i == s->n_layers - 1) && !s->pool[i];
+    // a pool that follows the layer is fused into the layer's epilogue when a tiled kernel runs it
+    const bool fuse = s->pool[i] && !(s->flags & PCONV_KERNEL_SIMPLE) &&
+                      pconv::tiled_supported(L, s->n, ch, cw);
+    const bool last_op = (i == s->n_layers - 1) && (!s->pool[i] || fuse);
     void* dst = last_op ? y : s->act[which];
-    pconv_status st = pconv_forward_ws(s->layers[i], cur, s->bias[i], dst, s->n, ch, cw, s->flags,
-                                       s->ws, s->ws_bytes, stream);
+    pconv_status st = pconv_forward_ws(s->layers[i], cur, s->bias[i], dst, s->n, ch, cw,
+                                       s->flags | (fuse ? PCONV_POOL2X2 : 0u), s->ws, s->ws_bytes, stream);
     if (st != PCONV_OK) return st;
     ch = (ch - 1) / L.stride + 1;
     cw = (cw - 1) / L.stride + 1;
     cur = dst;
     which ^= 1;
-    if (s->pool[i]) {
+    if (fuse) {
+      ch /= 2;
+      cw /= 2;
+    } else if (s->pool[i]) {
       void* pd = (i == s->n_layers - 1) ? y : s->act[which];
       st = pconv_maxpool2x2(cur, pd, s->n, L.c_out, ch, cw, s->storage, stream);
       if (st != PCONV_OK) return st;

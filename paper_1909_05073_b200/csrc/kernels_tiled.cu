@@ -71,6 +71,7 @@ struct Geo {
   int stages, x_stage_bytes, stage_bytes, tab_off, desc_off, stage_off;
   int ks, cps;           // channel splits (grid.z) and chunks per split
   int relu, is_half;
+  int pool, h_y, w_y;     // fused 2x2 max-pool: y holds [h_y][w_y] = [h_out/2][w_out/2] maps
 };
 
 // ---- PTX helpers ----------------------------------------------------------------------------------
@@ -440,6 +441,29 @@ __device__ __forceinline__ LaneOut lane_outputs(const DeviceLayer& L, const Geo&
   return r;
 }
 
+// The same for the pooled output: a lane in an even column writes, for each of its two pixels,
+// the two pooled rows that its four conv rows give (bit 0/1 = A/B upper, bit 2/3 = A/B lower);
+// rows are w_y elements apart.  A pooled position inside the pooled map has all four of its
+// sources inside the conv map, so no source needs masking.
+__device__ __forceinline__ LaneOut lane_outputs_pooled(const DeviceLayer& L, const Geo& g,
+                                                       const SubTile* tab, int slot, int col) {
+  const SubTile A = tab[2 * slot], B = tab[2 * slot + 1];
+  const int px_a = (A.x0 + col) >> 1, px_b = (B.x0 + col) >> 1;
+  const bool even = (col & 1) == 0;
+  const bool col_a = even && A.valid && px_a < g.w_y, col_b = even && B.valid && px_b < g.w_y;
+  const long long plane = (long long)g.h_y * g.w_y;
+  LaneOut r;
+  r.base_a = (long long)A.n * L.c_out * plane + (long long)(A.y0 >> 1) * g.w_y + px_a;
+  r.base_b = (long long)B.n * L.c_out * plane + (long long)(B.y0 >> 1) * g.w_y + px_b;
+  r.mask = 0;
+#pragma unroll
+  for (int k = 0; k < 2; ++k) {
+    if (col_a && (A.y0 >> 1) + k < g.h_y) r.mask |= 1u << (2 * k);
+    if (col_b && (B.y0 >> 1) + k < g.h_y) r.mask |= 2u << (2 * k);
+  }
+  return r;
+}
+
 template <bool HALF, bool RELU>
 __device__ __forceinline__ void store_out(void* __restrict__ y, long long i, float v) {
   if (RELU) v = fmaxf(v, 0.f);
@@ -479,6 +503,22 @@ __device__ __forceinline__ void emit_slot(const Geo& g, const LaneOut& lo, void*
   }
 }
 
+// 2x2 max over a slot's 8 values (rows pairwise inside the lane, columns with the neighbour
+// lane), bias and activation after the max (both are monotone), stored by the even lane.  Must be
+// called by the whole warp.
+template <bool HALF, bool RELU>
+__device__ __forceinline__ void emit_slot_pooled(const Geo& g, const LaneOut& lp, void* __restrict__ y,
+                                                 long long fbase, float bv, const float (&v)[8]) {
+  float m[4] = {fmaxf(v[0], v[2]), fmaxf(v[1], v[3]), fmaxf(v[4], v[6]), fmaxf(v[5], v[7])};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) m[i] = fmaxf(m[i], __shfl_xor_sync(0xffffffffu, m[i], 1));
+  const long long ia = fbase + lp.base_a, ib = fbase + lp.base_b;
+  if (lp.mask & 1u) store_out<HALF, RELU>(y, ia, m[0] + bv);
+  if (lp.mask & 2u) store_out<HALF, RELU>(y, ib, m[1] + bv);
+  if (lp.mask & 4u) store_out<HALF, RELU>(y, ia + g.w_y, m[2] + bv);
+  if (lp.mask & 8u) store_out<HALF, RELU>(y, ib + g.w_y, m[3] + bv);
+}
+
 // Which accumulators a consumer warp writes out: filter slots [a0, a1) of the `zs` column sets
 // that start at TMEM address `t0` (128 columns apart), summed.  zs = 1: the warp's own 16 slots.
 struct OutRange {
@@ -508,11 +548,23 @@ __device__ __forceinline__ void tmem_sum4(uint32_t (&v)[4][8], const OutRange& r
 // Outputs of one consumer warp (filter slots x 4 rows x {A,B} per lane).  `my_o` / `my_b` hold, in
 // lane a < 16, the original filter index and the bias of slot a (loaded at kernel start).
 template <bool GENERIC, int MODE, bool HALF, bool RELU>
-__device__ __forceinline__ void write_outputs(const Geo& g, const LaneOut& lo, void* __restrict__ y,
-                                              float* __restrict__ ws,
+__device__ __forceinline__ void write_outputs(const Geo& g, const LaneOut& lo, const LaneOut& lp,
+                                              void* __restrict__ y, float* __restrict__ ws,
                                               const u64 (&acc)[GENERIC ? kGroup : 1][4],
                                               const OutRange& r, int my_o, float my_b) {
   const long long plane = (long long)g.h_out * g.w_out;
+  const long long plane_y = (long long)g.h_y * g.w_y;
+  // one filter slot: plain stores / atomics, or the fused 2x2 max-pool (warp-uniform choice)
+  auto emit = [&](int o, float bv, const uint32_t (&v)[8]) {
+    if (MODE == 0 && g.pool) {
+      float f[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[e]);
+      emit_slot_pooled<HALF, RELU>(g, lp, y, (long long)o * plane_y, bv, f);
+    } else {
+      emit_slot<MODE, HALF, RELU>(g, lo, y, ws, (long long)o * plane, bv, v);
+    }
+  };
   if constexpr (GENERIC) {
 #pragma unroll
     for (int a = 0; a < kGroup; ++a) {
@@ -524,7 +576,7 @@ __device__ __forceinline__ void write_outputs(const Geo& g, const LaneOut& lo, v
       }
       const int o = __shfl_sync(0xffffffffu, my_o, a);
       const float bv = __shfl_sync(0xffffffffu, my_b, a);
-      if (o >= 0) emit_slot<MODE, HALF, RELU>(g, lo, y, ws, (long long)o * plane, bv, v);
+      if (o >= 0) emit(o, bv, v);
     }
   } else {
 #pragma unroll 1
@@ -535,7 +587,7 @@ __device__ __forceinline__ void write_outputs(const Geo& g, const LaneOut& lo, v
       for (int b = 0; b < 4; ++b) {
         const int o = __shfl_sync(0xffffffffu, my_o, a + b);
         const float bv = __shfl_sync(0xffffffffu, my_b, a + b);
-        if (o >= 0) emit_slot<MODE, HALF, RELU>(g, lo, y, ws, (long long)o * plane, bv, v[b]);
+        if (o >= 0) emit(o, bv, v[b]);
       }
     }
   }
@@ -544,20 +596,23 @@ __device__ __forceinline__ void write_outputs(const Geo& g, const LaneOut& lo, v
 // The last split to finish a warp's part of an output tile: workspace -> y, leaving the workspace
 // zeroed.  Four filter slots (32 independent loads per lane) are in flight at once.
 template <bool HALF, bool RELU>
-__device__ __forceinline__ void finalize_outputs(const Geo& g, const LaneOut& lo, void* __restrict__ y,
-                                                 float* __restrict__ ws, int a_begin, int a_end,
-                                                 int my_o, float my_b) {
+__device__ __forceinline__ void finalize_outputs(const Geo& g, const LaneOut& lo, const LaneOut& lp,
+                                                 void* __restrict__ y, float* __restrict__ ws,
+                                                 int a_begin, int a_end, int my_o, float my_b) {
   const long long plane = (long long)g.h_out * g.w_out;
+  const long long plane_y = (long long)g.h_y * g.w_y;
   constexpr int kBatch = 4;
 #pragma unroll 1
   for (int a0 = a_begin; a0 < a_end; a0 += kBatch) {
     float v[kBatch][8];
     long long fb[kBatch];
+    int fo[kBatch];
     float bv[kBatch];
 #pragma unroll
     for (int b = 0; b < kBatch; ++b) {
       const int o = __shfl_sync(0xffffffffu, my_o, a0 + b);
       bv[b] = __shfl_sync(0xffffffffu, my_b, a0 + b);
+      fo[b] = o;
       fb[b] = (o < 0) ? -1 : (long long)o * plane;
       const long long ia = fb[b] + lo.base_a, ib = fb[b] + lo.base_b;
       const uint32_t m = (o < 0) ? 0u : lo.mask;
@@ -572,6 +627,16 @@ __device__ __forceinline__ void finalize_outputs(const Geo& g, const LaneOut& lo
     for (int b = 0; b < kBatch; ++b) {
       if (fb[b] < 0) continue;
       const long long ia = fb[b] + lo.base_a, ib = fb[b] + lo.base_b;
+      if (g.pool) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int row = k * g.w_out;
+          if (lo.mask >> (2 * k) & 1u) ws[ia + row] = 0.f;
+          if (lo.mask >> (2 * k + 1) & 1u) ws[ib + row] = 0.f;
+        }
+        emit_slot_pooled<HALF, RELU>(g, lp, y, (long long)fo[b] * plane_y, bv[b], v[b]);
+        continue;
+      }
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         const int row = k * g.w_out;
@@ -837,15 +902,16 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
     }
     if (active && ok) {
       const LaneOut lo = lane_outputs(L, g, tab, slot, col);
+      const LaneOut lp = g.pool ? lane_outputs_pooled(L, g, tab, slot, col) : lo;
       bool split = false;
       if constexpr (!GENERIC) split = g.ks > 1;
       if (!split) {
         with_flags(g, [&](auto half, auto relu) {
-          write_outputs<GENERIC, 0, decltype(half)::value, decltype(relu)::value>(g, lo, y, ws, acc, orng,
-                                                                                   my_o, my_b);
+          write_outputs<GENERIC, 0, decltype(half)::value, decltype(relu)::value>(g, lo, lp, y, ws, acc,
+                                                                                   orng, my_o, my_b);
         });
       } else {
-        write_outputs<GENERIC, 1, false, false>(g, lo, y, ws, acc, orng, my_o, my_b);
+        write_outputs<GENERIC, 1, false, false>(g, lo, lp, y, ws, acc, orng, my_o, my_b);
         PCONV_MARK(4)
         PCONV_MARK_MAX(10)
         // Every warp owns the same part of the output tile in each of the ks splits, and takes a
@@ -865,8 +931,8 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
         if (t == g.ks - 1) {
           __threadfence();
           with_flags(g, [&](auto half, auto relu) {
-            finalize_outputs<decltype(half)::value, decltype(relu)::value>(g, lo, y, ws, orng.a0, orng.a1,
-                                                                          my_o, my_b);
+            finalize_outputs<decltype(half)::value, decltype(relu)::value>(g, lo, lp, y, ws, orng.a0,
+                                                                          orng.a1, my_o, my_b);
           });
         }
       }
@@ -968,6 +1034,9 @@ bool geo_for(const DeviceLayer& L, int n, int h, int w, int zs, Geo* out) {
   }
   if (g.stages < 1) return false;
   g.relu = 0;
+  g.pool = 0;
+  g.h_y = g.h_out;
+  g.w_y = g.w_out;
   g.is_half = (L.storage == PCONV_F16);
   *out = g;
   return true;
@@ -1119,7 +1188,7 @@ bool tiled_plan(const DeviceLayer& L, int n, int h, int w, bool generic_taps, bo
 }
 
 cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias, void* y, int n, int h,
-                         int w, bool relu, bool generic_taps, void* ws, size_t ws_bytes,
+                         int w, bool relu, bool pool, bool generic_taps, void* ws, size_t ws_bytes,
                          cudaStream_t stream) {
   if (!generic_taps && !L.codes_s) generic_taps = true;
   Geo g;
@@ -1128,6 +1197,12 @@ cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias,
   if (!(generic_taps ? make_geo<true>(L, n, h, w, false, &g) : make_geo<false>(L, n, h, w, split, &g)))
     return cudaErrorInvalidValue;
   g.relu = relu ? 1 : 0;
+  if (pool) {
+    if (g.h_out < 2 || g.w_out < 2) return cudaErrorInvalidValue;
+    g.pool = 1;
+    g.h_y = g.h_out / 2;
+    g.w_y = g.w_out / 2;
+  }
   float* wsf = nullptr;
   int* counters = nullptr;
   if (g.ks > 1) {

@@ -231,6 +231,54 @@ def test_channel_split_path_matches_the_oracle(case, storage):
     layer.close()
 
 
+POOL_CASES = [  # (c_in, c_out, h, w, n, stride, keep): even and odd maps, narrow tiles, stride 2
+    (8, 24, 12, 12, 2, 1, 0.5), (6, 20, 9, 11, 2, 1, 0.6), (16, 16, 37, 33, 1, 1, 0.3),
+    (12, 40, 4, 4, 5, 1, 0.5), (12, 20, 28, 28, 2, 2, 0.4), (128, 96, 28, 28, 1, 1, 0.3),
+    (256, 64, 14, 14, 1, 1, 0.3), (5, 8, 2, 3, 3, 1, 0.8),
+]
+
+
+@pytest.mark.parametrize("storage", ["f32", "f16"])
+@pytest.mark.parametrize("kernel", ["tiled", "generic", "auto"])
+@pytest.mark.parametrize("case", POOL_CASES, ids=lambda c: "x".join(str(v) for v in c))
+def test_fused_maxpool_matches_conv_then_pool(case, kernel, storage):
+    c_in, c_out, h, w, n, stride, keep = case
+    spec = synth.LayerSpec("t", c_in, c_out, h, w, stride, keep)
+    wt, bias, _ = synth.gen_weights(spec, 31 + c_in)
+    x = synth.gen_input(spec, n, 31 + c_in)
+    layer = B.Layer(wt, synth.PATTERNS8, stride, B.F16 if storage == "f16" else B.F32, bias)
+    xt = torch.from_numpy(x).cuda()
+    if storage == "f16":
+        xt = xt.half()
+    for relu in (True, False):
+        ref = oracle.maxpool2x2(oracle_layer(wt, bias, x, stride, storage, relu))
+        for split in (False, True):
+            y = layer.forward(xt, relu=relu, kernel=KERNELS[kernel], split=split, pool=True)
+            torch.cuda.synchronize()
+            assert tuple(y.shape) == ref.shape
+            check_close(y.float().cpu().numpy(), ref, storage, "fused pool %s relu=%s split=%s" % (case, relu, split))
+    ws = getattr(layer, "_ws", None)
+    if ws is not None:
+        assert not ws.any()
+    assert B.pconv_device_status(layer.handle)[0] == 0
+    layer.close()
+
+
+def test_fused_maxpool_is_refused_where_it_cannot_run():
+    spec = synth.LayerSpec("t", 4, 8, 6, 6, 1, 0.5)
+    wt, bias, _ = synth.gen_weights(spec, 5)
+    layer = B.Layer(wt, synth.PATTERNS8, 1, B.F32, bias)
+    x = torch.zeros(1, 4, 6, 6, device="cuda")
+    with pytest.raises(B.PconvError) as e:
+        layer.forward(x, kernel=B.KERNEL_SIMPLE, pool=True)
+    assert "PCONV_ERR_UNSUPPORTED" in str(e.value)
+    x1 = torch.zeros(1, 4, 1, 6, device="cuda")          # a one-row map cannot be pooled
+    with pytest.raises(B.PconvError) as e:
+        B.pconv_forward(layer.handle, x1, layer.bias, torch.zeros(1, 8, 1, 3, device="cuda"), B.POOL2X2)
+    assert "PCONV_ERR_SHAPE" in str(e.value)
+    layer.close()
+
+
 PLAN_CASES = [  # shapes that make the library use each way of sharing the consumer warps
     (16, 128, 32, 32, 74, 1, 0.5),    # as many tiles as SMs: one warp per unit
     (64, 64, 224, 224, 1, 1, 0.3),    # one large image
