@@ -202,23 +202,21 @@ def run_ours(args):
     acts = []
     a = x
     for layer, pool in zip(conv_layers, pools):
-        o = torch.empty(layer.out_shape(a.shape), dtype=torch.float32, device="cuda")
+        n_, c_, h_, w_ = layer.out_shape(a.shape)
+        o = torch.empty((n_, c_, h_ // 2, w_ // 2) if pool else (n_, c_, h_, w_), dtype=torch.float32,
+                        device="cuda")
         acts.append((a, o))
         a = o
-        if pool:
-            p = torch.empty(o.shape[0], o.shape[1], o.shape[2] // 2, o.shape[3] // 2,
-                            dtype=torch.float32, device="cuda")
-            B.pconv_maxpool2x2(o, p)
-            a = p
     conv_ms = [0.0] * len(conv_layers)
     wss = [layer.workspace(xi.shape) for layer, (xi, _) in zip(conv_layers, acts)]
     for _ in range(args.steps):
         flush.zero_()
         pairs = []
-        for layer, (xi, oi), ws in zip(conv_layers, acts, wss):
+        for layer, (xi, oi), ws, pool in zip(conv_layers, acts, wss, pools):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            B.pconv_forward(layer.handle, xi, layer.bias, oi, B.RELU, workspace=ws)
+            B.pconv_forward(layer.handle, xi, layer.bias, oi, B.RELU | (B.POOL2X2 if pool else 0),
+                            workspace=ws)
             e1.record()
             pairs.append((e0, e1))
         torch.cuda.synchronize()
@@ -260,7 +258,11 @@ def run_ours(args):
         err = np.abs(got - a_ref)
         parity_ok = bool((err <= 1e-4 * (1 + np.abs(a_ref))).all())
         conv_time_ms = sum(conv_ms)
-        achieved = flops / (conv_time_ms * 1e-3) / 1e12
+        # The timed region launches nothing but the 13 conv kernels (pools fused), so its duration
+        # is theirs, overlap between consecutive launches included; the launches timed one by one
+        # (no overlap) are reported beside it.
+        achieved = flops / (ms_step * 1e-3) / 1e12
+        achieved_alone = flops / (conv_time_ms * 1e-3) / 1e12
         value = world * flops / (ms_step * 1e-3) / 1e12
         out = {
             "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world,
@@ -284,7 +286,7 @@ def run_ours(args):
                          "frac": achieved / ALU_PEAK_TFLOPS,
                          "peak_source": "148 SMs x 128 FP32 lanes x 2 x 1.965 GHz (derived; "
                                         "no FP32 figure in MEASURED_PEAKS.json)",
-                         "launch_ms_sum": conv_time_ms,
+                         "launch_ms_sum": conv_time_ms, "achieved_launches_timed_alone": achieved_alone,
                          # dram__bytes_read + dram__bytes_write of the 13 conv launches of one
                          # step, from the ncu capture summarised in profiles/
                          "traffic": 63.8e6,
