@@ -318,6 +318,30 @@ __device__ __forceinline__ void stage_blocks_async(const DeviceLayer& L, const G
   }
 }
 
+// The same for fp16 storage: the values are widened on the way (loaded, converted, stored).
+__device__ __forceinline__ void stage_blocks_half(const DeviceLayer& L, const Geo& g, const uint4* desc,
+                                                  const uint8_t* codes, uint32_t stage_base, int kk,
+                                                  int ptid) {
+  const uint32_t wbase = stage_base + g.x_stage_bytes;
+  const uint32_t cbase = wbase + g.ng * kWSlot;
+  for (int j = 0; j < g.ng; ++j) {
+    const uint4 d = desc[2 * (j * g.cps + kk)];
+    if ((uint32_t)ptid < d.y) {
+      const uint2 raw = __ldg(reinterpret_cast<const uint2*>(L.wvals) + d.x + ptid);
+      const __half2 lo = *reinterpret_cast<const __half2*>(&raw.x);
+      const __half2 hi = *reinterpret_cast<const __half2*>(&raw.y);
+      sts128f(wbase + j * kWSlot + ptid * 16, __low2float(lo), __high2float(lo), __low2float(hi),
+              __high2float(hi));
+    }
+    if ((uint32_t)ptid * 16 < d.w) {
+      const uint4 cv = __ldg(reinterpret_cast<const uint4*>(codes + d.z) + ptid);
+      asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(cbase + j * kCodeSlot + ptid * 16),
+                   "r"(cv.x), "r"(cv.y), "r"(cv.z), "r"(cv.w)
+                   : "memory");
+    }
+  }
+}
+
 // fp32 storage: everything is fetched with cp.async (zero-fill outside the image), so the producer
 // never waits for data and several chunks are in flight; each thread's arrival on the stage's full
 // barrier fires when its own copies have landed.
@@ -326,7 +350,7 @@ __device__ __forceinline__ void produce_chunk_async(const DeviceLayer& L, const 
                                                     const float* __restrict__ x, const SubTile* tab,
                                                     const StagedElem (&pre)[kPreElems], const uint4* desc,
                                                     const uint8_t* codes, uint32_t stage_base, int k, int kk,
-                                                    int ptid) {
+                                                    int ptid, bool with_blocks) {
   const int c0 = k * kChunk;
   const int nc = min(kChunk, L.c_in - c0);
   const size_t hw = (size_t)g.h * g.w;
@@ -351,7 +375,7 @@ __device__ __forceinline__ void produce_chunk_async(const DeviceLayer& L, const 
     if (pre[i].dst != kSkipElem) copy_elem(pre[i], (size_t)c0 * hw);
   for (int e = ptid + kPreElems * kProducerThreads; e < n_elem; e += kProducerThreads)
     copy_elem(staged_elem<S>(L, g, tab, e, c0), 0);
-  stage_blocks_async(L, g, desc, codes, stage_base, kk, ptid);
+  if (with_blocks) stage_blocks_async(L, g, desc, codes, stage_base, kk, ptid);
 }
 
 // fp16 storage: loads, converts to fp32 and stores (the interleaved fp32 layout cannot be produced
@@ -362,7 +386,7 @@ __device__ __forceinline__ void produce_chunk_half(const DeviceLayer& L, const G
                                                    const __half* __restrict__ x, const SubTile* tab,
                                                    const StagedElem (&pre)[kPreElems], const uint4* desc,
                                                    const uint8_t* codes, uint32_t stage_base, int k, int kk,
-                                                   int ptid) {
+                                                   int ptid, bool with_blocks) {
   const int c0 = k * kChunk;
   const int nc = min(kChunk, L.c_in - c0);
   const size_t hw = (size_t)g.h * g.w;
@@ -392,24 +416,7 @@ __device__ __forceinline__ void produce_chunk_half(const DeviceLayer& L, const G
     const StagedElem s1 = two ? staged_elem<S>(L, g, tab, e + kProducerThreads, 0) : s0;
     copy_two(s0, s1, two);
   }
-  const uint32_t wbase = stage_base + g.x_stage_bytes;
-  const uint32_t cbase = wbase + g.ng * kWSlot;
-  for (int j = 0; j < g.ng; ++j) {
-    const uint4 d = desc[2 * (j * g.cps + kk)];
-    if ((uint32_t)ptid < d.y) {
-      const uint2 raw = __ldg(reinterpret_cast<const uint2*>(L.wvals) + d.x + ptid);
-      const __half2 lo = *reinterpret_cast<const __half2*>(&raw.x);
-      const __half2 hi = *reinterpret_cast<const __half2*>(&raw.y);
-      sts128f(wbase + j * kWSlot + ptid * 16, __low2float(lo), __high2float(lo), __low2float(hi),
-              __high2float(hi));
-    }
-    if ((uint32_t)ptid * 16 < d.w) {
-      const uint4 cv = __ldg(reinterpret_cast<const uint4*>(codes + d.z) + ptid);
-      asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(cbase + j * kCodeSlot + ptid * 16),
-                   "r"(cv.x), "r"(cv.y), "r"(cv.z), "r"(cv.w)
-                   : "memory");
-    }
-  }
+  if (with_blocks) stage_blocks_half(L, g, desc, codes, stage_base, kk, ptid);
 }
 
 __device__ __forceinline__ void red_add_f32(float* p, float v) {
@@ -724,9 +731,9 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   // Everything above reads only the packed layer.  When launched with programmatic stream
-  // serialisation the kernel has started before the previous one in the stream finished: wait
-  // for it here, before x is read and before y, workspace or tickets are written.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // serialisation the kernel has started before the previous one in the stream finished: each
+  // role waits for it (griddepcontrol.wait) below, after what it can do from the packed layer
+  // alone and before x or the bias is read and y, workspace or tickets are written.
   PCONV_MARK(1)
   const uint32_t tmem_base = GENERIC ? 0u : *tmem_base_s;
 
@@ -760,10 +767,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   // lane a < 16 keeps the original filter index and bias of slot a for the epilogue
   int my_o = -1;
   float my_b = 0.f;
-  if (warp < kCW && active && lane < kGroup) {
-    my_o = __ldg(L.perm + gi * kGroup + lane);
-    if (bias && my_o >= 0) my_b = __ldg(bias + my_o);
-  }
+  if (warp < kCW && active && lane < kGroup) my_o = __ldg(L.perm + gi * kGroup + lane);
   u64 acc[GENERIC ? kGroup : 1][4];
   bool ok = true;
 
@@ -774,15 +778,26 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
     const uint8_t* codes = GENERIC ? L.codes_g : L.codes_s;
     StagedElem pre[kPreElems];
     if (S == 1) precompute_elems<1>(pre, L, g, tab, ptid); else precompute_elems<2>(pre, L, g, tab, ptid);
+    // the weight records and codes of the first ring-full of chunks do not depend on the previous
+    // kernel: fetch them while it finishes
+    const int n_early = min(g.stages, nk);
+    for (int kk = 0; kk < n_early; ++kk) {
+      const uint32_t stage_base = sbase + g.stage_off + kk * g.stage_bytes;
+      if (g.is_half) stage_blocks_half(L, g, desc, codes, stage_base, kk, ptid);
+      else stage_blocks_async(L, g, desc, codes, stage_base, kk, ptid);
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int kk = 0; kk < nk; ++kk) {
       const int s = kk % g.stages, it = kk / g.stages;
       if (it > 0 && !mbar_wait(sbase + 8 * (kMaxStages + s), (it - 1) & 1, L.err, 1)) break;
       const uint32_t stage_base = sbase + g.stage_off + s * g.stage_bytes;
       if (g.is_half) {
-        produce_chunk_half<S>(L, g, (const __half*)x, tab, pre, desc, codes, stage_base, k0 + kk, kk, ptid);
+        produce_chunk_half<S>(L, g, (const __half*)x, tab, pre, desc, codes, stage_base, k0 + kk, kk, ptid,
+                              kk >= n_early);
         mbar_arrive(sbase + 8 * s);
       } else {
-        produce_chunk_async<S>(L, g, (const float*)x, tab, pre, desc, codes, stage_base, k0 + kk, kk, ptid);
+        produce_chunk_async<S>(L, g, (const float*)x, tab, pre, desc, codes, stage_base, k0 + kk, kk, ptid,
+                               kk >= n_early);
         cp_async_arrive(sbase + 8 * s);
       }
     }
@@ -799,6 +814,8 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
       for (int a = 0; a < kGroup; ++a) tmem_st8_zero(tq + a * 8);
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
     }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (bias && my_o >= 0) my_b = __ldg(bias + my_o);
 
 #ifdef PCONV_TRACE
     long long t_wait = 0, t_work = 0;
