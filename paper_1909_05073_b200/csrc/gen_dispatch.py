@@ -23,18 +23,15 @@ issue as few such instructions as it can: one 16-byte load for a kernel's four w
 out of four registers), one TMEM load and one TMEM store of 8 columns, and nine 16-byte loads per
 channel window (the staged tile is stored column-major so that two rows come with one load).
 
-Operands of the asm statement (all u32): %0 code pointer (first record of the warp's channel
-range), %1 weight pointer (its first kernel), %2 window pointer (one channel before the chunk),
-%3 channel stride, %4 column stride of the staged tile, %5 offset of the middle window column
-(bytes, shared-memory addresses), %6 TMEM address of the warp's slot 0, %7 the entry code
-((first channel + 1) << 4: the advance that leads to the range's first channel), %8 the number
-of quarter ends (code 10) after which the warp stops.
+Operands of the asm statement (all u32): %0 code pointer (the block's first record), %1 weight
+pointer (its first kernel), %2 window pointer (one channel before the chunk), %3 channel stride,
+%4 column stride of the staged tile, %5 offset of the middle window column (bytes, shared-memory
+addresses), %6 TMEM address of the warp's slot 0, %7 the entry code ((first channel + 1) << 4: the
+advance that leads to the block's first channel).
 
 Byte codes (specialised stream, 16-byte records): low nibble 0..7 = kernel with that canonical
 pattern, high nibble = filter slot; low nibble 8 = advance (high nibble, may be 0) channels, reload
-the register window and fetch the next record; 10 = the same, and a quarter of the block's kernels
-ends here (a warp that shares the block with others stops at the end of its last quarter); 9 = end
-of the (group, chunk) block.
+the register window and fetch the next record; 9 = end of the (group, chunk) block.
 """
 import os
 import sys
@@ -58,19 +55,17 @@ def gen(stride):
     emit(".reg .b64 w0, w1, w2, w3;")
     emit(".reg .b32 r0, r1, r2, r3;")          # raw weights of the next kernel
     emit(".reg .b32 c0, c1, c2, c3;")          # the current record of byte codes
-    emit(".reg .u32 code, idx, cp, wp, xp, ra, ta, tn, tq, xe;")
-    emit(".reg .pred pe;")
-    emit("TS: .branchtargets " + ", ".join(["P%d" % p for p in range(8)] + ["ADV", "END", "SUB"]) + ";")
+    emit(".reg .u32 code, idx, cp, wp, xp, ra, ta, tn, tq;")
+    emit("TS: .branchtargets " + ", ".join(["P%d" % p for p in range(8)] + ["ADV", "END"]) + ";")
     emit("mov.u32 cp, %0;")
     emit("mov.u32 wp, %1;")
     emit("mov.u32 xp, %2;")
     emit("mov.u32 tq, %6;")
     emit("mov.u32 code, %7;")
-    emit("mov.u32 xe, %8;")
     emit("ld.shared.v4.b32 {r0, r1, r2, r3}, [wp];")
     emit("add.u32 wp, wp, 16;")
     emit("tcgen05.wait::st.sync.aligned;")
-    emit("bra.uni ADV;")                      # the entry code leads to the range's first channel
+    emit("bra.uni ADV;")                      # the entry code leads to the block's first channel
 
     A8 = "{a0, a1, a2, a3, a4, a5, a6, a7}"
     S8 = "{s0, s1, s2, s3, s4, s5, s6, s7}"
@@ -122,11 +117,6 @@ def gen(stride):
 
     # Advance: `code` >> 4 channels further, reload the window (column-major tile: two rows per
     # 16-byte load) and fetch the next record of codes.
-    # Quarter end: stop after the last of this warp's quarters, else advance.
-    emit("SUB:")
-    emit("sub.u32 xe, xe, 1;")
-    emit("setp.eq.u32 pe, xe, 0;")
-    emit("@pe bra.uni END;")
     emit("ADV:")
     emit("tcgen05.wait::ld.sync.aligned;")  # the speculative load issued before this jump
     emit("tcgen05.wait::st.sync.aligned;")  # a slot may come back in the next channel

@@ -50,7 +50,7 @@ __host__ __device__ constexpr int cta_threads(bool generic) {
 constexpr int kTmemCols = 512;  // whole TMEM of the SM: 16 warps x 16 slots x 8 columns
 constexpr int kMaxStages = 8;
 constexpr int kWSlot = kMaxBlockKernels * 16 + 16;  // bytes per (group, stage): 4 fp32 per kernel
-constexpr int kCodeSlot = 320;                 // bytes per (group, stage)
+constexpr int kCodeSlot = 288;                 // bytes per (group, stage)
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr int kSmemLimit = 227 * 1024;
 constexpr int kNumSMs = 148;
@@ -171,20 +171,18 @@ struct Win {
 template <int S>
 __device__ __forceinline__ void dispatch_chunk(uint32_t cp, uint32_t wp, uint32_t xptr,
                                                uint32_t chan_b, uint32_t col_b, uint32_t off_mid,
-                                               uint32_t tq, uint32_t entry_code, uint32_t n_quarters) {
+                                               uint32_t tq, uint32_t entry_code) {
   if (S == 1) {
     asm volatile(
 #include "dispatch_s1.inc"
         :
-        : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(col_b), "r"(off_mid), "r"(tq), "r"(entry_code),
-          "r"(n_quarters)
+        : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(col_b), "r"(off_mid), "r"(tq), "r"(entry_code)
         : "memory");
   } else {
     asm volatile(
 #include "dispatch_s2.inc"
         :
-        : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(col_b), "r"(off_mid), "r"(tq), "r"(entry_code),
-          "r"(n_quarters)
+        : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(col_b), "r"(off_mid), "r"(tq), "r"(entry_code)
         : "memory");
   }
 }
@@ -712,7 +710,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   const int k0 = blockIdx.z * g.cps;                       // this CTA's chunk range
   const int nk = min(L.n_chunks, k0 + g.cps) - k0;
   // Block descriptors of the CTA's groups and chunks, two 16-byte words each:
-  // {first kernel record, records, code offset, code bytes}, {-, -, quarter entries}.
+  // {first kernel record, records, code offset, code bytes}, {-, -, first channel, -}.
   uint4* desc = reinterpret_cast<uint4*>(smem + g.desc_off);
   for (int i = tid; i < g.ng * g.cps; i += kThreads) {
     const int j = i / g.cps, kk = i - j * g.cps;
@@ -846,20 +844,9 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
         uint32_t wp = stage_base + g.x_stage_bytes + wgi * kWSlot;
         uint32_t cp = stage_base + g.x_stage_bytes + g.ng * kWSlot + wgi * kCodeSlot;
         if constexpr (!GENERIC) {
-          // enter at the first quarter that has a kernel; run through the others
-          const uint4 d1 = desc[2 * (wgi * g.cps + kk) + 1];
-          const u64 quarters = ((u64)d1.w << 32) | d1.z;
-          uint32_t ent = kQuarterEmpty, n_q = 0;
-          for (int q = kQuarters - 1; q >= 0; --q) {
-            const uint32_t e = (uint32_t)(quarters >> (16 * q)) & 0xFFFFu;
-            if (!(e & kQuarterEmpty)) {
-              ent = e;
-              ++n_q;
-            }
-          }
-          if (n_q)
-            dispatch_chunk<S>(cp + (ent & 31u) * 16u, wp + ((ent >> 5) & 127u) * 16u, xptr, chan_b, col_b,
-                              off_mid, tq, (((ent >> 12) & 7u) + 1u) << 4, n_q);
+          const uint4 d0 = desc[2 * (wgi * g.cps + kk)], d1 = desc[2 * (wgi * g.cps + kk) + 1];
+          if (d0.y)  // the block has kernels: enter at its first channel
+            dispatch_chunk<S>(cp, wp, xptr, chan_b, col_b, off_mid, tq, (d1.z + 1u) << 4);
         } else {
           u64 win[Win<S>::kRows][3];
 #pragma unroll
@@ -906,7 +893,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
     orng.a1 = kGroup;
     if constexpr (!GENERIC) {
       if (zs > 1) {
-        // The warps of a unit hold partial sums over their own quarters in their own TMEM columns
+        // The warps of a unit hold partial sums over the chunks they drew in their own TMEM columns
         // of the same lanes; once all have finished, each adds up and writes 16 / zs filter slots.
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         asm volatile("bar.sync 1, %0;" ::"n"(32 * kCW) : "memory");

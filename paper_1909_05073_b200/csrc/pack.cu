@@ -243,23 +243,17 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
         bd.cg_off = (uint32_t)codes_g.size();
         // Specialised stream: 16-byte records, each a run of kernel codes closed by a terminator
         // (advance to another channel's window, or end); the kernel reads a record with one load.
-        // The block's kernels are cut in kQuarters runs of equal length (in stream order, so a cut
-        // may fall inside a channel); a run begins on a record boundary and its entry point is kept
-        // in the descriptor, so that several warps can share one block with equal work.
+        // Nothing precedes the first kernel: the descriptor names its channel (`first_ch`).
         std::vector<uint8_t> rec;
-        int n_rec = 0;
         auto close_record = [&](uint8_t terminator) {
           rec.push_back(terminator);
           while (rec.size() < 16) rec.push_back((uint8_t)kCodeEnd);
           codes_s.insert(codes_s.end(), rec.begin(), rec.end());
           rec.clear();
-          ++n_rec;
         };
-        for (int q = 0; q < kQuarters; ++q) bd.quarter[q] = kQuarterEmpty;
+        bd.first_ch = items.empty() ? 0u : (uint32_t)(items.front().c - c0);
         int pos_s = -1;      // channel whose window the specialised stream has loaded (-1: none yet)
         int pos_g = c0 - 1;  // the same for the generic stream
-        int n_item = 0, q_prev = -1;
-        const int n_total = (int)items.size();
         for (const Item& it : items) {
           if (it.c != pos_g) {
             const int adv = it.c - pos_g;  // 1..kChunk
@@ -268,15 +262,9 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
             codes_g.push_back((uint8_t)(cg >> 8));
             pos_g = it.c;
           }
-          const int qn = (int)((long long)(n_item + 1) * kQuarters - 1) / n_total;  // run of item n_item
-          const bool new_quarter = n_item == 0 || qn != q_prev;
-          if (it.c != pos_s || new_quarter) {
-            if (pos_s >= 0)
-              close_record((uint8_t)(((it.c - pos_s) << 4) | (new_quarter ? kCodeSub : kCodeNext)));
-            if (new_quarter)
-              bd.quarter[qn] = (uint16_t)(n_rec | (n_item << 5) | ((it.c - c0) << 12));
+          if (it.c != pos_s) {
+            if (pos_s >= 0) close_record((uint8_t)(((it.c - pos_s) << 4) | kCodeNext));
             pos_s = it.c;
-            q_prev = qn;
           }
           if (rec.size() == 15) close_record((uint8_t)kCodeNext);  // same channel, next record
           const int canon = h->canon_id[it.r->pid];
@@ -288,7 +276,6 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
             wv16.insert(wv16.end(), it.r->hv, it.r->hv + 4);
           else
             wv32.insert(wv32.end(), it.r->v, it.r->v + 4);
-          ++n_item;
         }
         close_record((uint8_t)kCodeEnd);
         codes_g.push_back((uint8_t)(kGenEnd & 0xFF));

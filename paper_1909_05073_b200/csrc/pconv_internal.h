@@ -20,19 +20,10 @@ constexpr int kMaxBlockKernels = kGroup * kChunk;
 //   low nibble 8      terminator: advance (high nibble, 0..8) channels inside the chunk, load that
 //                     channel's window and continue with the next record
 //   9                 terminator: end of the block
-//   low nibble 10     the same as 8 (the advance may be 0), and a quarter of the block ends here
-// A block's kernels are cut, in stream order, in kQuarters runs of equal length.  A run's first
-// kernel opens a record, and the block descriptor keeps the run's entry point, so the consumer
-// warps that share a block can each take some of its quarters (a warp stops at the code-10
-// terminator that closes its last quarter).  Nothing precedes a quarter's first kernel: whoever
-// enters there loads the window of the entry's channel first.
+// Nothing precedes a block's first kernel: the block descriptor names its channel, and the kernel
+// loads that channel's window before it reads the first record.
 constexpr int kCodeNext = 8;
 constexpr int kCodeEnd = 9;
-constexpr int kCodeSub = 10;
-constexpr int kQuarters = 4;
-// Quarter entry: record index in the block (bits 0-4), kernel index in the block (bits 5-11),
-// channel inside the chunk (bits 12-14); bit 15 = the quarter has no kernel.
-constexpr uint16_t kQuarterEmpty = 0x8000;
 // Generic code stream (two bytes per entry) -- any 4-of-9 mask.
 //   (g << 9) | mask   kernel with run-time mask;   0x2000 | (adv-1)   advance;   0x4000   end
 constexpr int kGenNext = 0x2000;
@@ -48,7 +39,8 @@ struct BlockDesc {      // one per (group, chunk); 32 bytes
   uint32_t cs_len;      // specialised code bytes including the end code
   uint32_t cg_off;      // byte offset of the generic codes (16-byte aligned)
   uint32_t cg_len;      // generic code bytes including the end code
-  uint16_t quarter[kQuarters];  // entry points into the specialised stream
+  uint32_t first_ch;    // channel (inside the chunk) of the block's first kernel
+  uint32_t pad0;
 };
 
 struct DeviceLayer {         // device pointers of one packed layer (passed to kernels by value)
