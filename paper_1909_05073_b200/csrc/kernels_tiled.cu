@@ -20,7 +20,8 @@
 //    The hot code (~4 KB) stays inside the per-scheduler instruction cache and the jump latency is
 //    covered by the other warps (see gen_dispatch.py for the measurements behind this).
 //  * any 4-of-9 masks (GENERIC = true): 8 consumer warps with register accumulators, a switch on
-//    the filter slot and nine warp-uniform tap tests per kernel.
+//    the filter slot and nine warp-uniform tap tests per kernel (no register re-allocation between
+//    the roles: 384 threads leave 168 registers each, which the accumulators fit).
 //
 // Producer warps stage, per chunk of 8 input channels, the halo'd sub-tiles (zero-filled outside
 // the image, converted from fp16 when the storage type is fp16) and the chunk's weight records
@@ -51,7 +52,12 @@ constexpr int kTmemCols = 512;  // whole TMEM of the SM: 16 warps x 16 slots x 8
 constexpr int kMaxStages = 8;
 constexpr int kWSlot = kMaxBlockKernels * 16 + 16;  // bytes per (group, stage): 4 fp32 per kernel
 constexpr int kCodeSlot = 288;                 // bytes per (group, stage)
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr int kWRawSlot = kMaxBlockKernels * 8;  // fp16 weight records of one (group, chunk)
+constexpr int kRawStages = 3;
+constexpr uint32_t kSpinLimit = 1u << 20;
+// A waiting warp is suspended by the hardware for up to this long per try (it is woken when the
+// phase completes), so that waiting warps leave the issue slots to the warps that have work.
+constexpr uint32_t kWaitHintNs = 2000;
 constexpr int kSmemLimit = 227 * 1024;
 constexpr int kNumSMs = 148;
 
@@ -69,6 +75,9 @@ struct Geo {
   int colstride;         // bytes between staged columns (rows are contiguous float2)
   int substride, chan_stride;  // bytes per (sub-tile pair, channel) and per channel
   int stages, x_stage_bytes, stage_bytes, tab_off, desc_off, stage_off;
+  // fp16 storage with an even image width: raw copies of the chunk (fp16, row-major, fetched with
+  // cp.async) wait in a ring of raw_stages slots until the producers widen them into a stage
+  int raw_stages, raw_off, raw_slot, raw_pitch, raw_x_bytes;
   int ks, cps;           // channel splits (grid.z) and chunks per split
   int relu, is_half;
   int pool, h_y, w_y;     // fused 2x2 max-pool: y holds [h_y][w_y] = [h_out/2][w_out/2] maps
@@ -127,10 +136,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(kWaitHintNs)
       : "memory");
   return ok != 0;
 }
@@ -316,28 +325,39 @@ __device__ __forceinline__ void stage_blocks_async(const DeviceLayer& L, const G
   }
 }
 
-// The same for fp16 storage: the values are widened on the way (loaded, converted, stored).
+// The same for fp16 storage: the values are widened on the way (loaded, converted, stored).  All
+// groups' loads are issued before the first store, so a chunk costs two round trips, not 2 x ng.
 __device__ __forceinline__ void stage_blocks_half(const DeviceLayer& L, const Geo& g, const uint4* desc,
                                                   const uint8_t* codes, uint32_t stage_base, int kk,
                                                   int ptid) {
+  constexpr int kMaxNg = 16;
   const uint32_t wbase = stage_base + g.x_stage_bytes;
   const uint32_t cbase = wbase + g.ng * kWSlot;
+  // codes need no conversion: asynchronous copies, issued first and waited for at the end (the
+  // caller's plain barrier arrival does not cover them)
   for (int j = 0; j < g.ng; ++j) {
     const uint4 d = desc[2 * (j * g.cps + kk)];
-    if ((uint32_t)ptid < d.y) {
-      const uint2 raw = __ldg(reinterpret_cast<const uint2*>(L.wvals) + d.x + ptid);
-      const __half2 lo = *reinterpret_cast<const __half2*>(&raw.x);
-      const __half2 hi = *reinterpret_cast<const __half2*>(&raw.y);
+    if ((uint32_t)ptid * 16 < d.w) cp_async16(cbase + j * kCodeSlot + ptid * 16, codes + d.z + ptid * 16);
+  }
+  uint2 raw[kMaxNg];
+#pragma unroll
+  for (int j = 0; j < kMaxNg; ++j) {
+    raw[j] = make_uint2(0u, 0u);
+    if (j < g.ng) {
+      const uint4 d = desc[2 * (j * g.cps + kk)];
+      if ((uint32_t)ptid < d.y) raw[j] = __ldg(reinterpret_cast<const uint2*>(L.wvals) + d.x + ptid);
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < kMaxNg; ++j) {
+    if (j < g.ng) {
+      const __half2 lo = *reinterpret_cast<const __half2*>(&raw[j].x);
+      const __half2 hi = *reinterpret_cast<const __half2*>(&raw[j].y);
       sts128f(wbase + j * kWSlot + ptid * 16, __low2float(lo), __high2float(lo), __low2float(hi),
               __high2float(hi));
     }
-    if ((uint32_t)ptid * 16 < d.w) {
-      const uint4 cv = __ldg(reinterpret_cast<const uint4*>(codes + d.z) + ptid);
-      asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(cbase + j * kCodeSlot + ptid * 16),
-                   "r"(cv.x), "r"(cv.y), "r"(cv.z), "r"(cv.w)
-                   : "memory");
-    }
   }
+  asm volatile("cp.async.wait_all;" ::: "memory");
 }
 
 // fp32 storage: everything is fetched with cp.async (zero-fill outside the image), so the producer
@@ -376,45 +396,245 @@ __device__ __forceinline__ void produce_chunk_async(const DeviceLayer& L, const 
   if (with_blocks) stage_blocks_async(L, g, desc, codes, stage_base, kk, ptid);
 }
 
-// fp16 storage: loads, converts to fp32 and stores (the interleaved fp32 layout cannot be produced
-// by an asynchronous copy of 2-byte elements).  Two staged elements (32 loads) are in flight per
-// thread at a time.
+// ---- fp16 storage, even image width: raw ring ----------------------------------------------------
+// A chunk is first copied as it is (fp16, each sub-tile row-major with a two-column margin so that
+// every 4-byte unit starts on an even column and lies wholly inside or outside the image) into a
+// slot of the raw ring with cp.async -- no registers held, several chunks in flight -- together
+// with its fp16 weight records and its codes.  When the copies have landed the producer warps widen
+// the slot into a stage (shared memory to shared memory) in the layout the consumers read.
+
+// Byte offsets of a staged element's A and B halves inside a raw slot (channel 0) and of its
+// place in the stage, in the fields of a StagedElem (off_a, off_b, dst).
 template <int S>
-__device__ __forceinline__ void produce_chunk_half(const DeviceLayer& L, const Geo& g,
-                                                   const __half* __restrict__ x, const SubTile* tab,
-                                                   const StagedElem (&pre)[kPreElems], const uint4* desc,
-                                                   const uint8_t* codes, uint32_t stage_base, int k, int kk,
-                                                   int ptid, bool with_blocks) {
+__device__ __forceinline__ StagedElem raw_elem(const Geo& g, int e) {
+  constexpr int kRows = (S == 1) ? 6 : 9;
+  const int q = e / g.pitch, i = e - q * g.pitch;   // q = pair * rows + row
+  const int p = q / kRows, r = q - p * kRows;
+  const int hidx = staged_dx<S>(i, g.tw) + 2;        // column inside the raw row
+  const int row_b = g.raw_pitch * 2;
+  StagedElem se;
+  se.off_a = ((long long)(2 * p) * kChunk * kRows + r) * row_b + hidx * 2;
+  se.off_b = ((long long)(2 * p + 1) * kChunk * kRows + r) * row_b + hidx * 2;
+  se.dst = (uint32_t)(p * g.substride + i * g.colstride + r * 8);
+  return se;
+}
+
+template <int S>
+__device__ __forceinline__ void issue_raw(const DeviceLayer& L, const Geo& g, const __half* __restrict__ x,
+                                          const SubTile* tab, const uint4* desc, const uint8_t* codes,
+                                          uint32_t raw_base, int k, int kk, int ptid) {
+  constexpr int kRows = (S == 1) ? 6 : 9;
   const int c0 = k * kChunk;
   const int nc = min(kChunk, L.c_in - c0);
   const size_t hw = (size_t)g.h * g.w;
+  const int units_row = g.raw_pitch / 2;
+  const int n_units = g.pairs * 2 * kRows * units_row;
+  const uint32_t chan_b = (uint32_t)(kRows * g.raw_pitch * 2);
+  for (int v = ptid; v < n_units; v += kProducerThreads) {
+    const int q = v / units_row, u = v - q * units_row;   // q = sub-tile * rows + row
+    const int ps = q / kRows, r = q - ps * kRows;
+    const SubTile T = tab[ps];
+    const int iy = T.y0 * S - 1 + r, ix = T.x0 * S - 2 + 2 * u;
+    const bool in = T.valid && iy >= 0 && iy < g.h && ix >= 0 && ix < g.w;
+    const __half* src = in ? x + (((size_t)T.n * L.c_in + c0) * g.h + iy) * g.w + ix : x;
+    const size_t step = in ? hw : 0;
+    uint32_t dst = raw_base + (uint32_t)((ps * kChunk * kRows + r) * g.raw_pitch * 2 + u * 4);
+    for (int cc = 0; cc < kChunk; ++cc) {
+      cp_async4(dst, src, (in && cc < nc) ? 4u : 0u);
+      src += step;
+      dst += chan_b;
+    }
+  }
+  const uint32_t wbase = raw_base + g.raw_x_bytes;
+  const uint32_t cbase = wbase + g.ng * kWRawSlot;
+  for (int j = 0; j < g.ng; ++j) {
+    const uint4 d = desc[2 * (j * g.cps + kk)];
+    if ((uint32_t)ptid < d.y)
+      asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(wbase + j * kWRawSlot + ptid * 8),
+                   "l"(reinterpret_cast<const uint2*>(L.wvals) + d.x + ptid)
+                   : "memory");
+    if ((uint32_t)ptid * 16 < d.w) cp_async16(cbase + j * kCodeSlot + ptid * 16, codes + d.z + ptid * 16);
+  }
+}
+
+template <int S>
+__device__ __forceinline__ void widen_raw(const Geo& g, const StagedElem (&pre)[kPreElems],
+                                          const uint4* desc, uint32_t raw_base, uint32_t stage_base,
+                                          int kk, int ptid) {
+  constexpr int kRows = (S == 1) ? 6 : 9;
   const int n_elem = g.pairs * g.rows * g.pitch;
-  const size_t chan_off = (size_t)c0 * hw;
-  auto copy_two = [&](const StagedElem& s0, const StagedElem& s1, bool two) {
-    float va[2][kChunk], vb[2][kChunk];
+  const uint32_t raw_chan = (uint32_t)(kRows * g.raw_pitch * 2);
+  auto widen = [&](const StagedElem& se) {
+    uint32_t va[kChunk], vb[kChunk];
 #pragma unroll
     for (int cc = 0; cc < kChunk; ++cc) {
-      va[0][cc] = (s0.off_a >= 0 && cc < nc) ? ldg_f(x + s0.off_a + chan_off + cc * hw) : 0.f;
-      vb[0][cc] = (s0.off_b >= 0 && cc < nc) ? ldg_f(x + s0.off_b + chan_off + cc * hw) : 0.f;
-      va[1][cc] = (two && s1.off_a >= 0 && cc < nc) ? ldg_f(x + s1.off_a + chan_off + cc * hw) : 0.f;
-      vb[1][cc] = (two && s1.off_b >= 0 && cc < nc) ? ldg_f(x + s1.off_b + chan_off + cc * hw) : 0.f;
+      va[cc] = lds_u16(raw_base + (uint32_t)se.off_a + cc * raw_chan);
+      vb[cc] = lds_u16(raw_base + (uint32_t)se.off_b + cc * raw_chan);
     }
 #pragma unroll
     for (int cc = 0; cc < kChunk; ++cc) {
-      sts64f(stage_base + s0.dst + (uint32_t)(cc * g.chan_stride), va[0][cc], vb[0][cc]);
-      if (two) sts64f(stage_base + s1.dst + (uint32_t)(cc * g.chan_stride), va[1][cc], vb[1][cc]);
+      const uint32_t pk = va[cc] | (vb[cc] << 16);
+      const __half2 h = *reinterpret_cast<const __half2*>(&pk);
+      sts64f(stage_base + se.dst + (uint32_t)(cc * g.chan_stride), __low2float(h), __high2float(h));
     }
   };
 #pragma unroll
-  for (int i = 0; i < kPreElems; i += 2)
-    if (pre[i].dst != kSkipElem) copy_two(pre[i], pre[i + 1], pre[i + 1].dst != kSkipElem);
-  for (int e = ptid + kPreElems * kProducerThreads; e < n_elem; e += 2 * kProducerThreads) {
-    const StagedElem s0 = staged_elem<S>(L, g, tab, e, 0);
-    const bool two = e + kProducerThreads < n_elem;
-    const StagedElem s1 = two ? staged_elem<S>(L, g, tab, e + kProducerThreads, 0) : s0;
-    copy_two(s0, s1, two);
+  for (int i = 0; i < kPreElems; ++i)
+    if (pre[i].dst != kSkipElem) widen(pre[i]);
+  for (int e = ptid + kPreElems * kProducerThreads; e < n_elem; e += kProducerThreads) widen(raw_elem<S>(g, e));
+  const uint32_t rw = raw_base + g.raw_x_bytes, rc = rw + g.ng * kWRawSlot;
+  const uint32_t wbase = stage_base + g.x_stage_bytes, cbase = wbase + g.ng * kWSlot;
+  for (int j = 0; j < g.ng; ++j) {
+    const uint4 d = desc[2 * (j * g.cps + kk)];
+    if ((uint32_t)ptid < d.y) {
+      const u64 raw = lds64(rw + j * kWRawSlot + ptid * 8);
+      const uint32_t lo32 = (uint32_t)raw, hi32 = (uint32_t)(raw >> 32);
+      const __half2 lo = *reinterpret_cast<const __half2*>(&lo32);
+      const __half2 hi = *reinterpret_cast<const __half2*>(&hi32);
+      sts128f(wbase + j * kWSlot + ptid * 16, __low2float(lo), __high2float(lo), __low2float(hi),
+              __high2float(hi));
+    }
+    if ((uint32_t)ptid * 16 < d.w) {
+      uint32_t c0, c1, c2, c3;
+      asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                   : "=r"(c0), "=r"(c1), "=r"(c2), "=r"(c3)
+                   : "r"(rc + j * kCodeSlot + ptid * 16));
+      asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(cbase + j * kCodeSlot + ptid * 16),
+                   "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+                   : "memory");
+    }
   }
-  if (with_blocks) stage_blocks_half(L, g, desc, codes, stage_base, kk, ptid);
+}
+
+// The producers' loop of the raw-ring path.  Every producer thread passes through every named
+// barrier of every chunk, also after a bounded wait ran out (it then does no more work), so the
+// barrier counts always match.
+template <int S>
+__device__ __forceinline__ void produce_raw_stream(const DeviceLayer& L, const Geo& g,
+                                                   const __half* __restrict__ x, const SubTile* tab,
+                                                   const StagedElem (&pre)[kPreElems], const uint4* desc,
+                                                   const uint8_t* codes, uint32_t sbase, int k0, int nk,
+                                                   int ptid) {
+  const int R = g.raw_stages;
+  bool ok = true;
+  auto raw_base = [&](int kk) { return sbase + g.raw_off + (kk % R) * g.raw_slot; };
+  auto producers_sync = [] { asm volatile("bar.sync 2, %0;" ::"n"(kProducerThreads) : "memory"); };
+  // one cp.async group per chunk (empty past the last chunk), R - 1 chunks ahead of the one being
+  // widened, so "all but the newest R - 1 groups" is exactly "chunk kk has landed"
+  for (int j = 0; j < R - 1; ++j) {
+    if (j < nk) issue_raw<S>(L, g, x, tab, desc, codes, raw_base(j), k0 + j, j, ptid);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  }
+  for (int kk = 0; kk < nk; ++kk) {
+    const int ahead = kk + R - 1;
+    if (ok && ahead < nk) issue_raw<S>(L, g, x, tab, desc, codes, raw_base(ahead), k0 + ahead, ahead, ptid);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    if (R >= 3) asm volatile("cp.async.wait_group 2;" ::: "memory");
+    else if (R == 2) asm volatile("cp.async.wait_group 1;" ::: "memory");
+    else asm volatile("cp.async.wait_group 0;" ::: "memory");
+    producers_sync();   // everybody's copies of chunk kk have landed
+    const int s = kk % g.stages, it = kk / g.stages;
+    if (ok && it > 0) ok = mbar_wait(sbase + 8 * (kMaxStages + s), (it - 1) & 1, L.err, 1);
+    if (ok) {
+      widen_raw<S>(g, pre, desc, raw_base(kk), sbase + g.stage_off + s * g.stage_bytes, kk, ptid);
+      mbar_arrive(sbase + 8 * s);
+    }
+    producers_sync();   // the raw slot may be overwritten
+  }
+}
+
+// fp16 storage: loads, converts to fp32 and stores (the interleaved fp32 layout cannot be produced
+// by an asynchronous copy of 2-byte elements).  The loads of a batch (two staged elements x 8
+// channels x {A,B}) are issued before the previous batch is converted and stored, across chunk
+// boundaries too, so a thread always has loads in flight; the ring slot is only waited for when a
+// chunk's first store is due.  Returns false if a bounded wait ran out.
+struct HalfBatch {
+  uint32_t raw[2][kChunk];   // {A, B} halves of one staged element and channel
+  uint32_t dst[2];           // byte offset in the channel's staged block, kSkipElem = none
+};
+
+template <int S>
+__device__ __forceinline__ bool produce_half_stream(const DeviceLayer& L, const Geo& g,
+                                                    const __half* __restrict__ x, const SubTile* tab,
+                                                    const StagedElem (&pre)[kPreElems], const uint4* desc,
+                                                    const uint8_t* codes, uint32_t sbase, int k0, int nk,
+                                                    int n_early, int ptid) {
+  const size_t hw = (size_t)g.h * g.w;
+  const int n_elem = g.pairs * g.rows * g.pitch;
+  const int nb = ((n_elem + kProducerThreads - 1) / kProducerThreads + 1) / 2;  // batches per chunk
+  const unsigned short* xs = reinterpret_cast<const unsigned short*>(x);
+  auto issue = [&](HalfBatch& bt, int kk, int b) {
+    const int c0 = (k0 + kk) * kChunk;
+    const int nc = min(kChunk, L.c_in - c0);
+    const size_t chan_off = (size_t)c0 * hw;
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int i = 2 * b + u, e = ptid + i * kProducerThreads;
+      StagedElem se;
+      se.off_a = se.off_b = -1;
+      se.dst = kSkipElem;
+      if (e < n_elem) {
+        if (i < kPreElems) {
+#pragma unroll
+          for (int j = 0; j < kPreElems; ++j)   // static indices keep `pre` in registers
+            if (i == j) se = pre[j];
+        } else {
+          se = staged_elem<S>(L, g, tab, e, 0);
+        }
+      }
+      bt.dst[u] = se.dst;
+#pragma unroll
+      for (int cc = 0; cc < kChunk; ++cc) {
+        const uint32_t va = (se.off_a >= 0 && cc < nc) ? (uint32_t)__ldg(xs + se.off_a + chan_off + cc * hw) : 0u;
+        const uint32_t vb = (se.off_b >= 0 && cc < nc) ? (uint32_t)__ldg(xs + se.off_b + chan_off + cc * hw) : 0u;
+        bt.raw[u][cc] = va | (vb << 16);
+      }
+    }
+  };
+  auto store = [&](const HalfBatch& bt, uint32_t stage_base) {
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      if (bt.dst[u] == kSkipElem) continue;
+#pragma unroll
+      for (int cc = 0; cc < kChunk; ++cc) {
+        const __half2 h = *reinterpret_cast<const __half2*>(&bt.raw[u][cc]);
+        sts64f(stage_base + bt.dst[u] + (uint32_t)(cc * g.chan_stride), __low2float(h), __high2float(h));
+      }
+    }
+  };
+  HalfBatch cur, nxt;
+#ifdef PCONV_TRACE
+  long long t_pwait = 0;
+  const long long t_p0 = clock64();
+#endif
+  issue(cur, 0, 0);
+  for (int kk = 0; kk < nk; ++kk) {
+    const int s = kk % g.stages, it = kk / g.stages;
+    const uint32_t stage_base = sbase + g.stage_off + s * g.stage_bytes;
+    for (int b = 0; b < nb; ++b) {
+      const bool last = b + 1 == nb;
+      const int kk2 = last ? kk + 1 : kk, b2 = last ? 0 : b + 1;
+      if (kk2 < nk) issue(nxt, kk2, b2);
+#ifdef PCONV_TRACE
+      const long long tw0 = clock64();
+#endif
+      if (b == 0 && it > 0 && !mbar_wait(sbase + 8 * (kMaxStages + s), (it - 1) & 1, L.err, 1)) return false;
+#ifdef PCONV_TRACE
+      t_pwait += clock64() - tw0;
+#endif
+      store(cur, stage_base);
+      cur = nxt;
+    }
+    if (kk >= n_early) stage_blocks_half(L, g, desc, codes, stage_base, kk, ptid);
+    mbar_arrive(sbase + 8 * s);
+  }
+#ifdef PCONV_TRACE
+  if (ptid == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {
+    ((unsigned long long*)(L.err + 2))[4] = (unsigned long long)t_pwait;
+    ((unsigned long long*)(L.err + 2))[6] = (unsigned long long)(clock64() - t_p0);
+  }
+#endif
+  return true;
 }
 
 __device__ __forceinline__ void red_add_f32(float* p, float v) {
@@ -771,38 +991,46 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
 
   if (warp >= kCW) {
     // ===================================== producer warps =====================================
-    if (GENERIC) asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
     const int ptid = (warp - kCW) * 32 + lane;
     const uint8_t* codes = GENERIC ? L.codes_g : L.codes_s;
     StagedElem pre[kPreElems];
-    if (S == 1) precompute_elems<1>(pre, L, g, tab, ptid); else precompute_elems<2>(pre, L, g, tab, ptid);
-    // the weight records and codes of the first ring-full of chunks do not depend on the previous
-    // kernel: fetch them while it finishes
-    const int n_early = min(g.stages, nk);
-    for (int kk = 0; kk < n_early; ++kk) {
-      const uint32_t stage_base = sbase + g.stage_off + kk * g.stage_bytes;
-      if (g.is_half) stage_blocks_half(L, g, desc, codes, stage_base, kk, ptid);
-      else stage_blocks_async(L, g, desc, codes, stage_base, kk, ptid);
-    }
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    for (int kk = 0; kk < nk; ++kk) {
-      const int s = kk % g.stages, it = kk / g.stages;
-      if (it > 0 && !mbar_wait(sbase + 8 * (kMaxStages + s), (it - 1) & 1, L.err, 1)) break;
-      const uint32_t stage_base = sbase + g.stage_off + s * g.stage_bytes;
+    if (g.raw_stages > 0) {
+      const int n_elem = g.pairs * g.rows * g.pitch;
+#pragma unroll
+      for (int i = 0; i < kPreElems; ++i) {
+        const int e = ptid + i * kProducerThreads;
+        pre[i] = raw_elem<S>(g, e < n_elem ? e : 0);
+        if (e >= n_elem) pre[i].dst = kSkipElem;
+      }
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      produce_raw_stream<S>(L, g, (const __half*)x, tab, pre, desc, codes, sbase, k0, nk, ptid);
+    } else {
+      precompute_elems<S>(pre, L, g, tab, ptid);
+      // the weight records and codes of the first ring-full of chunks do not depend on the previous
+      // kernel: fetch them while it finishes
+      const int n_early = min(g.stages, nk);
+      for (int kk = 0; kk < n_early; ++kk) {
+        const uint32_t stage_base = sbase + g.stage_off + kk * g.stage_bytes;
+        if (g.is_half) stage_blocks_half(L, g, desc, codes, stage_base, kk, ptid);
+        else stage_blocks_async(L, g, desc, codes, stage_base, kk, ptid);
+      }
+      asm volatile("griddepcontrol.wait;" ::: "memory");
       if (g.is_half) {
-        produce_chunk_half<S>(L, g, (const __half*)x, tab, pre, desc, codes, stage_base, k0 + kk, kk, ptid,
-                              kk >= n_early);
-        mbar_arrive(sbase + 8 * s);
+        produce_half_stream<S>(L, g, (const __half*)x, tab, pre, desc, codes, sbase, k0, nk, n_early, ptid);
       } else {
-        produce_chunk_async<S>(L, g, (const float*)x, tab, pre, desc, codes, stage_base, k0 + kk, kk, ptid,
-                               kk >= n_early);
-        cp_async_arrive(sbase + 8 * s);
+        for (int kk = 0; kk < nk; ++kk) {
+          const int s = kk % g.stages, it = kk / g.stages;
+          if (it > 0 && !mbar_wait(sbase + 8 * (kMaxStages + s), (it - 1) & 1, L.err, 1)) break;
+          const uint32_t stage_base = sbase + g.stage_off + s * g.stage_bytes;
+          produce_chunk_async<S>(L, g, (const float*)x, tab, pre, desc, codes, stage_base, k0 + kk, kk, ptid,
+                                 kk >= n_early);
+          cp_async_arrive(sbase + 8 * s);
+        }
       }
     }
     asm volatile("cp.async.wait_all;" ::: "memory");
   } else {
     // ===================================== consumer warps =====================================
-    if (GENERIC) asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
     if constexpr (GENERIC) {
 #pragma unroll
       for (int a = 0; a < kGroup; ++a)
@@ -956,6 +1184,27 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   PCONV_MARK_MAX(7)
 }
 
+// Places descriptors, the raw ring (if any) and the stages for `cps` chunks per CTA, and picks the
+// ring depth; false if nothing fits.
+int pick_stages(int fit, int zs, int cps);
+bool place_stages(Geo* g, int n_chunks_total, int cps, bool want_raw, int stride) {
+  g->stage_off = g->desc_off + g->ng * cps * 32;
+  g->raw_stages = 0;
+  g->raw_off = g->stage_off;
+  g->raw_slot = g->raw_pitch = g->raw_x_bytes = 0;
+  if (want_raw) {
+    g->raw_pitch = (stride == 1) ? g->tw + 4 : 2 * g->tw + 2;   // halves per raw row (even)
+    g->raw_x_bytes = g->pairs * 2 * kChunk * g->rows * g->raw_pitch * 2;
+    g->raw_slot = (g->raw_x_bytes + g->ng * (kWRawSlot + kCodeSlot) + 15) & ~15;
+    g->raw_stages = kRawStages < cps ? kRawStages : cps;
+    g->stage_off += g->raw_stages * g->raw_slot;
+  }
+  (void)n_chunks_total;
+  g->stages = pick_stages((kSmemLimit - g->stage_off) / g->stage_bytes, g->zs, cps);
+  if (g->stages < 1 && want_raw) return place_stages(g, n_chunks_total, cps, false, stride);
+  return g->stages >= 1;
+}
+
 // Depth of the staging ring when `fit` stages fit in shared memory (0 = the geometry is not
 // usable).  The zs warps of a unit work on different chunks at the same time, so the ring holds at
 // least zs (then a warp that draws chunk k knows that chunk k - stages has been consumed, which
@@ -1024,9 +1273,7 @@ bool geo_for(const DeviceLayer& L, int n, int h, int w, int zs, Geo* out) {
     g.x_stage_bytes = kChunk * g.chan_stride;
     g.stage_bytes = (g.x_stage_bytes + g.ng * (kWSlot + kCodeSlot) + 15) & ~15;
     g.desc_off = (g.tab_off + 2 * g.pairs * (int)sizeof(SubTile) + 15) & ~15;
-    g.stage_off = g.desc_off + g.ng * L.n_chunks * 32;
-    g.stages = pick_stages((kSmemLimit - g.stage_off) / g.stage_bytes, zs, g.cps);
-    if (g.stages > 0) break;
+    if (place_stages(&g, L.n_chunks, g.cps, L.storage == PCONV_F16 && (w % 2) == 0, L.stride)) break;
     if (g.wy > 1) {
       g.wy /= 2;          // fewer pixel sets (the other warp rows idle)
     } else if (g.ng > 1) {
@@ -1056,9 +1303,7 @@ void set_split(const DeviceLayer& L, Geo* g, int ks) {
   if (ks > L.n_chunks) ks = L.n_chunks;
   g->cps = (L.n_chunks + ks - 1) / ks;
   g->ks = (L.n_chunks + g->cps - 1) / g->cps;
-  g->stage_off = g->desc_off + g->ng * g->cps * 32;
-  const int stages = pick_stages((kSmemLimit - g->stage_off) / g->stage_bytes, g->zs, g->cps);
-  g->stages = stages;
+  if (!place_stages(g, L.n_chunks, g->cps, g->raw_stages > 0, L.stride)) g->stages = 0;
 }
 
 // Estimated duration of a launch in units of one kernel (4 taps on a warp's 256 pixels, about
