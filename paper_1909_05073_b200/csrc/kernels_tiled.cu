@@ -57,7 +57,7 @@ constexpr int kRawStages = 3;
 constexpr uint32_t kSpinLimit = 1u << 20;
 // A waiting warp is suspended by the hardware for up to this long per try (it is woken when the
 // phase completes), so that waiting warps leave the issue slots to the warps that have work.
-constexpr uint32_t kWaitHintNs = 2000;
+constexpr uint32_t kWaitHintNs = 200;
 constexpr int kSmemLimit = 227 * 1024;
 constexpr int kNumSMs = 148;
 
