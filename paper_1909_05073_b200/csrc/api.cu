@@ -85,10 +85,10 @@ extern "C" pconv_status pconv_forward_ws(const pconv_handle* h, const void* x, c
     e = launch_simple(L, x, bias, y, n, h_in, w_in, relu, stream);
   } else if (sel == PCONV_KERNEL_TILED || sel == PCONV_KERNEL_GENERIC_TAPS) {
     if (!tiled_supported(L, n, h_in, w_in)) return PCONV_ERR_UNSUPPORTED;
-    const bool generic = (sel == PCONV_KERNEL_GENERIC_TAPS) || !h->canonical;
+    const bool generic = (sel == PCONV_KERNEL_GENERIC_TAPS);
     e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, pool, generic, ws, ws_bytes, stream);
   } else if (tiled_supported(L, n, h_in, w_in)) {
-    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, pool, !h->canonical, ws, ws_bytes, stream);
+    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, pool, false, ws, ws_bytes, stream);
   } else {
     e = launch_simple(L, x, bias, y, n, h_in, w_in, relu, stream);
   }

@@ -51,7 +51,7 @@ __host__ __device__ constexpr int cta_threads(bool generic) {
 constexpr int kTmemCols = 512;  // whole TMEM of the SM: 16 warps x 16 slots x 8 columns
 constexpr int kMaxStages = 8;
 constexpr int kWSlot = kMaxBlockKernels * 16 + 16;  // bytes per (group, stage): 4 fp32 per kernel
-constexpr int kCodeSlot = 288;                 // bytes per (group, stage)
+constexpr int kCodeSlot = 400;                 // bytes per (group, stage): <= 24 records of 7 codes
 constexpr int kWRawSlot = kMaxBlockKernels * 8;  // fp16 weight records of one (group, chunk)
 constexpr int kRawStages = 3;
 constexpr uint32_t kSpinLimit = 1u << 20;
@@ -190,6 +190,26 @@ __device__ __forceinline__ void dispatch_chunk(uint32_t cp, uint32_t wp, uint32_
   } else {
     asm volatile(
 #include "dispatch_s2.inc"
+        :
+        : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(col_b), "r"(off_mid), "r"(tq), "r"(entry_code)
+        : "memory");
+  }
+}
+// The same loop for wide codes (a body for every 4-of-9 mask); only the kernel instantiations for
+// non-canonical pattern sets contain it, so the canonical kernels stay compact.
+template <int S>
+__device__ __forceinline__ void dispatch_chunk_wide(uint32_t cp, uint32_t wp, uint32_t xptr,
+                                                 uint32_t chan_b, uint32_t col_b, uint32_t off_mid,
+                                                 uint32_t tq, uint32_t entry_code) {
+  if (S == 1) {
+    asm volatile(
+#include "dispatch_s1w.inc"
+        :
+        : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(col_b), "r"(off_mid), "r"(tq), "r"(entry_code)
+        : "memory");
+  } else {
+    asm volatile(
+#include "dispatch_s2w.inc"
         :
         : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(col_b), "r"(off_mid), "r"(tq), "r"(entry_code)
         : "memory");
@@ -878,7 +898,7 @@ __device__ __forceinline__ void finalize_outputs(const Geo& g, const LaneOut& lo
   }
 }
 
-template <int S, bool GENERIC>
+template <int S, bool GENERIC, bool WIDE>
 __global__ void __launch_bounds__(cta_threads(GENERIC), 1)
 tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
              const float* __restrict__ bias, void* __restrict__ y, float* __restrict__ ws,
@@ -1073,8 +1093,10 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
         uint32_t cp = stage_base + g.x_stage_bytes + g.ng * kWSlot + wgi * kCodeSlot;
         if constexpr (!GENERIC) {
           const uint4 d0 = desc[2 * (wgi * g.cps + kk)], d1 = desc[2 * (wgi * g.cps + kk) + 1];
-          if (d0.y)  // the block has kernels: enter at its first channel
-            dispatch_chunk<S>(cp, wp, xptr, chan_b, col_b, off_mid, tq, (d1.z + 1u) << 4);
+          if (d0.y) {  // the block has kernels: enter at its first channel
+            if constexpr (WIDE) dispatch_chunk_wide<S>(cp, wp, xptr, chan_b, col_b, off_mid, tq, (d1.z + 1u) << 8);
+            else dispatch_chunk<S>(cp, wp, xptr, chan_b, col_b, off_mid, tq, (d1.z + 1u) << 4);
+          }
         } else {
           u64 win[Win<S>::kRows][3];
 #pragma unroll
@@ -1368,14 +1390,14 @@ bool make_geo(const DeviceLayer& L, int n, int h, int w, bool allow_split, Geo* 
   return found;
 }
 
-template <int S, bool GENERIC>
+template <int S, bool GENERIC, bool WIDE>
 cudaError_t launch_one(const DeviceLayer& L, Geo g, const void* x, const float* bias, void* y, float* ws,
                        int* counters, cudaStream_t stream) {
   int smem = g.stage_off + g.stages * g.stage_bytes;
   // the TMEM variant must be alone on its SM (it takes all 512 columns): make sure two CTAs can
   // never be co-resident by asking for more than half of the shared memory
   if (!GENERIC && smem < 120 * 1024) smem = 120 * 1024;
-  cudaError_t e = cudaFuncSetAttribute(tiled_kernel<S, GENERIC>,
+  cudaError_t e = cudaFuncSetAttribute(tiled_kernel<S, GENERIC, WIDE>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
   if (e != cudaSuccess) return e;
   const long long ctas_x = ((long long)g.q_total + 2 * g.pairs - 1) / (2 * g.pairs);
@@ -1391,7 +1413,7 @@ cudaError_t launch_one(const DeviceLayer& L, Geo g, const void* x, const float* 
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, tiled_kernel<S, GENERIC>, L, g, x, bias, y, ws, counters);
+  return cudaLaunchKernelEx(&cfg, tiled_kernel<S, GENERIC, WIDE>, L, g, x, bias, y, ws, counters);
 }
 
 size_t out_elems(const DeviceLayer& L, int n, int h, int w) {
@@ -1458,11 +1480,15 @@ cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias,
     wsf = (float*)ws;
     counters = (int*)((char*)ws + ((out_elems(L, n, h, w) * 4 + 255) & ~(size_t)255));
   }
-  if (L.stride == 1)
-    return generic_taps ? launch_one<1, true>(L, g, x, bias, y, wsf, counters, stream)
-                        : launch_one<1, false>(L, g, x, bias, y, wsf, counters, stream);
-  return generic_taps ? launch_one<2, true>(L, g, x, bias, y, wsf, counters, stream)
-                      : launch_one<2, false>(L, g, x, bias, y, wsf, counters, stream);
+  const bool wide = L.wide_codes != 0;
+  if (L.stride == 1) {
+    if (generic_taps) return launch_one<1, true, false>(L, g, x, bias, y, wsf, counters, stream);
+    return wide ? launch_one<1, false, true>(L, g, x, bias, y, wsf, counters, stream)
+                : launch_one<1, false, false>(L, g, x, bias, y, wsf, counters, stream);
+  }
+  if (generic_taps) return launch_one<2, true, false>(L, g, x, bias, y, wsf, counters, stream);
+  return wide ? launch_one<2, false, true>(L, g, x, bias, y, wsf, counters, stream)
+              : launch_one<2, false, false>(L, g, x, bias, y, wsf, counters, stream);
 }
 
 }  // namespace pconv

@@ -160,10 +160,8 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
     h->canonical = true;
     for (int p = 0; p < n_patterns; ++p) {
       h->patterns[p] = patterns[p];
-      h->canon_id[p] = -1;
-      for (int q = 0; q < 8; ++q)
-        if (kCanonMasks[q] == patterns[p]) h->canon_id[p] = q;
-      if (h->canon_id[p] < 0) h->canonical = false;
+      h->body_id[p] = body_index(patterns[p]);
+      if (h->body_id[p] >= 8) h->canonical = false;
     }
     h->n_kept = n_kept;
 
@@ -237,18 +235,24 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
         std::memset(&bd, 0, sizeof(bd));
         bd.w_off = (uint32_t)((storage == PCONV_F16 ? wv16.size() : wv32.size()) / 4);
         bd.n_k = (uint32_t)items.size();
-        while (codes_s.size() % 16) codes_s.push_back(kCodeEnd);
         while (codes_g.size() % 16) codes_g.push_back(0);
         bd.cs_off = (uint32_t)codes_s.size();
         bd.cg_off = (uint32_t)codes_g.size();
         // Specialised stream: 16-byte records, each a run of kernel codes closed by a terminator
         // (advance to another channel's window, or end); the kernel reads a record with one load.
         // Nothing precedes the first kernel: the descriptor names its channel (`first_ch`).
-        std::vector<uint8_t> rec;
-        auto close_record = [&](uint8_t terminator) {
+        // Canonical sets use one-byte codes (15 to a record), any other set two-byte codes (7 to a
+        // record) that can name every mask's body.
+        const bool wide = !h->canonical;
+        const int per_record = wide ? kWideCodesPerRecord : kCodesPerRecord;
+        std::vector<uint16_t> rec;
+        auto close_record = [&](uint16_t terminator) {
           rec.push_back(terminator);
-          while (rec.size() < 16) rec.push_back((uint8_t)kCodeEnd);
-          codes_s.insert(codes_s.end(), rec.begin(), rec.end());
+          while ((int)rec.size() < per_record) rec.push_back((uint16_t)(wide ? kWideEnd : kCodeEnd));
+          for (uint16_t c : rec) {
+            codes_s.push_back((uint8_t)(c & 0xFF));
+            if (wide) codes_s.push_back((uint8_t)(c >> 8));
+          }
           rec.clear();
         };
         bd.first_ch = items.empty() ? 0u : (uint32_t)(items.front().c - c0);
@@ -263,12 +267,15 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
             pos_g = it.c;
           }
           if (it.c != pos_s) {
-            if (pos_s >= 0) close_record((uint8_t)(((it.c - pos_s) << 4) | kCodeNext));
+            if (pos_s >= 0)
+              close_record(wide ? (uint16_t)(((it.c - pos_s) << 8) | kWideAdv)
+                                : (uint16_t)(((it.c - pos_s) << 4) | kCodeNext));
             pos_s = it.c;
           }
-          if (rec.size() == 15) close_record((uint8_t)kCodeNext);  // same channel, next record
-          const int canon = h->canon_id[it.r->pid];
-          rec.push_back((uint8_t)((it.slot << 4) | (canon < 0 ? 0 : canon)));
+          if ((int)rec.size() == per_record - 1)   // same channel, next record
+            close_record((uint16_t)(wide ? kWideCont : kCodeNext));
+          rec.push_back(wide ? (uint16_t)((it.slot << 8) | (kWideBody0 + h->body_id[it.r->pid]))
+                             : (uint16_t)((it.slot << 4) | h->body_id[it.r->pid]));
           const uint16_t cg = (uint16_t)((it.slot << 9) | patterns[it.r->pid]);
           codes_g.push_back((uint8_t)(cg & 0xFF));
           codes_g.push_back((uint8_t)(cg >> 8));
@@ -277,7 +284,7 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
           else
             wv32.insert(wv32.end(), it.r->v, it.r->v + 4);
         }
-        close_record((uint8_t)kCodeEnd);
+        close_record((uint16_t)(wide ? kWideEnd : kCodeEnd));
         codes_g.push_back((uint8_t)(kGenEnd & 0xFF));
         codes_g.push_back((uint8_t)(kGenEnd >> 8));
         bd.cs_len = (uint32_t)codes_s.size() - bd.cs_off;
@@ -285,7 +292,7 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
       }
     }
     // slack so that a staged block may be read in whole 16-byte pieces
-    for (int i = 0; i < 32; ++i) { codes_s.push_back(kCodeEnd); codes_g.push_back(0); }
+    for (int i = 0; i < 32; ++i) { codes_s.push_back(0); codes_s.push_back(0); codes_g.push_back(0); }
     for (int i = 0; i < 8; ++i) { wv32.push_back(0.f); wv16.push_back(0); }
 
     // ---- one device allocation, sub-buffers 256-byte aligned ------------------------------------
@@ -341,7 +348,8 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
     d.csr_val = (const float*)(dev + parts[i_cv].off);
     d.blocks = (const BlockDesc*)(dev + parts[i_bl].off);
     d.wvals = dev + parts[i_wv].off;
-    d.codes_s = h->canonical ? (const uint8_t*)(dev + parts[i_cs].off) : nullptr;
+    d.codes_s = (const uint8_t*)(dev + parts[i_cs].off);
+    d.wide_codes = h->canonical ? 0 : 1;
     d.codes_g = (const uint8_t*)(dev + parts[i_cg].off);
     d.perm = (const int*)(dev + parts[i_pm].off);
     d.err = (int*)(dev + parts[i_er].off);

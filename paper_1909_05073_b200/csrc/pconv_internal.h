@@ -13,24 +13,54 @@ constexpr int kGroup = 16;         // filters per group (accumulator slots of on
 constexpr int kChunk = 8;          // input channels per pipeline stage
 constexpr int kMaxBlockKernels = kGroup * kChunk;
 
-// Specialised code stream -- valid when the pattern set is a subset of the eight masks the tiled
-// kernel has straight-line bodies for.  A (group, chunk) block is a sequence of 16-byte records;
-// a record is a run of kernel codes closed by one terminator (unused bytes repeat the end code):
+// Specialised code stream (the tiled kernel with Tensor-Memory accumulators).  A (group, chunk) block
+// is a sequence of 16-byte records; a record is a run of kernel codes closed by one terminator.
+// Nothing precedes a block's first kernel: the block descriptor names its channel, and the kernel
+// loads that channel's window before it reads the first record.
+//
+// Narrow codes (one byte, 15 kernels to a record) -- pattern sets inside the canonical eight:
 //   low nibble 0..7   kernel: canonical pattern id; high nibble = filter slot
 //   low nibble 8      terminator: advance (high nibble, 0..8) channels inside the chunk, load that
 //                     channel's window and continue with the next record
-//   9                 terminator: end of the block
-// Nothing precedes a block's first kernel: the block descriptor names its channel, and the kernel
-// loads that channel's window before it reads the first record.
+//   9                 terminator: end of the block (also fills unused bytes)
 constexpr int kCodeNext = 8;
 constexpr int kCodeEnd = 9;
+constexpr int kCodesPerRecord = 16;
+// Wide codes (two bytes, 7 kernels to a record) -- any other set of 4-of-9 masks:
+//   low byte 0        terminator: advance (high byte, 0..8) channels, load that channel's window
+//                     and continue with the next record
+//   low byte 1        terminator: end of the block (also fills unused entries)
+//   low byte 2        terminator: the channel's kernels continue in the next record
+//   low byte 3..128   kernel: kWideBody0 + index of the body for its mask (body_index()); high
+//                     byte = filter slot
+constexpr int kWideAdv = 0;
+constexpr int kWideEnd = 1;
+constexpr int kWideCont = 2;
+constexpr int kWideBody0 = 3;
+constexpr int kWideCodesPerRecord = 8;
 // Generic code stream (two bytes per entry) -- any 4-of-9 mask.
 //   (g << 9) | mask   kernel with run-time mask;   0x2000 | (adv-1)   advance;   0x4000   end
 constexpr int kGenNext = 0x2000;
 constexpr int kGenEnd = 0x4000;
 
-// The eight masks with specialised bodies, in canonical order (bit 3u+v).
+// The eight masks whose bodies come first, in canonical order (bit 3u+v); the bodies of all other
+// masks with four bits follow in ascending order of the mask (the generated dispatch code
+// enumerates them the same way).
 constexpr uint16_t kCanonMasks[8] = {0x03A, 0x09A, 0x0B8, 0x0B2, 0x01B, 0x036, 0x0D8, 0x1B0};
+inline int body_index(uint16_t mask) {
+  for (int q = 0; q < 8; ++q)
+    if (kCanonMasks[q] == mask) return q;
+  int idx = 8;
+  for (int m = 0; m < 512; ++m) {
+    if (__builtin_popcount(m) != 4) continue;
+    bool canon = false;
+    for (int q = 0; q < 8; ++q) canon = canon || kCanonMasks[q] == m;
+    if (canon) continue;
+    if (m == mask) return idx;
+    ++idx;
+  }
+  return -1;
+}
 
 struct BlockDesc {      // one per (group, chunk); 32 bytes
   uint32_t w_off;       // first kernel record of the block in the value stream
@@ -51,11 +81,12 @@ struct DeviceLayer {         // device pointers of one packed layer (passed to k
   // grouped / chunked streams (tiled kernel)
   const BlockDesc* blocks;   // [n_groups][n_chunks]
   const void* wvals;         // 4 values per kernel: fp32 (16 B) or fp16 (8 B)
-  const uint8_t* codes_s;    // specialised codes (may be null)
+  const uint8_t* codes_s;    // specialised codes (narrow or wide, see wide_codes)
   const uint8_t* codes_g;    // generic codes
   const int* perm;           // [n_groups * kGroup] original filter index or -1
   int* err;                  // device status word (0 = fine)
   int c_out, c_in, stride, storage, n_groups, n_chunks;
+  int wide_codes;            // 0 = narrow codes (canonical set), 1 = wide codes
   long long n_kept;          // surviving kernels of the layer
 };
 
@@ -66,8 +97,8 @@ struct pconv_handle {
   int device;
   int n_patterns;
   uint16_t patterns[PCONV_MAX_PATTERNS];
-  int canon_id[PCONV_MAX_PATTERNS];  // canonical index of each pattern or -1
-  bool canonical;
+  int body_id[PCONV_MAX_PATTERNS];   // body index of each pattern
+  bool canonical;                    // every pattern is one of the canonical eight
   pconv_stats_t stats;
   long long n_kept;
   size_t wvals_bytes, codes_s_bytes, codes_g_bytes;

@@ -1,5 +1,8 @@
 """One synthetic layer, a warm-up launch and `reps` timed launches: the small case used for ncu
-captures (`python -m paper_1909_05073_b200.profile_case 64 64 56 32 1 0.35 [tiled|generic|simple] [f32|f16]`)."""
+captures and for the pattern-count sweep
+(`python -m paper_1909_05073_b200.profile_case 64 64 56 32 1 0.35 [tiled|generic|simple|auto] [f32|f16] [4|8|12]`;
+the last argument is the number of patterns in the set: the four designed ones, the canonical
+eight, or those plus four arbitrary masks, which only the run-time-mask kernel serves)."""
 import sys
 
 import numpy as np
@@ -9,20 +12,21 @@ from paper_1909_05073_b200 import binding as B
 from paper_1909_05073_b200 import synth
 
 
-def run(c_in, c_out, h, n, stride, keep, kernel="tiled", storage="f32", reps=3):
+def run(c_in, c_out, h, n, stride, keep, kernel="tiled", storage="f32", n_patterns=8, reps=3):
     sel = {"tiled": B.KERNEL_TILED, "generic": B.KERNEL_GENERIC_TAPS, "simple": B.KERNEL_SIMPLE,
            "auto": 0}[kernel]
     st = B.F16 if storage == "f16" else B.F32
     spec = synth.LayerSpec("p", c_in, c_out, h, h, stride, keep)
-    w, b, ids = synth.gen_weights(spec, 1)
-    layer = B.Layer(w, synth.PATTERNS8, stride, st, b)
+    patterns = {4: synth.SCP4, 8: synth.PATTERNS8, 12: synth.PATTERNS12}[int(n_patterns)]
+    w, b, ids = synth.gen_weights(spec, 1, patterns)
+    layer = B.Layer(w, patterns, stride, st, b)
     x = torch.from_numpy(synth.gen_input(spec, n, 1)).cuda()
     if st == B.F16:
         x = x.half()
     y = layer.forward(x, kernel=sel)
     torch.cuda.synchronize()
     us = []
-    for _ in range(reps):
+    for _ in range(int(reps)):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         layer.forward(x, kernel=sel, out=y)

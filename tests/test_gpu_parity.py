@@ -115,14 +115,43 @@ def test_empty_filters_and_no_bias(kernel):
     assert not got.any()
 
 
-@pytest.mark.parametrize("kernel", ["simple", "generic", "auto"])
-def test_twelve_patterns_and_noncanonical_sets(kernel):
-    spec = synth.LayerSpec("t", 24, 40, 18, 21, 1, 0.4, probs=(1 / 12,) * 12)
+@pytest.mark.parametrize("stride", [1, 2])
+@pytest.mark.parametrize("kernel", ["simple", "tiled", "generic", "auto"])
+def test_twelve_patterns_and_noncanonical_sets(kernel, stride):
+    spec = synth.LayerSpec("t", 24, 40, 18, 21, stride, 0.4, probs=(1 / 12,) * 12)
     wt, bias, ids = synth.gen_weights(spec, 5, synth.PATTERNS12)
     assert ids.max() == 11
     x = synth.gen_input(spec, 2, 5)
-    got = run_layer(wt, bias, x, kernel=kernel, patterns=synth.PATTERNS12)
-    check_close(got, oracle_layer(wt, bias, x), "f32", "12 patterns")
+    got = run_layer(wt, bias, x, stride=stride, kernel=kernel, patterns=synth.PATTERNS12)
+    check_close(got, oracle_layer(wt, bias, x, stride), "f32", "12 patterns")
+
+
+def all_masks_with_four_taps():
+    return [m for m in range(512) if bin(m).count("1") == 4]
+
+
+@pytest.mark.parametrize("stride", [1, 2])
+def test_every_one_of_the_126_masks_has_a_correct_body(stride):
+    """The tiled kernel holds one straight-line body per 4-of-9 mask: run them all, 14 masks to a
+    layer (pattern sets hold at most 16), every kernel carrying one tap weight per tap."""
+    masks = all_masks_with_four_taps()
+    assert len(masks) == 126
+    rng = np.random.default_rng(126 + stride)
+    for lo in range(0, len(masks), 14):
+        pats = tuple(masks[lo:lo + 14])
+        c_in, c_out, h, w, n = 10, 2 * len(pats), 9, 13, 2
+        wt = np.zeros((c_out, c_in, 3, 3), np.float32)
+        for o in range(c_out):
+            for c in range(c_in):
+                if rng.random() < 0.6:
+                    m = pats[(o + c) % len(pats)]
+                    for t in range(9):
+                        if m >> t & 1:
+                            wt[o, c, t // 3, t % 3] = rng.uniform(0.5, 1.5) * rng.choice([-1.0, 1.0])
+        bias = rng.normal(0, 0.1, c_out).astype(np.float32)
+        x = rng.uniform(-1, 1, (n, c_in, h, w)).astype(np.float32)
+        got = run_layer(wt, bias, x, stride=stride, kernel="tiled", patterns=pats)
+        check_close(got, oracle_layer(wt, bias, x, stride), "f32", "masks %d.." % lo)
 
 
 @pytest.mark.parametrize("storage", ["f32", "f16"])
