@@ -65,8 +65,10 @@ enum {
    * tests and benchmarks can pin one implementation; they never change the result beyond
    * summation order. */
   PCONV_KERNEL_SIMPLE = 0x100u, /* one thread per output, walks the per-filter kernel list */
-  PCONV_KERNEL_TILED = 0x200u,  /* shared-memory halo tiles, register-blocked FFMA2 path */
-  PCONV_KERNEL_GENERIC_TAPS = 0x400u /* tiled path with run-time 9-bit masks (any pattern set) */
+  PCONV_KERNEL_TILED = 0x200u,  /* shared-memory halo tiles, packed FMAs, one straight-line body per
+                                   pattern mask (any set of 4-of-9 masks); the default */
+  PCONV_KERNEL_GENERIC_TAPS = 0x400u /* tiled path that tests the 9 mask bits at run time; slower,
+                                        kept as a cross-check of the per-mask bodies */
 };
 
 #define PCONV_MAX_PATTERNS 16
@@ -200,7 +202,7 @@ pconv_status pconv_unpack(const pconv_handle* h, float* w_oihw_host_out);
 /* How the tiled kernel would run one forward (the paper has no counterpart: its tuning step picks
  * tile sizes off line; here the library picks them per call from the shape). */
 typedef struct pconv_plan_t {
-  int generic_taps;      /* 1 = run-time masks (the pattern set is not the canonical eight, or asked) */
+  int generic_taps;      /* 1 = run-time masks (asked for with PCONV_KERNEL_GENERIC_TAPS) */
   int warps_per_unit;    /* consumer warps that share one (pixels, filter group) and split each chunk's
                             channels among themselves: 1, 2 or 4 */
   int channel_splits;    /* CTAs that share one output tile through the workspace (1 = none) */
