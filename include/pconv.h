@@ -81,7 +81,7 @@ typedef struct {
   int n_groups, group_size;                     /* filter groups of the tiled layout */
   long long max_group_kernels, min_group_kernels; /* load balance of the grouping */
   long long packed_bytes;                       /* device bytes held by the handle */
-  int canonical_patterns;                       /* 1 if the set is served by the specialised code */
+  int canonical_patterns;                       /* 1 if every pattern is one of the canonical eight (one-byte codes) */
 } pconv_stats_t;
 
 /*
