@@ -233,6 +233,14 @@ pconv_status pconv_filter_order(const pconv_handle* h, int* perm_out);
  * internal wait id), else PCONV_OK. */
 pconv_status pconv_device_status(const pconv_handle* h, int* where);
 
+/* Development aid (no counterpart in the paper): synchronises the device and copies the first
+ * n_words (<= PCONV_TRACE_WORDS) 64-bit trace words of the handle to the HOST.  A library built
+ * with -DPCONV_TRACE makes the tiled kernel leave timestamps of its phases there (nanoseconds of
+ * the global timer for words 0-10, SM cycles for 11-12; the meaning of each word is listed where
+ * the kernel writes them); in a normal build the words stay zero. */
+#define PCONV_TRACE_WORDS 14
+pconv_status pconv_trace_read(const pconv_handle* h, unsigned long long* words_host, int n_words);
+
 /* Constant, NUL-terminated description of a status. */
 const char* pconv_status_str(pconv_status s);
 

@@ -25,7 +25,7 @@ STATUS_NAMES = ["PCONV_OK", "PCONV_ERR_NULL", "PCONV_ERR_SHAPE", "PCONV_ERR_PATT
 
 EXPORTS = ["pconv_pack", "pconv_forward", "pconv_forward_ws", "pconv_forward_static_ws", "pconv_workspace_bytes", "pconv_plan",
            "pconv_free", "pconv_maxpool2x2", "pconv_unpack",
-           "pconv_stats", "pconv_filter_order", "pconv_device_status", "pconv_status_str",
+           "pconv_stats", "pconv_filter_order", "pconv_device_status", "pconv_trace_read", "pconv_status_str",
            "pconv_stack_create", "pconv_stack_out_shape", "pconv_stack_forward",
            "pconv_stack_forward_host", "pconv_stack_free"]
 
@@ -83,6 +83,7 @@ def lib():
         L.pconv_stats.argtypes = [vp, ctypes.POINTER(Stats)]
         L.pconv_filter_order.argtypes = [vp, vp]
         L.pconv_device_status.argtypes = [vp, ip]
+        L.pconv_trace_read.argtypes = [vp, ctypes.POINTER(ctypes.c_ulonglong), ci]
         L.pconv_status_str.argtypes = [ci]
         L.pconv_status_str.restype = ctypes.c_char_p
         L.pconv_stack_create.argtypes = [vp, vp, vp, ci, ci, ci, ci, cu, ctypes.POINTER(vp)]
@@ -145,6 +146,16 @@ def pconv_plan(handle, n, h, w, flags=0, with_workspace=False):
     _check(lib().pconv_plan(handle, n, h, w, int(flags), int(bool(with_workspace)), ctypes.byref(p)),
            "pconv_plan")
     return {k: int(getattr(p, k)) for k, _ in Plan._fields_}
+
+
+TRACE_WORDS = 14
+
+
+def pconv_trace_read(handle):
+    """The handle's trace words (all zero unless the library was built with -DPCONV_TRACE)."""
+    buf = (ctypes.c_ulonglong * TRACE_WORDS)()
+    _check(lib().pconv_trace_read(handle, buf, TRACE_WORDS), "pconv_trace_read")
+    return list(buf)
 
 
 def pconv_workspace_bytes(handle, n, h, w):

@@ -6,6 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpconv.so")
+TRACE_LIB = os.path.join(HERE, "libpconv_trace.so")
 SOURCES = ["pack.cu", "api.cu", "kernels_simple.cu", "kernels_tiled.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC"]
@@ -21,28 +22,33 @@ def generate():
         sys.path.remove(CSRC)
 
 
-def _stale():
-    if not os.path.exists(LIB):
+def _stale(lib=None):
+    lib = lib or LIB
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if not f.endswith(".inc")]
     deps.append(os.path.join(HERE, "..", "include", "pconv.h"))
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force=False, verbose=False):
-    """Compile the CUDA library if it is missing or older than its sources; returns its path."""
-    if not force and not _stale():
-        return LIB
+def build(force=False, verbose=False, trace=False):
+    """Compile the CUDA library if it is missing or older than its sources; returns its path.
+    trace=True builds libpconv_trace.so instead: the same library with -DPCONV_TRACE (the tiled
+    kernel records phase timestamps, and PCONV_FORCE_ZS / PCONV_FORCE_KS in the environment
+    override the launch plan); see trace_case.py."""
+    lib = TRACE_LIB if trace else LIB
+    if not force and not _stale(lib):
+        return lib
     generate()
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    tmp = LIB + ".tmp%d" % os.getpid()
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + \
-          [os.path.join(CSRC, s) for s in SOURCES]
+    tmp = lib + ".tmp%d" % os.getpid()
+    cmd = [nvcc] + NVCC_FLAGS + (["-DPCONV_TRACE"] if trace else []) + \
+          (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES]
     subprocess.check_call(cmd)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, trace="--trace" in sys.argv))

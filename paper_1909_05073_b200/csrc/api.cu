@@ -172,6 +172,18 @@ extern "C" pconv_status pconv_device_status(const pconv_handle* h, int* where) {
   return PCONV_OK;
 }
 
+extern "C" pconv_status pconv_trace_read(const pconv_handle* h, unsigned long long* words, int n_words) {
+  if (!h || !words) return PCONV_ERR_NULL;
+  if (n_words < 0 || n_words > pconv::kTraceWords) return PCONV_ERR_SHAPE;
+  if (cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpy(words, pconv::trace_words(h->d), (size_t)n_words * 8, cudaMemcpyDeviceToHost) !=
+          cudaSuccess) {
+    cudaGetLastError();
+    return PCONV_ERR_CUDA;
+  }
+  return PCONV_OK;
+}
+
 // ---- stacks ---------------------------------------------------------------------------------------
 
 struct pconv_stack {

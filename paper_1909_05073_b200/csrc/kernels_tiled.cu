@@ -151,19 +151,24 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* er
   return false;
 }
 
+// Built with -DPCONV_TRACE (build.py: build(trace=True) -> libpconv_trace.so) the kernel leaves
+// timestamps in the trace words of the handle's status block (pconv_trace_read):
+//   0 start, 1 set-up done, 2 warp 0's first chunk landed, 3 loop end, 4 partial sums issued (split only),
+//   5 epilogue end, 6 after the CTA's last barrier -- thread 0 of CTA (0,0,0), globaltimer ns;
+//   7 end, 8 start, 9 loop end, 10 partial sums issued -- latest over all CTAs;
+//   11 / 12 cycles warp 0 of CTA (0,0,0) spent waiting for chunks / working on them, 13 its chunks.
 #ifdef PCONV_TRACE
 #define PCONV_MARK(i)                                                         \
   if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) { \
     unsigned long long t_;                                                    \
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                    \
-    ((unsigned long long*)(L.err + 2))[i] = t_;                               \
+    trace_words(L)[i] = t_;                                                   \
   }
-// latest time at which any CTA passed this point (slot i of the trace words)
 #define PCONV_MARK_MAX(i)                                                     \
   if (threadIdx.x == 0) {                                                     \
     unsigned long long t_;                                                    \
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                    \
-    atomicMax((unsigned long long*)(L.err + 2) + i, t_);                      \
+    atomicMax(trace_words(L) + i, t_);                                        \
   }
 #else
 #define PCONV_MARK(i)
@@ -623,10 +628,6 @@ __device__ __forceinline__ bool produce_half_stream(const DeviceLayer& L, const 
     }
   };
   HalfBatch cur, nxt;
-#ifdef PCONV_TRACE
-  long long t_pwait = 0;
-  const long long t_p0 = clock64();
-#endif
   issue(cur, 0, 0);
   for (int kk = 0; kk < nk; ++kk) {
     const int s = kk % g.stages, it = kk / g.stages;
@@ -635,25 +636,13 @@ __device__ __forceinline__ bool produce_half_stream(const DeviceLayer& L, const 
       const bool last = b + 1 == nb;
       const int kk2 = last ? kk + 1 : kk, b2 = last ? 0 : b + 1;
       if (kk2 < nk) issue(nxt, kk2, b2);
-#ifdef PCONV_TRACE
-      const long long tw0 = clock64();
-#endif
       if (b == 0 && it > 0 && !mbar_wait(sbase + 8 * (kMaxStages + s), (it - 1) & 1, L.err, 1)) return false;
-#ifdef PCONV_TRACE
-      t_pwait += clock64() - tw0;
-#endif
       store(cur, stage_base);
       cur = nxt;
     }
     if (kk >= n_early) stage_blocks_half(L, g, desc, codes, stage_base, kk, ptid);
     mbar_arrive(sbase + 8 * s);
   }
-#ifdef PCONV_TRACE
-  if (ptid == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {
-    ((unsigned long long*)(L.err + 2))[4] = (unsigned long long)t_pwait;
-    ((unsigned long long*)(L.err + 2))[6] = (unsigned long long)(clock64() - t_p0);
-  }
-#endif
   return true;
 }
 
@@ -1085,7 +1074,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
 #ifdef PCONV_TRACE
       const long long tc1 = clock64();
 #endif
-      if (kk == 0) { PCONV_MARK(2) }
+      if (next_kk == 1) { PCONV_MARK(2) }   // this warp's first chunk has landed
       if (active) {
         const uint32_t stage_base = sbase + g.stage_off + s * g.stage_bytes;
         uint32_t xptr = stage_base + lane_off - chan_b;  // one channel before the chunk
@@ -1127,9 +1116,9 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
     }
 #ifdef PCONV_TRACE
     if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {
-      ((unsigned long long*)(L.err + 2))[11] = (unsigned long long)t_wait;
-      ((unsigned long long*)(L.err + 2))[12] = (unsigned long long)t_work;
-      ((unsigned long long*)(L.err + 2))[13] = (unsigned long long)nk;
+      trace_words(L)[11] = (unsigned long long)t_wait;
+      trace_words(L)[12] = (unsigned long long)t_work;
+      trace_words(L)[13] = (unsigned long long)nk;
     }
 #endif
 

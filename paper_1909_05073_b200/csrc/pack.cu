@@ -315,8 +315,8 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
     const int i_cs = add(codes_s.data(), codes_s.size());
     const int i_cg = add(codes_g.data(), codes_g.size());
     const int i_pm = add(perm.data(), perm.size() * 4);
-    const int zero = 0;
-    const int i_er = add(&zero, 4);
+    const std::vector<unsigned char> zero_block(kStatusBlockBytes, 0);
+    const int i_er = add(zero_block.data(), zero_block.size());
 
     char* dev = nullptr;
     if (cudaMalloc((void**)&dev, total) != cudaSuccess) {

@@ -84,11 +84,19 @@ struct DeviceLayer {         // device pointers of one packed layer (passed to k
   const uint8_t* codes_s;    // specialised codes (narrow or wide, see wide_codes)
   const uint8_t* codes_g;    // generic codes
   const int* perm;           // [n_groups * kGroup] original filter index or -1
-  int* err;                  // device status word (0 = fine)
+  int* err;                  // device status block: word 0 = status (0 = fine), then trace words
   int c_out, c_in, stride, storage, n_groups, n_chunks;
   int wide_codes;            // 0 = narrow codes (canonical set), 1 = wide codes
   long long n_kept;          // surviving kernels of the layer
 };
+
+// Status block: one status word, one pad word, kTraceWords 64-bit trace words (written only by
+// builds with -DPCONV_TRACE).
+constexpr int kTraceWords = 14;
+constexpr int kStatusBlockBytes = 8 + 8 * kTraceWords;
+__host__ __device__ inline unsigned long long* trace_words(const DeviceLayer& L) {
+  return reinterpret_cast<unsigned long long*>(L.err + 2);
+}
 
 }  // namespace pconv
 
