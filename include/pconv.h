@@ -244,6 +244,33 @@ pconv_status pconv_trace_read(const pconv_handle* h, unsigned long long* words_h
 /* Constant, NUL-terminated description of a status. */
 const char* pconv_status_str(pconv_status s);
 
+/* ---- producing PCONV weights from dense ones --------------------------------------------------- */
+
+/*
+ * pconv_project -- projection of dense 3x3 kernels onto the PCONV constraint set, the step of the
+ * paper's training framework that "assigns patterns to each kernel or prunes specific kernels"
+ * (section on the ADMM-based framework; its formulas are in a supplement that is not available, so
+ * the Euclidean projection is this build's reading).  Not part of the forward pass.
+ *
+ * For each kernel the pattern that retains the largest sum of squares is chosen (lowest pattern id
+ * on ties); the k = round(keep * n_kernels) kernels with the largest retained sum survive,
+ * together with every kernel that ties with the k-th; everything else becomes zero.  The sums are
+ * formed in fp32, tap after tap in ascending tap order, multiply and add separately.
+ *
+ *  w_dev           [n_kernels][9] fp32, DEVICE (an OIHW tensor with n_kernels = c_out * c_in).
+ *  patterns        n_patterns masks, HOST, as for pconv_pack.
+ *  keep            fraction of kernels to keep, 0..1.
+ *  w_out_dev       [n_kernels][9] fp32, DEVICE; may be w_dev (in place).
+ *  pattern_id_dev  [n_kernels] int8, DEVICE: the chosen pattern, -1 for pruned kernels.
+ *  ws_dev          DEVICE scratch of pconv_project_workspace_bytes(n_kernels) bytes, 256-byte
+ *                  aligned; contents irrelevant before and after.
+ * Asynchronous on `stream`; allocates nothing.  PCONV_ERR_WORKSPACE if ws_bytes is too small.
+ */
+pconv_status pconv_project_workspace_bytes(long long n_kernels, size_t* bytes);
+pconv_status pconv_project(const float* w_dev, long long n_kernels, const uint16_t* patterns,
+                           int n_patterns, double keep, float* w_out_dev,
+                           signed char* pattern_id_dev, void* ws_dev, size_t ws_bytes, void* stream);
+
 /* ---- layer stacks ---------------------------------------------------------------------------- */
 
 /*

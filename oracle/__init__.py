@@ -12,7 +12,9 @@ pattern of the set -- exactly 4 of them in strict mode --, every pruned kernel i
 "Sparse Convolution Pattern" section, and the 2.25x = 9/4 pattern rate of the pattern-count
 tables).
 
-Pins: see tests/test_oracle_pins.py.  No function here is "parity unpinned".
+Pins: see tests/test_oracle_pins.py.  `project` (the projection that produces PCONV weights from
+dense ones; not part of the forward pass) is "parity unpinned": the paper's formulas for it are in
+a supplement that is not available, and only its defining properties are tested.
 """
 import ctypes
 import os
@@ -133,3 +135,44 @@ def check_invariants(w, patterns, strict4=True):
         nnz = (np.asarray(w) != 0).sum(axis=(2, 3))
         assert set(np.unique(nnz)) <= {0, 4}, "a kernel has a non-zero count other than 0 or 4"
     return ids
+
+
+def project(w, patterns, keep):
+    """Projection of dense 3x3 kernels onto the PCONV constraint set: the step that turns trained
+    weights into pattern- and connectivity-pruned ones ("assign patterns to each kernel, or prune
+    specific kernels", section on the ADMM-based training framework; the paper's own formulas are
+    in a supplement that is not available, so this is a reading of that sentence: the Euclidean
+    projection -- parity unpinned beyond the properties tested in tests/test_oracle_pins.py).
+
+    For each kernel the pattern that retains the largest sum of squares is chosen (lowest pattern
+    id on ties); then the k = round(keep * kernels) kernels with the largest retained sum of
+    squares survive, together with every kernel that ties with the k-th.  The sums that take
+    these decisions are formed in fp32, one tap after the other in ascending tap order with a
+    separate multiply and add (both sides of a comparison use the same precision).
+
+    w: [c_out, c_in, 3, 3] float32.  Returns (projected weights float32, pattern ids int8 with -1
+    for pruned kernels)."""
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    c_out, c_in = w.shape[:2]
+    flat = w.reshape(c_out * c_in, 9)
+    n = flat.shape[0]
+    scores = np.zeros((len(patterns), n), np.float32)
+    for p, mask in enumerate(patterns):
+        s = np.zeros(n, np.float32)
+        for t in range(9):
+            if mask >> t & 1:
+                s = (s + (flat[:, t] * flat[:, t]).astype(np.float32)).astype(np.float32)
+        scores[p] = s
+    pid = np.argmax(scores, axis=0)                    # first maximum = lowest id on ties
+    best = scores[pid, np.arange(n)]
+    k = int(np.floor(keep * n + 0.5))
+    k = min(max(k, 0), n)
+    if k == 0:
+        kept = np.zeros(n, bool)
+    else:
+        threshold = np.sort(best)[n - k]              # the k-th largest value
+        kept = best >= threshold
+    masks = np.array([[(m >> t) & 1 for t in range(9)] for m in patterns], np.float32)
+    out = flat * masks[pid] * kept[:, None]
+    ids = np.where(kept, pid, -1).astype(np.int8)
+    return out.reshape(w.shape).astype(np.float32), ids.reshape(c_out, c_in)

@@ -27,7 +27,8 @@ EXPORTS = ["pconv_pack", "pconv_forward", "pconv_forward_ws", "pconv_forward_sta
            "pconv_free", "pconv_maxpool2x2", "pconv_unpack",
            "pconv_stats", "pconv_filter_order", "pconv_device_status", "pconv_trace_read", "pconv_status_str",
            "pconv_stack_create", "pconv_stack_out_shape", "pconv_stack_forward",
-           "pconv_stack_forward_host", "pconv_stack_free"]
+           "pconv_stack_forward_host", "pconv_stack_free",
+           "pconv_project", "pconv_project_workspace_bytes"]
 
 
 class PconvError(RuntimeError):
@@ -83,6 +84,9 @@ def lib():
         L.pconv_stats.argtypes = [vp, ctypes.POINTER(Stats)]
         L.pconv_filter_order.argtypes = [vp, vp]
         L.pconv_device_status.argtypes = [vp, ip]
+        L.pconv_project_workspace_bytes.argtypes = [ctypes.c_longlong, ctypes.POINTER(ctypes.c_size_t)]
+        L.pconv_project.argtypes = [vp, ctypes.c_longlong, vp, ci, ctypes.c_double, vp, vp, vp,
+                                    ctypes.c_size_t, vp]
         L.pconv_trace_read.argtypes = [vp, ctypes.POINTER(ctypes.c_ulonglong), ci]
         L.pconv_status_str.argtypes = [ci]
         L.pconv_status_str.restype = ctypes.c_char_p
@@ -146,6 +150,27 @@ def pconv_plan(handle, n, h, w, flags=0, with_workspace=False):
     _check(lib().pconv_plan(handle, n, h, w, int(flags), int(bool(with_workspace)), ctypes.byref(p)),
            "pconv_plan")
     return {k: int(getattr(p, k)) for k, _ in Plan._fields_}
+
+
+def pconv_project(w, patterns, keep, out=None, stream=None):
+    """Projects a CUDA fp32 tensor [c_out, c_in, 3, 3] onto the pattern set / keep rate.
+    Returns (projected weights, int8 pattern ids [c_out, c_in] with -1 = pruned)."""
+    import torch
+    if not (w.is_cuda and w.is_contiguous() and w.dtype == torch.float32 and tuple(w.shape[2:]) == (3, 3)):
+        raise ValueError("w must be a contiguous CUDA float32 tensor [c_out, c_in, 3, 3]")
+    n = w.shape[0] * w.shape[1]
+    need = ctypes.c_size_t(0)
+    _check(lib().pconv_project_workspace_bytes(n, ctypes.byref(need)), "pconv_project_workspace_bytes")
+    ws = torch.empty(max(int(need.value), 256), dtype=torch.uint8, device=w.device)
+    if out is None:
+        out = torch.empty_like(w)
+    ids = torch.empty((w.shape[0], w.shape[1]), dtype=torch.int8, device=w.device)
+    pats = (ctypes.c_uint16 * len(patterns))(*patterns)
+    _check(lib().pconv_project(ctypes.c_void_p(w.data_ptr()), n, pats, len(patterns), float(keep),
+                               ctypes.c_void_p(out.data_ptr()), ctypes.c_void_p(ids.data_ptr()),
+                               ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream_ptr(stream)),
+           "pconv_project")
+    return out, ids
 
 
 TRACE_WORDS = 14

@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpconv.so")
 TRACE_LIB = os.path.join(HERE, "libpconv_trace.so")
-SOURCES = ["pack.cu", "api.cu", "kernels_simple.cu", "kernels_tiled.cu"]
+SOURCES = ["pack.cu", "api.cu", "kernels_simple.cu", "kernels_tiled.cu", "project.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC"]
 

@@ -230,3 +230,59 @@ def test_config_shapes_match_the_benchmark_definitions():
     assert c4.batch == 256 and c4.storage == "f16" and c4.layers[-1].h == 2
     # connectivity rate of the ImageNet VGG-16 table (3.1x) is close to keep = 0.3
     assert abs(1 / 3.1 - 0.3) < 0.03
+
+
+# ---- projection onto the pattern / connectivity constraint set -------------------------------------
+
+def _brute_force_project(w, patterns, keep):
+    """Exhaustive search in fp64 on a tiny tensor: every assignment of a pattern or 'pruned' to
+    every kernel with exactly k survivors; returns the largest retained energy."""
+    import itertools
+    c_out, c_in = w.shape[:2]
+    flat = w.reshape(-1, 9).astype(np.float64)
+    n = flat.shape[0]
+    k = int(np.floor(keep * n + 0.5))
+    best_per_kernel = np.array([max(sum(flat[i, t] ** 2 for t in range(9) if m >> t & 1) for m in patterns)
+                                for i in range(n)])
+    best = -1.0
+    for chosen in itertools.combinations(range(n), k):
+        best = max(best, float(best_per_kernel[list(chosen)].sum()))
+    return best, k
+
+
+def test_projection_is_the_energy_maximising_choice_on_tiny_tensors():
+    rng = np.random.default_rng(11)
+    for trial in range(6):
+        w = rng.normal(0, 1, (2, 3, 3, 3)).astype(np.float32)
+        for keep in (0.0, 0.34, 0.5, 1.0):
+            out, ids = oracle.project(w, synth.PATTERNS8, keep)
+            energy, k = _brute_force_project(w, synth.PATTERNS8, keep)
+            assert int((ids >= 0).sum()) == k
+            assert abs(float((out.astype(np.float64) ** 2).sum()) - energy) <= 1e-5 * (1 + energy)
+
+
+def test_projection_output_satisfies_the_pconv_invariants_and_keeps_values():
+    rng = np.random.default_rng(12)
+    w = rng.normal(0, 1, (16, 24, 3, 3)).astype(np.float32)
+    out, ids = oracle.project(w, synth.PATTERNS8, 0.3)
+    oracle.check_invariants(out, synth.PATTERNS8, strict4=True)
+    assert int((ids >= 0).sum()) == round(0.3 * 16 * 24)
+    nz = out != 0
+    assert np.array_equal(out[nz], w[nz])                      # survivors keep their values
+    got_ids = oracle.classify(out, synth.PATTERNS8)
+    assert np.array_equal(got_ids, ids)
+    # idempotent: projecting a projected tensor with the same keep rate changes nothing
+    again, ids2 = oracle.project(out, synth.PATTERNS8, 0.3)
+    assert np.array_equal(again, out) and np.array_equal(ids2, ids)
+
+
+def test_projection_ties_and_degenerate_inputs():
+    w = np.zeros((2, 2, 3, 3), np.float32)
+    w[0, 0] = 1.0                                              # every pattern retains 4: lowest id wins
+    w[1, 1] = 1.0
+    out, ids = oracle.project(w, synth.PATTERNS8, 0.25)        # k = 1 but two kernels tie: both kept
+    assert ids[0, 0] == 0 and ids[1, 1] == 0 and int((ids >= 0).sum()) == 2
+    out, ids = oracle.project(w, synth.PATTERNS8, 0.0)
+    assert not out.any() and (ids == -1).all()
+    out, ids = oracle.project(w, synth.PATTERNS8, 1.0)         # zero kernels tie at 0 and are "kept"
+    assert (ids >= 0).all() and int((out != 0).sum()) == 8
