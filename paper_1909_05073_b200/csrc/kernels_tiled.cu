@@ -1318,14 +1318,20 @@ void set_split(const DeviceLayer& L, Geo* g, int ks) {
 }
 
 // Estimated duration of a launch in units of one kernel (4 taps on a warp's 256 pixels, about
-// 0.18 us), from measurements of batch-1 layers: a CTA pays a fixed start (first chunk in flight)
-// and an epilogue that shrinks with the warps sharing a unit; CTAs run in waves of one per SM; a
-// channel split across CTAs adds the atomic traffic of every CTA's whole tile and its draining.
+// 0.17 us), from measurements of batch-1 and small-map layers: a CTA pays a fixed start (first
+// chunk in flight) and an epilogue that shrinks with the warps sharing a unit; a chunk takes the
+// consumers its kernels plus a fixed part, and the four producer warps a time that grows with the
+// staged elements (measured 0.5 us + 4 ns per element), zs chunks being consumed at a time; CTAs
+// run in waves of one per SM; a channel split across CTAs adds the atomic traffic of every CTA's
+// tile and its draining.
 double geo_cost(const DeviceLayer& L, const Geo& g) {
   const double k_unit = (double)L.n_kept / (L.n_groups > 0 ? L.n_groups : 1);  // kernels of one group
   const double per_chunk = 1.5;                                                // barrier, entry, exit
   const int turns = (g.cps + g.zs - 1) / g.zs;                                 // chunks per warp
-  const double loop = turns * (k_unit / L.n_chunks + per_chunk);
+  const double consume = k_unit / L.n_chunks + per_chunk;
+  const double produce = 3.0 + 0.024 * (g.pairs * g.rows * g.pitch);
+  const double chunk = consume > g.zs * produce ? consume : g.zs * produce;
+  const double loop = turns * chunk;
   const double fixed = 28.0 + 17.0 / g.zs;
   const long long ctas = geo_tiles(L, g) * g.ks;
   const double waves = (double)((ctas + kNumSMs - 1) / kNumSMs);
