@@ -64,6 +64,11 @@ enum {
   /* Kernel selection (forward).  Default: the library picks per shape.  These bits exist so that
    * tests and benchmarks can pin one implementation; they never change the result beyond
    * summation order. */
+  PCONV_REPRODUCIBLE = 8u, /* forward: the same call gives bit-identical outputs every time: the
+                              warps that share a tile take their chunks in a fixed order and the
+                              channel range is not split across thread blocks (a workspace, if
+                              given, is left untouched).  Without it the grouping of the fp32 partial
+                              sums -- not the result beyond rounding -- may vary from run to run. */
   PCONV_KERNEL_SIMPLE = 0x100u, /* one thread per output, walks the per-filter kernel list */
   PCONV_KERNEL_TILED = 0x200u,  /* shared-memory halo tiles, packed FMAs, one straight-line body per
                                    pattern mask (any set of 4-of-9 masks); the default */
@@ -117,7 +122,7 @@ pconv_status pconv_pack(const float* w_oihw_host, int c_out, int c_in, const uin
  *  bias_dev  [c_out] fp32, DEVICE, or NULL for no bias.
  *  y_dev     [n][c_out][h_out][w_out], DEVICE, same storage type, 16-byte aligned, must not
  *            overlap x.  h_out = (h_in - 1) / stride + 1, likewise w_out.
- *  flags     PCONV_RELU, PCONV_POOL2X2 and/or one PCONV_KERNEL_* bit.  With PCONV_POOL2X2 the
+ *  flags     PCONV_RELU, PCONV_POOL2X2, PCONV_REPRODUCIBLE and/or one PCONV_KERNEL_* bit.  With PCONV_POOL2X2 the
  *            layer's output is max-pooled before it is stored (the VGG stacks of the evaluation
  *            pool after conv2/4/7/10): y_dev is [n][c_out][h_out/2][w_out/2] (odd trailing row
  *            and column dropped, as pconv_maxpool2x2 does), h_out and w_out must be >= 2, and the

@@ -14,7 +14,7 @@ LIB_PATH = os.path.join(HERE, "libpconv.so")
 
 OK = 0
 F32, F16 = 0, 1
-RELU, STRICT4, POOL2X2 = 1, 2, 4
+RELU, STRICT4, POOL2X2, REPRODUCIBLE = 1, 2, 4, 8
 KERNEL_SIMPLE, KERNEL_TILED, KERNEL_GENERIC_TAPS = 0x100, 0x200, 0x400
 MAX_PATTERNS = 16
 

@@ -55,7 +55,7 @@ extern "C" pconv_status pconv_forward_ws(const pconv_handle* h, const void* x, c
   if (!h || !x || !y) return PCONV_ERR_NULL;
   if (n < 0 || h_in <= 0 || w_in <= 0) return PCONV_ERR_SHAPE;
   const unsigned known =
-      PCONV_RELU | PCONV_POOL2X2 | PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED | PCONV_KERNEL_GENERIC_TAPS;
+      PCONV_RELU | PCONV_POOL2X2 | PCONV_REPRODUCIBLE | PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED | PCONV_KERNEL_GENERIC_TAPS;
   if (flags & ~known) return PCONV_ERR_UNSUPPORTED;
   const unsigned sel = flags & (PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED | PCONV_KERNEL_GENERIC_TAPS);
   if (sel & (sel - 1)) return PCONV_ERR_UNSUPPORTED;  // at most one selection bit
@@ -78,6 +78,7 @@ extern "C" pconv_status pconv_forward_ws(const pconv_handle* h, const void* x, c
   cudaStream_t stream = (cudaStream_t)stream_v;
   const bool relu = flags & PCONV_RELU;
   const bool pool = flags & PCONV_POOL2X2;
+  const bool repro = flags & PCONV_REPRODUCIBLE;
   cudaError_t e;
   if (pool && (sel == PCONV_KERNEL_SIMPLE || !tiled_supported(L, n, h_in, w_in)))
     return PCONV_ERR_UNSUPPORTED;  // only the tiled kernels fuse the pool
@@ -86,9 +87,9 @@ extern "C" pconv_status pconv_forward_ws(const pconv_handle* h, const void* x, c
   } else if (sel == PCONV_KERNEL_TILED || sel == PCONV_KERNEL_GENERIC_TAPS) {
     if (!tiled_supported(L, n, h_in, w_in)) return PCONV_ERR_UNSUPPORTED;
     const bool generic = (sel == PCONV_KERNEL_GENERIC_TAPS);
-    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, pool, generic, ws, ws_bytes, stream);
+    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, pool, repro, generic, ws, ws_bytes, stream);
   } else if (tiled_supported(L, n, h_in, w_in)) {
-    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, pool, false, ws, ws_bytes, stream);
+    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, pool, repro, false, ws, ws_bytes, stream);
   } else {
     e = launch_simple(L, x, bias, y, n, h_in, w_in, relu, stream);
   }

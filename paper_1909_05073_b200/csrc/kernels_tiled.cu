@@ -81,6 +81,7 @@ struct Geo {
   int ks, cps;           // channel splits (grid.z) and chunks per split
   int relu, is_half;
   int pool, h_y, w_y;     // fused 2x2 max-pool: y holds [h_y][w_y] = [h_out/2][w_out/2] maps
+  int fixed_turns;        // 1 = the warps of a unit take the chunks in a fixed order (reproducible sums)
 };
 
 // ---- PTX helpers ----------------------------------------------------------------------------------
@@ -1056,13 +1057,19 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
     long long t_wait = 0, t_work = 0;
 #endif
     // The warps of a unit draw the chunks from the unit's counter, so a warp that got a heavier
-    // chunk (or started later) simply takes fewer.
+    // chunk (or started later) simply takes fewer -- or, when reproducible sums are asked for,
+    // take them in turn (warp z: chunks z, z + zs, ...; the ring depth is then a multiple of zs,
+    // so a slot always comes back to the same warps).
     int next_kk = 0;
     while (ok) {
       int kk = next_kk++;
       if (zs > 1) {
-        if (lane == 0) kk = atomicAdd(unit_ctr + unit, 1);
-        kk = __shfl_sync(0xffffffffu, kk, 0);
+        if (g.fixed_turns) {
+          kk = z + kk * zs;
+        } else {
+          if (lane == 0) kk = atomicAdd(unit_ctr + unit, 1);
+          kk = __shfl_sync(0xffffffffu, kk, 0);
+        }
       }
       if (kk >= nk) break;
       const int s = kk % g.stages;
@@ -1296,6 +1303,7 @@ bool geo_for(const DeviceLayer& L, int n, int h, int w, int zs, Geo* out) {
   }
   if (g.stages < 1) return false;
   g.relu = 0;
+  g.fixed_turns = 0;
   g.pool = 0;
   g.h_y = g.h_out;
   g.w_y = g.w_out;
@@ -1454,15 +1462,20 @@ bool tiled_plan(const DeviceLayer& L, int n, int h, int w, bool generic_taps, bo
 }
 
 cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias, void* y, int n, int h,
-                         int w, bool relu, bool pool, bool generic_taps, void* ws, size_t ws_bytes,
-                         cudaStream_t stream) {
+                         int w, bool relu, bool pool, bool reproducible, bool generic_taps, void* ws,
+                         size_t ws_bytes, cudaStream_t stream) {
   if (!generic_taps && !L.codes_s) generic_taps = true;
   Geo g;
   const size_t need = generic_taps ? 0 : tiled_workspace_bytes(L, n, h, w);
-  const bool split = need > 0 && ws && ws_bytes >= need;
+  const bool split = !reproducible && need > 0 && ws && ws_bytes >= need;
   if (!(generic_taps ? make_geo<true>(L, n, h, w, false, &g) : make_geo<false>(L, n, h, w, split, &g)))
     return cudaErrorInvalidValue;
   g.relu = relu ? 1 : 0;
+  if (reproducible && g.zs > 1) {
+    g.fixed_turns = 1;
+    if (g.stages < g.cps) g.stages = g.stages / g.zs * g.zs;   // >= zs by pick_stages
+    if (g.stages < 1) return cudaErrorInvalidValue;
+  }
   if (pool) {
     if (g.h_out < 2 || g.w_out < 2) return cudaErrorInvalidValue;
     g.pool = 1;

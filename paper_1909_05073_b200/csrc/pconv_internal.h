@@ -119,8 +119,8 @@ namespace pconv {
 cudaError_t launch_simple(const DeviceLayer& L, const void* x, const float* bias, void* y, int n,
                           int h, int w, bool relu, cudaStream_t stream);
 cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias, void* y, int n,
-                         int h, int w, bool relu, bool pool, bool generic_taps, void* ws,
-                         size_t ws_bytes, cudaStream_t stream);
+                         int h, int w, bool relu, bool pool, bool reproducible, bool generic_taps,
+                         void* ws, size_t ws_bytes, cudaStream_t stream);
 size_t tiled_workspace_bytes(const DeviceLayer& L, int n, int h, int w);
 bool tiled_supported(const DeviceLayer& L, int n, int h, int w);
 bool tiled_plan(const DeviceLayer& L, int n, int h, int w, bool generic_taps, bool with_workspace,

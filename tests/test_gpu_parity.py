@@ -308,6 +308,35 @@ def test_fused_maxpool_is_refused_where_it_cannot_run():
     layer.close()
 
 
+@pytest.mark.parametrize("case", [(64, 128, 56, 56, 1, 1, 0.3), (256, 256, 14, 14, 1, 1, 0.3),
+                                  (128, 128, 28, 28, 2, 2, 0.35), (512, 512, 7, 7, 1, 1, 0.3)],
+                         ids=lambda c: "x".join(str(v) for v in c))
+def test_reproducible_flag_gives_bit_identical_runs(case):
+    c_in, c_out, h, w, n, stride, keep = case
+    spec = synth.LayerSpec("t", c_in, c_out, h, w, stride, keep)
+    wt, bias, _ = synth.gen_weights(spec, 55 + c_in)
+    x = synth.gen_input(spec, n, 55 + c_in)
+    layer = B.Layer(wt, synth.PATTERNS8, stride, B.F32, bias)
+    assert B.pconv_plan(layer.handle, n, h, w, 0, False)["warps_per_unit"] > 1   # several warps share a tile
+    xt = torch.from_numpy(x).cuda()
+    ws = layer.workspace(xt.shape)
+    ref = oracle_layer(wt, bias, x, stride, "f32", True)
+    first = None
+    for _ in range(6):
+        y = torch.empty(layer.out_shape(xt.shape), device="cuda")
+        B.pconv_forward(layer.handle, xt, layer.bias, y, B.RELU | B.REPRODUCIBLE, workspace=ws)
+        torch.cuda.synchronize()
+        got = y.cpu().numpy()
+        check_close(got, ref, "f32", "reproducible %s" % (case,))
+        if first is None:
+            first = got
+        assert np.array_equal(got, first)
+    if ws is not None:
+        assert not ws.any()            # the flag keeps the channel range in one thread block
+    assert B.pconv_device_status(layer.handle)[0] == 0
+    layer.close()
+
+
 PLAN_CASES = [  # shapes that make the library use each way of sharing the consumer warps
     (16, 128, 32, 32, 74, 1, 0.5),    # as many tiles as SMs: one warp per unit
     (64, 64, 224, 224, 1, 1, 0.3),    # one large image
