@@ -226,6 +226,13 @@ typedef struct pconv_plan_t {
 pconv_status pconv_plan(const pconv_handle* h, int n, int h_in, int w_in, unsigned flags,
                         int with_workspace, pconv_plan_t* plan);
 
+/* The same without a handle (host arithmetic only, needs no device): the plan for a layer of the
+ * given shape with `kept_kernels` surviving kernels; canonical_patterns != 0 = the pattern set lies
+ * inside the canonical eight. */
+pconv_status pconv_plan_shape(int c_out, int c_in, long long kept_kernels, int stride, int storage,
+                              int canonical_patterns, int n, int h_in, int w_in, unsigned flags,
+                              int with_workspace, pconv_plan_t* plan);
+
 /* Fills *out with the layer's structure counts. */
 pconv_status pconv_stats(const pconv_handle* h, pconv_stats_t* out);
 

@@ -23,7 +23,7 @@ STATUS_NAMES = ["PCONV_OK", "PCONV_ERR_NULL", "PCONV_ERR_SHAPE", "PCONV_ERR_PATT
                 "PCONV_ERR_ALIGN", "PCONV_ERR_ALLOC", "PCONV_ERR_CUDA",
                 "PCONV_ERR_DEVICE_TIMEOUT", "PCONV_ERR_WORKSPACE"]
 
-EXPORTS = ["pconv_pack", "pconv_forward", "pconv_forward_ws", "pconv_forward_static_ws", "pconv_workspace_bytes", "pconv_plan",
+EXPORTS = ["pconv_pack", "pconv_forward", "pconv_forward_ws", "pconv_forward_static_ws", "pconv_workspace_bytes", "pconv_plan", "pconv_plan_shape",
            "pconv_free", "pconv_maxpool2x2", "pconv_unpack",
            "pconv_stats", "pconv_filter_order", "pconv_device_status", "pconv_trace_read", "pconv_status_str",
            "pconv_stack_create", "pconv_stack_out_shape", "pconv_stack_forward",
@@ -77,6 +77,8 @@ def lib():
         L.pconv_forward_static_ws.argtypes = [vp, vp, vp, vp, ci, ci, ci, cu, vp]
         L.pconv_workspace_bytes.argtypes = [vp, ci, ci, ci, ctypes.POINTER(ctypes.c_size_t)]
         L.pconv_plan.argtypes = [vp, ci, ci, ci, cu, ci, ctypes.POINTER(Plan)]
+        L.pconv_plan_shape.argtypes = [ci, ci, ctypes.c_longlong, ci, ci, ci, ci, ci, ci, cu, ci,
+                                       ctypes.POINTER(Plan)]
         L.pconv_free.argtypes = [vp]
         L.pconv_free.restype = None
         L.pconv_maxpool2x2.argtypes = [vp, vp, ci, ci, ci, ci, ci, vp]
@@ -181,6 +183,14 @@ def pconv_trace_read(handle):
     buf = (ctypes.c_ulonglong * TRACE_WORDS)()
     _check(lib().pconv_trace_read(handle, buf, TRACE_WORDS), "pconv_trace_read")
     return list(buf)
+
+
+def pconv_plan_shape(c_out, c_in, kept, stride, storage, canonical, n, h, w, flags=0, with_workspace=False):
+    """pconv_plan for a shape alone (host arithmetic; works without a GPU)."""
+    p = Plan()
+    _check(lib().pconv_plan_shape(c_out, c_in, int(kept), stride, storage, int(bool(canonical)), n, h, w,
+                                  int(flags), int(bool(with_workspace)), ctypes.byref(p)), "pconv_plan_shape")
+    return {k: int(getattr(p, k)) for k, _ in Plan._fields_}
 
 
 def pconv_workspace_bytes(handle, n, h, w):

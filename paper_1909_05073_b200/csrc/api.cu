@@ -43,6 +43,30 @@ extern "C" pconv_status pconv_plan(const pconv_handle* h, int n, int h_in, int w
   return PCONV_OK;
 }
 
+extern "C" pconv_status pconv_plan_shape(int c_out, int c_in, long long kept_kernels, int stride,
+                                         int storage, int n_patterns_canonical, int n, int h_in,
+                                         int w_in, unsigned flags, int with_workspace,
+                                         pconv_plan_t* plan) {
+  if (!plan) return PCONV_ERR_NULL;
+  if (c_out <= 0 || c_in <= 0 || kept_kernels < 0 || n <= 0 || h_in <= 0 || w_in <= 0) return PCONV_ERR_SHAPE;
+  if ((stride != 1 && stride != 2) || (storage != PCONV_F32 && storage != PCONV_F16)) return PCONV_ERR_UNSUPPORTED;
+  pconv::DeviceLayer L;
+  std::memset(&L, 0, sizeof(L));
+  L.c_out = c_out;
+  L.c_in = c_in;
+  L.stride = stride;
+  L.storage = storage;
+  L.n_groups = (c_out + pconv::kGroup - 1) / pconv::kGroup;
+  L.n_chunks = (c_in + pconv::kChunk - 1) / pconv::kChunk;
+  L.n_kept = kept_kernels;
+  L.wide_codes = n_patterns_canonical ? 0 : 1;
+  L.codes_s = reinterpret_cast<const uint8_t*>(&L);   // only tested for presence by the planner
+  std::memset(plan, 0, sizeof(*plan));
+  if (!tiled_plan(L, n, h_in, w_in, (flags & PCONV_KERNEL_GENERIC_TAPS) != 0, with_workspace != 0, plan))
+    return PCONV_ERR_UNSUPPORTED;
+  return PCONV_OK;
+}
+
 extern "C" pconv_status pconv_forward(const pconv_handle* h, const void* x, const float* bias,
                                       void* y, int n, int h_in, int w_in, unsigned flags,
                                       void* stream_v) {

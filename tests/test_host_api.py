@@ -91,3 +91,42 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libpconv.so")
     with pytest.raises(RuntimeError, match="only implementation"):
         binding.lib()
+
+
+def test_launch_plans_are_well_formed_over_many_shapes(lib):
+    """The planner is host arithmetic: for thousands of shapes the chosen geometry must fit the
+    hardware (shared memory, ring depth, grid limits) and follow its own rules."""
+    rng = np.random.default_rng(2024)
+    seen_zs, seen_split = set(), set()
+    for _ in range(4000):
+        c_in = int(rng.choice([1, 3, 8, 16, 40, 64, 100, 128, 256, 512, 1024, 2048]))
+        c_out = int(rng.choice([1, 8, 16, 33, 64, 128, 256, 512, 1000]))
+        h = int(rng.choice([1, 2, 4, 7, 8, 14, 16, 28, 32, 56, 112, 224, 300]))
+        w = int(rng.choice([1, 2, 3, 4, 7, 8, 14, 15, 16, 28, 32, 56, 112, 224, 333]))
+        n = int(rng.choice([1, 1, 2, 8, 32, 256]))
+        stride = int(rng.choice([1, 2]))
+        storage = int(rng.choice([binding.F32, binding.F16]))
+        keep = float(rng.choice([0.05, 0.3, 0.5, 1.0]))
+        canonical = bool(rng.random() < 0.7)
+        generic = bool(rng.random() < 0.15)
+        ws = bool(rng.random() < 0.5)
+        kept = int(keep * c_in * c_out)
+        flags = binding.KERNEL_GENERIC_TAPS if generic else 0
+        p = binding.pconv_plan_shape(c_out, c_in, kept, stride, storage, canonical, n, h, w, flags, ws)
+        what = (c_out, c_in, h, w, n, stride, storage, keep, canonical, generic, ws, p)
+        assert p["smem_bytes"] <= 227 * 1024, what
+        assert p["stages"] >= 1 and p["ctas"] >= 1, what
+        assert p["warps_per_unit"] in (1, 2, 4) and p["tile_width"] in (2, 4, 8, 16, 32), what
+        n_chunks = (c_in + 7) // 8
+        assert 1 <= p["channel_splits"] <= n_chunks, what
+        if generic:
+            assert p["generic_taps"] == 1 and p["warps_per_unit"] == 1 and p["channel_splits"] == 1, what
+        if not ws:
+            assert p["channel_splits"] == 1, what
+        chunks_per_cta = -(-n_chunks // p["channel_splits"])
+        # a ring shallower than the warps sharing a unit is only allowed when no slot is reused
+        assert p["stages"] >= min(p["warps_per_unit"], chunks_per_cta) or p["stages"] == chunks_per_cta, what
+        assert p["groups_per_cta"] * p["pixel_sets"] * p["warps_per_unit"] <= (8 if generic else 16), what
+        seen_zs.add(p["warps_per_unit"])
+        seen_split.add(p["channel_splits"] > 1)
+    assert seen_zs == {1, 2, 4} and seen_split == {False, True}
