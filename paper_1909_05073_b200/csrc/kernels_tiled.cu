@@ -1141,8 +1141,9 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
       if (zs > 1) {
         // The warps of a unit hold partial sums over the chunks they drew in their own TMEM columns
         // of the same lanes; once all have finished, each adds up and writes 16 / zs filter slots.
+        // (a barrier of the unit's own zs warps: units do not wait for one another)
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        asm volatile("bar.sync 1, %0;" ::"n"(32 * kCW) : "memory");
+        asm volatile("bar.sync %0, %1;" ::"r"(3 + unit), "r"(32 * zs) : "memory");
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         orng.t0 = tquad + (uint32_t)(((warp >> 2) - z) * (kGroup * 8));
         orng.zs = zs;
