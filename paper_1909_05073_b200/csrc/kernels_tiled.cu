@@ -394,15 +394,61 @@ __device__ __forceinline__ void produce_chunk_async(const DeviceLayer& L, const 
                                                     const float* __restrict__ x, const SubTile* tab,
                                                     const StagedElem (&pre)[kPreElems], const uint4* desc,
                                                     const uint8_t* codes, uint32_t stage_base, int k, int kk,
-                                                    int ptid, bool with_blocks) {
+                                                    int ptid, bool with_x, bool with_blocks) {
+  const int c0 = k * kChunk;
+  const int nc = min(kChunk, L.c_in - c0);
+  const size_t hw = (size_t)g.h * g.w;
+  const int n_elem = with_x ? g.pairs * g.rows * g.pitch : 0;
+  const uint32_t chan_b = (uint32_t)g.chan_stride;
+  auto copy_elem = [&](const StagedElem& se, size_t chan_off) {
+    const float* sa = se.off_a >= 0 ? x + se.off_a + chan_off : x;
+    const float* sb = se.off_b >= 0 ? x + se.off_b + chan_off : x;
+    const size_t step_a = se.off_a >= 0 ? hw : 0, step_b = se.off_b >= 0 ? hw : 0;
+    const uint32_t na = se.off_a >= 0 ? 4u : 0u, nb = se.off_b >= 0 ? 4u : 0u;
+    uint32_t dst = stage_base + se.dst;
+    if (nc == kChunk) {   // a whole chunk: straight-line copies
+#pragma unroll
+      for (int cc = 0; cc < kChunk; ++cc) {
+        cp_async4(dst + cc * chan_b, sa + cc * step_a, na);
+        cp_async4(dst + cc * chan_b + 4, sb + cc * step_b, nb);
+      }
+    } else {
+      for (int cc = 0; cc < nc; ++cc) {
+        cp_async4(dst, sa, na);
+        cp_async4(dst + 4, sb, nb);
+        sa += step_a;
+        sb += step_b;
+        dst += chan_b;
+      }
+    }
+  };
+  if (with_x) {
+#pragma unroll
+    for (int i = 0; i < kPreElems; ++i)
+      if (pre[i].dst != kSkipElem) copy_elem(pre[i], (size_t)c0 * hw);
+  }
+  for (int e = ptid + kPreElems * kProducerThreads; e < n_elem; e += kProducerThreads)
+    copy_elem(staged_elem<S>(L, g, tab, e, c0), 0);
+  if (with_blocks) stage_blocks_async(L, g, desc, codes, stage_base, kk, ptid);
+}
+
+// The x part of one chunk copied by `n_threads` threads (thread `t` of them): used by the
+// consumer warps, which have nothing else to do yet, for the first chunks of a launch.  A warp can
+// keep only a few cp.async in flight, so twenty warps fill a chunk several times faster than the
+// four producer warps.
+template <int S>
+__device__ __forceinline__ void fill_chunk_x(const DeviceLayer& L, const Geo& g, const float* __restrict__ x,
+                                             const SubTile* tab, uint32_t stage_base, int k, int t,
+                                             int n_threads) {
   const int c0 = k * kChunk;
   const int nc = min(kChunk, L.c_in - c0);
   const size_t hw = (size_t)g.h * g.w;
   const int n_elem = g.pairs * g.rows * g.pitch;
   const uint32_t chan_b = (uint32_t)g.chan_stride;
-  auto copy_elem = [&](const StagedElem& se, size_t chan_off) {
-    const float* sa = se.off_a >= 0 ? x + se.off_a + chan_off : x;
-    const float* sb = se.off_b >= 0 ? x + se.off_b + chan_off : x;
+  for (int e = t; e < n_elem; e += n_threads) {
+    const StagedElem se = staged_elem<S>(L, g, tab, e, c0);
+    const float* sa = se.off_a >= 0 ? x + se.off_a : x;
+    const float* sb = se.off_b >= 0 ? x + se.off_b : x;
     const size_t step_a = se.off_a >= 0 ? hw : 0, step_b = se.off_b >= 0 ? hw : 0;
     const uint32_t na = se.off_a >= 0 ? 4u : 0u, nb = se.off_b >= 0 ? 4u : 0u;
     uint32_t dst = stage_base + se.dst;
@@ -413,13 +459,7 @@ __device__ __forceinline__ void produce_chunk_async(const DeviceLayer& L, const 
       sb += step_b;
       dst += chan_b;
     }
-  };
-#pragma unroll
-  for (int i = 0; i < kPreElems; ++i)
-    if (pre[i].dst != kSkipElem) copy_elem(pre[i], (size_t)c0 * hw);
-  for (int e = ptid + kPreElems * kProducerThreads; e < n_elem; e += kProducerThreads)
-    copy_elem(staged_elem<S>(L, g, tab, e, c0), 0);
-  if (with_blocks) stage_blocks_async(L, g, desc, codes, stage_base, kk, ptid);
+  }
 }
 
 // ---- fp16 storage, even image width: raw ring ----------------------------------------------------
@@ -998,6 +1038,9 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   if (warp < kCW && active && lane < kGroup) my_o = __ldg(L.perm + gi * kGroup + lane);
   u64 acc[GENERIC ? kGroup : 1][4];
   bool ok = true;
+  // fp32 element-wise staging: the consumer warps copy the x part of the first chunks themselves
+  // (one per warp of a unit), the producers only their weight blocks
+  const int n_coop = (!g.is_half && g.raw_stages == 0) ? min(min(zs, g.stages), nk) : 0;
 
   if (warp >= kCW) {
     // ===================================== producer warps =====================================
@@ -1033,7 +1076,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
           if (it > 0 && !mbar_wait(sbase + 8 * (kMaxStages + s), (it - 1) & 1, L.err, 1)) break;
           const uint32_t stage_base = sbase + g.stage_off + s * g.stage_bytes;
           produce_chunk_async<S>(L, g, (const float*)x, tab, pre, desc, codes, stage_base, k0 + kk, kk, ptid,
-                                 kk >= n_early);
+                                 kk >= n_coop, kk >= n_early);
           cp_async_arrive(sbase + 8 * s);
         }
       }
@@ -1051,6 +1094,13 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (n_coop > 0) {
+      for (int kk = 0; kk < n_coop; ++kk)
+        fill_chunk_x<S>(L, g, (const float*)x, tab, sbase + g.stage_off + kk * g.stage_bytes, k0 + kk,
+                        warp * 32 + lane, 32 * kCW);
+      asm volatile("cp.async.wait_all;" ::: "memory");
+      asm volatile("bar.sync 11, %0;" ::"n"(32 * kCW) : "memory");   // every consumer's copies have landed
+    }
     if (bias && my_o >= 0) my_b = __ldg(bias + my_o);
 
 #ifdef PCONV_TRACE
