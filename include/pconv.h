@@ -314,7 +314,16 @@ pconv_status pconv_stack_forward_host(pconv_stack* s, const void* x_host, void* 
                                       void* stream);
 
 /* Releases the stack (not the handles).  NULL is allowed. */
+/* Captures one forward from x_dev to y_dev into a CUDA graph kept by the stack (replacing an
+ * earlier one), on a stream that allows capture (not the legacy default stream:
+ * PCONV_ERR_UNSUPPORTED); the launches keep their programmatic dependencies inside the graph.
+ * pconv_stack_replay launches it; x_dev and y_dev must then still be the same buffers.
+ * pconv_stack_forward_host captures and replays on its own buffers where it can. */
+pconv_status pconv_stack_capture(pconv_stack* s, const void* x_dev, void* y_dev, void* stream);
+pconv_status pconv_stack_replay(pconv_stack* s, void* stream);
+
 void pconv_stack_free(pconv_stack* s);
+
 
 #ifdef __cplusplus
 }

@@ -27,7 +27,7 @@ EXPORTS = ["pconv_pack", "pconv_forward", "pconv_forward_ws", "pconv_forward_sta
            "pconv_free", "pconv_maxpool2x2", "pconv_unpack",
            "pconv_stats", "pconv_filter_order", "pconv_device_status", "pconv_trace_read", "pconv_status_str",
            "pconv_stack_create", "pconv_stack_out_shape", "pconv_stack_forward",
-           "pconv_stack_forward_host", "pconv_stack_free",
+           "pconv_stack_forward_host", "pconv_stack_free", "pconv_stack_capture", "pconv_stack_replay",
            "pconv_project", "pconv_project_workspace_bytes"]
 
 
@@ -96,6 +96,8 @@ def lib():
         L.pconv_stack_out_shape.argtypes = [vp, ip, ip, ip, ip]
         L.pconv_stack_forward.argtypes = [vp, vp, vp, vp]
         L.pconv_stack_forward_host.argtypes = [vp, vp, vp, vp]
+        L.pconv_stack_capture.argtypes = [vp, vp, vp, vp]
+        L.pconv_stack_replay.argtypes = [vp, vp]
         L.pconv_stack_free.argtypes = [vp]
         L.pconv_stack_free.restype = None
         _lib = L
@@ -353,6 +355,15 @@ class Stack:
         _check(lib().pconv_stack_forward(self.ptr, ctypes.c_void_p(x.data_ptr()),
                                          ctypes.c_void_p(y.data_ptr()), _stream_ptr(stream)),
                "pconv_stack_forward")
+
+    def capture(self, x, y, stream):
+        """Captures one forward x -> y into a CUDA graph (stream: a non-default torch stream)."""
+        _check(lib().pconv_stack_capture(self.ptr, ctypes.c_void_p(x.data_ptr()),
+                                         ctypes.c_void_p(y.data_ptr()), _stream_ptr(stream)),
+               "pconv_stack_capture")
+
+    def replay(self, stream=None):
+        _check(lib().pconv_stack_replay(self.ptr, _stream_ptr(stream)), "pconv_stack_replay")
 
     def forward_host(self, x_host, y_host, stream=None):
         """x_host / y_host: CPU torch tensors or numpy arrays (pinned memory makes it async)."""

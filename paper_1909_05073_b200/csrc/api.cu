@@ -223,6 +223,12 @@ struct pconv_stack {
   void* io[2];    // device input / output used by the host entry point
   void* ws;       // channel-split workspace shared by the layers (kept zeroed between launches)
   size_t ws_bytes;
+  // a captured forward (pconv_stack_capture) and the buffers it was captured for
+  cudaGraphExec_t graph_exec;
+  const void* graph_x;
+  void* graph_y;
+  cudaGraphExec_t host_exec;   // the host entry point's own graph (io[0] -> io[1])
+  bool host_graph_failed;      // its capture was tried and is not possible on the stream given
 };
 
 extern "C" void pconv_stack_free(pconv_stack* s) {
@@ -232,6 +238,8 @@ extern "C" void pconv_stack_free(pconv_stack* s) {
     if (s->io[i]) cudaFree(s->io[i]);
   }
   if (s->ws) cudaFree(s->ws);
+  if (s->graph_exec) cudaGraphExecDestroy(s->graph_exec);
+  if (s->host_exec) cudaGraphExecDestroy(s->host_exec);
   delete[] s->layers;
   delete[] s->bias;
   delete[] s->pool;
@@ -357,15 +365,78 @@ extern "C" pconv_status pconv_stack_forward(pconv_stack* s, const void* x, void*
   return PCONV_OK;
 }
 
+static pconv_status capture_forward(pconv_stack* s, const void* x, void* y, void* stream_v,
+                                    cudaGraphExec_t* exec) {
+  cudaStream_t stream = (cudaStream_t)stream_v;
+  if (*exec) {
+    cudaGraphExecDestroy(*exec);
+    *exec = nullptr;
+  }
+  // the legacy default stream cannot be captured
+  if (stream == nullptr || stream == cudaStreamLegacy) return PCONV_ERR_UNSUPPORTED;
+  if (cudaStreamBeginCapture(stream, cudaStreamCaptureModeRelaxed) != cudaSuccess) {
+    cudaGetLastError();
+    return PCONV_ERR_CUDA;
+  }
+  const pconv_status st = pconv_stack_forward(s, x, y, stream_v);
+  cudaGraph_t graph = nullptr;
+  const cudaError_t e = cudaStreamEndCapture(stream, &graph);
+  if (st != PCONV_OK || e != cudaSuccess || !graph) {
+    cudaGetLastError();
+    if (graph) cudaGraphDestroy(graph);
+    return st != PCONV_OK ? st : PCONV_ERR_CUDA;
+  }
+  const cudaError_t ei = cudaGraphInstantiate(exec, graph, 0);
+  cudaGraphDestroy(graph);
+  if (ei != cudaSuccess) {
+    cudaGetLastError();
+    *exec = nullptr;
+    return PCONV_ERR_CUDA;
+  }
+  return PCONV_OK;
+}
+
+extern "C" pconv_status pconv_stack_capture(pconv_stack* s, const void* x, void* y, void* stream_v) {
+  if (!s || !x || !y) return PCONV_ERR_NULL;
+  const pconv_status st = capture_forward(s, x, y, stream_v, &s->graph_exec);
+  s->graph_x = st == PCONV_OK ? x : nullptr;
+  s->graph_y = st == PCONV_OK ? y : nullptr;
+  return st;
+}
+
+extern "C" pconv_status pconv_stack_replay(pconv_stack* s, void* stream_v) {
+  if (!s) return PCONV_ERR_NULL;
+  if (!s->graph_exec) return PCONV_ERR_UNSUPPORTED;
+  if (cudaGraphLaunch(s->graph_exec, (cudaStream_t)stream_v) != cudaSuccess) {
+    cudaGetLastError();
+    return PCONV_ERR_CUDA;
+  }
+  return PCONV_OK;
+}
+
 extern "C" pconv_status pconv_stack_forward_host(pconv_stack* s, const void* x_host, void* y_host,
                                                  void* stream_v) {
   if (!s || !x_host || !y_host) return PCONV_ERR_NULL;
   cudaStream_t stream = (cudaStream_t)stream_v;
+  // the device part always runs on the stack's own input / output buffers: replay it from a graph
+  // captured on first use where the stream allows capture
+  if (!s->host_exec && !s->host_graph_failed &&
+      capture_forward(s, s->io[0], s->io[1], stream_v, &s->host_exec) != PCONV_OK)
+    s->host_graph_failed = true;
+  const bool replay = s->host_exec != nullptr;
   if (cudaMemcpyAsync(s->io[0], x_host, s->in_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
     cudaGetLastError();
     return PCONV_ERR_CUDA;
   }
-  pconv_status st = pconv_stack_forward(s, s->io[0], s->io[1], stream_v);
+  pconv_status st = PCONV_OK;
+  if (replay) {
+    if (cudaGraphLaunch(s->host_exec, stream) != cudaSuccess) {
+      cudaGetLastError();
+      st = PCONV_ERR_CUDA;
+    }
+  } else {
+    st = pconv_stack_forward(s, s->io[0], s->io[1], stream_v);
+  }
   if (st != PCONV_OK) return st;
   if (cudaMemcpyAsync(y_host, s->io[1], s->out_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
       cudaStreamSynchronize(stream) != cudaSuccess) {

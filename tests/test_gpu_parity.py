@@ -412,3 +412,40 @@ def test_stack_matches_the_chained_oracle(storage):
     assert torch.equal(y_host, y.cpu()) or storage == "f32" and np.allclose(
         y_host.numpy(), y.cpu().numpy(), rtol=0, atol=1e-5)
     stack.close()
+
+
+def test_stack_graph_replay_matches_the_eager_forward():
+    chans = [(3, 16), (16, 32), (32, 32), (32, 48)]
+    pools = [False, True, False, True]
+    h = 24
+    layers = []
+    for i, (ci, co) in enumerate(chans):
+        spec = synth.LayerSpec("g%d" % i, ci, co, h, h, 1, 1.0 if i == 0 else 0.5, sigma=None, x_dist="uniform_01")
+        w, b, _ = synth.gen_weights(spec, 700 + i)
+        layers.append(B.Layer(w, synth.PATTERNS8, 1, B.F32, b))
+    stack = B.Stack(layers, pools, 1, h, h, B.RELU)
+    x = torch.rand(1, 3, h, h, device="cuda")
+    y_eager = torch.empty(stack.out_shape, device="cuda")
+    y_graph = torch.zeros(stack.out_shape, device="cuda")
+    stack.forward(x, y_eager)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    with pytest.raises(B.PconvError):
+        stack.replay(side)                      # nothing captured yet
+    stack.capture(x, y_graph, side)
+    for _ in range(3):                          # replays reuse the (zeroed) workspace correctly
+        y_graph.zero_()
+        side.synchronize()
+        stack.replay(side)
+        side.synchronize()
+        assert torch.equal(y_graph, y_eager) or torch.allclose(y_graph, y_eager, rtol=1e-5, atol=1e-6)
+    # the host entry point captures on its own buffers when the stream allows it
+    xh = x.cpu().pin_memory()
+    yh = torch.empty(stack.out_shape).pin_memory()
+    for _ in range(2):
+        stack.forward_host(xh, yh, side)
+        assert torch.allclose(yh, y_eager.cpu(), rtol=1e-5, atol=1e-6)
+    stack.forward_host(xh, yh)                  # default stream: eager path
+    assert torch.allclose(yh, y_eager.cpu(), rtol=1e-5, atol=1e-6)
+    assert B.pconv_device_status(layers[0].handle)[0] == 0
+    stack.close()
