@@ -1,34 +1,37 @@
 // Tiled pattern-sparse 3x3 convolution for sm_100a.
 //
-// One CTA = consumer warps + 4 producer warps (warp-specialised).  The consumer warps form a
-// (wy x ng) grid: ng filter groups of 16 filters that share the staged input, wy independent sets
-// of pixel sub-tiles.  Lanes are pixels: a lane owns a column of 4 output rows in each of two
-// sub-tiles ("A" and "B"), and the two are interleaved as float2 in shared memory so that every
-// multiply-add is a packed fma.rn.f32x2 (one issue slot per two FMAs) on naturally aligned
-// register pairs:  acc[g][k].{A,B} += {w,w} * win[row][col].{A,B}.
+// One CTA = consumer warps + 4 producer warps (warp-specialised), one CTA per SM.  Lanes are pixels:
+// a lane owns a column of 4 output rows in each of two sub-tiles ("A" and "B"), and the two are
+// interleaved as float2 in shared memory so that every multiply-add is a packed fma.rn.f32x2 (one
+// issue slot per two FMAs) on naturally aligned register pairs:
+//     acc[slot][k].{A,B} += {w,w} * win[row][col].{A,B}.
+// A consumer warp works for one unit = (256 pixels, a group of 16 filters).  Per input channel a
+// lane loads its register window once (6x3 float2 at stride 1, 9x3 at stride 2) and reuses it for
+// every surviving kernel of the unit's 16 filters on that channel.  Which kernels survive, for which
+// filter slot and with which pattern, is a code stream written by the packer; pruned kernels cost
+// nothing and no lane ever diverges.
 //
-// Per input channel a lane loads its register window once (6x3 float2 at stride 1, 9x3 at stride 2)
-// and reuses it for every surviving kernel of the warp's 16 filters on that channel.  Which kernels
-// survive, for which filter slot and with which pattern, is a byte-code stream written by the
-// packer; pruned kernels cost nothing and no lane ever diverges.
-//
-// Two consumer variants:
-//  * canonical pattern sets (GENERIC = false): 16 consumer warps whose accumulators live in Tensor
-//    Memory.  TMEM is addressed at run time, so the filter slot is data, not code: a warp-uniform
-//    indexed jump selects one of 8 straight-line bodies specialised on the pattern only (exactly 4
-//    taps), which reads the slot's 8 accumulator columns, runs 16 packed FMAs and writes them back.
-//    The hot code (~4 KB) stays inside the per-scheduler instruction cache and the jump latency is
-//    covered by the other warps (see gen_dispatch.py for the measurements behind this).
-//  * any 4-of-9 masks (GENERIC = true): 8 consumer warps with register accumulators, a switch on
-//    the filter slot and nine warp-uniform tap tests per kernel (no register re-allocation between
-//    the roles: 384 threads leave 168 registers each, which the accumulators fit).
+// Consumer variants (template parameters GENERIC, WIDE):
+//  * Tensor-Memory accumulators (GENERIC = false): 16 consumer warps.  TMEM is addressed at run
+//    time, so the filter slot is data, not code: a warp-uniform indexed jump selects a straight-line
+//    body specialised on the 4-tap mask only, which reads the slot's 8 accumulator columns, runs 16
+//    packed FMAs and writes them back (gen_dispatch.py).  WIDE = false: the eight canonical masks,
+//    one-byte codes; WIDE = true: a body for each of the 126 masks, two-byte codes.
+//    zs = 1, 2 or 4 warps of one TMEM lane quadrant may share a unit: they draw the chunks of the
+//    channel range from a counter, accumulate in their own columns, and add the column sets up
+//    before the epilogue.  The channel range can also be split across CTAs (grid.z), with fp32
+//    atomics into a workspace and per-warp tickets that elect who finishes each part of a tile.
+//  * run-time masks (GENERIC = true): 8 consumer warps with register accumulators, a switch on the
+//    filter slot and nine warp-uniform tap tests per kernel (384 threads leave 168 registers each,
+//    which the accumulators fit); a slower cross-check of the generated bodies.
 //
 // Producer warps stage, per chunk of 8 input channels, the halo'd sub-tiles (zero-filled outside
-// the image, converted from fp16 when the storage type is fp16) and the chunk's weight records
-// (duplicated to {w,w} pairs) and codes, through a ring of shared-memory stages guarded by
-// full/empty mbarriers.  Every wait is bounded; a wait that runs out records its id in the
-// layer's status word and the warp stops working but still reaches the common exit, where the
-// TMEM allocation is released.
+// the image; fp16 storage goes through a raw ring and is widened from shared memory) and the
+// chunk's weight records and codes, through a ring of shared-memory stages guarded by full/empty
+// mbarriers.  Every wait is bounded; a wait that runs out records its id in the layer's status word
+// and the warp stops working but still reaches every barrier and the common exit, where the TMEM
+// allocation is released.  Launches use programmatic stream serialisation: set-up runs while the
+// previous kernel finishes, and griddepcontrol.wait precedes the first access to activations.
 #include <cuda_fp16.h>
 
 #include <type_traits>
@@ -51,7 +54,7 @@ __host__ __device__ constexpr int cta_threads(bool generic) {
 constexpr int kTmemCols = 512;  // whole TMEM of the SM: 16 warps x 16 slots x 8 columns
 constexpr int kMaxStages = 8;
 constexpr int kWSlot = kMaxBlockKernels * 16 + 16;  // bytes per (group, stage): 4 fp32 per kernel
-constexpr int kCodeSlot = 400;                 // bytes per (group, stage): <= 24 records of 7 codes
+constexpr int kCodeSlot = 400;                 // bytes per (group, stage): <= 24 records of 7 wide codes
 constexpr int kWRawSlot = kMaxBlockKernels * 8;  // fp16 weight records of one (group, chunk)
 constexpr int kRawStages = 3;
 constexpr uint32_t kSpinLimit = 1u << 20;
