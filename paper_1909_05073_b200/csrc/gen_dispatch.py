@@ -13,8 +13,7 @@ Why PTX text, and why this shape (all measured on B200):
  * so the filter slot is taken out of the code: accumulators live in Tensor Memory (TMEM), which is
    addressed at run time.  A body is specialised on the pattern only: it waits for
    the slot's 8 accumulator columns (requested by the previous body), runs the 16 packed FMAs of
-   the 4 taps, writes the columns back in two halves and refills each half's registers with the
-   next kernel's columns at once, then jumps.
+   the 4 taps, writes the columns back, requests the next kernel's columns, then jumps.
 
 Shared-memory loads, TMEM loads and TMEM stores all pass through one memory-instruction queue
 that retires roughly one instruction per 7-9 cycles per scheduler, whatever its width; with 16
