@@ -1069,17 +1069,20 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
         const uint32_t stage_base = sbase + g.stage_off + kk * g.stage_bytes;
         if (g.is_half) stage_blocks_half(L, g, desc, codes, stage_base, kk, ptid);
         else stage_blocks_async(L, g, desc, codes, stage_base, kk, ptid);
+        // chunks whose x the consumers copy are complete, for the producers, once their blocks have
+        // landed: arrive now, so that the barrier does not also wait for the later chunks' blocks
+        if (kk < n_coop) cp_async_arrive(sbase + 8 * kk);
       }
       asm volatile("griddepcontrol.wait;" ::: "memory");
       if (g.is_half) {
         produce_half_stream<S>(L, g, (const __half*)x, tab, pre, desc, codes, sbase, k0, nk, n_early, ptid);
       } else {
-        for (int kk = 0; kk < nk; ++kk) {
+        for (int kk = n_coop; kk < nk; ++kk) {
           const int s = kk % g.stages, it = kk / g.stages;
           if (it > 0 && !mbar_wait(sbase + 8 * (kMaxStages + s), (it - 1) & 1, L.err, 1)) break;
           const uint32_t stage_base = sbase + g.stage_off + s * g.stage_bytes;
           produce_chunk_async<S>(L, g, (const float*)x, tab, pre, desc, codes, stage_base, k0 + kk, kk, ptid,
-                                 kk >= n_coop, kk >= n_early);
+                                 true, kk >= n_early);
           cp_async_arrive(sbase + 8 * s);
         }
       }
