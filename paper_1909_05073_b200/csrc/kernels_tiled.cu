@@ -53,6 +53,7 @@ __host__ __device__ constexpr int cta_threads(bool generic) {
 }
 constexpr int kTmemCols = 512;  // whole TMEM of the SM: 16 warps x 16 slots x 8 columns
 constexpr int kMaxStages = 8;
+constexpr int kMaxCoop = 4;   // chunks whose x the consumer warps copy at the start of a launch
 constexpr int kWSlot = kMaxBlockKernels * 16 + 16;  // bytes per (group, stage): 4 fp32 per kernel
 constexpr int kCodeSlot = 400;                 // bytes per (group, stage): <= 24 records of 7 wide codes
 constexpr int kWRawSlot = kMaxBlockKernels * 8;  // fp16 weight records of one (group, chunk)
@@ -953,7 +954,9 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   // grid to finish before it touches activations, see below).
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (tid < kCW) unit_ctr[tid] = 0;
+  const uint32_t coop_bar = sbase + 8 * 2 * kMaxStages + 16 + 64;   // kMaxCoop barriers
   if (tid == 0) {
+    for (int j = 0; j < kMaxCoop; ++j) mbar_init(coop_bar + 8 * j, 32 * kCW);
     for (int s = 0; s < g.stages; ++s) {
       mbar_init(sbase + 8 * s, 32 * kProducerWarps);
       mbar_init(sbase + 8 * (kMaxStages + s), kCW / (GENERIC ? 1 : g.zs));
@@ -1043,7 +1046,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   bool ok = true;
   // fp32 element-wise staging: the consumer warps copy the x part of the first chunks themselves
   // (one per warp of a unit), the producers only their weight blocks
-  const int n_coop = (!g.is_half && g.raw_stages == 0) ? min(min(zs, g.stages), nk) : 0;
+  const int n_coop = (!g.is_half && g.raw_stages == 0) ? min(min(zs, g.stages), min(nk, kMaxCoop)) : 0;
 
   if (warp >= kCW) {
     // ===================================== producer warps =====================================
@@ -1100,12 +1103,12 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (n_coop > 0) {
-      for (int kk = 0; kk < n_coop; ++kk)
-        fill_chunk_x<S>(L, g, (const float*)x, tab, sbase + g.stage_off + kk * g.stage_bytes, k0 + kk,
-                        warp * 32 + lane, 32 * kCW);
-      asm volatile("cp.async.wait_all;" ::: "memory");
-      asm volatile("bar.sync 11, %0;" ::"n"(32 * kCW) : "memory");   // every consumer's copies have landed
+    // (each consumer thread arrives on the chunk's own barrier when its copies for that chunk
+    // have landed; a warp waits for that barrier as well as for the producers' before the chunk)
+    for (int kk = 0; kk < n_coop; ++kk) {
+      fill_chunk_x<S>(L, g, (const float*)x, tab, sbase + g.stage_off + kk * g.stage_bytes, k0 + kk,
+                      warp * 32 + lane, 32 * kCW);
+      cp_async_arrive(coop_bar + 8 * kk);
     }
     if (bias && my_o >= 0) my_b = __ldg(bias + my_o);
 
@@ -1133,6 +1136,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
       const long long tc0 = clock64();
 #endif
       ok = mbar_wait(sbase + 8 * s, (kk / g.stages) & 1, L.err, 2);
+      if (ok && kk < n_coop) ok = mbar_wait(coop_bar + 8 * kk, 0, L.err, 3);
       if (!ok) break;
 #ifdef PCONV_TRACE
       const long long tc1 = clock64();
@@ -1338,7 +1342,7 @@ bool geo_for(const DeviceLayer& L, int n, int h, int w, int zs, Geo* out) {
   g.substride = g.pitch * g.colstride;
   if (g.tw == 4) while (g.substride % 128 != 64) g.substride += 16;
   if (g.tw == 2) while (g.substride % 128 != 32) g.substride += 16;
-  g.tab_off = 8 * 2 * kMaxStages + 16 + 64;  // barriers, the TMEM base address word, unit counters
+  g.tab_off = 8 * 2 * kMaxStages + 16 + 64 + 8 * kMaxCoop;  // barriers, TMEM base word, unit counters, first-chunk barriers
   if (L.n_chunks > 512) return false;   // descriptor table budget (c_in <= 4096)
   g.ks = 1;
   g.cps = L.n_chunks;
