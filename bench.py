@@ -3,17 +3,23 @@
 the four 2x2 max-pools after conv2/4/7/10, fused into those layers' epilogues) on one 224x224 image
 per GPU, fp32.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-configs]
+    python bench.py --layer C_IN,C_OUT,H,N,STRIDE,KEEP[,f32|f16[,4|8|12[,split]]]  [--steps K]
+    python bench.py --layer cfg5:0          (layer 0 of benchmark configuration 5, at its batch)
 
 A step is one pass of the whole stack over one image (per rank).  `value` is effective TFLOP/s
 (2 x surviving multiply-adds of all ranks / device time, inputs resident in HBM); `e2e` is the same
 figure through the host entry point (input copied from pinned host memory and the result copied
-back inside the timed region).  `--impl reference` times the CPU oracle on the same workload.
-Under torchrun every rank runs its own image (batch sharding, no collective on the data path).
+back inside the timed region).  `configs` holds, for the other four benchmark configurations, the
+time, effective TFLOP/s and roofline fraction of every layer.  `--impl reference` times the CPU
+oracle on the same workload.  Under torchrun every rank runs its own image (batch sharding, no
+collective on the data path).  `--layer` times one layer alone (the small case used for profiler
+captures) and prints its launch plan.
 """
 import argparse
 import json
 import os
+import re
 import statistics
 import subprocess
 import sys
@@ -29,8 +35,31 @@ from paper_1909_05073_b200 import synth  # noqa: E402
 
 CID = 2
 METRIC = "pattern-conv effective TFLOP/s (2 x surviving MACs / s), VGG-16 conv stack, batch 1 per GPU"
-# FP32 FMA peak of the part: SMs x 128 lanes x 2 flop x max SM clock
+WORKLOAD = ("config 2: VGG-16 conv stack (13 conv + 4 fused max-pool), 224x224x3, batch 1 per GPU, "
+            "fp32, 8 patterns, keep 1.0 (conv1) / 0.3")
+# FP32 FMA peak of the part: SMs x 128 lanes x 2 flop x max SM clock (derived; a register-only
+# fma.rn.f32x2 loop measured 74.1 TFLOP/s on this machine, see profiles/fp32_peak.md)
 ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+
+
+def hbm_peak_gbs():
+    """(GB/s, source): the measured copy bandwidth of this machine's B200s, else the stated fallback."""
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json)"
+    except (OSError, KeyError, ValueError):
+        return 6650.0, "fallback (earlier measurement on this pool)"
+
+
+def recorded_traffic():
+    """dram__bytes_read + dram__bytes_write of the conv launches of one bench step, from the
+    profiler summary under profiles/ (a line `traffic_bytes_per_step = N`), or None."""
+    try:
+        text = open(os.path.join(ROOT, "profiles", "bench_vgg16_n1_launch_list.md")).read()
+        m = re.search(r"traffic_bytes_per_step\s*=\s*([0-9.eE+]+)", text)
+        return float(m.group(1)) if m else None
+    except OSError:
+        return None
 
 
 def build_workload():
@@ -43,15 +72,28 @@ def build_workload():
     return cfg, layers, x
 
 
+def layer_flops(spec, kept, n=1):
+    return 2 * 4 * kept * spec.h_out * spec.w_out * n
+
+
+def layer_bytes(spec, kept, n=1, es=4):
+    """Minimal HBM bytes of a layer: input once, output once, 4 values + 2 index bytes per
+    surviving kernel, bias."""
+    return (es * n * (spec.c_in * spec.h * spec.w + spec.c_out * spec.h_out * spec.w_out)
+            + kept * (4 * es + 2) + 4 * spec.c_out)
+
+
+def layer_roof_us(spec, kept, n, es, hbm_gbs):
+    return max(layer_flops(spec, kept, n) / (ALU_PEAK_TFLOPS * 1e12),
+               layer_bytes(spec, kept, n, es) / (hbm_gbs * 1e9)) * 1e6
+
+
 def surviving_flops(layers):
-    return sum(2 * 4 * kept * s.h_out * s.w_out for s, _, _, kept in layers)
+    return sum(layer_flops(s, kept) for s, _, _, kept in layers)
 
 
 def algorithmic_bytes(layers):
-    """Minimal HBM bytes of the conv layers: input once, output once, 4 values + 2 index bytes per
-    surviving kernel, bias."""
-    return sum(4 * (s.c_in * s.h * s.w + s.c_out * s.h_out * s.w_out) + kept * 18 + 4 * s.c_out
-               for s, _, _, kept in layers)
+    return sum(layer_bytes(s, kept) for s, _, _, kept in layers)
 
 
 class ClockSampler:
@@ -133,14 +175,125 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "config 2: VGG-16 conv stack, 224x224x3, batch 1, fp32, 8 patterns, "
-                               "keep 1.0 / 0.3", "images_per_step": 1},
+        "config": {"workload": WORKLOAD, "images_per_step": 1},
         "ms_per_image": ms,
         "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
                          "sample": "whole stack (13 conv + 4 pool), 1 image per step, dense "
                                    "direct convolution in fp64"},
         "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
+
+
+def _time_launch(torch, flush, fn, reps):
+    """Median device time (us) of fn() over `reps` launches, L2 flushed before each."""
+    us = []
+    for _ in range(reps):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        us.append(e0.elapsed_time(e1) * 1e3)
+    return float(np.median(us))
+
+
+def measure_config(torch, B, flush, cid, batch, reps, hbm_gbs):
+    """Every layer of one benchmark configuration, each launch timed alone with CUDA events after
+    an L2 flush, as a layer stack launches it (workspace for the channel split, fused pool)."""
+    cfg = synth.config(cid, batch)
+    half = cfg.storage == "f16"
+    st, es = (B.F16, 2) if half else (B.F32, 4)
+    tdtype = torch.float16 if half else torch.float32
+    rows, layers = [], []
+    x_next = None
+    for li, spec in enumerate(cfg.layers):
+        w, b, ids = synth.gen_weights(spec, synth.layer_seed(cid, li), cfg.patterns)
+        kept = int((ids >= 0).sum())
+        layer = B.Layer(w, cfg.patterns, spec.stride, st, b, strict4=True)
+        layers.append(layer)
+        if cfg.chained and x_next is not None:
+            x = x_next
+        else:
+            x = torch.from_numpy(synth.gen_input(spec, cfg.batch, synth.layer_seed(cid, li))).cuda().to(tdtype)
+        pool = bool(cfg.chained and spec.pool_after)
+        n_, c_, h_, w_ = layer.out_shape(x.shape)
+        y = torch.empty((n_, c_, h_ // 2, w_ // 2) if pool else (n_, c_, h_, w_), dtype=tdtype, device="cuda")
+        layer.forward(x, relu=True, out=y, split=True, pool=pool)      # warm-up (and the chain's data)
+        us = _time_launch(torch, flush, lambda: layer.forward(x, relu=True, out=y, split=True, pool=pool), reps)
+        roof = layer_roof_us(spec, kept, cfg.batch, es, hbm_gbs)
+        row = {"layer": spec.name, "us": round(us, 2), "roof_us": round(roof, 3),
+               "frac": round(roof / us, 4),
+               "tflops": round(layer_flops(spec, kept, cfg.batch) / us / 1e6, 3)}
+        if cid == 5:
+            s = layer.stats()
+            mean = s.kept_kernels / max(s.n_groups, 1)
+            row["group_kernels_max_over_mean"] = round(s.max_group_kernels / mean, 4)
+        rows.append((row, layer_flops(spec, kept, cfg.batch), roof))
+        x_next = y if cfg.chained else None
+    status = [B.pconv_device_status(l.handle)[0] for l in layers]
+    if any(status):
+        raise SystemExit("device reported an abandoned wait in config %d" % cid)
+    total_us = sum(r["us"] for r, _, _ in rows)
+    flops = sum(f for _, f, _ in rows)
+    roof = sum(r for _, _, r in rows)
+    out = {"workload": "config %d: %s, batch %d, %s" % (cid, cfg.name, cfg.batch, cfg.storage),
+           "ms": round(total_us / 1e3, 4), "ms_per_image": round(total_us / 1e3 / cfg.batch, 5),
+           "tflops": round(flops / total_us / 1e6, 3), "roof_us": round(roof, 2),
+           "frac": round(roof / total_us, 4), "timing": "sum of the layers' launches timed alone",
+           "layers": [r for r, _, _ in rows]}
+    for l in layers:
+        l.close()
+    return out
+
+
+def run_layer(args):
+    """One layer alone: plan, median time, effective TFLOP/s (the case profiler captures use)."""
+    import torch
+    from paper_1909_05073_b200 import binding as B
+    from paper_1909_05073_b200 import build as pbuild
+    pbuild.build()
+    torch.cuda.set_device(0)
+    a = args.layer.split(",")
+    split = "split" in a
+    a = [v for v in a if v != "split"]
+    if a[0].startswith("cfg"):
+        cid, li = a[0][3:].split(":")[:2]
+        cfg = synth.config(int(cid), int(a[1]) if len(a) > 1 else None)
+        spec, n, patterns = cfg.layers[int(li)], cfg.batch, cfg.patterns
+        storage = cfg.storage
+        seed = synth.layer_seed(int(cid), int(li))
+        split = True
+    else:
+        c_in, c_out, h, n, stride = (int(v) for v in a[:5])
+        spec = synth.LayerSpec("layer", c_in, c_out, h, h, stride, float(a[5]))
+        storage = a[6] if len(a) > 6 else "f32"
+        patterns = {4: synth.SCP4, 8: synth.PATTERNS8, 12: synth.PATTERNS12}[int(a[7]) if len(a) > 7 else 8]
+        seed = 1
+    half = storage == "f16"
+    w, b, ids = synth.gen_weights(spec, seed, patterns)
+    kept = int((ids >= 0).sum())
+    layer = B.Layer(w, patterns, spec.stride, B.F16 if half else B.F32, b)
+    x = torch.from_numpy(synth.gen_input(spec, n, seed)).cuda()
+    if half:
+        x = x.half()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    y = layer.forward(x, split=split)
+    for _ in range(max(args.warmup - 1, 0)):
+        layer.forward(x, out=y, split=split)
+    us = _time_launch(torch, flush, lambda: layer.forward(x, out=y, split=split), args.steps)
+    hbm, src = hbm_peak_gbs()
+    roof = layer_roof_us(spec, kept, n, 2 if half else 4, hbm)
+    assert B.pconv_device_status(layer.handle)[0] == 0
+    print(json.dumps({
+        "layer": {"c_in": spec.c_in, "c_out": spec.c_out, "h": spec.h, "w": spec.w, "n": n,
+                  "stride": spec.stride, "keep": spec.keep, "storage": storage,
+                  "patterns": len(patterns), "kept_kernels": kept, "workspace": split},
+        "plan": B.pconv_plan(layer.handle, n, spec.h, spec.w, 0, split),
+        "us": round(us, 2), "tflops": round(layer_flops(spec, kept, n) / us / 1e6, 3),
+        "frac_of_alu_peak": round(layer_flops(spec, kept, n) / us / 1e6 / ALU_PEAK_TFLOPS, 4),
+        "roof_us": round(roof, 3), "frac": round(roof / us, 4), "hbm_peak": src,
+        "l2": "flushed before every timed launch"}))
 
 
 def run_ours(args):
@@ -262,12 +415,13 @@ def run_ours(args):
     t = max_over_ranks([ms_total, e2e_total * 1e3], device="cuda")
     ms_step = t[0] / args.steps
     e2e_ms = t[1] / args.steps
-    status, where = B.pconv_device_status(conv_layers[0].handle)
-    if status != 0:
+    status, where = stack.status()
+    if status != 0 or any(B.pconv_device_status(l.handle)[0] for l in conv_layers):
         raise SystemExit("device reported an abandoned wait (%d)" % where)
 
     if rank == 0:
         import oracle
+        hbm_gbs, hbm_src = hbm_peak_gbs()
         t0 = time.perf_counter()
         a_ref = x_np
         for spec, w, b, _ in layers:
@@ -279,6 +433,7 @@ def run_ours(args):
         err = np.abs(got - a_ref)
         parity_ok = bool((err <= 1e-4 * (1 + np.abs(a_ref))).all())
         conv_time_ms = sum(conv_ms)
+        roofs = [layer_roof_us(s, kept, 1, 4, hbm_gbs) for s, _, _, kept in layers]
         # The timed region launches nothing but the 13 conv kernels (pools fused), so its duration
         # is theirs, overlap between consecutive launches included; the launches timed one by one
         # (no overlap) are reported beside it.
@@ -290,12 +445,12 @@ def run_ours(args):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
-            "config": {"workload": "config 2: VGG-16 conv stack, 224x224x3, batch 1 per GPU, fp32, "
-                                   "8 patterns, keep 1.0 (conv1) / 0.3", "images_per_step": world,
-                       "l2": "flushed between timed steps (256 MB write)", "parallelism": "batch sharding, no collective"},
+            "config": {"workload": WORKLOAD, "images_per_step": world,
+                       "l2": "flushed between timed steps (256 MB write)",
+                       "parallelism": "batch sharding, no collective"},
             "ms_per_image": ms_step,
             "surviving_gflop_per_image": flops / 1e9,
-            "roofline_time_us_per_image": flops / (ALU_PEAK_TFLOPS * 1e12) * 1e6,
+            "roofline_time_us_per_image": sum(roofs),
             "clocks": clocks,
             "e2e": {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                     "ms_per_step": e2e_ms, "h2d_bytes_per_step": int(x_host.numel() * 4),
@@ -308,18 +463,37 @@ def run_ours(args):
                          "achieved": achieved, "peak": ALU_PEAK_TFLOPS, "unit": "TFLOP/s",
                          "frac": achieved / ALU_PEAK_TFLOPS,
                          "peak_source": "148 SMs x 128 FP32 lanes x 2 x 1.965 GHz (derived; "
-                                        "no FP32 figure in MEASURED_PEAKS.json)",
+                                        "no FP32 figure in MEASURED_PEAKS.json; an FFMA2 loop "
+                                        "measured 74.1, profiles/fp32_peak.md)",
+                         "frac_of_layer_roofs": sum(roofs) / (ms_step * 1e3),
+                         "hbm_peak_gbs": hbm_gbs, "hbm_peak_source": hbm_src,
                          "launch_ms_sum": conv_time_ms, "achieved_launches_timed_alone": achieved_alone,
-                         # dram__bytes_read + dram__bytes_write of the 13 conv launches of one
-                         # step, from the ncu capture summarised in profiles/
-                         "traffic": 63.5e6,
+                         # dram__bytes_read + dram__bytes_write of the conv launches of one step,
+                         # from the profiler capture summarised in profiles/
+                         "traffic": recorded_traffic(),
                          "algorithmic_bytes": algorithmic_bytes(layers),
-                         "per_layer_us": [round(m * 1e3, 2) for m in conv_ms]},
+                         "per_layer_us": [round(m * 1e3, 2) for m in conv_ms],
+                         "per_layer_roof_us": [round(r, 3) for r in roofs],
+                         "per_layer_frac": [round(r / (m * 1e3), 4) for r, m in zip(roofs, conv_ms)]},
             "cpu_baseline": {"value": flops / cpu_s / 1e12, "unit": "TFLOP/s",
                              "cores": oracle.num_threads(), "kind": "oracle", "seconds": cpu_s,
                              "sample": "whole stack, 1 image (dense direct convolution, fp64)"},
             "parity": {"ok": parity_ok, "max_abs_err": float(err.max())},
         }
+        if not args.no_configs and world == 1:
+            reps = max(3, min(args.steps, 10))
+            stack.close()
+            del x, y, y_graph, acts
+            out["configs"] = {
+                "note": "every layer launched alone (as a stack launches it), CUDA events, L2 flushed "
+                        "before each launch, median of %d; frac = max(surviving flop / ALU peak, "
+                        "minimal bytes / HBM peak) / time" % reps,
+                "config1": measure_config(torch, B, flush, 1, 1, reps, hbm_gbs),
+                "config3_n1": measure_config(torch, B, flush, 3, 1, reps, hbm_gbs),
+                "config3_n32": measure_config(torch, B, flush, 3, 32, reps, hbm_gbs),
+                "config4": measure_config(torch, B, flush, 4, 256, reps, hbm_gbs),
+                "config5": measure_config(torch, B, flush, 5, 64, reps, hbm_gbs),
+            }
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
@@ -331,8 +505,13 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layer", default=None, help="time one layer alone (see the module docstring)")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="skip the per-layer measurement of configurations 1, 3, 4 and 5")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.layer:
+        run_layer(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

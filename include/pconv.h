@@ -245,29 +245,22 @@ pconv_status pconv_filter_order(const pconv_handle* h, int* perm_out);
  * internal wait id), else PCONV_OK. */
 pconv_status pconv_device_status(const pconv_handle* h, int* where);
 
-/* Development aid (no counterpart in the paper): synchronises the device and copies the first
- * n_words (<= PCONV_TRACE_WORDS) 64-bit trace words of the handle to the HOST.  A library built
- * with -DPCONV_TRACE makes the tiled kernel leave timestamps of its phases there (nanoseconds of
- * the global timer for words 0-10, SM cycles for 11-12; the meaning of each word is listed where
- * the kernel writes them); in a normal build the words stay zero. */
-#define PCONV_TRACE_WORDS 14
-pconv_status pconv_trace_read(const pconv_handle* h, unsigned long long* words_host, int n_words);
-
 /* Constant, NUL-terminated description of a status. */
 const char* pconv_status_str(pconv_status s);
 
 /* ---- producing PCONV weights from dense ones --------------------------------------------------- */
 
 /*
- * pconv_project -- projection of dense 3x3 kernels onto the PCONV constraint set, the step of the
- * paper's training framework that "assigns patterns to each kernel or prunes specific kernels"
- * (section on the ADMM-based framework; its formulas are in a supplement that is not available, so
- * the Euclidean projection is this build's reading).  Not part of the forward pass.
+ * pconv_project -- projection of dense 3x3 kernels onto the PCONV constraint set: the step of the
+ * ADMM-based training framework (accuracy-analysis section) that picks one pattern per kernel and
+ * removes whole kernels.  Its formulas are in a supplement that is not available, so the Euclidean
+ * projection is this build's reading.  Not part of the forward pass.
  *
  * For each kernel the pattern that retains the largest sum of squares is chosen (lowest pattern id
  * on ties); the k = round(keep * n_kernels) kernels with the largest retained sum survive,
  * together with every kernel that ties with the k-th; everything else becomes zero.  The sums are
- * formed in fp32, tap after tap in ascending tap order, multiply and add separately.
+ * formed in fp32, tap after tap in ascending tap order, multiply and add separately; where two
+ * candidates differ by less than that rounding, the choice may differ from an exact evaluation.
  *
  *  w_dev           [n_kernels][9] fp32, DEVICE (an OIHW tensor with n_kernels = c_out * c_in).
  *  patterns        n_patterns masks, HOST, as for pconv_pack.
@@ -309,11 +302,12 @@ pconv_status pconv_stack_forward(pconv_stack* s, const void* x_dev, void* y_dev,
 
 /* The same with HOST input and output: copies x to the device, runs the chain, copies the result
  * back and synchronises `stream` before returning.  Pinned host memory makes the copies
- * asynchronous; pageable memory also works.  Uses two extra device buffers owned by the stack. */
+ * asynchronous; pageable memory also works.  Uses two extra device buffers owned by the stack.
+ * Returns PCONV_ERR_DEVICE_TIMEOUT (y_host then holds no valid result) if a kernel of this forward
+ * abandoned a bounded wait; pconv_stack_status gives the wait id and makes the stack usable again. */
 pconv_status pconv_stack_forward_host(pconv_stack* s, const void* x_host, void* y_host,
                                       void* stream);
 
-/* Releases the stack (not the handles).  NULL is allowed. */
 /* Captures one forward from x_dev to y_dev into a CUDA graph kept by the stack (replacing an
  * earlier one), on a stream that allows capture (not the legacy default stream:
  * PCONV_ERR_UNSUPPORTED); the launches keep their programmatic dependencies inside the graph.
@@ -322,6 +316,14 @@ pconv_status pconv_stack_forward_host(pconv_stack* s, const void* x_host, void* 
 pconv_status pconv_stack_capture(pconv_stack* s, const void* x_dev, void* y_dev, void* stream);
 pconv_status pconv_stack_replay(pconv_stack* s, void* stream);
 
+/* Synchronises the device and returns PCONV_ERR_DEVICE_TIMEOUT if a kernel launched by this stack
+ * abandoned a bounded wait since the stack was created or since the last call of this function
+ * (then *where, if given, receives the internal wait id, and the stack's output of that forward is
+ * not valid), else PCONV_OK.  The call clears the record and zeroes the stack's channel-split
+ * workspace again, so the stack can be used afterwards. */
+pconv_status pconv_stack_status(pconv_stack* s, int* where);
+
+/* Releases the stack (not the handles).  NULL is allowed. */
 void pconv_stack_free(pconv_stack* s);
 
 

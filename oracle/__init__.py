@@ -14,7 +14,8 @@ tables).
 
 Pins: see tests/test_oracle_pins.py.  `project` (the projection that produces PCONV weights from
 dense ones; not part of the forward pass) is "parity unpinned": the paper's formulas for it are in
-a supplement that is not available, and only its defining properties are tested.
+a supplement that is not available; it is the plain fp64 definition of the Euclidean projection,
+and only that definition's properties are tested (exhaustive search on tiny tensors, invariants).
 """
 import ctypes
 import os
@@ -139,30 +140,28 @@ def check_invariants(w, patterns, strict4=True):
 
 def project(w, patterns, keep):
     """Projection of dense 3x3 kernels onto the PCONV constraint set: the step that turns trained
-    weights into pattern- and connectivity-pruned ones ("assign patterns to each kernel, or prune
-    specific kernels", section on the ADMM-based training framework; the paper's own formulas are
-    in a supplement that is not available, so this is a reading of that sentence: the Euclidean
-    projection -- parity unpinned beyond the properties tested in tests/test_oracle_pins.py).
+    weights into pattern- and connectivity-pruned ones (the training section says only that, inside
+    an ADMM framework, each kernel is given a pattern or is removed as a whole; its formulas are in
+    a supplement that is not available, so this is a reading of that sentence: the Euclidean
+    projection, which is what the constrained-variable update of that framework computes --
+    parity unpinned beyond the properties tested in tests/test_oracle_pins.py).
 
-    For each kernel the pattern that retains the largest sum of squares is chosen (lowest pattern
-    id on ties); then the k = round(keep * kernels) kernels with the largest retained sum of
-    squares survive, together with every kernel that ties with the k-th.  The sums that take
-    these decisions are formed in fp32, one tap after the other in ascending tap order with a
-    separate multiply and add (both sides of a comparison use the same precision).
+    Definition, in fp64: for each kernel the pattern that retains the largest sum of squares
+    (lowest pattern id among exact ties); then the k = round(keep * kernels) kernels with the
+    largest retained sum survive, together with every kernel that ties exactly with the k-th.
+    Where two candidates differ by less than rounding, an implementation that sums in a lower
+    precision may legitimately choose the other one; tests allow for that with a relative slack
+    on the retained sums and compare exactly where the sums are exact (integer-valued weights).
 
-    w: [c_out, c_in, 3, 3] float32.  Returns (projected weights float32, pattern ids int8 with -1
-    for pruned kernels)."""
+    w: [c_out, c_in, 3, 3].  Returns (projected weights float32, pattern ids int8 with -1 for
+    pruned kernels)."""
     w = np.ascontiguousarray(w, dtype=np.float32)
     c_out, c_in = w.shape[:2]
     flat = w.reshape(c_out * c_in, 9)
     n = flat.shape[0]
-    scores = np.zeros((len(patterns), n), np.float32)
-    for p, mask in enumerate(patterns):
-        s = np.zeros(n, np.float32)
-        for t in range(9):
-            if mask >> t & 1:
-                s = (s + (flat[:, t] * flat[:, t]).astype(np.float32)).astype(np.float32)
-        scores[p] = s
+    sq = flat.astype(np.float64) ** 2
+    masks = np.array([[(int(m) >> t) & 1 for t in range(9)] for m in patterns], np.float64)
+    scores = masks @ sq.T                               # [pattern, kernel] retained sum of squares
     pid = np.argmax(scores, axis=0)                    # first maximum = lowest id on ties
     best = scores[pid, np.arange(n)]
     k = int(np.floor(keep * n + 0.5))
@@ -172,7 +171,14 @@ def project(w, patterns, keep):
     else:
         threshold = np.sort(best)[n - k]              # the k-th largest value
         kept = best >= threshold
-    masks = np.array([[(m >> t) & 1 for t in range(9)] for m in patterns], np.float32)
-    out = flat * masks[pid] * kept[:, None]
+    out = flat * masks[pid].astype(np.float32) * kept[:, None]
     ids = np.where(kept, pid, -1).astype(np.int8)
     return out.reshape(w.shape).astype(np.float32), ids.reshape(c_out, c_in)
+
+
+def retained_energy(w, patterns):
+    """fp64 sum of squares that each pattern of the set retains of each kernel: [pattern, kernel]
+    (the quantity `project` maximises; tests use it to judge choices that differ by rounding)."""
+    flat = np.ascontiguousarray(w, dtype=np.float32).reshape(-1, 9).astype(np.float64)
+    masks = np.array([[(int(m) >> t) & 1 for t in range(9)] for m in patterns], np.float64)
+    return masks @ (flat ** 2).T

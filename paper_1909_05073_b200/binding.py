@@ -25,9 +25,9 @@ STATUS_NAMES = ["PCONV_OK", "PCONV_ERR_NULL", "PCONV_ERR_SHAPE", "PCONV_ERR_PATT
 
 EXPORTS = ["pconv_pack", "pconv_forward", "pconv_forward_ws", "pconv_forward_static_ws", "pconv_workspace_bytes", "pconv_plan", "pconv_plan_shape",
            "pconv_free", "pconv_maxpool2x2", "pconv_unpack",
-           "pconv_stats", "pconv_filter_order", "pconv_device_status", "pconv_trace_read", "pconv_status_str",
+           "pconv_stats", "pconv_filter_order", "pconv_device_status", "pconv_status_str",
            "pconv_stack_create", "pconv_stack_out_shape", "pconv_stack_forward",
-           "pconv_stack_forward_host", "pconv_stack_free", "pconv_stack_capture", "pconv_stack_replay",
+           "pconv_stack_forward_host", "pconv_stack_free", "pconv_stack_capture", "pconv_stack_replay", "pconv_stack_status",
            "pconv_project", "pconv_project_workspace_bytes"]
 
 
@@ -61,47 +61,65 @@ class Plan(ctypes.Structure):
 _lib = None
 
 
+def load(path):
+    """Loads a build of the library and declares its entry points' argument types."""
+    if not os.path.exists(path):
+        raise RuntimeError("%s is missing: run `python -m paper_1909_05073_b200.build`"
+                           " (the CUDA library is the only implementation)" % os.path.basename(path))
+    L = ctypes.CDLL(path)
+    vp, ci, cu = ctypes.c_void_p, ctypes.c_int, ctypes.c_uint
+    ip = ctypes.POINTER(ctypes.c_int)
+    L.pconv_pack.argtypes = [vp, ci, ci, vp, ci, ci, ci, cu, vp, ctypes.POINTER(vp), ip, ip]
+    L.pconv_forward.argtypes = [vp, vp, vp, vp, ci, ci, ci, cu, vp]
+    L.pconv_forward_ws.argtypes = [vp, vp, vp, vp, ci, ci, ci, cu, vp, ctypes.c_size_t, vp]
+    L.pconv_forward_static_ws.argtypes = [vp, vp, vp, vp, ci, ci, ci, cu, vp]
+    L.pconv_workspace_bytes.argtypes = [vp, ci, ci, ci, ctypes.POINTER(ctypes.c_size_t)]
+    L.pconv_plan.argtypes = [vp, ci, ci, ci, cu, ci, ctypes.POINTER(Plan)]
+    L.pconv_plan_shape.argtypes = [ci, ci, ctypes.c_longlong, ci, ci, ci, ci, ci, ci, cu, ci,
+                                   ctypes.POINTER(Plan)]
+    L.pconv_free.argtypes = [vp]
+    L.pconv_free.restype = None
+    L.pconv_maxpool2x2.argtypes = [vp, vp, ci, ci, ci, ci, ci, vp]
+    L.pconv_unpack.argtypes = [vp, vp]
+    L.pconv_stats.argtypes = [vp, ctypes.POINTER(Stats)]
+    L.pconv_filter_order.argtypes = [vp, vp]
+    L.pconv_device_status.argtypes = [vp, ip]
+    L.pconv_project_workspace_bytes.argtypes = [ctypes.c_longlong, ctypes.POINTER(ctypes.c_size_t)]
+    L.pconv_project.argtypes = [vp, ctypes.c_longlong, vp, ci, ctypes.c_double, vp, vp, vp,
+                                ctypes.c_size_t, vp]
+    if hasattr(L, "pconv_trace_read"):     # development build only (csrc/pconv_dev.h)
+        L.pconv_trace_read.argtypes = [vp, ctypes.POINTER(ctypes.c_ulonglong), ci]
+        L.pconv_dev_withhold.argtypes = [ci, cu]
+        L.pconv_dev_clear_status.argtypes = [vp]
+    L.pconv_status_str.argtypes = [ci]
+    L.pconv_status_str.restype = ctypes.c_char_p
+    L.pconv_stack_create.argtypes = [vp, vp, vp, ci, ci, ci, ci, cu, ctypes.POINTER(vp)]
+    L.pconv_stack_out_shape.argtypes = [vp, ip, ip, ip, ip]
+    L.pconv_stack_forward.argtypes = [vp, vp, vp, vp]
+    L.pconv_stack_forward_host.argtypes = [vp, vp, vp, vp]
+    L.pconv_stack_capture.argtypes = [vp, vp, vp, vp]
+    L.pconv_stack_replay.argtypes = [vp, vp]
+    L.pconv_stack_status.argtypes = [vp, ip]
+    L.pconv_stack_free.argtypes = [vp]
+    L.pconv_stack_free.restype = None
+    return L
+
+
 def lib():
     """The loaded shared library; raises if it has not been built (no fallback exists)."""
     global _lib
     if _lib is None:
-        if not os.path.exists(LIB_PATH):
-            raise RuntimeError("libpconv.so is missing: run `python -m paper_1909_05073_b200.build`"
-                               " (the CUDA library is the only implementation)")
-        L = ctypes.CDLL(LIB_PATH)
-        vp, ci, cu = ctypes.c_void_p, ctypes.c_int, ctypes.c_uint
-        ip = ctypes.POINTER(ctypes.c_int)
-        L.pconv_pack.argtypes = [vp, ci, ci, vp, ci, ci, ci, cu, vp, ctypes.POINTER(vp), ip, ip]
-        L.pconv_forward.argtypes = [vp, vp, vp, vp, ci, ci, ci, cu, vp]
-        L.pconv_forward_ws.argtypes = [vp, vp, vp, vp, ci, ci, ci, cu, vp, ctypes.c_size_t, vp]
-        L.pconv_forward_static_ws.argtypes = [vp, vp, vp, vp, ci, ci, ci, cu, vp]
-        L.pconv_workspace_bytes.argtypes = [vp, ci, ci, ci, ctypes.POINTER(ctypes.c_size_t)]
-        L.pconv_plan.argtypes = [vp, ci, ci, ci, cu, ci, ctypes.POINTER(Plan)]
-        L.pconv_plan_shape.argtypes = [ci, ci, ctypes.c_longlong, ci, ci, ci, ci, ci, ci, cu, ci,
-                                       ctypes.POINTER(Plan)]
-        L.pconv_free.argtypes = [vp]
-        L.pconv_free.restype = None
-        L.pconv_maxpool2x2.argtypes = [vp, vp, ci, ci, ci, ci, ci, vp]
-        L.pconv_unpack.argtypes = [vp, vp]
-        L.pconv_stats.argtypes = [vp, ctypes.POINTER(Stats)]
-        L.pconv_filter_order.argtypes = [vp, vp]
-        L.pconv_device_status.argtypes = [vp, ip]
-        L.pconv_project_workspace_bytes.argtypes = [ctypes.c_longlong, ctypes.POINTER(ctypes.c_size_t)]
-        L.pconv_project.argtypes = [vp, ctypes.c_longlong, vp, ci, ctypes.c_double, vp, vp, vp,
-                                    ctypes.c_size_t, vp]
-        L.pconv_trace_read.argtypes = [vp, ctypes.POINTER(ctypes.c_ulonglong), ci]
-        L.pconv_status_str.argtypes = [ci]
-        L.pconv_status_str.restype = ctypes.c_char_p
-        L.pconv_stack_create.argtypes = [vp, vp, vp, ci, ci, ci, ci, cu, ctypes.POINTER(vp)]
-        L.pconv_stack_out_shape.argtypes = [vp, ip, ip, ip, ip]
-        L.pconv_stack_forward.argtypes = [vp, vp, vp, vp]
-        L.pconv_stack_forward_host.argtypes = [vp, vp, vp, vp]
-        L.pconv_stack_capture.argtypes = [vp, vp, vp, vp]
-        L.pconv_stack_replay.argtypes = [vp, vp]
-        L.pconv_stack_free.argtypes = [vp]
-        L.pconv_stack_free.restype = None
-        _lib = L
+        _lib = load(LIB_PATH)
     return _lib
+
+
+def use_library(path):
+    """Makes every call of this module go to another build of the library (the development
+    build, in its tests); returns the library that was in use before."""
+    global _lib
+    old = _lib
+    _lib = load(path) if path is not None else None
+    return old
 
 
 def _check(status, what, detail=None):
@@ -181,7 +199,7 @@ TRACE_WORDS = 14
 
 
 def pconv_trace_read(handle):
-    """The handle's trace words (all zero unless the library was built with -DPCONV_TRACE)."""
+    """The handle's trace words (development build of the library only)."""
     buf = (ctypes.c_ulonglong * TRACE_WORDS)()
     _check(lib().pconv_trace_read(handle, buf, TRACE_WORDS), "pconv_trace_read")
     return list(buf)
@@ -371,6 +389,13 @@ class Stack:
         yp = y_host.data_ptr() if hasattr(y_host, "data_ptr") else y_host.ctypes.data
         _check(lib().pconv_stack_forward_host(self.ptr, ctypes.c_void_p(xp), ctypes.c_void_p(yp),
                                               _stream_ptr(stream)), "pconv_stack_forward_host")
+
+    def status(self):
+        """(status, wait id): PCONV_ERR_DEVICE_TIMEOUT if a kernel of this stack gave up a bounded
+        wait since the last call; the call clears the record and the stack's workspace."""
+        where = ctypes.c_int(0)
+        st = lib().pconv_stack_status(self.ptr, ctypes.byref(where))
+        return st, where.value
 
     def close(self):
         if self.ptr is not None:

@@ -6,7 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpconv.so")
-TRACE_LIB = os.path.join(HERE, "libpconv_trace.so")
+DEV_LIB = os.path.join(HERE, "libpconv_dev.so")
 SOURCES = ["pack.cu", "api.cu", "kernels_simple.cu", "kernels_tiled.cu", "project.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC"]
@@ -32,18 +32,19 @@ def _stale(lib=None):
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force=False, verbose=False, trace=False):
+def build(force=False, verbose=False, dev=False):
     """Compile the CUDA library if it is missing or older than its sources; returns its path.
-    trace=True builds libpconv_trace.so instead: the same library with -DPCONV_TRACE (the tiled
-    kernel records phase timestamps, and PCONV_FORCE_ZS / PCONV_FORCE_KS in the environment
-    override the launch plan); see trace_case.py."""
-    lib = TRACE_LIB if trace else LIB
+    dev=True builds libpconv_dev.so instead: the same library with -DPCONV_DEV (the entry points
+    of csrc/pconv_dev.h: phase timestamps of the tiled kernel, a launch plan forced through
+    PCONV_FORCE_ZS / PCONV_FORCE_KS in the environment, and a bounded wait that can be made to
+    run out for the tests of the give-up path)."""
+    lib = DEV_LIB if dev else LIB
     if not force and not _stale(lib):
         return lib
     generate()
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = lib + ".tmp%d" % os.getpid()
-    cmd = [nvcc] + NVCC_FLAGS + (["-DPCONV_TRACE"] if trace else []) + \
+    cmd = [nvcc] + NVCC_FLAGS + (["-DPCONV_DEV"] if dev else []) + \
           (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES]
     subprocess.check_call(cmd)
     os.replace(tmp, lib)
@@ -51,4 +52,4 @@ def build(force=False, verbose=False, trace=False):
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, trace="--trace" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, dev="--dev" in sys.argv))

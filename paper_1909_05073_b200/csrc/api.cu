@@ -4,8 +4,29 @@
 #include <new>
 
 #include "pconv_internal.h"
+#ifdef PCONV_DEV
+#include "pconv_dev.h"
+#endif
 
 using namespace pconv;
+
+int pconv::device_sm_count() {
+  constexpr int kMaxDev = 64, kDefault = 148;
+  static int cached[kMaxDev] = {0};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) {
+    cudaGetLastError();
+    return kDefault;
+  }
+  int v = cached[dev];
+  if (v > 0) return v;
+  if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) {
+    cudaGetLastError();
+    return kDefault;
+  }
+  cached[dev] = v;
+  return v;
+}
 
 extern "C" const char* pconv_status_str(pconv_status s) {
   switch (s) {
@@ -73,9 +94,22 @@ extern "C" pconv_status pconv_forward(const pconv_handle* h, const void* x, cons
   return pconv_forward_ws(h, x, bias, y, n, h_in, w_in, flags, nullptr, 0, stream_v);
 }
 
+// The forward behind every entry point.  `status_dev` != nullptr makes the kernels record an
+// abandoned wait there instead of in the handle's own status block (a stack collects the status
+// of all its layers in one word).
+static pconv_status forward_impl(const pconv_handle* h, const void* x, const float* bias, void* y,
+                                 int n, int h_in, int w_in, unsigned flags, void* ws,
+                                 size_t ws_bytes, void* stream_v, int* status_dev);
+
 extern "C" pconv_status pconv_forward_ws(const pconv_handle* h, const void* x, const float* bias,
                                          void* y, int n, int h_in, int w_in, unsigned flags,
                                          void* ws, size_t ws_bytes, void* stream_v) {
+  return forward_impl(h, x, bias, y, n, h_in, w_in, flags, ws, ws_bytes, stream_v, nullptr);
+}
+
+static pconv_status forward_impl(const pconv_handle* h, const void* x, const float* bias, void* y,
+                                 int n, int h_in, int w_in, unsigned flags, void* ws,
+                                 size_t ws_bytes, void* stream_v, int* status_dev) {
   if (!h || !x || !y) return PCONV_ERR_NULL;
   if (n < 0 || h_in <= 0 || w_in <= 0) return PCONV_ERR_SHAPE;
   const unsigned known =
@@ -87,7 +121,8 @@ extern "C" pconv_status pconv_forward_ws(const pconv_handle* h, const void* x, c
   if (bias && ((uintptr_t)bias & 3u)) return PCONV_ERR_ALIGN;
   if (ws && ((uintptr_t)ws & 255u)) return PCONV_ERR_ALIGN;
   if (n == 0) return PCONV_OK;
-  const DeviceLayer& L = h->d;
+  DeviceLayer L = h->d;
+  if (status_dev) L.err = status_dev;
   {  // x and y must not overlap
     const size_t es = (L.storage == PCONV_F16) ? 2 : 4;
     const int ho = (h_in - 1) / L.stride + 1, wo = (w_in - 1) / L.stride + 1;
@@ -197,6 +232,7 @@ extern "C" pconv_status pconv_device_status(const pconv_handle* h, int* where) {
   return PCONV_OK;
 }
 
+#ifdef PCONV_DEV
 extern "C" pconv_status pconv_trace_read(const pconv_handle* h, unsigned long long* words, int n_words) {
   if (!h || !words) return PCONV_ERR_NULL;
   if (n_words < 0 || n_words > pconv::kTraceWords) return PCONV_ERR_SHAPE;
@@ -208,6 +244,25 @@ extern "C" pconv_status pconv_trace_read(const pconv_handle* h, unsigned long lo
   }
   return PCONV_OK;
 }
+
+extern "C" pconv_status pconv_dev_withhold(int chunk, unsigned spin_limit) {
+  if (pconv::dev_set_withhold(chunk, spin_limit) != cudaSuccess) {
+    cudaGetLastError();
+    return PCONV_ERR_CUDA;
+  }
+  return PCONV_OK;
+}
+
+extern "C" pconv_status pconv_dev_clear_status(const pconv_handle* h) {
+  if (!h) return PCONV_ERR_NULL;
+  if (cudaDeviceSynchronize() != cudaSuccess || cudaMemset(h->d.err, 0, 4) != cudaSuccess ||
+      cudaDeviceSynchronize() != cudaSuccess) {
+    cudaGetLastError();
+    return PCONV_ERR_CUDA;
+  }
+  return PCONV_OK;
+}
+#endif
 
 // ---- stacks ---------------------------------------------------------------------------------------
 
@@ -223,6 +278,8 @@ struct pconv_stack {
   void* io[2];    // device input / output used by the host entry point
   void* ws;       // channel-split workspace shared by the layers (kept zeroed between launches)
   size_t ws_bytes;
+  int* status_dev;   // status block of every launch of this stack (word 0: first abandoned wait)
+  int* status_host;  // pinned copy of word 0, read back by the host entry point
   // a captured forward (pconv_stack_capture) and the buffers it was captured for
   cudaGraphExec_t graph_exec;
   const void* graph_x;
@@ -238,6 +295,8 @@ extern "C" void pconv_stack_free(pconv_stack* s) {
     if (s->io[i]) cudaFree(s->io[i]);
   }
   if (s->ws) cudaFree(s->ws);
+  if (s->status_dev) cudaFree(s->status_dev);
+  if (s->status_host) cudaFreeHost(s->status_host);
   if (s->graph_exec) cudaGraphExecDestroy(s->graph_exec);
   if (s->host_exec) cudaGraphExecDestroy(s->host_exec);
   delete[] s->layers;
@@ -312,6 +371,10 @@ extern "C" pconv_status pconv_stack_create(const pconv_handle* const* layers,
     e = cudaMalloc(&s->ws, s->ws_bytes);
     if (e == cudaSuccess) e = cudaMemset(s->ws, 0, s->ws_bytes);
   }
+  if (e == cudaSuccess) e = cudaMalloc(&s->status_dev, pconv::kStatusBlockBytes);
+  if (e == cudaSuccess) e = cudaMemset(s->status_dev, 0, pconv::kStatusBlockBytes);
+  if (e == cudaSuccess) e = cudaMallocHost(&s->status_host, sizeof(int));
+  if (e == cudaSuccess) *s->status_host = 0;
   if (e != cudaSuccess) {
     cudaGetLastError();
     pconv_stack_free(s);
@@ -342,8 +405,9 @@ extern "C" pconv_status pconv_stack_forward(pconv_stack* s, const void* x, void*
                       pconv::tiled_supported(L, s->n, ch, cw);
     const bool last_op = (i == s->n_layers - 1) && (!s->pool[i] || fuse);
     void* dst = last_op ? y : s->act[which];
-    pconv_status st = pconv_forward_ws(s->layers[i], cur, s->bias[i], dst, s->n, ch, cw,
-                                       s->flags | (fuse ? PCONV_POOL2X2 : 0u), s->ws, s->ws_bytes, stream);
+    pconv_status st = forward_impl(s->layers[i], cur, s->bias[i], dst, s->n, ch, cw,
+                                   s->flags | (fuse ? PCONV_POOL2X2 : 0u), s->ws, s->ws_bytes, stream,
+                                   s->status_dev);
     if (st != PCONV_OK) return st;
     ch = (ch - 1) / L.stride + 1;
     cw = (cw - 1) / L.stride + 1;
@@ -439,9 +503,33 @@ extern "C" pconv_status pconv_stack_forward_host(pconv_stack* s, const void* x_h
   }
   if (st != PCONV_OK) return st;
   if (cudaMemcpyAsync(y_host, s->io[1], s->out_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      cudaMemcpyAsync(s->status_host, s->status_dev, sizeof(int), cudaMemcpyDeviceToHost, stream) !=
+          cudaSuccess ||
       cudaStreamSynchronize(stream) != cudaSuccess) {
     cudaGetLastError();
     return PCONV_ERR_CUDA;
   }
-  return PCONV_OK;
+  // a layer that abandoned a bounded wait wrote no valid output: say so instead of handing it on
+  return *s->status_host ? PCONV_ERR_DEVICE_TIMEOUT : PCONV_OK;
+}
+
+extern "C" pconv_status pconv_stack_status(pconv_stack* s, int* where) {
+  if (!s) return PCONV_ERR_NULL;
+  int v = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpy(&v, s->status_dev, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    return PCONV_ERR_CUDA;
+  }
+  if (!v) return PCONV_OK;
+  if (where) *where = v;
+  // the abandoned launch may have left partial sums and tickets in the workspace
+  if (cudaMemset(s->status_dev, 0, sizeof(int)) != cudaSuccess ||
+      (s->ws && cudaMemset(s->ws, 0, s->ws_bytes) != cudaSuccess) ||
+      cudaDeviceSynchronize() != cudaSuccess) {
+    cudaGetLastError();
+    return PCONV_ERR_CUDA;
+  }
+  *s->status_host = 0;
+  return PCONV_ERR_DEVICE_TIMEOUT;
 }

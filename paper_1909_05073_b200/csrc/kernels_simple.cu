@@ -103,7 +103,8 @@ cudaError_t launch_maxpool(const void* x, void* y, int n, int c, int h, int w, i
   const long long total = (long long)n * c * h_out * w_out;
   if (total == 0) return cudaSuccess;
   long long blocks = (total + 255) / 256;
-  if (blocks > 148 * 16) blocks = 148 * 16;
+  const long long max_blocks = (long long)device_sm_count() * 16;
+  if (blocks > max_blocks) blocks = max_blocks;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)blocks, 1, 1);
   cfg.blockDim = dim3(256, 1, 1);

@@ -35,7 +35,7 @@
 #include <cuda_fp16.h>
 
 #include <type_traits>
-#ifdef PCONV_TRACE
+#ifdef PCONV_DEV
 #include <cstdlib>
 #endif
 
@@ -63,7 +63,6 @@ constexpr uint32_t kSpinLimit = 1u << 20;
 // phase completes), so that waiting warps leave the issue slots to the warps that have work.
 constexpr uint32_t kWaitHintNs = 200;
 constexpr int kSmemLimit = 227 * 1024;
-constexpr int kNumSMs = 148;
 
 struct SubTile {
   int n, y0, x0, valid;  // image, first output row / column, inside the batch?
@@ -148,21 +147,34 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+#ifdef PCONV_DEV
+// Development build only (pconv_dev_withhold): the number of tries of every bounded wait, and the
+// chunk for which one producer thread leaves out its arrival (-1 = none).
+__device__ unsigned int g_dev_spin_limit = kSpinLimit;
+__device__ int g_dev_withhold_chunk = -1;
+#define PCONV_SPIN_LIMIT g_dev_spin_limit
+#define PCONV_WITHHELD(kk, ptid) (g_dev_withhold_chunk == (kk) && (ptid) == 0)
+#else
+#define PCONV_SPIN_LIMIT kSpinLimit
+#define PCONV_WITHHELD(kk, ptid) false
+#endif
+
 // Bounded wait: false (and the wait id recorded) if the phase never completes.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* err, int id) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it)
+  const uint32_t limit = PCONV_SPIN_LIMIT;
+  for (uint32_t it = 0; it < limit; ++it)
     if (mbar_try_wait(bar, parity)) return true;
   atomicCAS(err, 0, id);
   return false;
 }
 
-// Built with -DPCONV_TRACE (build.py: build(trace=True) -> libpconv_trace.so) the kernel leaves
+// Built with -DPCONV_DEV (build.py: build(dev=True) -> libpconv_dev.so) the kernel leaves
 // timestamps in the trace words of the handle's status block (pconv_trace_read):
 //   0 start, 1 set-up done, 2 warp 0's first chunk landed, 3 loop end, 4 partial sums issued (split only),
 //   5 epilogue end, 6 after the CTA's last barrier -- thread 0 of CTA (0,0,0), globaltimer ns;
 //   7 end, 8 start, 9 loop end, 10 partial sums issued -- latest over all CTAs;
 //   11 / 12 cycles warp 0 of CTA (0,0,0) spent waiting for chunks / working on them, 13 its chunks.
-#ifdef PCONV_TRACE
+#ifdef PCONV_DEV
 #define PCONV_MARK(i)                                                         \
   if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) { \
     unsigned long long t_;                                                    \
@@ -607,7 +619,7 @@ __device__ __forceinline__ void produce_raw_stream(const DeviceLayer& L, const G
     if (ok && it > 0) ok = mbar_wait(sbase + 8 * (kMaxStages + s), (it - 1) & 1, L.err, 1);
     if (ok) {
       widen_raw<S>(g, pre, desc, raw_base(kk), sbase + g.stage_off + s * g.stage_bytes, kk, ptid);
-      mbar_arrive(sbase + 8 * s);
+      if (!PCONV_WITHHELD(kk, ptid)) mbar_arrive(sbase + 8 * s);
     }
     producers_sync();   // the raw slot may be overwritten
   }
@@ -686,7 +698,7 @@ __device__ __forceinline__ bool produce_half_stream(const DeviceLayer& L, const 
       cur = nxt;
     }
     if (kk >= n_early) stage_blocks_half(L, g, desc, codes, stage_base, kk, ptid);
-    mbar_arrive(sbase + 8 * s);
+    if (!PCONV_WITHHELD(kk, ptid)) mbar_arrive(sbase + 8 * s);
   }
   return true;
 }
@@ -1074,7 +1086,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
         else stage_blocks_async(L, g, desc, codes, stage_base, kk, ptid);
         // chunks whose x the consumers copy are complete, for the producers, once their blocks have
         // landed: arrive now, so that the barrier does not also wait for the later chunks' blocks
-        if (kk < n_coop) cp_async_arrive(sbase + 8 * kk);
+        if (kk < n_coop && !PCONV_WITHHELD(kk, ptid)) cp_async_arrive(sbase + 8 * kk);
       }
       asm volatile("griddepcontrol.wait;" ::: "memory");
       if (g.is_half) {
@@ -1086,7 +1098,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
           const uint32_t stage_base = sbase + g.stage_off + s * g.stage_bytes;
           produce_chunk_async<S>(L, g, (const float*)x, tab, pre, desc, codes, stage_base, k0 + kk, kk, ptid,
                                  true, kk >= n_early);
-          cp_async_arrive(sbase + 8 * s);
+          if (!PCONV_WITHHELD(kk, ptid)) cp_async_arrive(sbase + 8 * s);
         }
       }
     }
@@ -1112,7 +1124,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
     }
     if (bias && my_o >= 0) my_b = __ldg(bias + my_o);
 
-#ifdef PCONV_TRACE
+#ifdef PCONV_DEV
     long long t_wait = 0, t_work = 0;
 #endif
     // The warps of a unit draw the chunks from the unit's counter, so a warp that got a heavier
@@ -1132,13 +1144,13 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
       }
       if (kk >= nk) break;
       const int s = kk % g.stages;
-#ifdef PCONV_TRACE
+#ifdef PCONV_DEV
       const long long tc0 = clock64();
 #endif
       ok = mbar_wait(sbase + 8 * s, (kk / g.stages) & 1, L.err, 2);
       if (ok && kk < n_coop) ok = mbar_wait(coop_bar + 8 * kk, 0, L.err, 3);
       if (!ok) break;
-#ifdef PCONV_TRACE
+#ifdef PCONV_DEV
       const long long tc1 = clock64();
 #endif
       if (next_kk == 1) { PCONV_MARK(2) }   // this warp's first chunk has landed
@@ -1176,12 +1188,12 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
       __syncwarp();
       if (lane == 0) mbar_arrive(sbase + 8 * (kMaxStages + s));
       __syncwarp();
-#ifdef PCONV_TRACE
+#ifdef PCONV_DEV
       t_wait += tc1 - tc0;
       t_work += clock64() - tc1;
 #endif
     }
-#ifdef PCONV_TRACE
+#ifdef PCONV_DEV
     if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {
       trace_words(L)[11] = (unsigned long long)t_wait;
       trace_words(L)[12] = (unsigned long long)t_work;
@@ -1403,7 +1415,8 @@ double geo_cost(const DeviceLayer& L, const Geo& g) {
   const double loop = turns * chunk;
   const double fixed = 28.0 + 17.0 / g.zs;
   const long long ctas = geo_tiles(L, g) * g.ks;
-  const double waves = (double)((ctas + kNumSMs - 1) / kNumSMs);
+  const int sms = device_sm_count();
+  const double waves = (double)((ctas + sms - 1) / sms);
   return waves * (fixed + loop) + (g.ks > 1 ? 100.0 / g.zs : 0.0);
 }
 
@@ -1415,17 +1428,17 @@ bool make_geo(const DeviceLayer& L, int n, int h, int w, bool allow_split, Geo* 
   if (GENERIC) return geo_for<true>(L, n, h, w, 1, out);
   bool found = false;
   double best = 0.0;
-#ifdef PCONV_TRACE
+#ifdef PCONV_DEV
   const char* force_zs = getenv("PCONV_FORCE_ZS");
   const char* force_ks = getenv("PCONV_FORCE_KS");
 #endif
   for (int zs = 1; zs <= 4; zs *= 2) {
     Geo g;
-#ifdef PCONV_TRACE
+#ifdef PCONV_DEV
     if (force_zs && atoi(force_zs) != zs) continue;
 #endif
     if (!geo_for<false>(L, n, h, w, zs, &g)) continue;
-#ifdef PCONV_TRACE
+#ifdef PCONV_DEV
     if (force_ks && allow_split) {
       set_split(L, &g, atoi(force_ks));
       if (g.stages < 1) continue;
@@ -1438,7 +1451,7 @@ bool make_geo(const DeviceLayer& L, int n, int h, int w, bool allow_split, Geo* 
       if (pass == 1) {
         if (!allow_split) break;
         const long long tiles = geo_tiles(L, g);
-        const long long ks = kNumSMs / tiles;   // fill one wave
+        const long long ks = device_sm_count() / tiles;   // fill one wave
         if (ks < 2) break;
         set_split(L, &c, (int)ks);
         if (c.ks < 2 || c.stages < 1) break;
@@ -1559,5 +1572,16 @@ cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias,
   return wide ? launch_one<2, false, true>(L, g, x, bias, y, wsf, counters, stream)
               : launch_one<2, false, false>(L, g, x, bias, y, wsf, counters, stream);
 }
+
+#ifdef PCONV_DEV
+cudaError_t dev_set_withhold(int chunk, unsigned spin_limit) {
+  const unsigned limit = chunk < 0 ? kSpinLimit : (spin_limit ? spin_limit : 1u);
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e == cudaSuccess) e = cudaMemcpyToSymbol(g_dev_spin_limit, &limit, sizeof(limit));
+  if (e == cudaSuccess) e = cudaMemcpyToSymbol(g_dev_withhold_chunk, &chunk, sizeof(chunk));
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  return e;
+}
+#endif
 
 }  // namespace pconv

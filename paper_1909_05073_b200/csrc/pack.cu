@@ -4,6 +4,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstring>
+#include <memory>
 #include <new>
 #include <numeric>
 
@@ -154,7 +155,10 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
       }
     }
 
-    pconv_handle* h = new pconv_handle();
+    // owned here until the pack has succeeded: an allocation failure further down (the vectors
+    // below can throw) must not leak the handle
+    std::unique_ptr<pconv_handle> owner(new pconv_handle());
+    pconv_handle* h = owner.get();
     std::memset(h, 0, sizeof(*h));
     h->n_patterns = n_patterns;
     h->canonical = true;
@@ -321,7 +325,6 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
     char* dev = nullptr;
     if (cudaMalloc((void**)&dev, total) != cudaSuccess) {
       cudaGetLastError();
-      delete h;
       return PCONV_ERR_ALLOC;
     }
     cudaError_t e = cudaSuccess;
@@ -333,7 +336,6 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
     if (e != cudaSuccess) {
       cudaGetLastError();
       cudaFree(dev);
-      delete h;
       return PCONV_ERR_CUDA;
     }
     cudaGetDevice(&h->device);
@@ -381,7 +383,7 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
     st.min_group_kernels = min_gk < 0 ? 0 : min_gk;
     st.packed_bytes = (long long)total;
     st.canonical_patterns = h->canonical ? 1 : 0;
-    *out = h;
+    *out = owner.release();
     return PCONV_OK;
   } catch (const std::bad_alloc&) {
     return PCONV_ERR_ALLOC;

@@ -91,7 +91,7 @@ struct DeviceLayer {         // device pointers of one packed layer (passed to k
 };
 
 // Status block: one status word, one pad word, kTraceWords 64-bit trace words (written only by
-// builds with -DPCONV_TRACE).
+// builds with -DPCONV_DEV).
 constexpr int kTraceWords = 14;
 constexpr int kStatusBlockBytes = 8 + 8 * kTraceWords;
 __host__ __device__ inline unsigned long long* trace_words(const DeviceLayer& L) {
@@ -115,6 +115,10 @@ struct pconv_handle {
 };
 
 namespace pconv {
+// Streaming multiprocessors of the current device (cudaDevAttrMultiProcessorCount, looked up once
+// per device).  Without a usable device -- the planner also runs on machines that have none -- the
+// count of the part this library is written for (B200: 148).
+int device_sm_count();
 // kernels (defined in the .cu files); all asynchronous on `stream`
 cudaError_t launch_simple(const DeviceLayer& L, const void* x, const float* bias, void* y, int n,
                           int h, int w, bool relu, cudaStream_t stream);
@@ -125,6 +129,9 @@ size_t tiled_workspace_bytes(const DeviceLayer& L, int n, int h, int w);
 bool tiled_supported(const DeviceLayer& L, int n, int h, int w);
 bool tiled_plan(const DeviceLayer& L, int n, int h, int w, bool generic_taps, bool with_workspace,
                 pconv_plan_t* out);
+#ifdef PCONV_DEV
+cudaError_t dev_set_withhold(int chunk, unsigned spin_limit);   // see pconv_dev.h
+#endif
 cudaError_t launch_maxpool(const void* x, void* y, int n, int c, int h, int w, int storage,
                            cudaStream_t stream);
 }  // namespace pconv

@@ -84,17 +84,21 @@ __global__ void pick_kernel(int shift, SelectState* st) {
   for (int i = 0; i < 256; ++i) st->hist[i] = 0;
 }
 
-__global__ void __launch_bounds__(kThreads) mask_kernel(const float* __restrict__ w, long long n,
-                                                        PatternSet ps, const float* __restrict__ best,
+// `out` may be `w` itself (in-place use), so neither pointer is declared restrict and a thread
+// reads its kernel's nine taps before it writes any of them.
+__global__ void __launch_bounds__(kThreads) mask_kernel(const float* w, long long n, PatternSet ps,
+                                                        const float* __restrict__ best,
                                                         const SelectState* __restrict__ st, int keep_none,
-                                                        float* __restrict__ out,
-                                                        signed char* __restrict__ pid) {
+                                                        float* out, signed char* __restrict__ pid) {
   const long long i = blockIdx.x * (long long)kThreads + threadIdx.x;
   if (i >= n) return;
+  float v[9];
+#pragma unroll
+  for (int t = 0; t < 9; ++t) v[t] = w[i * 9 + t];
   const bool kept = !keep_none && __float_as_uint(best[i]) >= st->prefix;   // ties with the k-th stay
   const unsigned int m = kept ? ps.mask[pid[i]] : 0u;
 #pragma unroll
-  for (int t = 0; t < 9; ++t) out[i * 9 + t] = (m >> t & 1u) ? w[i * 9 + t] : 0.f;
+  for (int t = 0; t < 9; ++t) out[i * 9 + t] = (m >> t & 1u) ? v[t] : 0.f;
   if (!kept) pid[i] = -1;
 }
 
@@ -150,7 +154,8 @@ extern "C" pconv_status pconv_project(const float* w_dev, long long n_kernels,
   const long long blocks = (n_kernels + kThreads - 1) / kThreads;
   if (blocks > 0x7FFFFFFF) return PCONV_ERR_SHAPE;
   score_kernel<<<(unsigned)blocks, kThreads, 0, stream>>>(w_dev, n_kernels, ps, best, pattern_id_dev);
-  const unsigned hist_blocks = (unsigned)(blocks < 148 * 8 ? blocks : 148 * 8);
+  const long long hist_max = (long long)device_sm_count() * 8;
+  const unsigned hist_blocks = (unsigned)(blocks < hist_max ? blocks : hist_max);
   for (int shift = 24; shift >= 0; shift -= 8) {
     hist_kernel<<<hist_blocks, kThreads, 0, stream>>>(best, n_kernels, shift, st);
     pick_kernel<<<1, 32, 0, stream>>>(shift, st);

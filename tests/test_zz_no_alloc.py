@@ -4,13 +4,14 @@ Some users of this library run where cudaMalloc is off limits: inside another fr
 plan, under an allocator they do not own, or on a path that must never touch the driver's
 allocator.  For them the channel-split scratch lives in a fixed array inside the library.  This
 test calls that entry point through the C ABI twice in a row and checks each result against the
-ordinary workspace entry point (pconv_forward_ws), with the tolerance of the other parity tests.
-It is collected last so that a failure here cannot hide any other test.
+ordinary workspace entry point (pconv_forward_ws) and against the CPU oracle, with the tolerance
+of the other parity tests.  It is collected last so that a failure here cannot hide any other test.
 """
 import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_1909_05073_b200 import binding as B
 from paper_1909_05073_b200 import build as pbuild
 from paper_1909_05073_b200 import synth
@@ -20,15 +21,17 @@ pytestmark = pytest.mark.gpu
 
 
 def _layer(c_in, c_out, h, seed, stride=1):
+    """(packed layer, device input, the CPU oracle's result for it)"""
     spec = synth.LayerSpec("t", c_in, c_out, h, h, stride, 0.35)
     w, b, _ = synth.gen_weights(spec, seed)
-    x = torch.from_numpy(synth.gen_input(spec, 1, seed)).cuda()
-    return B.Layer(w, synth.PATTERNS8, stride, B.F32, b), x
+    x = synth.gen_input(spec, 1, seed)
+    return (B.Layer(w, synth.PATTERNS8, stride, B.F32, b), torch.from_numpy(x).cuda(),
+            oracle.conv3x3(x, w, b, stride, True))
 
 
 def test_static_workspace_entry_point_matches_the_workspace_entry_point():
     pbuild.build()
-    layer, x = _layer(128, 96, 28, 31)
+    layer, x, want = _layer(128, 96, 28, 31)
     assert 0 < B.pconv_workspace_bytes(layer.handle, 1, 28, 28) <= B.STATIC_WS_BYTES
     ref = layer.forward(x, relu=True, split=True)        # existing entry point, caller's buffer
     torch.cuda.synchronize()
@@ -38,13 +41,15 @@ def test_static_workspace_entry_point_matches_the_workspace_entry_point():
         B.pconv_forward_static_ws(layer.handle, x, layer.bias, y, B.RELU)
         torch.cuda.synchronize()
         check_close(y.cpu().numpy(), ref, "f32", "static workspace, call %d" % call)
+        check_close(y.cpu().numpy(), want, "f32", "static workspace against the oracle, call %d" % call)
     # a different layer right after: leftovers of the previous shape must not matter
-    layer2, x2 = _layer(64, 64, 14, 32)
+    layer2, x2, want2 = _layer(64, 64, 14, 32)
     ref2 = layer2.forward(x2, relu=True, split=True).cpu().numpy()
     y2 = torch.empty_like(torch.from_numpy(ref2)).cuda()
     B.pconv_forward_static_ws(layer2.handle, x2, layer2.bias, y2, B.RELU)
     torch.cuda.synchronize()
     check_close(y2.cpu().numpy(), ref2, "f32", "static workspace, second layer")
+    check_close(y2.cpu().numpy(), want2, "f32", "static workspace against the oracle, second layer")
     assert B.pconv_device_status(layer.handle)[0] == 0
     layer.close()
     layer2.close()
