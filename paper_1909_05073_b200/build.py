@@ -7,6 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpconv.so")
 DEV_LIB = os.path.join(HERE, "libpconv_dev.so")
+# (fp32_peak.cu is a stand-alone measuring program, see build_peak)
 SOURCES = ["pack.cu", "api.cu", "kernels_simple.cu", "kernels_tiled.cu", "project.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC"]
@@ -51,5 +52,17 @@ def build(force=False, verbose=False, dev=False):
     return lib
 
 
+def build_peak():
+    """Compiles the stand-alone FP32-peak measurement (csrc/fp32_peak.cu) to ./fp32_peak."""
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    exe = os.path.join(HERE, "fp32_peak")
+    subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-o", exe,
+                           os.path.join(CSRC, "fp32_peak.cu")])
+    return exe
+
+
 if __name__ == "__main__":
+    if "--peak" in sys.argv:
+        print(build_peak())
+        sys.exit(0)
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, dev="--dev" in sys.argv))
