@@ -72,8 +72,16 @@ enum {
   PCONV_KERNEL_SIMPLE = 0x100u, /* one thread per output, walks the per-filter kernel list */
   PCONV_KERNEL_TILED = 0x200u,  /* shared-memory halo tiles, packed FMAs, one straight-line body per
                                    pattern mask (any set of 4-of-9 masks); the default */
-  PCONV_KERNEL_GENERIC_TAPS = 0x400u /* tiled path that tests the 9 mask bits at run time; slower,
-                                        kept as a cross-check of the per-mask bodies */
+  PCONV_KERNEL_GENERIC_TAPS = 0x400u, /* tiled path that tests the 9 mask bits at run time; slower,
+                                         kept as a cross-check of the per-mask bodies */
+  PCONV_KERNEL_TENSOR = 0x800u /* fp16 storage, stride 1 only: the layer as a dense implicit GEMM over
+                                  the zero-inserted weights on the tensor cores (tcgen05.mma, fp32
+                                  accumulators in Tensor Memory).  It multiplies the pruned zeros too
+                                  -- 9 / (4 x keep rate) times the surviving multiply-adds -- and is
+                                  still several times faster for fp16 at the benchmark's keep rates,
+                                  so the library picks it by default when the batch gives it enough
+                                  tiles; fp16 products are exact in fp32, so the result differs from
+                                  the sparse kernels by summation order only.  No fused max-pool. */
 };
 
 #define PCONV_MAX_PATTERNS 16
@@ -217,6 +225,9 @@ typedef struct pconv_plan_t {
   int stages;            /* depth of the staging ring */
   int smem_bytes;        /* dynamic shared memory the geometry needs */
   long long ctas;        /* CTAs launched */
+  int tensor_path;       /* 1 = a default forward of this shape (no kernel-selection flag, no fused
+                            pool) runs the dense tensor-core kernel instead of the tiled one; the
+                            fields above still describe the tiled kernel */
 } pconv_plan_t;
 
 /* Test / tuning aid: fills *plan with the geometry a tiled forward of this shape would use;

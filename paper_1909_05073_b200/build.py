@@ -8,7 +8,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpconv.so")
 DEV_LIB = os.path.join(HERE, "libpconv_dev.so")
 # (fp32_peak.cu is a stand-alone measuring program, see build_peak)
-SOURCES = ["pack.cu", "api.cu", "kernels_simple.cu", "kernels_tiled.cu", "project.cu"]
+SOURCES = ["pack.cu", "api.cu", "kernels_simple.cu", "kernels_tiled.cu", "kernels_tensor.cu", "project.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC"]
 

@@ -61,6 +61,7 @@ extern "C" pconv_status pconv_plan(const pconv_handle* h, int n, int h_in, int w
   std::memset(plan, 0, sizeof(*plan));
   if (!tiled_plan(h->d, n, h_in, w_in, (flags & PCONV_KERNEL_GENERIC_TAPS) != 0, with_workspace != 0, plan))
     return PCONV_ERR_UNSUPPORTED;
+  plan->tensor_path = tensor_preferred(h->d, n, h_in, w_in) ? 1 : 0;
   return PCONV_OK;
 }
 
@@ -113,9 +114,11 @@ static pconv_status forward_impl(const pconv_handle* h, const void* x, const flo
   if (!h || !x || !y) return PCONV_ERR_NULL;
   if (n < 0 || h_in <= 0 || w_in <= 0) return PCONV_ERR_SHAPE;
   const unsigned known =
-      PCONV_RELU | PCONV_POOL2X2 | PCONV_REPRODUCIBLE | PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED | PCONV_KERNEL_GENERIC_TAPS;
+      PCONV_RELU | PCONV_POOL2X2 | PCONV_REPRODUCIBLE | PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED |
+      PCONV_KERNEL_GENERIC_TAPS | PCONV_KERNEL_TENSOR;
   if (flags & ~known) return PCONV_ERR_UNSUPPORTED;
-  const unsigned sel = flags & (PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED | PCONV_KERNEL_GENERIC_TAPS);
+  const unsigned sel = flags & (PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED | PCONV_KERNEL_GENERIC_TAPS |
+                                PCONV_KERNEL_TENSOR);
   if (sel & (sel - 1)) return PCONV_ERR_UNSUPPORTED;  // at most one selection bit
   if (((uintptr_t)x | (uintptr_t)y) & 15u) return PCONV_ERR_ALIGN;
   if (bias && ((uintptr_t)bias & 3u)) return PCONV_ERR_ALIGN;
@@ -141,7 +144,12 @@ static pconv_status forward_impl(const pconv_handle* h, const void* x, const flo
   cudaError_t e;
   if (pool && (sel == PCONV_KERNEL_SIMPLE || !tiled_supported(L, n, h_in, w_in)))
     return PCONV_ERR_UNSUPPORTED;  // only the tiled kernels fuse the pool
-  if (sel == PCONV_KERNEL_SIMPLE) {
+  if (sel == PCONV_KERNEL_TENSOR) {
+    if (pool || !tensor_supported(L, n, h_in, w_in)) return PCONV_ERR_UNSUPPORTED;
+    e = launch_tensor(L, x, bias, y, n, h_in, w_in, relu, stream);
+  } else if (sel == 0 && !pool && tensor_preferred(L, n, h_in, w_in)) {
+    e = launch_tensor(L, x, bias, y, n, h_in, w_in, relu, stream);
+  } else if (sel == PCONV_KERNEL_SIMPLE) {
     e = launch_simple(L, x, bias, y, n, h_in, w_in, relu, stream);
   } else if (sel == PCONV_KERNEL_TILED || sel == PCONV_KERNEL_GENERIC_TAPS) {
     if (!tiled_supported(L, n, h_in, w_in)) return PCONV_ERR_UNSUPPORTED;
@@ -401,7 +409,12 @@ extern "C" pconv_status pconv_stack_forward(pconv_stack* s, const void* x, void*
   for (int i = 0; i < s->n_layers; ++i) {
     const pconv::DeviceLayer& L = s->layers[i]->d;
     // a pool that follows the layer is fused into the layer's epilogue when a tiled kernel runs it
-    const bool fuse = s->pool[i] && !(s->flags & PCONV_KERNEL_SIMPLE) &&
+    // (not when the layer takes the dense tensor-core kernel, which has no pooled epilogue: the
+    // plain max-pool kernel follows it)
+    const unsigned sel_bits = PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED | PCONV_KERNEL_GENERIC_TAPS | PCONV_KERNEL_TENSOR;
+    const bool tensor = (s->flags & PCONV_KERNEL_TENSOR) ||
+                        (!(s->flags & sel_bits) && pconv::tensor_preferred(L, s->n, ch, cw));
+    const bool fuse = s->pool[i] && !(s->flags & PCONV_KERNEL_SIMPLE) && !tensor &&
                       pconv::tiled_supported(L, s->n, ch, cw);
     const bool last_op = (i == s->n_layers - 1) && (!s->pool[i] || fuse);
     void* dst = last_op ? y : s->act[which];

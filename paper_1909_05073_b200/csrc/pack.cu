@@ -299,10 +299,38 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
     for (int i = 0; i < 32; ++i) { codes_s.push_back(0); codes_s.push_back(0); codes_g.push_back(0); }
     for (int i = 0; i < 8; ++i) { wv32.push_back(0.f); wv16.push_back(0); }
 
+    // ---- zero-inserted dense weights for the tensor-core path (fp16 storage, stride 1) ----------
+    // Filters in original order, tiles of 64 (layers of up to 64 filters) or 128; channels padded to
+    // a multiple of 16 with zeros.  Left out for layers whose dense form would exceed 64 MB.
+    std::vector<uint16_t> wdense;
+    int dense_nt = 0;
+    if (storage == PCONV_F16 && stride == 1) {
+      const int nt = c_out <= 64 ? 64 : 128;
+      const size_t n_tiles = (size_t)(c_out + nt - 1) / nt, k_steps = (size_t)(c_in + 15) / 16;
+      const size_t halves = n_tiles * k_steps * 9 * nt * 16;
+      if (halves * 2 <= ((size_t)64 << 20)) {
+        dense_nt = nt;
+        wdense.assign(halves, 0);
+        for (int o = 0; o < c_out; ++o) {
+          const size_t tile = (size_t)o / nt, on = (size_t)o % nt;
+          for (const KernelRec& r : per_filter[o]) {
+            const size_t ks = (size_t)r.c / 16, kc = (size_t)r.c % 16;
+            int s = 0;
+            for (int t = 0; t < 9; ++t) {
+              if (!(patterns[r.pid] >> t & 1)) continue;
+              const size_t idx = ((((tile * k_steps + ks) * 9 + t) * 2 + kc / 8) * (nt / 8) + on / 8) * 64 +
+                                 (on % 8) * 8 + kc % 8;
+              wdense[idx] = r.hv[s++];
+            }
+          }
+        }
+      }
+    }
+
     // ---- one device allocation, sub-buffers 256-byte aligned ------------------------------------
     struct Part { const void* src; size_t bytes; size_t off; };
     auto align256 = [](size_t v) { return (v + 255) & ~(size_t)255; };
-    Part parts[9];
+    Part parts[10];
     int np = 0;
     size_t total = 0;
     auto add = [&](const void* src, size_t bytes) {
@@ -321,6 +349,7 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
     const int i_pm = add(perm.data(), perm.size() * 4);
     const std::vector<unsigned char> zero_block(kStatusBlockBytes, 0);
     const int i_er = add(zero_block.data(), zero_block.size());
+    const int i_wd = dense_nt ? add(wdense.data(), wdense.size() * 2) : -1;
 
     char* dev = nullptr;
     if (cudaMalloc((void**)&dev, total) != cudaSuccess) {
@@ -355,6 +384,8 @@ extern "C" pconv_status pconv_pack(const float* w, int c_out, int c_in, const ui
     d.codes_g = (const uint8_t*)(dev + parts[i_cg].off);
     d.perm = (const int*)(dev + parts[i_pm].off);
     d.err = (int*)(dev + parts[i_er].off);
+    d.wdense = i_wd >= 0 ? dev + parts[i_wd].off : nullptr;
+    d.dense_nt = dense_nt;
     d.c_out = c_out;
     d.c_in = c_in;
     d.stride = stride;

@@ -88,6 +88,11 @@ struct DeviceLayer {         // device pointers of one packed layer (passed to k
   int c_out, c_in, stride, storage, n_groups, n_chunks;
   int wide_codes;            // 0 = narrow codes (canonical set), 1 = wide codes
   long long n_kept;          // surviving kernels of the layer
+  // zero-inserted dense fp16 weights for the tensor-core path (fp16 storage, stride 1; else null):
+  // per (filter tile of dense_nt, 16-channel step) nine [dense_nt x 16] matrices in the K-major
+  // core-matrix order of tcgen05 shared-memory descriptors: [tap][k half][filter / 8][filter % 8][k % 8]
+  const void* wdense;
+  int dense_nt;
 };
 
 // Status block: one status word, one pad word, kTraceWords 64-bit trace words (written only by
@@ -125,6 +130,10 @@ cudaError_t launch_simple(const DeviceLayer& L, const void* x, const float* bias
 cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias, void* y, int n,
                          int h, int w, bool relu, bool pool, bool reproducible, bool generic_taps,
                          void* ws, size_t ws_bytes, cudaStream_t stream);
+cudaError_t launch_tensor(const DeviceLayer& L, const void* x, const float* bias, void* y, int n,
+                          int h, int w, bool relu, cudaStream_t stream);
+bool tensor_supported(const DeviceLayer& L, int n, int h, int w);
+bool tensor_preferred(const DeviceLayer& L, int n, int h, int w);
 size_t tiled_workspace_bytes(const DeviceLayer& L, int n, int h, int w);
 bool tiled_supported(const DeviceLayer& L, int n, int h, int w);
 bool tiled_plan(const DeviceLayer& L, int n, int h, int w, bool generic_taps, bool with_workspace,
