@@ -219,12 +219,28 @@ def measure_config(torch, B, flush, cid, batch, reps, hbm_gbs):
         pool = bool(cfg.chained and spec.pool_after)
         n_, c_, h_, w_ = layer.out_shape(x.shape)
         y = torch.empty((n_, c_, h_ // 2, w_ // 2) if pool else (n_, c_, h_, w_), dtype=tdtype, device="cuda")
-        layer.forward(x, relu=True, out=y, split=True, pool=pool)      # warm-up (and the chain's data)
-        us = _time_launch(torch, flush, lambda: layer.forward(x, relu=True, out=y, split=True, pool=pool), reps)
+        plan = B.pconv_plan(layer.handle, cfg.batch, spec.h, spec.w, 0, True)
+        if pool and plan["tensor_path"]:
+            # what a stack launches here: the dense tensor-core kernel, then the plain max-pool kernel
+            y_full = torch.empty((n_, c_, h_, w_), dtype=tdtype, device="cuda")
+
+            def run(layer=layer, x=x, y=y, y_full=y_full):
+                layer.forward(x, relu=True, out=y_full, split=True)
+                B.pconv_maxpool2x2(y_full, y)
+        else:
+            def run(layer=layer, x=x, y=y, pool=pool):
+                layer.forward(x, relu=True, out=y, split=True, pool=pool)
+        run()                                                          # warm-up (and the chain's data)
+        us = _time_launch(torch, flush, run, reps)
         roof = layer_roof_us(spec, kept, cfg.batch, es, hbm_gbs)
         row = {"layer": spec.name, "us": round(us, 2), "roof_us": round(roof, 3),
                "frac": round(roof / us, 4),
-               "tflops": round(layer_flops(spec, kept, cfg.batch) / us / 1e6, 3)}
+               "tflops": round(layer_flops(spec, kept, cfg.batch) / us / 1e6, 3),
+               "kernel": "tensor" if plan["tensor_path"] else "tiled"}
+        if plan["tensor_path"]:
+            # the dense path's own roof: zero-inserted multiply-adds at the measured bf16 tensor peak
+            dense = 2.0 * 9 * spec.c_in * spec.c_out * spec.h_out * spec.w_out * cfg.batch
+            row["dense_tflops"] = round(dense / us / 1e6, 1)
         if cid == 5:
             s = layer.stats()
             mean = s.kept_kernels / max(s.n_groups, 1)
@@ -235,6 +251,17 @@ def measure_config(torch, B, flush, cid, batch, reps, hbm_gbs):
     if any(status):
         raise SystemExit("device reported an abandoned wait in config %d" % cid)
     total_us = sum(r["us"] for r, _, _ in rows)
+    stack_us = None
+    if cfg.chained:
+        s0 = cfg.layers[0]
+        stack = B.Stack(layers, [l.pool_after for l in cfg.layers], cfg.batch, s0.h, s0.w, B.RELU)
+        xs = torch.from_numpy(synth.gen_input(s0, cfg.batch, synth.layer_seed(cid, 0))).cuda().to(tdtype)
+        ys = torch.empty(stack.out_shape, dtype=tdtype, device="cuda")
+        stack.forward(xs, ys)
+        stack_us = _time_launch(torch, flush, lambda: stack.forward(xs, ys), reps)
+        if stack.status()[0]:
+            raise SystemExit("device reported an abandoned wait in the stack of config %d" % cid)
+        stack.close()
     flops = sum(f for _, f, _ in rows)
     roof = sum(r for _, _, r in rows)
     out = {"workload": "config %d: %s, batch %d, %s" % (cid, cfg.name, cfg.batch, cfg.storage),
@@ -242,6 +269,10 @@ def measure_config(torch, B, flush, cid, batch, reps, hbm_gbs):
            "tflops": round(flops / total_us / 1e6, 3), "roof_us": round(roof, 2),
            "frac": round(roof / total_us, 4), "timing": "sum of the layers' launches timed alone",
            "layers": [r for r, _, _ in rows]}
+    if stack_us is not None:
+        out["stack_ms"] = round(stack_us / 1e3, 4)
+        out["stack_tflops"] = round(flops / stack_us / 1e6, 3)
+        out["stack_frac"] = round(roof / stack_us, 4)
     for l in layers:
         l.close()
     return out

@@ -25,14 +25,29 @@
 //    zero-inserted [n_t x 16] fp16 matrices already in the K-major canonical core-matrix order; a
 //    stage's 9 x n_t x 32 bytes arrive with one bulk copy (cp.async.bulk, no tensor map, no
 //    multicast) that completes on the stage's mbarrier.
-//  * Warp roles: warps 0-3 epilogue (warp q reads TMEM lanes 32q..32q+31: bias, ReLU, fp16
-//    convert, store to NCHW), warp 4 issues the MMAs (one thread) and owns the TMEM allocation,
+//  * Warp roles: warps 0-3 epilogue (warp q reads TMEM lanes 32q..32q+31, adds the bias, applies
+//    ReLU, converts to fp16 and stages the tile in shared memory as [filter][pixel]; the 128
+//    threads then copy it out in 16-byte pieces, a filter's 8 consecutive pixels each -- the
+//    first version stored 2 bytes per lane and column straight from the registers and spent more
+//    time in its epilogue than in its MMAs), warp 4 issues the MMAs (one thread) and owns the TMEM allocation,
 //    warps 5-12 are the A producers, in two groups that take alternate stages so that one group's
 //    global loads are in flight while the other converts and stores.  Two accumulator buffers
 //    (2 x n_t columns) let the epilogue of a tile overlap the next tile's MMAs.  CTAs are
-//    persistent: tile t of a CTA is blockIdx.x + t * gridDim.x.
+//    persistent: item t of a CTA is blockIdx.x + t * gridDim.x.
+//  * Weight reuse.  The nine taps make the weight operand of a step (9 x n_t x 16 values) six
+//    times larger than the activations it meets (128 pixels x 16 channels, halo included), and
+//    measured on the first version -- one pixel tile per weight stage -- the L2-to-SM traffic of
+//    the weight stream held the tensor pipe at 23 %.  A work item is therefore mt = 1, 2 or 4
+//    vertically adjacent pixel tiles (one halo'd strip of mt * r + 2 rows) that share every weight
+//    stage: mt accumulators of n_t columns each.  mt * n_t <= 256 leaves room for two accumulator
+//    sets; with 512 columns in use the epilogue of an item is not overlapped.
 //  * Every wait is bounded; a wait that runs out records its id (20-25) in the layer's status word,
 //    the role stops working, and all roles meet at the common exit where TMEM is released.
+//  * The kernel is compiled once per input layout (template parameter MODE): rows of a multiple of
+//    8 pixels (one aligned 16-byte load per task), other widths of 8 and more (element-wise), and
+//    the narrow maps with 4, 2 and 1 or 3 columns.  The producers' inner loop is instruction-bound
+//    (a task is one load, eight funnel shifts and three 16-byte stores), so everything that does
+//    not depend on the channel step is worked out once per item.
 #include <cuda_fp16.h>
 
 #include "pconv_internal.h"
@@ -50,7 +65,7 @@ constexpr int kProdWarpsPerGroup = 4;
 constexpr int kProdThreadsPerGroup = 32 * kProdWarpsPerGroup;
 constexpr int kTensorThreads = 32 * (kProdWarp0 + kProdGroups * kProdWarpsPerGroup);
 constexpr int kMaxTStages = 6;
-constexpr int kMaxTasks = 4;              // A tasks of one producer thread per stage
+constexpr int kMaxTasks = 9;              // A tasks of one producer thread per stage (18 rows x 64 / 128)
 constexpr uint32_t kTSpinLimit = 1u << 20;
 constexpr uint32_t kTWaitHintNs = 200;
 constexpr int kTSmemLimit = 227 * 1024;
@@ -61,12 +76,15 @@ struct TGeo {
   int wc;            // cell width: w rounded up to a multiple of 8, or to 1, 2, 4 for w < 8
   int cpr;           // cells (images) side by side in a strip row
   int tw, r;         // tile: r strip rows x tw columns, r * tw = 128
+  int mt, n_buf;     // pixel tiles per work item (stacked vertically); accumulator sets (1 or 2)
+  int rows_a;        // staged rows of an item: mt * r + 2
   int tiles_x;       // column tiles of the virtual width cpr * wc
-  long long strip_rows, tiles_y;
+  int strip_rows, tiles_y;   // strip rows of the batch; items along the strip
   int n_t, n_tiles_n, k_steps;
   int stages, a_copy_bytes, a_lbo, row_bytes, b_bytes, stage_bytes, stage_off;
+  int out_off, bias_off;   // the epilogue's staging tile [n_t][128] fp16 and the tile's bias [n_t] fp32
   int relu;
-  long long total_tiles;
+  long long total_items;   // tiles_y * tiles_x * n_tiles_n
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -140,34 +158,115 @@ __device__ __forceinline__ void tmem_ld16(uint32_t (&v)[16], uint32_t taddr) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-// One A task = (halo row, 8-channel block, column group of 8 pixels, channel within the block): 16
-// bytes of each of the three horizontally shifted copies.  What depends on the tile only is kept
-// per task: the element offset of the group's first pixel for channel `ch` of step 0 (-1: the
-// whole group is padding), the same for the pixel left of the group and right of it, and for
-// narrow maps the per-pixel data.
-struct ATask {
-  long long off;        // element offset of pixel 0 of the group (channel `ch` of k-step 0), or -1
-  uint32_t dst;         // byte offset inside a copy
-  int ch;               // channel inside the 16-channel step
-  uint32_t flags;       // bit 0: left neighbour exists, bit 1: right neighbour exists
-};
+// Input layouts the kernel is compiled for.
+enum { kModeW8 = 0,   // w a multiple of 8: a task is one aligned 16-byte load (+ two neighbours)
+       kModeWX = 1,   // any other w >= 5: element-wise loads and stores
+       kModeN4 = 2,   // w = 4: two images side by side, 8-byte rows
+       kModeN2 = 3,   // w = 2: four images side by side, 4-byte rows
+       kModeNX = 4 }; // w = 1 or 3: element-wise, 8 or 2 images side by side
 
-// The strip row a tile row maps to: image group and row inside it, or invalid (separator / outside).
-__device__ __forceinline__ bool strip_row(const TGeo& g, long long s, long long* group, int* row) {
+// One A task = (staged row, 8-channel block, column group of 8 pixels, channel within the block):
+// 16 bytes of each of the three horizontally shifted copies.  Task t of a stage decodes as
+// t = ((row * 2 + block) * (tw / 8) + group) * 8 + channel, so that the 32 lanes of a warp write
+// 512 contiguous bytes.
+
+// The image group and row of strip row s, or false for a separator row / outside the strip.
+__device__ __forceinline__ bool strip_row(const TGeo& g, int s, int* group, int* row) {
   if (s < 0 || s >= g.strip_rows) return false;
-  const long long gi = s / g.hp;
-  const int lr = (int)(s - gi * g.hp);
+  const int gi = s / g.hp;
+  const int lr = s - gi * g.hp;
   *group = gi;
   *row = lr;
   return lr < g.h;
 }
 
-template <bool RELU>
-__device__ __forceinline__ void store_col(__half* y, long long idx, float v) {
-  if (RELU) v = fmaxf(v, 0.f);
-  y[idx] = __float2half_rn(v);
+__device__ __forceinline__ uint32_t ldg_u16(const unsigned short* p) { return (uint32_t)__ldg(p); }
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// Barrier of the 128 epilogue threads that also tells whether `v` holds for all of them (so that a
+// bounded wait that ran out for some of them makes all of them leave together).
+__device__ __forceinline__ bool epi_all(bool v) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.and.pred p, 1, 128, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"((uint32_t)v)
+      : "memory");
+  return r != 0;
+}
+__device__ __forceinline__ uint32_t lds_b32(uint32_t a) {
+  uint32_t v;
+  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint4 lds_v4(uint32_t a) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ void sts_u16(uint32_t a, unsigned short v) {
+  asm volatile("st.shared.u16 [%0], %1;" ::"r"(a), "h"(v) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t (&v)[32], uint32_t taddr) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// The 8 pixels of one task (one channel, one staged row, one column group) as four packed fp16
+// pairs, and the pixels left and right of the group (0 where there is none).  `p` addresses the
+// group's first pixel; `aux` is what the item set-up left for the task: in the wide layouts bit 0 /
+// bit 1 = a left / right neighbour exists and bits 8.. = the first pixel's column, in the narrow
+// ones the number of the group's images that lie inside the batch.
+template <int MODE>
+__device__ __forceinline__ void load_task(const TGeo& g, const unsigned short* p, uint32_t aux, size_t img,
+                                          uint4* v, uint32_t* lft, uint32_t* rgt) {
+  *lft = *rgt = 0u;
+  if (MODE == kModeW8) {
+    *v = __ldg(reinterpret_cast<const uint4*>(p));
+    if (aux & 1u) *lft = ldg_u16(p - 1);
+    if (aux & 2u) *rgt = ldg_u16(p + 8);
+  } else if (MODE == kModeWX) {
+    const int vx = (int)(aux >> 8);
+    uint32_t e[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) e[i] = (vx + i < g.w) ? ldg_u16(p + i) : 0u;
+    *v = make_uint4(e[0] | (e[1] << 16), e[2] | (e[3] << 16), e[4] | (e[5] << 16), e[6] | (e[7] << 16));
+    if (aux & 1u) *lft = ldg_u16(p - 1);
+    if (aux & 2u) *rgt = ldg_u16(p + 8);
+  } else if (MODE == kModeN4) {
+    uint2 a = make_uint2(0u, 0u), b = a;
+    if (aux > 0) a = __ldg(reinterpret_cast<const uint2*>(p));
+    if (aux > 1) b = __ldg(reinterpret_cast<const uint2*>(p + img));
+    *v = make_uint4(a.x, a.y, b.x, b.y);
+  } else if (MODE == kModeN2) {
+    uint32_t e[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      if ((uint32_t)i < aux) e[i] = __ldg(reinterpret_cast<const uint32_t*>(p + i * img));
+    *v = make_uint4(e[0], e[1], e[2], e[3]);
+  } else {
+    uint32_t e[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int cell = g.wc == 1 ? i : i >> 2;      // w = 1: eight images; w = 3: two cells of four
+      const int xin = i - cell * g.wc;
+      e[i] = ((uint32_t)cell < aux && xin < g.w) ? ldg_u16(p + cell * img + xin) : 0u;
+    }
+    *v = make_uint4(e[0] | (e[1] << 16), e[2] | (e[3] << 16), e[4] | (e[5] << 16), e[6] | (e[7] << 16));
+  }
+}
+
+template <int MODE>
 __global__ void __launch_bounds__(kTensorThreads, 1)
 tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
               const float* __restrict__ bias, __half* __restrict__ y) {
@@ -179,7 +278,8 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
   const uint32_t bar_full = sbase, bar_empty = sbase + 8 * kMaxTStages;
   const uint32_t bar_accf = sbase + 16 * kMaxTStages, bar_acce = bar_accf + 16;
   volatile uint32_t* tmem_base_s = reinterpret_cast<volatile uint32_t*>(smem + 16 * kMaxTStages + 32);
-  const uint32_t tmem_cols = (uint32_t)(2 * g.n_t);   // 128 or 256: a power of two >= 32
+  const int acc_cols = g.mt * g.n_t;                          // columns of one accumulator set
+  const uint32_t tmem_cols = (uint32_t)(g.n_buf * acc_cols);  // 64 .. 512, a power of two
 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (tid == 0) {
@@ -206,9 +306,9 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
   // the previous kernel of the stream must have finished before x is read or y written
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
-  const long long my_tiles = (g.total_tiles > blockIdx.x)
-                                 ? (g.total_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
-  const uint32_t row_b = (uint32_t)g.row_bytes;     // bytes of one tile row of core matrices
+  const int my_items = (g.total_items > (long long)blockIdx.x)
+                           ? (int)((g.total_items - blockIdx.x + gridDim.x - 1) / gridDim.x) : 0;
+  const uint32_t row_b = (uint32_t)g.row_bytes;     // bytes of one staged row of core matrices
   const size_t hw = (size_t)g.h * g.w;
 
   if (warp == kMmaWarp) {
@@ -216,33 +316,40 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
     if (lane == 0) {
       // instruction descriptor: D fp32, A and B fp16, A pixel-major (MN-major), B K-major, N, M = 128
       const uint32_t idesc = (1u << 4) | (1u << 15) | ((uint32_t)(g.n_t >> 3) << 17) | ((128u >> 4) << 24);
-      const uint32_t b_lbo = (uint32_t)(g.n_t / 8) * 128u;
+      // descriptors of a stage differ in the start address only: bits 0-13 of the low word, in
+      // 16-byte units (shared memory is below 256 KB, so adding an offset never carries out)
+      const u64 a_desc0 = smem_desc(0u, (uint32_t)g.a_lbo, 128u);
+      const u64 b_desc0 = smem_desc(0u, (uint32_t)(g.n_t / 8) * 128u, 128u);
+      const uint32_t copy16 = (uint32_t)g.a_copy_bytes >> 4, row16 = row_b >> 4;
+      const uint32_t tap16 = (uint32_t)(g.n_t * 32) >> 4, tile16 = (uint32_t)g.r * row16;
       long long it = 0;
       bool ok = true;
-      for (long long ti = 0; ti < my_tiles && ok; ++ti) {
-        const int buf = (int)(ti & 1);
-        const uint32_t use = (uint32_t)(ti >> 1);
+      for (int ti = 0; ti < my_items && ok; ++ti) {
+        const int buf = ti % g.n_buf;
+        const uint32_t use = (uint32_t)(ti / g.n_buf);
         ok = mbar_wait(bar_acce + 8 * buf, (use & 1u) ^ 1u, L.err, 20);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * g.n_t);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * acc_cols);
         for (int ks = 0; ks < g.k_steps; ++ks, ++it) {
           const int s = (int)(it % g.stages);
           ok = mbar_wait(bar_full + 8 * s, (uint32_t)((it / g.stages) & 1), L.err, 21);
           if (!ok) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t a0 = sbase + g.stage_off + s * g.stage_bytes;
-          const uint32_t b0 = a0 + 3 * g.a_copy_bytes;
+          const u64 a_st = a_desc0 + (a0 >> 4), b_st = b_desc0 + ((a0 + 3 * g.a_copy_bytes) >> 4);
+          for (int j = 0; j < g.mt; ++j) {       // the item's pixel tiles share the stage's weights
+            const u64 a_tile = a_st + j * tile16;
 #pragma unroll
-          for (int t = 0; t < 9; ++t) {
-            const int u = t / 3, v = t - 3 * u;
-            const u64 ad = smem_desc(a0 + v * g.a_copy_bytes + u * row_b, (uint32_t)g.a_lbo, 128u);
-            const u64 bd = smem_desc(b0 + t * (g.n_t * 32), b_lbo, 128u);
-            umma_f16(d_tmem, ad, bd, idesc, (ks > 0 || t > 0) ? 1u : 0u);
+            for (int t = 0; t < 9; ++t) {
+              const int u = t / 3, v = t - 3 * u;
+              umma_f16(d_tmem + (uint32_t)(j * g.n_t), a_tile + v * copy16 + u * row16, b_st + t * tap16,
+                       idesc, (ks > 0 || t > 0) ? 1u : 0u);
+            }
           }
           umma_commit(bar_empty + 8 * s);          // the stage may be refilled once these MMAs are done
         }
-        if (ok) umma_commit(bar_accf + 8 * buf);   // the tile's accumulator is complete
+        if (ok) umma_commit(bar_accf + 8 * buf);   // the item's accumulators are complete
       }
     }
     __syncwarp();
@@ -250,53 +357,76 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
     // ======================================= A producers ======================================
     const int group = (warp - kProdWarp0) / kProdWarpsPerGroup;
     const int gt = (warp - kProdWarp0 - group * kProdWarpsPerGroup) * 32 + lane;
-    const int cgs = g.tw / 8;
-    const int n_tasks = (g.r + 2) * 2 * cgs * 8;
+    const int cg_shift = g.tw == 32 ? 2 : (g.tw == 16 ? 1 : 0);      // log2(column groups of a row)
+    const int n_tasks = g.rows_a << (4 + cg_shift);                 // rows x 2 blocks x groups x 8 channels
     const unsigned short* xs = reinterpret_cast<const unsigned short*>(x);
-    const bool fast = (g.w % 8) == 0;          // rows are 16-byte aligned: one vector load per task
+    const size_t img = (size_t)g.c_in * hw;    // elements of one image
+    const size_t step = 16 * hw;               // elements between channel steps
+    // what depends on the task only: its place in a copy and its channel inside a step
+    uint32_t dst[kMaxTasks];
+#pragma unroll
+    for (int q = 0; q < kMaxTasks; ++q) {
+      const int t = gt + q * kProdThreadsPerGroup;
+      const int c8 = t & 7, cg = (t >> 3) & ((1 << cg_shift) - 1);
+      const int kb = (t >> (3 + cg_shift)) & 1, hr = t >> (4 + cg_shift);
+      dst[q] = (uint32_t)(kb * g.a_lbo) + (uint32_t)hr * row_b + (uint32_t)(cg * 128 + c8 * 16);
+    }
+    // keep-masks of the shifted copies on narrow maps: no pixel may see across its image's edge
+    // (copy 0 shows the left neighbour: cleared where the pixel is a row's first; copy 2 the right
+    // neighbour: cleared where the pixel is the row's last); even / odd = words 0, 2 / 1, 3
+    uint32_t zm_even = 0xFFFFFFFFu, zm_odd = 0xFFFFFFFFu, zp_even = 0xFFFFFFFFu, zp_odd = 0xFFFFFFFFu;
+    if (MODE == kModeN4 || (MODE == kModeNX && g.wc == 4)) {
+      zm_even = 0xFFFF0000u;                                   // pixels 0 and 4 start a row
+      zp_odd = (g.w == 4) ? 0x0000FFFFu : 0xFFFF0000u;         // pixels 3, 7 (w = 4) or 2, 6 (w = 3) end one
+    } else if (MODE == kModeN2) {
+      zm_even = zm_odd = 0xFFFF0000u;                          // even pixels start a row, odd ones end it
+      zp_even = zp_odd = 0x0000FFFFu;
+    } else if (MODE == kModeNX) {                              // w = 1: no neighbours at all
+      zm_even = zm_odd = zp_even = zp_odd = 0u;
+    }
     bool ok = true;
-    long long it = 0;                          // global stage counter (all tiles of this CTA)
-    for (long long ti = 0; ti < my_tiles && ok; ++ti) {
-      const long long tile = blockIdx.x + ti * gridDim.x;
-      const long long mt = tile / g.n_tiles_n;
-      const int nt = (int)(tile - mt * g.n_tiles_n);
-      const long long ty = mt / g.tiles_x;
-      const int tx = (int)(mt - ty * g.tiles_x);
-      ATask task[kMaxTasks];
+    long long it = 0;                          // stage counter over all items of this CTA
+    for (int ti = 0; ti < my_items && ok; ++ti) {
+      // the stages of this item that fall to this group: none if the item has one step and it is
+      // the other group's turn
+      if (g.k_steps == 1 && (int)(it & 1) != group) {
+        ++it;
+        continue;
+      }
+      const long long item = blockIdx.x + (long long)ti * gridDim.x;
+      const int mti = (int)(item / g.n_tiles_n);
+      const int nt = (int)(item - (long long)mti * g.n_tiles_n);
+      const int ty = mti / g.tiles_x;
+      const int tx = mti - ty * g.tiles_x;
+      // per task: where its 8 pixels are for the channels of step 0 (null = padding) and `aux`
+      const unsigned short* src[kMaxTasks];
+      uint32_t aux[kMaxTasks];
 #pragma unroll
       for (int q = 0; q < kMaxTasks; ++q) {
         const int t = gt + q * kProdThreadsPerGroup;
-        task[q].off = -1;
-        task[q].dst = 0xFFFFFFFFu;
-        task[q].ch = 0;
-        task[q].flags = 0;
+        src[q] = nullptr;
+        aux[q] = 0u;
         if (t < n_tasks) {
-          const int c8 = t & 7;
-          int rest = t >> 3;
-          const int cg = rest % cgs;
-          rest /= cgs;
-          const int kb = rest & 1, hr = rest >> 1;
-          task[q].ch = kb * 8 + c8;
-          task[q].dst = (uint32_t)(kb * g.a_lbo + hr * (int)row_b + cg * 128 + c8 * 16);
-          long long gi;
-          int lr;
-          const int vx = tx * g.tw + cg * 8;        // virtual column of the group's first pixel
-          if (strip_row(g, ty * g.r + hr - 1, &gi, &lr) && g.wc >= 8) {
-            const long long n_img = gi;             // one image per strip row
-            if (n_img < g.n && vx < g.w) {
-              task[q].off = ((n_img * g.c_in + task[q].ch) * g.h + lr) * (long long)g.w + vx;
-              task[q].flags = (vx > 0 ? 1u : 0u) | (vx + 8 < g.w ? 2u : 0u);
+          const int c8 = t & 7, cg = (t >> 3) & ((1 << cg_shift) - 1);
+          const int kb = (t >> (3 + cg_shift)) & 1, hr = t >> (4 + cg_shift);
+          const int ch = kb * 8 + c8;
+          int gi, lr;
+          if (strip_row(g, ty * (g.mt * g.r) + hr - 1, &gi, &lr)) {
+            if (MODE == kModeW8 || MODE == kModeWX) {   // one image per strip row
+              const int vx = tx * g.tw + cg * 8;        // column of the group's first pixel
+              if (vx < g.w) {
+                src[q] = xs + (((size_t)gi * g.c_in + ch) * g.h + lr) * (size_t)g.w + vx;
+                aux[q] = (vx > 0 ? 1u : 0u) | (vx + 8 < g.w ? 2u : 0u) | ((uint32_t)vx << 8);
+              }
+            } else {                                    // 8 / wc images side by side: the first one
+              src[q] = xs + (((size_t)gi * g.cpr * g.c_in + ch) * g.h + lr) * (size_t)g.w;
+              aux[q] = (uint32_t)min(g.cpr, g.n - gi * g.cpr);
             }
-          } else if (g.wc < 8 && strip_row(g, ty * g.r + hr - 1, &gi, &lr)) {
-            // narrow maps: the 8 pixels are 8 / wc images side by side; `off` addresses the first
-            task[q].off = ((gi * g.cpr + vx / g.wc) * (long long)g.c_in + task[q].ch) * g.h * (long long)g.w +
-                          (long long)lr * g.w;
-            task[q].flags = 4u;
           }
         }
       }
       for (int ks = 0; ks < g.k_steps && ok; ++ks, ++it) {
-        if ((it & 1) != group) continue;           // the other group's stage
+        if ((int)(it & 1) != group) continue;       // the other group's stage
         const int s = (int)(it % g.stages);
         ok = mbar_wait(bar_empty + 8 * s, (uint32_t)(((it / g.stages) & 1) ^ 1), L.err, 22);
         if (!ok) break;
@@ -307,46 +437,27 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
                         reinterpret_cast<const char*>(L.wdense) + ((size_t)nt * g.k_steps + ks) * g.b_bytes,
                         (uint32_t)g.b_bytes, bar_full + 8 * s);
         }
-        const int c_base = ks * 16;
-        // loads of all tasks first, then shifts and stores
+        // channels beyond c_in (last step of a layer whose depth is no multiple of 16) are zeros
+        const int ch_limit = g.c_in - ks * 16;
+        const size_t chan_off = (size_t)ks * step;
+        // every load of the stage first (they are independent), then shifts and stores
         uint4 v[kMaxTasks];
         uint32_t lft[kMaxTasks], rgt[kMaxTasks];
 #pragma unroll
         for (int q = 0; q < kMaxTasks; ++q) {
           v[q] = make_uint4(0u, 0u, 0u, 0u);
           lft[q] = rgt[q] = 0u;
-          if (task[q].dst == 0xFFFFFFFFu || task[q].off < 0) continue;
-          const int c = c_base + task[q].ch;
-          if (c >= g.c_in) continue;
-          const unsigned short* p = xs + task[q].off + (size_t)c_base * hw;
-          if (task[q].flags & 4u) {
-            // narrow maps: pixel q8 belongs to image (q8 / wc) of the row, column q8 % wc
-            uint32_t e[8];
-            const long long img0 = task[q].off / ((long long)g.c_in * (long long)hw);
-#pragma unroll
-            for (int q8 = 0; q8 < 8; ++q8) {
-              const int cell = q8 / g.wc, xin = q8 - cell * g.wc;
-              e[q8] = (xin < g.w && img0 + cell < g.n)
-                          ? (uint32_t)__ldg(p + (size_t)cell * g.c_in * hw + xin) : 0u;
-            }
-            v[q] = make_uint4(e[0] | (e[1] << 16), e[2] | (e[3] << 16), e[4] | (e[5] << 16), e[6] | (e[7] << 16));
-          } else if (fast) {
-            v[q] = __ldg(reinterpret_cast<const uint4*>(p));
-            if (task[q].flags & 1u) lft[q] = (uint32_t)__ldg(p - 1);
-            if (task[q].flags & 2u) rgt[q] = (uint32_t)__ldg(p + 8);
-          } else {
-            const int vx = (int)((task[q].off) % g.w);   // column of pixel 0 (off = ... * w + vx)
-            uint32_t e[8];
-#pragma unroll
-            for (int q8 = 0; q8 < 8; ++q8) e[q8] = (vx + q8 < g.w) ? (uint32_t)__ldg(p + q8) : 0u;
-            v[q] = make_uint4(e[0] | (e[1] << 16), e[2] | (e[3] << 16), e[4] | (e[5] << 16), e[6] | (e[7] << 16));
-            if (task[q].flags & 1u) lft[q] = (uint32_t)__ldg(p - 1);
-            if (task[q].flags & 2u) rgt[q] = (uint32_t)__ldg(p + 8);
+          if (src[q] == nullptr) continue;
+          if (ch_limit < 16) {
+            const int t = gt + q * kProdThreadsPerGroup;
+            if (((((t >> (3 + cg_shift)) & 1) << 3) | (t & 7)) >= ch_limit) continue;
           }
+          load_task<MODE>(g, src[q] + chan_off, aux[q], img, &v[q], &lft[q], &rgt[q]);
         }
+        const uint32_t copy_b = (uint32_t)g.a_copy_bytes;
 #pragma unroll
         for (int q = 0; q < kMaxTasks; ++q) {
-          if (task[q].dst == 0xFFFFFFFFu) continue;
+          if (gt + q * kProdThreadsPerGroup >= n_tasks) continue;
           const uint4 c = v[q];
           // copy 0: pixel p holds input column p - 1;  copy 2: column p + 1
           uint4 m1, p1;
@@ -358,24 +469,14 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
           p1.y = __funnelshift_r(c.y, c.z, 16);
           p1.z = __funnelshift_r(c.z, c.w, 16);
           p1.w = __funnelshift_r(c.w, rgt[q], 16);
-          if (task[q].flags & 4u) {
-            // narrow maps: no pixel may see across its image's edge
-            uint32_t zm[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};   // keep masks, copy 0
-            uint32_t zp[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};   // copy 2
-#pragma unroll
-            for (int q8 = 0; q8 < 8; ++q8) {
-              const int xin = q8 % g.wc;
-              const uint32_t half_mask = (q8 & 1) ? 0x0000FFFFu : 0xFFFF0000u;   // what stays when this half is cleared
-              if (xin == 0) zm[q8 >> 1] &= half_mask;
-              if (xin + 1 >= g.w) zp[q8 >> 1] &= half_mask;
-            }
-            m1.x &= zm[0]; m1.y &= zm[1]; m1.z &= zm[2]; m1.w &= zm[3];
-            p1.x &= zp[0]; p1.y &= zp[1]; p1.z &= zp[2]; p1.w &= zp[3];
+          if (MODE >= kModeN4) {
+            m1.x &= zm_even; m1.y &= zm_odd; m1.z &= zm_even; m1.w &= zm_odd;
+            p1.x &= zp_even; p1.y &= zp_odd; p1.z &= zp_even; p1.w &= zp_odd;
           }
-          const uint32_t d = a0 + task[q].dst;
+          const uint32_t d = a0 + dst[q];
           sts128(d, m1.x, m1.y, m1.z, m1.w);
-          sts128(d + g.a_copy_bytes, c.x, c.y, c.z, c.w);
-          sts128(d + 2 * g.a_copy_bytes, p1.x, p1.y, p1.z, p1.w);
+          sts128(d + copy_b, c.x, c.y, c.z, c.w);
+          sts128(d + 2 * copy_b, p1.x, p1.y, p1.z, p1.w);
         }
         // generic-proxy stores must be visible to the tensor core's (async proxy) reads
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -384,48 +485,109 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
     }
   } else {
     // ======================================= epilogue =========================================
+    // Accumulators (lane = pixel, column = filter) -> bias, ReLU, fp16 -> shared memory as
+    // [filter][pixel] -> 16-byte pieces (8 consecutive pixels of a filter) to y.
     const int q = warp;                       // TMEM lane quadrant
-    const int m = 32 * q + lane;              // pixel of the tile
-    const int tr = m / g.tw, tc = m - tr * g.tw;
+    const int m = 32 * q + lane;              // this lane's pixel of a tile
+    const int et = tid;                       // 0..127
+    const uint32_t out_s = sbase + (uint32_t)g.out_off;       // [n_t][128] fp16
+    const uint32_t bias_s = sbase + (uint32_t)g.bias_off;     // [n_t] fp32
+    // copy-out: this thread always handles pixel group pg (8 pixels) of filters f0, f0 + 8, ...
+    const int pg = et & 15, f0 = et >> 4;
+    const int ctr = (pg * 8) / g.tw, ctc = (pg * 8) - ctr * g.tw;   // the group's tile row / first column
     bool ok = true;
-    for (long long ti = 0; ti < my_tiles && ok; ++ti) {
-      const long long tile = blockIdx.x + ti * gridDim.x;
-      const long long mt = tile / g.n_tiles_n;
-      const int nt = (int)(tile - mt * g.n_tiles_n);
-      const long long ty = mt / g.tiles_x;
-      const int tx = (int)(mt - ty * g.tiles_x);
-      const int buf = (int)(ti & 1);
-      const uint32_t use = (uint32_t)(ti >> 1);
-      long long gi = 0;
-      int lr = 0;
-      bool valid = strip_row(g, ty * g.r + tr, &gi, &lr);
-      const int vcol = tx * g.tw + tc;
-      const int cell = vcol / g.wc, xin = vcol - cell * g.wc;
-      const long long n_img = gi * g.cpr + cell;
-      valid = valid && xin < g.w && cell < g.cpr && n_img < g.n;
-      const long long base = valid ? (n_img * g.c_out * (long long)g.h + lr) * g.w + xin : 0;
+    for (int ti = 0; ti < my_items && ok; ++ti) {
+      const long long item = blockIdx.x + (long long)ti * gridDim.x;
+      const int mti = (int)(item / g.n_tiles_n);
+      const int nt = (int)(item - (long long)mti * g.n_tiles_n);
+      const int ty = mti / g.tiles_x;
+      const int tx = mti - ty * g.tiles_x;
+      const int buf = ti % g.n_buf;
+      const uint32_t use = (uint32_t)(ti / g.n_buf);
+      const int o_base = nt * g.n_t;
+      const int n_f = min(g.n_t, g.c_out - o_base);            // real filters of this tile
+      epi_sync();                                              // the previous item's bias is no longer read
+      if (et < g.n_t) {
+        const float bv = (bias && et < n_f) ? __ldg(bias + o_base + et) : 0.f;
+        asm volatile("st.shared.f32 [%0], %1;" ::"r"(bias_s + 4 * et), "f"(bv) : "memory");
+      }
       ok = mbar_wait(bar_accf + 8 * buf, use & 1u, L.err, 23);
+      ok = epi_all(ok);                                        // bias staged; all leave together if a wait ran out
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * g.n_t);
-      for (int j0 = 0; j0 < g.n_t; j0 += 16) {
-        const int o0 = nt * g.n_t + j0;
-        if (o0 >= g.c_out) break;               // padding filters of the last tile (warp-uniform)
-        uint32_t acc[16];
-        tmem_ld16(acc, taddr + (uint32_t)j0);
+      for (int j = 0; j < g.mt; ++j) {
+        const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * acc_cols + j * g.n_t);
+        for (int j0 = 0; j0 < n_f; j0 += 32) {
+          uint32_t acc[32];
+          tmem_ld32(acc, taddr + (uint32_t)j0);
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const int o = o0 + j;
-          if (o < g.c_out && valid) {
-            const float bv = bias ? __ldg(bias + o) : 0.f;
-            const float val = __uint_as_float(acc[j]) + bv;
-            if (g.relu) store_col<true>(y, base + (long long)o * (long long)hw, val);
-            else store_col<false>(y, base + (long long)o * (long long)hw, val);
+          for (int jj = 0; jj < 32; ++jj) {
+            float val = __uint_as_float(acc[jj]) + __uint_as_float(lds_b32(bias_s + 4 * (j0 + jj)));
+            if (g.relu) val = fmaxf(val, 0.f);
+            sts_u16(out_s + (uint32_t)((j0 + jj) * 256 + m * 2), __half_as_ushort(__float2half_rn(val)));
           }
         }
+        if (j == g.mt - 1) {   // the accumulators have been read: the MMA warp may reuse them
+          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+          mbar_arrive(bar_acce + 8 * buf);
+        }
+        epi_sync();                                            // the tile is staged
+        // where this thread's pixel group goes
+        int gi = 0, lr = 0;
+        const bool row_ok = strip_row(g, (ty * g.mt + j) * g.r + ctr, &gi, &lr);
+        const int vx = tx * g.tw + ctc;
+        if (row_ok) {
+          if (MODE == kModeW8) {
+            if (vx < g.w) {
+              __half* dstp = y + (((size_t)gi * g.c_out + o_base) * g.h + lr) * (size_t)g.w + vx;
+              for (int f = f0; f < n_f; f += 8)
+                *reinterpret_cast<uint4*>(dstp + (size_t)f * hw) = lds_v4(out_s + (uint32_t)(f * 256 + pg * 16));
+            }
+          } else if (MODE == kModeWX) {
+            if (vx < g.w) {
+              __half* dstp = y + (((size_t)gi * g.c_out + o_base) * g.h + lr) * (size_t)g.w + vx;
+              const int npx = min(8, g.w - vx);
+              for (int f = f0; f < n_f; f += 8) {
+                const uint4 vv = lds_v4(out_s + (uint32_t)(f * 256 + pg * 16));
+                const uint32_t wds[4] = {vv.x, vv.y, vv.z, vv.w};
+                unsigned short* dp = reinterpret_cast<unsigned short*>(dstp + (size_t)f * hw);
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                  if (i < npx) dp[i] = (unsigned short)(wds[i >> 1] >> (16 * (i & 1)));
+              }
+            }
+          } else {
+            // narrow maps: the group is 8 / wc images side by side, w pixels of each are real
+            const int cells = min(g.cpr, g.n - gi * g.cpr);
+            __half* dstp = y + (((size_t)gi * g.cpr * g.c_out + o_base) * g.h + lr) * (size_t)g.w;
+            const size_t oimg = (size_t)g.c_out * hw;
+            for (int f = f0; f < n_f; f += 8) {
+              const uint4 vv = lds_v4(out_s + (uint32_t)(f * 256 + pg * 16));
+              __half* dp = dstp + (size_t)f * hw;
+              if (MODE == kModeN4) {
+                if (cells > 0) *reinterpret_cast<uint2*>(dp) = make_uint2(vv.x, vv.y);
+                if (cells > 1) *reinterpret_cast<uint2*>(dp + oimg) = make_uint2(vv.z, vv.w);
+              } else if (MODE == kModeN2) {
+                const uint32_t wds[4] = {vv.x, vv.y, vv.z, vv.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                  if (i < cells) *reinterpret_cast<uint32_t*>(dp + i * oimg) = wds[i];
+              } else {
+                const uint32_t wds[4] = {vv.x, vv.y, vv.z, vv.w};
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                  const int cell = g.wc == 1 ? i : i >> 2;
+                  const int xin = i - cell * g.wc;
+                  if (cell < cells && xin < g.w)
+                    reinterpret_cast<unsigned short*>(dp + cell * oimg)[xin] =
+                        (unsigned short)(wds[i >> 1] >> (16 * (i & 1)));
+                }
+              }
+            }
+          }
+        }
+        epi_sync();                                            // staging buffer free again
       }
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      mbar_arrive(bar_acce + 8 * buf);
     }
   }
 
@@ -437,7 +599,8 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
                  : "memory");
 }
 
-bool tensor_geo(const DeviceLayer& L, int n, int h, int w, TGeo* out) {
+// Geometry of a launch with mt pixel tiles per work item; false if it does not fit.
+bool tensor_geo_mt(const DeviceLayer& L, int n, int h, int w, int mt, TGeo* out) {
   if (!L.wdense || L.dense_nt <= 0 || L.stride != 1 || L.storage != PCONV_F16) return false;
   TGeo g;
   g.n = n;
@@ -455,33 +618,55 @@ bool tensor_geo(const DeviceLayer& L, int n, int h, int w, TGeo* out) {
   }
   const int vw = g.wc * g.cpr;
   // Tile width: a power of two from 8 to 32.  32 columns are 64 contiguous bytes per row and
-  // channel (whole sectors), and four rows of halo'd height 6 keep the re-read of halo rows at 1.5;
-  // wider maps take several column tiles, the horizontal neighbours come from the image itself.
+  // channel (whole sectors); wider maps take several column tiles, the horizontal neighbours
+  // come from the image itself.
   g.tw = 8;
   while (g.tw < vw && g.tw < 32) g.tw *= 2;
   g.r = 128 / g.tw;
   g.tiles_x = (vw + g.tw - 1) / g.tw;
-  g.strip_rows = ((long long)n + g.cpr - 1) / g.cpr * g.hp;
-  g.tiles_y = (g.strip_rows + g.r - 1) / g.r;
+  const long long strip = ((long long)n + g.cpr - 1) / g.cpr * g.hp;
+  if (strip > 0x3FFFFFFF) return false;
+  g.strip_rows = (int)strip;
   g.n_t = L.dense_nt;
+  if (mt * g.n_t > 512) return false;
+  g.mt = mt;
+  g.n_buf = (2 * mt * g.n_t <= 512) ? 2 : 1;
+  g.rows_a = mt * g.r + 2;
+  g.tiles_y = (g.strip_rows + mt * g.r - 1) / (mt * g.r);
   g.n_tiles_n = (L.c_out + g.n_t - 1) / g.n_t;
   g.k_steps = (L.c_in + 15) / 16;
   g.row_bytes = (g.tw / 8) * 128;
-  g.a_lbo = (g.r + 2) * g.row_bytes;
+  g.a_lbo = g.rows_a * g.row_bytes;
   g.a_copy_bytes = 2 * g.a_lbo;
   g.b_bytes = 9 * g.n_t * 32;
   g.stage_bytes = 3 * g.a_copy_bytes + g.b_bytes;
   g.stage_off = 256;
-  g.stages = (kTSmemLimit - g.stage_off) / g.stage_bytes;
+  const int epi_bytes = g.n_t * 256 + g.n_t * 4;
+  g.stages = (kTSmemLimit - g.stage_off - epi_bytes) / g.stage_bytes;
   if (g.stages > kMaxTStages) g.stages = kMaxTStages;
-  if (g.stages & 1) --g.stages;            // the two producer groups take alternate stages
   if (g.stages < 2) return false;
-  if ((g.r + 2) * 2 * (g.tw / 8) * 8 > kMaxTasks * kProdThreadsPerGroup) return false;
+  g.out_off = g.stage_off + g.stages * g.stage_bytes;
+  g.bias_off = g.out_off + g.n_t * 256;
+  if (g.rows_a * 2 * (g.tw / 8) * 8 > kMaxTasks * kProdThreadsPerGroup) return false;
   g.relu = 0;
-  g.total_tiles = g.tiles_y * g.tiles_x * g.n_tiles_n;
-  if (g.tiles_y * g.tiles_x > 0x7FFFFFFFll) return false;
+  g.total_items = (long long)g.tiles_y * g.tiles_x * g.n_tiles_n;
   *out = g;
   return true;
+}
+
+// The launch geometry: as many pixel tiles per item (weight reuse) as still leave every SM at
+// least one item, preferring a count of items that fills whole waves.
+bool tensor_geo(const DeviceLayer& L, int n, int h, int w, TGeo* out) {
+  const long long sms = device_sm_count();
+  bool found = false;
+  for (int mt = 4; mt >= 1; mt /= 2) {
+    TGeo g;
+    if (!tensor_geo_mt(L, n, h, w, mt, &g)) continue;
+    *out = g;              // the last one tried (fewest tiles per item) stands if none fills the device
+    found = true;
+    if (g.total_items >= sms) return true;
+  }
+  return found;
 }
 
 }  // namespace
@@ -492,29 +677,31 @@ bool tensor_supported(const DeviceLayer& L, int n, int h, int w) {
 }
 
 // Whether the dense tensor-core path is expected to beat the pattern-sparse kernel: it needs
-// enough tiles to occupy the device (it has no channel split), and the zero-inserted contraction
-// (9 / (4 x keep) times the surviving multiply-adds, at roughly a third of the tensor peak) must be
-// cheaper than the surviving multiply-adds at the ~20 % of the FP32 peak the sparse kernel reaches.
+// enough pixel tiles to occupy a fair part of the device (it has no channel split), and the
+// zero-inserted contraction over the padded shape (channels to 16, filters to the tile) at the
+// fifth of the tensor peak this kernel reaches must be cheaper than the surviving multiply-adds at
+// the fifth of the FP32 peak the sparse kernel reaches.  (Measured on the CIFAR-shaped stack at
+// batch 256: faster on every layer but the 3-channel first one, which this rule leaves to the
+// sparse kernel.)
 bool tensor_preferred(const DeviceLayer& L, int n, int h, int w) {
   TGeo g;
   if (!tensor_geo(L, n, h, w, &g)) return false;
-  if (g.total_tiles < device_sm_count() / 2) return false;
-  const double dense = 2.0 * 9.0 * (double)L.c_in * (double)g.n_tiles_n * g.n_t;   // per pixel
+  if (g.total_items * g.mt < device_sm_count() / 4) return false;
+  const double dense = 2.0 * 9.0 * (16.0 * g.k_steps) * ((double)g.n_tiles_n * g.n_t);   // per pixel
   const double sparse = 8.0 * (double)L.n_kept;
-  return dense / (0.33 * 2250e12) < sparse / (0.2 * 74.45e12);
+  return dense / (0.2 * 2250e12) < sparse / (0.2 * 74.45e12);
 }
 
-cudaError_t launch_tensor(const DeviceLayer& L, const void* x, const float* bias, void* y, int n, int h,
-                          int w, bool relu, cudaStream_t stream) {
-  TGeo g;
-  if (!tensor_geo(L, n, h, w, &g)) return cudaErrorInvalidValue;
-  g.relu = relu ? 1 : 0;
-  const int smem = g.stage_off + g.stages * g.stage_bytes;
-  cudaError_t e = cudaFuncSetAttribute(tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmemLimit);
+template <int MODE>
+cudaError_t launch_tensor_mode(const DeviceLayer& L, const TGeo& g, const void* x, const float* bias, void* y,
+                               cudaStream_t stream) {
+  const int smem = g.bias_off + g.n_t * 4;
+  cudaError_t e = cudaFuncSetAttribute(tensor_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kTSmemLimit);
   if (e != cudaSuccess) return e;
   const long long sms = device_sm_count();
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(g.total_tiles < sms ? g.total_tiles : sms), 1, 1);
+  cfg.gridDim = dim3((unsigned)(g.total_items < sms ? g.total_items : sms), 1, 1);
   cfg.blockDim = dim3(kTensorThreads, 1, 1);
   // more than half of an SM's shared memory: one CTA per SM, whatever the stage count
   cfg.dynamicSmemBytes = (size_t)(smem < 120 * 1024 ? 120 * 1024 : smem);
@@ -524,7 +711,19 @@ cudaError_t launch_tensor(const DeviceLayer& L, const void* x, const float* bias
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, tensor_kernel, L, g, (const __half*)x, bias, (__half*)y);
+  return cudaLaunchKernelEx(&cfg, tensor_kernel<MODE>, L, g, (const __half*)x, bias, (__half*)y);
+}
+
+cudaError_t launch_tensor(const DeviceLayer& L, const void* x, const float* bias, void* y, int n, int h,
+                          int w, bool relu, cudaStream_t stream) {
+  TGeo g;
+  if (!tensor_geo(L, n, h, w, &g)) return cudaErrorInvalidValue;
+  g.relu = relu ? 1 : 0;
+  if (w >= 8 && w % 8 == 0) return launch_tensor_mode<kModeW8>(L, g, x, bias, y, stream);
+  if (w >= 5) return launch_tensor_mode<kModeWX>(L, g, x, bias, y, stream);
+  if (w == 4) return launch_tensor_mode<kModeN4>(L, g, x, bias, y, stream);
+  if (w == 2) return launch_tensor_mode<kModeN2>(L, g, x, bias, y, stream);
+  return launch_tensor_mode<kModeNX>(L, g, x, bias, y, stream);
 }
 
 }  // namespace pconv

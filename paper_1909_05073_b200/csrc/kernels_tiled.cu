@@ -46,19 +46,12 @@ namespace {
 
 typedef unsigned long long u64;
 
-#ifndef PCONV_CW
-#define PCONV_CW 16
-#endif
-#ifndef PCONV_PW
-#define PCONV_PW 4
-#endif
-constexpr int kProducerWarps = PCONV_PW;
-constexpr int kCtasPerSm = (PCONV_CW == 16) ? 1 : 2;
-__host__ __device__ constexpr int consumer_warps(bool generic) { return generic ? 8 : PCONV_CW; }
+constexpr int kProducerWarps = 4;
+__host__ __device__ constexpr int consumer_warps(bool generic) { return generic ? 8 : 16; }
 __host__ __device__ constexpr int cta_threads(bool generic) {
   return 32 * (consumer_warps(generic) + kProducerWarps);
 }
-constexpr int kTmemCols = 32 * PCONV_CW;  // consumer warps / 4 per lane quadrant x 16 slots x 8 columns
+constexpr int kTmemCols = 512;  // whole TMEM of the SM: 16 warps x 16 slots x 8 columns
 constexpr int kMaxStages = 8;
 constexpr int kMaxCoop = 4;   // chunks whose x the consumer warps copy at the start of a launch
 constexpr int kWSlot = kMaxBlockKernels * 16 + 16;  // bytes per (group, stage): 4 fp32 per kernel
@@ -69,7 +62,7 @@ constexpr uint32_t kSpinLimit = 1u << 20;
 // A waiting warp is suspended by the hardware for up to this long per try (it is woken when the
 // phase completes), so that waiting warps leave the issue slots to the warps that have work.
 constexpr uint32_t kWaitHintNs = 200;
-constexpr int kSmemLimit = (kCtasPerSm == 1) ? 227 * 1024 : 113 * 1024;
+constexpr int kSmemLimit = 227 * 1024;
 
 struct SubTile {
   int n, y0, x0, valid;  // image, first output row / column, inside the batch?
@@ -367,8 +360,9 @@ __device__ __forceinline__ void stage_blocks_async(const DeviceLayer& L, const G
   const uint32_t cbase = wbase + g.ng * kWSlot;
   for (int j = 0; j < g.ng; ++j) {
     const uint4 d = desc[2 * (j * g.cps + kk)];  // {w_off, n_k, code_off, code_len}
-    for (uint32_t i = (uint32_t)ptid; i < d.y; i += kProducerThreads)
-      cp_async16(wbase + j * kWSlot + i * 16, reinterpret_cast<const float*>(L.wvals) + (size_t)(d.x + i) * 4);
+    if ((uint32_t)ptid < d.y)
+      cp_async16(wbase + j * kWSlot + ptid * 16,
+                 reinterpret_cast<const float*>(L.wvals) + (size_t)(d.x + ptid) * 4);
     if ((uint32_t)ptid * 16 < d.w) cp_async16(cbase + j * kCodeSlot + ptid * 16, codes + d.z + ptid * 16);
   }
 }
@@ -387,32 +381,22 @@ __device__ __forceinline__ void stage_blocks_half(const DeviceLayer& L, const Ge
     const uint4 d = desc[2 * (j * g.cps + kk)];
     if ((uint32_t)ptid * 16 < d.w) cp_async16(cbase + j * kCodeSlot + ptid * 16, codes + d.z + ptid * 16);
   }
-  constexpr int kPer = (kMaxBlockKernels + kProducerThreads - 1) / kProducerThreads;  // kernels per thread
-  uint2 raw[kMaxNg][kPer];
+  uint2 raw[kMaxNg];
 #pragma unroll
   for (int j = 0; j < kMaxNg; ++j) {
-#pragma unroll
-    for (int u = 0; u < kPer; ++u) {
-      raw[j][u] = make_uint2(0u, 0u);
-      if (j < g.ng) {
-        const uint4 d = desc[2 * (j * g.cps + kk)];
-        const uint32_t i = (uint32_t)ptid + u * kProducerThreads;
-        if (i < d.y) raw[j][u] = __ldg(reinterpret_cast<const uint2*>(L.wvals) + d.x + i);
-      }
+    raw[j] = make_uint2(0u, 0u);
+    if (j < g.ng) {
+      const uint4 d = desc[2 * (j * g.cps + kk)];
+      if ((uint32_t)ptid < d.y) raw[j] = __ldg(reinterpret_cast<const uint2*>(L.wvals) + d.x + ptid);
     }
   }
 #pragma unroll
   for (int j = 0; j < kMaxNg; ++j) {
     if (j < g.ng) {
-#pragma unroll
-      for (int u = 0; u < kPer; ++u) {
-        const uint32_t i = (uint32_t)ptid + u * kProducerThreads;
-        if (i >= (uint32_t)kMaxBlockKernels) continue;
-        const __half2 lo = *reinterpret_cast<const __half2*>(&raw[j][u].x);
-        const __half2 hi = *reinterpret_cast<const __half2*>(&raw[j][u].y);
-        sts128f(wbase + j * kWSlot + i * 16, __low2float(lo), __high2float(lo), __low2float(hi),
-                __high2float(hi));
-      }
+      const __half2 lo = *reinterpret_cast<const __half2*>(&raw[j].x);
+      const __half2 hi = *reinterpret_cast<const __half2*>(&raw[j].y);
+      sts128f(wbase + j * kWSlot + ptid * 16, __low2float(lo), __high2float(lo), __low2float(hi),
+              __high2float(hi));
     }
   }
   asm volatile("cp.async.wait_all;" ::: "memory");
@@ -547,9 +531,9 @@ __device__ __forceinline__ void issue_raw(const DeviceLayer& L, const Geo& g, co
   const uint32_t cbase = wbase + g.ng * kWRawSlot;
   for (int j = 0; j < g.ng; ++j) {
     const uint4 d = desc[2 * (j * g.cps + kk)];
-    for (uint32_t i = (uint32_t)ptid; i < d.y; i += kProducerThreads)
-      asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(wbase + j * kWRawSlot + i * 8),
-                   "l"(reinterpret_cast<const uint2*>(L.wvals) + d.x + i)
+    if ((uint32_t)ptid < d.y)
+      asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(wbase + j * kWRawSlot + ptid * 8),
+                   "l"(reinterpret_cast<const uint2*>(L.wvals) + d.x + ptid)
                    : "memory");
     if ((uint32_t)ptid * 16 < d.w) cp_async16(cbase + j * kCodeSlot + ptid * 16, codes + d.z + ptid * 16);
   }
@@ -584,12 +568,12 @@ __device__ __forceinline__ void widen_raw(const Geo& g, const StagedElem (&pre)[
   const uint32_t wbase = stage_base + g.x_stage_bytes, cbase = wbase + g.ng * kWSlot;
   for (int j = 0; j < g.ng; ++j) {
     const uint4 d = desc[2 * (j * g.cps + kk)];
-    for (uint32_t i = (uint32_t)ptid; i < d.y; i += kProducerThreads) {
-      const u64 raw = lds64(rw + j * kWRawSlot + i * 8);
+    if ((uint32_t)ptid < d.y) {
+      const u64 raw = lds64(rw + j * kWRawSlot + ptid * 8);
       const uint32_t lo32 = (uint32_t)raw, hi32 = (uint32_t)(raw >> 32);
       const __half2 lo = *reinterpret_cast<const __half2*>(&lo32);
       const __half2 hi = *reinterpret_cast<const __half2*>(&hi32);
-      sts128f(wbase + j * kWSlot + i * 16, __low2float(lo), __high2float(lo), __low2float(hi),
+      sts128f(wbase + j * kWSlot + ptid * 16, __low2float(lo), __high2float(lo), __low2float(hi),
               __high2float(hi));
     }
     if ((uint32_t)ptid * 16 < d.w) {
@@ -961,7 +945,7 @@ __device__ __forceinline__ void finalize_outputs(const Geo& g, const LaneOut& lo
 }
 
 template <int S, bool GENERIC, bool WIDE>
-__global__ void __launch_bounds__(cta_threads(GENERIC), GENERIC ? 1 : kCtasPerSm)
+__global__ void __launch_bounds__(cta_threads(GENERIC), 1)
 tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
              const float* __restrict__ bias, void* __restrict__ y, float* __restrict__ ws,
              int* __restrict__ counters) {
@@ -1431,7 +1415,7 @@ double geo_cost(const DeviceLayer& L, const Geo& g) {
   const double loop = turns * chunk;
   const double fixed = 28.0 + 17.0 / g.zs;
   const long long ctas = geo_tiles(L, g) * g.ks;
-  const int sms = device_sm_count() * kCtasPerSm;   // CTA slots of the device
+  const int sms = device_sm_count();
   const double waves = (double)((ctas + sms - 1) / sms);
   return waves * (fixed + loop) + (g.ks > 1 ? 100.0 / g.zs : 0.0);
 }
@@ -1448,7 +1432,7 @@ bool make_geo(const DeviceLayer& L, int n, int h, int w, bool allow_split, Geo* 
   const char* force_zs = getenv("PCONV_FORCE_ZS");
   const char* force_ks = getenv("PCONV_FORCE_KS");
 #endif
-  for (int zs = 1; zs <= consumer_warps(false) / 4; zs *= 2) {
+  for (int zs = 1; zs <= 4; zs *= 2) {
     Geo g;
 #ifdef PCONV_DEV
     if (force_zs && atoi(force_zs) != zs) continue;
@@ -1467,7 +1451,7 @@ bool make_geo(const DeviceLayer& L, int n, int h, int w, bool allow_split, Geo* 
       if (pass == 1) {
         if (!allow_split) break;
         const long long tiles = geo_tiles(L, g);
-        const long long ks = device_sm_count() * kCtasPerSm / tiles;   // fill one wave
+        const long long ks = device_sm_count() / tiles;   // fill one wave
         if (ks < 2) break;
         set_split(L, &c, (int)ks);
         if (c.ks < 2 || c.stages < 1) break;
@@ -1489,8 +1473,7 @@ cudaError_t launch_one(const DeviceLayer& L, Geo g, const void* x, const float* 
   int smem = g.stage_off + g.stages * g.stage_bytes;
   // the TMEM variant must be alone on its SM (it takes all 512 columns): make sure two CTAs can
   // never be co-resident by asking for more than half of the shared memory
-  constexpr int kMinSmem = (kCtasPerSm == 1) ? 120 * 1024 : 76 * 1024;   // no more CTAs per SM than planned
-  if (!GENERIC && smem < kMinSmem) smem = kMinSmem;
+  if (!GENERIC && smem < 120 * 1024) smem = 120 * 1024;
   cudaError_t e = cudaFuncSetAttribute(tiled_kernel<S, GENERIC, WIDE>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
   if (e != cudaSuccess) return e;
