@@ -30,8 +30,9 @@
 //    threads then copy it out in 16-byte pieces, a filter's 8 consecutive pixels each -- the
 //    first version stored 2 bytes per lane and column straight from the registers and spent more
 //    time in its epilogue than in its MMAs), warp 4 issues the MMAs (one thread) and owns the TMEM allocation,
-//    warps 5-12 are the A producers, in two groups that take alternate stages so that one group's
-//    global loads are in flight while the other converts and stores.  Two accumulator buffers
+//    warps 5-12 are the A producers (each thread keeps the loads of the next two stages in
+//    flight in two register sets while it shifts and stores the current one), warp 13 streams
+//    the weights through a ring of their own (three taps per bulk copy).  Two accumulator buffers
 //    (2 x n_t columns) let the epilogue of a tile overlap the next tile's MMAs.  CTAs are
 //    persistent: item t of a CTA is blockIdx.x + t * gridDim.x.
 //  * Weight reuse.  The nine taps make the weight operand of a step (9 x n_t x 16 values) six
@@ -60,12 +61,14 @@ typedef unsigned long long u64;
 constexpr int kEpiWarps = 4;
 constexpr int kMmaWarp = 4;
 constexpr int kProdWarp0 = 5;
-constexpr int kProdGroups = 2;
-constexpr int kProdWarpsPerGroup = 4;
-constexpr int kProdThreadsPerGroup = 32 * kProdWarpsPerGroup;
-constexpr int kTensorThreads = 32 * (kProdWarp0 + kProdGroups * kProdWarpsPerGroup);
-constexpr int kMaxTStages = 6;
-constexpr int kMaxTasks = 9;              // A tasks of one producer thread per stage (18 rows x 64 / 128)
+constexpr int kProdWarps = 8;
+constexpr int kProdThreads = 32 * kProdWarps;
+constexpr int kBWarp = kProdWarp0 + kProdWarps;   // warp 13: streams the weights
+constexpr int kTensorThreads = 32 * (kBWarp + 1);
+constexpr int kMaxAStages = 6;            // ring of activation stages (one 16-channel step each)
+constexpr int kMaxBStages = 16;           // ring of weight sub-stages (three taps of a step each)
+constexpr int kTHeaderBytes = 512;        // barriers and the TMEM base word
+constexpr int kMaxTasks = 5;              // A tasks of one producer thread per stage (18 rows x 64 / 256)
 constexpr uint32_t kTSpinLimit = 1u << 20;
 constexpr uint32_t kTWaitHintNs = 200;
 constexpr int kTSmemLimit = 227 * 1024;
@@ -81,8 +84,11 @@ struct TGeo {
   int tiles_x;       // column tiles of the virtual width cpr * wc
   int strip_rows, tiles_y;   // strip rows of the batch; items along the strip
   int n_t, n_tiles_n, k_steps;
-  int stages, a_copy_bytes, a_lbo, row_bytes, b_bytes, stage_bytes, stage_off;
-  int out_off, bias_off;   // the epilogue's staging tile [n_t][128] fp16 and the tile's bias [n_t] fp32
+  int a_stages, b_stages;  // ring depths
+  int b_resident;          // 1: the layer's whole weight operand fits the ring and is loaded once per CTA
+  int a_copy_bytes, a_lbo, row_bytes, a_stage_bytes, a_off;
+  int b_bytes, b_sub_bytes, b_off;   // weights of a step (nine taps) / of a sub-stage (three taps)
+  int out_off, bias_off;   // the epilogue's staging tile [n_t / 2][128][2] fp16 and the tile's bias [n_t] fp32
   int relu;
   long long total_items;   // tiles_y * tiles_x * n_tiles_n
 };
@@ -143,20 +149,40 @@ __device__ __forceinline__ void umma_f16(uint32_t d_tmem, u64 a_desc, u64 b_desc
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// True in exactly one lane of the (converged) warp.  The MMA and weight-stream warps run their
+// loops with all 32 lanes, so that addresses and descriptors stay warp-uniform (the tensor-core
+// instructions take them from uniform registers), and only the issuing instruction is elected.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t p;
+  asm volatile(
+      "{\n\t.reg .pred P;\n\t"
+      "elect.sync _|P, 0xFFFFFFFF;\n\t"
+      "selp.u32 %0, 1, 0, P;\n\t}"
+      : "=r"(p));
+  return p != 0;
+}
 // The mbarrier receives one arrival when all MMAs issued so far by this thread have completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
                : "memory");
 }
-__device__ __forceinline__ void tmem_ld16(uint32_t (&v)[16], uint32_t taddr) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-      : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
+
+// Development build: CTA 0 leaves, in the layer's trace words, the cycles its roles spent waiting
+// and working (0 whole kernel; MMA warp: 1 waiting for free accumulators, 2 for activations, 3 for
+// weights, 4 issuing; producers' thread 0: 5 waiting for a free stage, 6 issuing loads, 7 shifting
+// and storing; weight stream: 8 waiting for a free sub-stage; epilogue thread 0: 9 waiting for
+// accumulators, 10 working).
+#ifdef PCONV_DEV
+#define T_NOW() clock64()
+#define T_ADD(i, t0) do { if (blockIdx.x == 0) tw_[i] += clock64() - (t0); } while (0)
+#define T_DECL long long tw_[14] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}
+#define T_FLUSH(lo, hi) do { if (blockIdx.x == 0) for (int i_ = (lo); i_ <= (hi); ++i_) trace_words(L)[i_] = (unsigned long long)tw_[i_]; } while (0)
+#else
+#define T_NOW() 0ll
+#define T_ADD(i, t0) do { (void)(t0); } while (0)
+#define T_DECL
+#define T_FLUSH(lo, hi)
+#endif
 
 // Input layouts the kernel is compiled for.
 enum { kModeW8 = 0,   // w a multiple of 8: a task is one aligned 16-byte load (+ two neighbours)
@@ -196,20 +222,14 @@ __device__ __forceinline__ bool epi_all(bool v) {
       : "memory");
   return r != 0;
 }
-__device__ __forceinline__ uint32_t lds_b32(uint32_t a) {
-  uint32_t v;
-  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(a));
-  return v;
-}
 __device__ __forceinline__ uint4 lds_v4(uint32_t a) {
   uint4 v;
   asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
   return v;
 }
-__device__ __forceinline__ void sts_u16(uint32_t a, unsigned short v) {
-  asm volatile("st.shared.u16 [%0], %1;" ::"r"(a), "h"(v) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t (&v)[32], uint32_t taddr) {
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// 32 accumulator columns of this warp's 32 lanes; the registers are valid after tmem_ld_wait().
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t (&v)[32], uint32_t taddr) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
@@ -219,7 +239,6 @@ __device__ __forceinline__ void tmem_ld32(uint32_t (&v)[32], uint32_t taddr) {
         "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
         "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
       : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
 // The 8 pixels of one task (one channel, one staged row, one column group) as four packed fp16
@@ -274,18 +293,24 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
   const uint32_t sbase = smem_u32(smem);
   const int tid = threadIdx.x, lane = tid & 31;
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
-  // barriers: full[s], empty[s] (s < stages), acc_full[2], acc_empty[2]; then the TMEM base word
-  const uint32_t bar_full = sbase, bar_empty = sbase + 8 * kMaxTStages;
-  const uint32_t bar_accf = sbase + 16 * kMaxTStages, bar_acce = bar_accf + 16;
-  volatile uint32_t* tmem_base_s = reinterpret_cast<volatile uint32_t*>(smem + 16 * kMaxTStages + 32);
+  // barriers: a_full / a_empty per activation stage, b_full / b_empty per weight sub-stage,
+  // acc_full[2], acc_empty[2]; then the TMEM base word
+  const uint32_t bar_afull = sbase, bar_aempty = sbase + 8 * kMaxAStages;
+  const uint32_t bar_bfull = sbase + 16 * kMaxAStages, bar_bempty = bar_bfull + 8 * kMaxBStages;
+  const uint32_t bar_accf = bar_bempty + 8 * kMaxBStages, bar_acce = bar_accf + 16;
+  volatile uint32_t* tmem_base_s = reinterpret_cast<volatile uint32_t*>(smem + 16 * (kMaxAStages + kMaxBStages) + 32);
   const int acc_cols = g.mt * g.n_t;                          // columns of one accumulator set
   const uint32_t tmem_cols = (uint32_t)(g.n_buf * acc_cols);  // 64 .. 512, a power of two
 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (tid == 0) {
-    for (int s = 0; s < g.stages; ++s) {
-      mbar_init(bar_full + 8 * s, kProdThreadsPerGroup + 1);   // a group's threads + the bulk copy's issuer
-      mbar_init(bar_empty + 8 * s, 1);                         // one tcgen05.commit
+    for (int s = 0; s < g.a_stages; ++s) {
+      mbar_init(bar_afull + 8 * s, kProdThreads);              // every producer thread
+      mbar_init(bar_aempty + 8 * s, 1);                        // one tcgen05.commit
+    }
+    for (int s = 0; s < g.b_stages; ++s) {
+      mbar_init(bar_bfull + 8 * s, 1);                         // the bulk copy's issuer (+ its bytes)
+      mbar_init(bar_bempty + 8 * s, 1);                        // one tcgen05.commit
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(bar_accf + 8 * b, 1);
@@ -313,7 +338,7 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
 
   if (warp == kMmaWarp) {
     // ======================================= MMA issuer =======================================
-    if (lane == 0) {
+    {
       // instruction descriptor: D fp32, A and B fp16, A pixel-major (MN-major), B K-major, N, M = 128
       const uint32_t idesc = (1u << 4) | (1u << 15) | ((uint32_t)(g.n_t >> 3) << 17) | ((128u >> 4) << 24);
       // descriptors of a stage differ in the start address only: bits 0-13 of the low word, in
@@ -321,52 +346,69 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
       const u64 a_desc0 = smem_desc(0u, (uint32_t)g.a_lbo, 128u);
       const u64 b_desc0 = smem_desc(0u, (uint32_t)(g.n_t / 8) * 128u, 128u);
       const uint32_t copy16 = (uint32_t)g.a_copy_bytes >> 4, row16 = row_b >> 4;
-      const uint32_t tap16 = (uint32_t)(g.n_t * 32) >> 4, tile16 = (uint32_t)g.r * row16;
-      long long it = 0;
+      const uint32_t tap16 = (uint32_t)(g.n_t * 32) >> 4;
+      long long ita = 0, itb = 0;    // activation stages and weight sub-stages consumed so far
       bool ok = true;
+      T_DECL;
+      const long long t_start = T_NOW();
       for (int ti = 0; ti < my_items && ok; ++ti) {
         const int buf = ti % g.n_buf;
         const uint32_t use = (uint32_t)(ti / g.n_buf);
+        long long t0 = T_NOW();
         ok = mbar_wait(bar_acce + 8 * buf, (use & 1u) ^ 1u, L.err, 20);
+        T_ADD(1, t0);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * acc_cols);
-        for (int ks = 0; ks < g.k_steps; ++ks, ++it) {
-          const int s = (int)(it % g.stages);
-          ok = mbar_wait(bar_full + 8 * s, (uint32_t)((it / g.stages) & 1), L.err, 21);
+        for (int ks = 0; ks < g.k_steps && ok; ++ks, ++ita) {
+          const int sa = (int)(ita % g.a_stages);
+          t0 = T_NOW();
+          ok = mbar_wait(bar_afull + 8 * sa, (uint32_t)((ita / g.a_stages) & 1), L.err, 21);
+          T_ADD(2, t0);
           if (!ok) break;
-          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t a0 = sbase + g.stage_off + s * g.stage_bytes;
-          const u64 a_st = a_desc0 + (a0 >> 4), b_st = b_desc0 + ((a0 + 3 * g.a_copy_bytes) >> 4);
-          for (int j = 0; j < g.mt; ++j) {       // the item's pixel tiles share the stage's weights
-            const u64 a_tile = a_st + j * tile16;
+          const u64 a_st = a_desc0 + ((sbase + g.a_off + sa * g.a_stage_bytes) >> 4);
+          for (int u = 0; u < 3; ++u, ++itb) {    // the three taps of kernel row u
+            const int sb = g.b_resident ? ks * 3 + u : (int)(itb % g.b_stages);
+            t0 = T_NOW();
+            ok = mbar_wait(bar_bfull + 8 * sb, g.b_resident ? 0u : (uint32_t)((itb / g.b_stages) & 1), L.err, 24);
+            T_ADD(3, t0);
+            if (!ok) break;
+            t0 = T_NOW();
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const u64 b_st = b_desc0 + ((sbase + g.b_off + sb * g.b_sub_bytes) >> 4);
+            for (int j = 0; j < g.mt; ++j) {      // the item's pixel tiles share the weights
+              const u64 a_tile = a_st + (uint32_t)(j * g.r + u) * row16;
 #pragma unroll
-            for (int t = 0; t < 9; ++t) {
-              const int u = t / 3, v = t - 3 * u;
-              umma_f16(d_tmem + (uint32_t)(j * g.n_t), a_tile + v * copy16 + u * row16, b_st + t * tap16,
-                       idesc, (ks > 0 || t > 0) ? 1u : 0u);
+              for (int v = 0; v < 3; ++v)
+                if (elect_one())
+                  umma_f16(d_tmem + (uint32_t)(j * g.n_t), a_tile + v * copy16, b_st + v * tap16, idesc,
+                           (ks > 0 || u > 0 || v > 0) ? 1u : 0u);
             }
+            // the sub-stage may be refilled once these MMAs are done
+            if (!g.b_resident && elect_one()) umma_commit(bar_bempty + 8 * sb);
+            T_ADD(4, t0);
           }
-          umma_commit(bar_empty + 8 * s);          // the stage may be refilled once these MMAs are done
+          if (ok && elect_one()) umma_commit(bar_aempty + 8 * sa);
         }
-        if (ok) umma_commit(bar_accf + 8 * buf);   // the item's accumulators are complete
+        if (ok && elect_one()) umma_commit(bar_accf + 8 * buf);   // the item's accumulators are complete
       }
+      T_ADD(0, t_start);
+      if (lane == 0) T_FLUSH(0, 4);
     }
     __syncwarp();
-  } else if (warp >= kProdWarp0) {
+  } else if (warp >= kProdWarp0 && warp < kBWarp) {
     // ======================================= A producers ======================================
-    const int group = (warp - kProdWarp0) / kProdWarpsPerGroup;
-    const int gt = (warp - kProdWarp0 - group * kProdWarpsPerGroup) * 32 + lane;
+    const int gt = (warp - kProdWarp0) * 32 + lane;                  // 0..255
     const int cg_shift = g.tw == 32 ? 2 : (g.tw == 16 ? 1 : 0);      // log2(column groups of a row)
     const int n_tasks = g.rows_a << (4 + cg_shift);                 // rows x 2 blocks x groups x 8 channels
     const unsigned short* xs = reinterpret_cast<const unsigned short*>(x);
     const size_t img = (size_t)g.c_in * hw;    // elements of one image
     const size_t step = 16 * hw;               // elements between channel steps
-    // what depends on the task only: its place in a copy and its channel inside a step
+    // what depends on the task only: its place in a copy
     uint32_t dst[kMaxTasks];
 #pragma unroll
     for (int q = 0; q < kMaxTasks; ++q) {
-      const int t = gt + q * kProdThreadsPerGroup;
+      const int t = gt + q * kProdThreads;
       const int c8 = t & 7, cg = (t >> 3) & ((1 << cg_shift) - 1);
       const int kb = (t >> (3 + cg_shift)) & 1, hr = t >> (4 + cg_shift);
       dst[q] = (uint32_t)(kb * g.a_lbo) + (uint32_t)hr * row_b + (uint32_t)(cg * 128 + c8 * 16);
@@ -384,26 +426,23 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
     } else if (MODE == kModeNX) {                              // w = 1: no neighbours at all
       zm_even = zm_odd = zp_even = zp_odd = 0u;
     }
-    bool ok = true;
-    long long it = 0;                          // stage counter over all items of this CTA
-    for (int ti = 0; ti < my_items && ok; ++ti) {
-      // the stages of this item that fall to this group: none if the item has one step and it is
-      // the other group's turn
-      if (g.k_steps == 1 && (int)(it & 1) != group) {
-        ++it;
-        continue;
-      }
+    // A thread's loads run two stages ahead of its stores, in two register sets: global-memory
+    // latency is then covered by two stage periods, whatever the ring still has free.
+    struct RegSet {
+      uint4 v[kMaxTasks];
+      uint32_t lft[kMaxTasks], rgt[kMaxTasks];
+    };
+    RegSet set0, set1;
+    const unsigned short* src[kMaxTasks];   // of the item being loaded: a task's 8 pixels at step 0 (null = padding)
+    uint32_t aux[kMaxTasks];
+    auto setup_item = [&](int ti) {
       const long long item = blockIdx.x + (long long)ti * gridDim.x;
       const int mti = (int)(item / g.n_tiles_n);
-      const int nt = (int)(item - (long long)mti * g.n_tiles_n);
       const int ty = mti / g.tiles_x;
       const int tx = mti - ty * g.tiles_x;
-      // per task: where its 8 pixels are for the channels of step 0 (null = padding) and `aux`
-      const unsigned short* src[kMaxTasks];
-      uint32_t aux[kMaxTasks];
 #pragma unroll
       for (int q = 0; q < kMaxTasks; ++q) {
-        const int t = gt + q * kProdThreadsPerGroup;
+        const int t = gt + q * kProdThreads;
         src[q] = nullptr;
         aux[q] = 0u;
         if (t < n_tasks) {
@@ -425,64 +464,119 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
           }
         }
       }
-      for (int ks = 0; ks < g.k_steps && ok; ++ks, ++it) {
-        if ((int)(it & 1) != group) continue;       // the other group's stage
-        const int s = (int)(it % g.stages);
-        ok = mbar_wait(bar_empty + 8 * s, (uint32_t)(((it / g.stages) & 1) ^ 1), L.err, 22);
-        if (!ok) break;
-        const uint32_t a0 = sbase + g.stage_off + s * g.stage_bytes;
-        if (gt == 0) {   // the stage's weights: one bulk copy, counted on the same barrier
-          mbar_arrive_expect_tx(bar_full + 8 * s, (uint32_t)g.b_bytes);
-          bulk_copy_g2s(a0 + 3 * g.a_copy_bytes,
-                        reinterpret_cast<const char*>(L.wdense) + ((size_t)nt * g.k_steps + ks) * g.b_bytes,
-                        (uint32_t)g.b_bytes, bar_full + 8 * s);
-        }
-        // channels beyond c_in (last step of a layer whose depth is no multiple of 16) are zeros
-        const int ch_limit = g.c_in - ks * 16;
-        const size_t chan_off = (size_t)ks * step;
-        // every load of the stage first (they are independent), then shifts and stores
-        uint4 v[kMaxTasks];
-        uint32_t lft[kMaxTasks], rgt[kMaxTasks];
+    };
+    // (l_ti, l_ks): the next stage to load; loading past the last stage does nothing
+    int l_ti = 0, l_ks = 0;
+    if (my_items > 0) setup_item(0);
+    auto load_next = [&](RegSet& rs) {
 #pragma unroll
-        for (int q = 0; q < kMaxTasks; ++q) {
-          v[q] = make_uint4(0u, 0u, 0u, 0u);
-          lft[q] = rgt[q] = 0u;
-          if (src[q] == nullptr) continue;
-          if (ch_limit < 16) {
-            const int t = gt + q * kProdThreadsPerGroup;
-            if (((((t >> (3 + cg_shift)) & 1) << 3) | (t & 7)) >= ch_limit) continue;
-          }
-          load_task<MODE>(g, src[q] + chan_off, aux[q], img, &v[q], &lft[q], &rgt[q]);
-        }
-        const uint32_t copy_b = (uint32_t)g.a_copy_bytes;
-#pragma unroll
-        for (int q = 0; q < kMaxTasks; ++q) {
-          if (gt + q * kProdThreadsPerGroup >= n_tasks) continue;
-          const uint4 c = v[q];
-          // copy 0: pixel p holds input column p - 1;  copy 2: column p + 1
-          uint4 m1, p1;
-          m1.x = __funnelshift_l(lft[q] << 16, c.x, 16);
-          m1.y = __funnelshift_l(c.x, c.y, 16);
-          m1.z = __funnelshift_l(c.y, c.z, 16);
-          m1.w = __funnelshift_l(c.z, c.w, 16);
-          p1.x = __funnelshift_r(c.x, c.y, 16);
-          p1.y = __funnelshift_r(c.y, c.z, 16);
-          p1.z = __funnelshift_r(c.z, c.w, 16);
-          p1.w = __funnelshift_r(c.w, rgt[q], 16);
-          if (MODE >= kModeN4) {
-            m1.x &= zm_even; m1.y &= zm_odd; m1.z &= zm_even; m1.w &= zm_odd;
-            p1.x &= zp_even; p1.y &= zp_odd; p1.z &= zp_even; p1.w &= zp_odd;
-          }
-          const uint32_t d = a0 + dst[q];
-          sts128(d, m1.x, m1.y, m1.z, m1.w);
-          sts128(d + copy_b, c.x, c.y, c.z, c.w);
-          sts128(d + 2 * copy_b, p1.x, p1.y, p1.z, p1.w);
-        }
-        // generic-proxy stores must be visible to the tensor core's (async proxy) reads
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        mbar_arrive(bar_full + 8 * s);
+      for (int q = 0; q < kMaxTasks; ++q) {
+        rs.v[q] = make_uint4(0u, 0u, 0u, 0u);
+        rs.lft[q] = rs.rgt[q] = 0u;
       }
+      if (l_ti >= my_items) return;
+      // channels beyond c_in (last step of a layer whose depth is no multiple of 16) are zeros
+      const int ch_limit = g.c_in - l_ks * 16;
+      const size_t chan_off = (size_t)l_ks * step;
+#pragma unroll
+      for (int q = 0; q < kMaxTasks; ++q) {
+        if (src[q] == nullptr) continue;
+        if (ch_limit < 16) {
+          const int t = gt + q * kProdThreads;
+          if (((((t >> (3 + cg_shift)) & 1) << 3) | (t & 7)) >= ch_limit) continue;
+        }
+        load_task<MODE>(g, src[q] + chan_off, aux[q], img, &rs.v[q], &rs.lft[q], &rs.rgt[q]);
+      }
+      if (++l_ks == g.k_steps) {
+        l_ks = 0;
+        if (++l_ti < my_items) setup_item(l_ti);
+      }
+    };
+    const uint32_t copy_b = (uint32_t)g.a_copy_bytes;
+    const long long n_stages = (long long)my_items * g.k_steps;
+    T_DECL;
+    auto store_stage = [&](const RegSet& rs, long long it) -> bool {
+      const int s = (int)(it % g.a_stages);
+      long long t0 = T_NOW();
+      const bool got = mbar_wait(bar_aempty + 8 * s, (uint32_t)(((it / g.a_stages) & 1) ^ 1), L.err, 22);
+      T_ADD(5, t0);
+      if (!got) return false;
+      t0 = T_NOW();
+      const uint32_t a0 = sbase + g.a_off + s * g.a_stage_bytes;
+#pragma unroll
+      for (int q = 0; q < kMaxTasks; ++q) {
+        if (gt + q * kProdThreads >= n_tasks) continue;
+        const uint4 c = rs.v[q];
+        // copy 0: pixel p holds input column p - 1;  copy 2: column p + 1
+        uint4 m1, p1;
+        m1.x = __funnelshift_l(rs.lft[q] << 16, c.x, 16);
+        m1.y = __funnelshift_l(c.x, c.y, 16);
+        m1.z = __funnelshift_l(c.y, c.z, 16);
+        m1.w = __funnelshift_l(c.z, c.w, 16);
+        p1.x = __funnelshift_r(c.x, c.y, 16);
+        p1.y = __funnelshift_r(c.y, c.z, 16);
+        p1.z = __funnelshift_r(c.z, c.w, 16);
+        p1.w = __funnelshift_r(c.w, rs.rgt[q], 16);
+        if (MODE >= kModeN4) {
+          m1.x &= zm_even; m1.y &= zm_odd; m1.z &= zm_even; m1.w &= zm_odd;
+          p1.x &= zp_even; p1.y &= zp_odd; p1.z &= zp_even; p1.w &= zp_odd;
+        }
+        const uint32_t d = a0 + dst[q];
+        sts128(d, m1.x, m1.y, m1.z, m1.w);
+        sts128(d + copy_b, c.x, c.y, c.z, c.w);
+        sts128(d + 2 * copy_b, p1.x, p1.y, p1.z, p1.w);
+      }
+      // generic-proxy stores must be visible to the tensor core's (async proxy) reads
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      mbar_arrive(bar_afull + 8 * s);
+      T_ADD(7, t0);
+      return true;
+    };
+    load_next(set0);
+    load_next(set1);
+    for (long long it = 0; it < n_stages; it += 2) {
+      if (!store_stage(set0, it)) break;
+      long long t0 = T_NOW();
+      load_next(set0);
+      T_ADD(6, t0);
+      if (it + 1 >= n_stages) break;
+      if (!store_stage(set1, it + 1)) break;
+      t0 = T_NOW();
+      load_next(set1);
+      T_ADD(6, t0);
     }
+    if (gt == 0) T_FLUSH(5, 7);
+  } else if (warp == kBWarp) {
+    // ======================================= weight stream ====================================
+    // One thread: per (item, step, kernel row) one bulk copy of three taps' [n_t x 16] matrices
+    // into the next free sub-stage, as far ahead of the MMAs as the ring allows.
+    {
+      bool ok = true;
+      long long itb = 0;
+      T_DECL;
+      for (int ti = 0; ti < (g.b_resident ? min(my_items, 1) : my_items) && ok; ++ti) {
+        const long long item = blockIdx.x + (long long)ti * gridDim.x;
+        const int nt = (int)(item % g.n_tiles_n);
+        const char* wsrc = reinterpret_cast<const char*>(L.wdense) + (size_t)nt * g.k_steps * g.b_bytes;
+        for (int ks = 0; ks < g.k_steps && ok; ++ks) {
+          for (int u = 0; u < 3; ++u, ++itb) {
+            const int sb = (int)(itb % g.b_stages);
+            const long long t0 = T_NOW();
+            ok = mbar_wait(bar_bempty + 8 * sb, (uint32_t)(((itb / g.b_stages) & 1) ^ 1), L.err, 25);
+            T_ADD(8, t0);
+            if (!ok) break;
+            if (elect_one()) {
+              mbar_arrive_expect_tx(bar_bfull + 8 * sb, (uint32_t)g.b_sub_bytes);
+              bulk_copy_g2s(sbase + g.b_off + sb * g.b_sub_bytes,
+                            wsrc + (size_t)ks * g.b_bytes + (size_t)u * g.b_sub_bytes,
+                            (uint32_t)g.b_sub_bytes, bar_bfull + 8 * sb);
+            }
+          }
+        }
+      }
+      if (lane == 0) T_FLUSH(8, 8);
+    }
+    __syncwarp();
   } else {
     // ======================================= epilogue =========================================
     // Accumulators (lane = pixel, column = filter) -> bias, ReLU, fp16 -> shared memory as
@@ -490,12 +584,12 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
     const int q = warp;                       // TMEM lane quadrant
     const int m = 32 * q + lane;              // this lane's pixel of a tile
     const int et = tid;                       // 0..127
-    const uint32_t out_s = sbase + (uint32_t)g.out_off;       // [n_t][128] fp16
-    const uint32_t bias_s = sbase + (uint32_t)g.bias_off;     // [n_t] fp32
-    // copy-out: this thread always handles pixel group pg (8 pixels) of filters f0, f0 + 8, ...
+    const uint32_t out_s = sbase + (uint32_t)g.out_off;       // [n_t / 2][128] pairs of fp16
+    // copy-out: this thread always handles pixel group pg (8 pixels) of filter pairs f0, f0 + 8, ...
     const int pg = et & 15, f0 = et >> 4;
     const int ctr = (pg * 8) / g.tw, ctc = (pg * 8) - ctr * g.tw;   // the group's tile row / first column
     bool ok = true;
+    T_DECL;
     for (int ti = 0; ti < my_items && ok; ++ti) {
       const long long item = blockIdx.x + (long long)ti * gridDim.x;
       const int mti = (int)(item / g.n_tiles_n);
@@ -505,75 +599,118 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
       const int buf = ti % g.n_buf;
       const uint32_t use = (uint32_t)(ti / g.n_buf);
       const int o_base = nt * g.n_t;
+      long long t0 = T_NOW();
       const int n_f = min(g.n_t, g.c_out - o_base);            // real filters of this tile
       epi_sync();                                              // the previous item's bias is no longer read
-      if (et < g.n_t) {
-        const float bv = (bias && et < n_f) ? __ldg(bias + o_base + et) : 0.f;
-        asm volatile("st.shared.f32 [%0], %1;" ::"r"(bias_s + 4 * et), "f"(bv) : "memory");
-      }
+      if (et < g.n_t)
+        reinterpret_cast<float*>(smem + g.bias_off)[et] = (bias && et < n_f) ? __ldg(bias + o_base + et) : 0.f;
       ok = mbar_wait(bar_accf + 8 * buf, use & 1u, L.err, 23);
       ok = epi_all(ok);                                        // bias staged; all leave together if a wait ran out
+      T_ADD(9, t0);
       if (!ok) break;
+      t0 = T_NOW();
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       for (int j = 0; j < g.mt; ++j) {
+        long long t1 = T_NOW();
         const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * acc_cols + j * g.n_t);
-        for (int j0 = 0; j0 < n_f; j0 += 32) {
-          uint32_t acc[32];
-          tmem_ld32(acc, taddr + (uint32_t)j0);
+        // Two adjacent filters of a pixel are converted together (the packed fp16 conversion runs
+        // at full rate, the scalar one at a quarter of it: it alone took longer than the MMAs of
+        // a tile) and staged as one 32-bit word: [filter pair][pixel].  Plain shared-memory
+        // accesses, not asm: the compiler may overlap the columns.  The TMEM load of the next 32
+        // columns is in flight while the current ones are converted.
+        auto stage_block = [&](const uint32_t (&acc)[32], int j0) {
+          // (the 32 bias values first: a load after a store to shared memory could not be moved up)
+          const float4* bias_p = reinterpret_cast<const float4*>(smem + g.bias_off + 4 * j0);
+          float bv[32];
 #pragma unroll
-          for (int jj = 0; jj < 32; ++jj) {
-            float val = __uint_as_float(acc[jj]) + __uint_as_float(lds_b32(bias_s + 4 * (j0 + jj)));
-            if (g.relu) val = fmaxf(val, 0.f);
-            sts_u16(out_s + (uint32_t)((j0 + jj) * 256 + m * 2), __half_as_ushort(__float2half_rn(val)));
+          for (int i = 0; i < 8; ++i) {
+            const float4 b4 = bias_p[i];
+            bv[4 * i] = b4.x;
+            bv[4 * i + 1] = b4.y;
+            bv[4 * i + 2] = b4.z;
+            bv[4 * i + 3] = b4.w;
+          }
+          __half2* out_p = reinterpret_cast<__half2*>(smem + g.out_off) + (size_t)(j0 >> 1) * 128 + m;
+#pragma unroll
+          for (int jj = 0; jj < 32; jj += 2) {
+            float v0 = __uint_as_float(acc[jj]) + bv[jj];
+            float v1 = __uint_as_float(acc[jj + 1]) + bv[jj + 1];
+            if (g.relu) {
+              v0 = fmaxf(v0, 0.f);
+              v1 = fmaxf(v1, 0.f);
+            }
+            out_p[(jj >> 1) * 128] = __floats2half2_rn(v0, v1);
+          }
+        };
+        uint32_t acc0[32], acc1[32];
+        tmem_ld32_issue(acc0, taddr);
+        tmem_ld_wait();
+        for (int j0 = 0; j0 < n_f; j0 += 64) {
+          if (j0 + 32 < n_f) tmem_ld32_issue(acc1, taddr + (uint32_t)(j0 + 32));
+          stage_block(acc0, j0);
+          tmem_ld_wait();
+          if (j0 + 32 < n_f) {
+            if (j0 + 64 < n_f) tmem_ld32_issue(acc0, taddr + (uint32_t)(j0 + 64));
+            stage_block(acc1, j0 + 32);
+            tmem_ld_wait();
           }
         }
         if (j == g.mt - 1) {   // the accumulators have been read: the MMA warp may reuse them
           asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
           mbar_arrive(bar_acce + 8 * buf);
         }
+        T_ADD(11, t1);
+        t1 = T_NOW();
         epi_sync();                                            // the tile is staged
+        T_ADD(12, t1);
+        t1 = T_NOW();
         // where this thread's pixel group goes
         int gi = 0, lr = 0;
         const bool row_ok = strip_row(g, (ty * g.mt + j) * g.r + ctr, &gi, &lr);
         const int vx = tx * g.tw + ctc;
-        if (row_ok) {
-          if (MODE == kModeW8) {
-            if (vx < g.w) {
-              __half* dstp = y + (((size_t)gi * g.c_out + o_base) * g.h + lr) * (size_t)g.w + vx;
-              for (int f = f0; f < n_f; f += 8)
-                *reinterpret_cast<uint4*>(dstp + (size_t)f * hw) = lds_v4(out_s + (uint32_t)(f * 256 + pg * 16));
-            }
-          } else if (MODE == kModeWX) {
-            if (vx < g.w) {
-              __half* dstp = y + (((size_t)gi * g.c_out + o_base) * g.h + lr) * (size_t)g.w + vx;
-              const int npx = min(8, g.w - vx);
-              for (int f = f0; f < n_f; f += 8) {
-                const uint4 vv = lds_v4(out_s + (uint32_t)(f * 256 + pg * 16));
-                const uint32_t wds[4] = {vv.x, vv.y, vv.z, vv.w};
-                unsigned short* dp = reinterpret_cast<unsigned short*>(dstp + (size_t)f * hw);
+        bool grp_ok = row_ok;
+        __half* dstp = y;
+        int cells = 0;
+        if (MODE == kModeW8 || MODE == kModeWX) {
+          grp_ok = grp_ok && vx < g.w;
+          if (grp_ok) dstp = y + (((size_t)gi * g.c_out + o_base) * g.h + lr) * (size_t)g.w + vx;
+        } else if (grp_ok) {
+          // narrow maps: the group is 8 / wc images side by side, w pixels of each are real
+          cells = min(g.cpr, g.n - gi * g.cpr);
+          dstp = y + (((size_t)gi * g.cpr * g.c_out + o_base) * g.h + lr) * (size_t)g.w;
+        }
+        if (grp_ok) {
+          const int npx = min(8, g.w - vx);                    // kModeWX: real pixels of the group
+          const size_t oimg = (size_t)g.c_out * hw;
+          for (int fp = f0; 2 * fp < n_f; fp += 8) {
+            // 8 pixels x {filter 2 fp, filter 2 fp + 1} -> 8 pixels of each filter
+            const uint4 a = lds_v4(out_s + (uint32_t)(fp * 512 + pg * 32));
+            const uint4 b = lds_v4(out_s + (uint32_t)(fp * 512 + pg * 32 + 16));
+            uint4 vv[2];
+            vv[0] = make_uint4(__byte_perm(a.x, a.y, 0x5410), __byte_perm(a.z, a.w, 0x5410),
+                               __byte_perm(b.x, b.y, 0x5410), __byte_perm(b.z, b.w, 0x5410));
+            vv[1] = make_uint4(__byte_perm(a.x, a.y, 0x7632), __byte_perm(a.z, a.w, 0x7632),
+                               __byte_perm(b.x, b.y, 0x7632), __byte_perm(b.z, b.w, 0x7632));
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const int f = 2 * fp + e;
+              if (f >= n_f) break;
+              __half* dp = dstp + (size_t)f * hw;
+              const uint32_t wds[4] = {vv[e].x, vv[e].y, vv[e].z, vv[e].w};
+              if (MODE == kModeW8) {
+                *reinterpret_cast<uint4*>(dp) = vv[e];
+              } else if (MODE == kModeWX) {
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
-                  if (i < npx) dp[i] = (unsigned short)(wds[i >> 1] >> (16 * (i & 1)));
-              }
-            }
-          } else {
-            // narrow maps: the group is 8 / wc images side by side, w pixels of each are real
-            const int cells = min(g.cpr, g.n - gi * g.cpr);
-            __half* dstp = y + (((size_t)gi * g.cpr * g.c_out + o_base) * g.h + lr) * (size_t)g.w;
-            const size_t oimg = (size_t)g.c_out * hw;
-            for (int f = f0; f < n_f; f += 8) {
-              const uint4 vv = lds_v4(out_s + (uint32_t)(f * 256 + pg * 16));
-              __half* dp = dstp + (size_t)f * hw;
-              if (MODE == kModeN4) {
-                if (cells > 0) *reinterpret_cast<uint2*>(dp) = make_uint2(vv.x, vv.y);
-                if (cells > 1) *reinterpret_cast<uint2*>(dp + oimg) = make_uint2(vv.z, vv.w);
+                  if (i < npx) reinterpret_cast<unsigned short*>(dp)[i] = (unsigned short)(wds[i >> 1] >> (16 * (i & 1)));
+              } else if (MODE == kModeN4) {
+                if (cells > 0) *reinterpret_cast<uint2*>(dp) = make_uint2(wds[0], wds[1]);
+                if (cells > 1) *reinterpret_cast<uint2*>(dp + oimg) = make_uint2(wds[2], wds[3]);
               } else if (MODE == kModeN2) {
-                const uint32_t wds[4] = {vv.x, vv.y, vv.z, vv.w};
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
                   if (i < cells) *reinterpret_cast<uint32_t*>(dp + i * oimg) = wds[i];
               } else {
-                const uint32_t wds[4] = {vv.x, vv.y, vv.z, vv.w};
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                   const int cell = g.wc == 1 ? i : i >> 2;
@@ -586,9 +723,12 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
             }
           }
         }
+        T_ADD(13, t1);
         epi_sync();                                            // staging buffer free again
       }
+      T_ADD(10, t0);
     }
+    if (et == 0) T_FLUSH(9, 13);
   }
 
   // ---- common exit ----------------------------------------------------------------------------
@@ -639,32 +779,64 @@ bool tensor_geo_mt(const DeviceLayer& L, int n, int h, int w, int mt, TGeo* out)
   g.a_lbo = g.rows_a * g.row_bytes;
   g.a_copy_bytes = 2 * g.a_lbo;
   g.b_bytes = 9 * g.n_t * 32;
-  g.stage_bytes = 3 * g.a_copy_bytes + g.b_bytes;
-  g.stage_off = 256;
+  g.b_sub_bytes = 3 * g.n_t * 32;
+  g.a_stage_bytes = 3 * g.a_copy_bytes;
+  // Shared memory: barriers, activation ring, weight ring, the epilogue's staging tile and bias.
+  // The producers keep two stages of loads in registers, so three activation stages are enough;
+  // the weight ring takes what is left (what matters is how many steps of MMAs it covers: a
+  // sub-stage comes back only after its MMAs have completed and a copy from L2 has landed, about
+  // 2 us, while a step of one tile is 0.3 us of MMAs), and what the weight ring cannot use goes
+  // back to the activations.
   const int epi_bytes = g.n_t * 256 + g.n_t * 4;
-  g.stages = (kTSmemLimit - g.stage_off - epi_bytes) / g.stage_bytes;
-  if (g.stages > kMaxTStages) g.stages = kMaxTStages;
-  if (g.stages < 2) return false;
-  g.out_off = g.stage_off + g.stages * g.stage_bytes;
+  const int avail = kTSmemLimit - kTHeaderBytes - epi_bytes;
+  g.a_stages = (3 * g.a_stage_bytes + 6 * g.b_sub_bytes <= avail) ? 3 : 2;
+  g.b_stages = (avail - g.a_stages * g.a_stage_bytes) / g.b_sub_bytes;
+  if (g.b_stages > kMaxBStages) g.b_stages = kMaxBStages;
+  if (g.b_stages < 3) return false;
+  // a layer with one filter tile whose weights all fit keeps them: nothing is streamed again
+  g.b_resident = 0;
+  if (g.n_tiles_n == 1 && 3 * g.k_steps <= kMaxBStages &&
+      2 * g.a_stage_bytes + 3 * g.k_steps * g.b_sub_bytes <= avail) {
+    g.b_resident = 1;
+    g.b_stages = 3 * g.k_steps;
+    g.a_stages = 2;
+  }
+  while (g.a_stages < kMaxAStages &&
+         (g.a_stages + 1) * g.a_stage_bytes + g.b_stages * g.b_sub_bytes <= avail)
+    ++g.a_stages;
+  g.a_off = kTHeaderBytes;
+  g.b_off = g.a_off + g.a_stages * g.a_stage_bytes;
+  g.out_off = g.b_off + g.b_stages * g.b_sub_bytes;
   g.bias_off = g.out_off + g.n_t * 256;
-  if (g.rows_a * 2 * (g.tw / 8) * 8 > kMaxTasks * kProdThreadsPerGroup) return false;
+  if (g.rows_a * 2 * (g.tw / 8) * 8 > kMaxTasks * kProdThreads) return false;
   g.relu = 0;
   g.total_items = (long long)g.tiles_y * g.tiles_x * g.n_tiles_n;
   *out = g;
   return true;
 }
 
-// The launch geometry: as many pixel tiles per item (weight reuse) as still leave every SM at
-// least one item, preferring a count of items that fills whole waves.
+// The launch geometry: pixel tiles per item chosen by an estimate of the launch's duration in
+// units of one MMA (128 x n_t x 16): a CTA runs ceil(items / SMs) items one after the other; a step
+// of an item issues 9 * mt MMAs and cannot be shorter than the hand-over of a stage between the
+// producers, the weight stream and the MMA warp (measured: about eighteen MMAs' time per step when
+// the step itself is shorter: the rings then cover less than the time a stage takes to come back); an item ends with the epilogue of its mt tiles, overlapped with the next item's steps
+// only if two accumulator sets fit.
 bool tensor_geo(const DeviceLayer& L, int n, int h, int w, TGeo* out) {
   const long long sms = device_sm_count();
   bool found = false;
+  double best = 0.0;
   for (int mt = 4; mt >= 1; mt /= 2) {
     TGeo g;
     if (!tensor_geo_mt(L, n, h, w, mt, &g)) continue;
-    *out = g;              // the last one tried (fewest tiles per item) stands if none fills the device
-    found = true;
-    if (g.total_items >= sms) return true;
+    const double waves = (double)((g.total_items + sms - 1) / sms);
+    const double step = 9.0 * mt > 18.0 ? 9.0 * mt : 18.0;
+    const double epilogue = 6.0 * mt;
+    const double cost = waves * (g.k_steps * step + (g.n_buf == 1 || waves == 1.0 ? epilogue : 0.0)) + epilogue;
+    if (!found || cost < best) {
+      found = true;
+      best = cost;
+      *out = g;
+    }
   }
   return found;
 }
