@@ -703,9 +703,6 @@ __device__ __forceinline__ bool produce_half_stream(const DeviceLayer& L, const 
   return true;
 }
 
-__device__ __forceinline__ void red_add_f32(float* p, float v) {
-  asm volatile("red.global.add.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
-}
 
 // Where a lane's outputs go: the element offsets (inside filter 0's plane of the A / B image) of
 // row 0 of its two pixels, and which of the 8 outputs lie inside the image and the batch
@@ -774,23 +771,32 @@ __device__ __forceinline__ void with_flags(const Geo& g, F f) {
   }
 }
 
-// The 8 outputs of one filter slot.  MODE 0: y = act(v + bias); MODE 1: workspace += v.
+__device__ __forceinline__ void red_add_v4(float* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("red.global.v4.f32.add [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(__uint_as_float(a)),
+               "f"(__uint_as_float(b)), "f"(__uint_as_float(c)), "f"(__uint_as_float(d))
+               : "memory");
+}
+
+// The 8 outputs of one filter slot.  MODE 0: y = act(v + bias); MODE 1: workspace += v, where
+// `ws` points at this lane's 8 floats of the slot in the warp's part of the workspace (the
+// workspace is laid out for the warps that write and read it, not like y: [tile][warp][slot]
+// [lane][8], so that a lane's partial sums go out as two 16-byte reductions and come back as two
+// 16-byte loads; lanes and rows outside the image carry zeros or garbage that nobody uses).
 template <int MODE, bool HALF, bool RELU>
 __device__ __forceinline__ void emit_slot(const Geo& g, const LaneOut& lo, void* __restrict__ y,
                                           float* __restrict__ ws, long long fbase, float bv,
                                           const uint32_t (&v)[8]) {
+  if (MODE == 1) {
+    red_add_v4(ws, v[0], v[1], v[2], v[3]);
+    red_add_v4(ws + 4, v[4], v[5], v[6], v[7]);
+    return;
+  }
   const long long ia = fbase + lo.base_a, ib = fbase + lo.base_b;
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
     const int row = k * g.w_out;
-    if (lo.mask >> (2 * k) & 1u) {
-      if (MODE == 1) red_add_f32(ws + ia + row, __uint_as_float(v[2 * k]));
-      else store_out<HALF, RELU>(y, ia + row, __uint_as_float(v[2 * k]) + bv);
-    }
-    if (lo.mask >> (2 * k + 1) & 1u) {
-      if (MODE == 1) red_add_f32(ws + ib + row, __uint_as_float(v[2 * k + 1]));
-      else store_out<HALF, RELU>(y, ib + row, __uint_as_float(v[2 * k + 1]) + bv);
-    }
+    if (lo.mask >> (2 * k) & 1u) store_out<HALF, RELU>(y, ia + row, __uint_as_float(v[2 * k]) + bv);
+    if (lo.mask >> (2 * k + 1) & 1u) store_out<HALF, RELU>(y, ib + row, __uint_as_float(v[2 * k + 1]) + bv);
   }
 }
 
@@ -856,6 +862,10 @@ __device__ __forceinline__ void write_outputs(const Geo& g, const LaneOut& lo, c
       emit_slot<MODE, HALF, RELU>(g, lo, y, ws, (long long)o * plane, bv, v);
     }
   };
+  // MODE 1: `ws` is the lane's first float of the warp's first slot (r.a0); slots are 256 floats apart
+  auto emit_ws = [&](int a, const uint32_t (&v)[8]) {
+    emit_slot<1, false, false>(g, lo, y, ws + (size_t)(a - r.a0) * 256, 0, 0.f, v);
+  };
   if constexpr (GENERIC) {
 #pragma unroll
     for (int a = 0; a < kGroup; ++a) {
@@ -878,14 +888,18 @@ __device__ __forceinline__ void write_outputs(const Geo& g, const LaneOut& lo, c
       for (int b = 0; b < 4; ++b) {
         const int o = __shfl_sync(0xffffffffu, my_o, a + b);
         const float bv = __shfl_sync(0xffffffffu, my_b, a + b);
-        if (o >= 0) emit(o, bv, v[b]);
+        if (o >= 0) {
+          if (MODE == 1) emit_ws(a + b, v[b]);
+          else emit(o, bv, v[b]);
+        }
       }
     }
   }
 }
 
 // The last split to finish a warp's part of an output tile: workspace -> y, leaving the workspace
-// zeroed.  Four filter slots (32 independent loads per lane) are in flight at once.
+// zeroed.  `ws` is the lane's first float of the warp's first slot (a_begin); a slot's 8 sums
+// come back as two 16-byte loads, four slots (eight loads per lane) in flight at once.
 template <bool HALF, bool RELU>
 __device__ __forceinline__ void finalize_outputs(const Geo& g, const LaneOut& lo, const LaneOut& lp,
                                                  void* __restrict__ y, float* __restrict__ ws,
@@ -896,49 +910,35 @@ __device__ __forceinline__ void finalize_outputs(const Geo& g, const LaneOut& lo
 #pragma unroll 1
   for (int a0 = a_begin; a0 < a_end; a0 += kBatch) {
     float v[kBatch][8];
-    long long fb[kBatch];
     int fo[kBatch];
     float bv[kBatch];
 #pragma unroll
     for (int b = 0; b < kBatch; ++b) {
-      const int o = __shfl_sync(0xffffffffu, my_o, a0 + b);
+      fo[b] = __shfl_sync(0xffffffffu, my_o, a0 + b);
       bv[b] = __shfl_sync(0xffffffffu, my_b, a0 + b);
-      fo[b] = o;
-      fb[b] = (o < 0) ? -1 : (long long)o * plane;
-      const long long ia = fb[b] + lo.base_a, ib = fb[b] + lo.base_b;
-      const uint32_t m = (o < 0) ? 0u : lo.mask;
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const int row = k * g.w_out;
-        v[b][2 * k] = (m >> (2 * k) & 1u) ? __ldcg(ws + ia + row) : 0.f;
-        v[b][2 * k + 1] = (m >> (2 * k + 1) & 1u) ? __ldcg(ws + ib + row) : 0.f;
-      }
+      float4* p = reinterpret_cast<float4*>(ws + (size_t)(a0 + b - a_begin) * 256);
+      const float4 lo4 = (fo[b] < 0) ? make_float4(0.f, 0.f, 0.f, 0.f) : __ldcg(p);
+      const float4 hi4 = (fo[b] < 0) ? make_float4(0.f, 0.f, 0.f, 0.f) : __ldcg(p + 1);
+      v[b][0] = lo4.x; v[b][1] = lo4.y; v[b][2] = lo4.z; v[b][3] = lo4.w;
+      v[b][4] = hi4.x; v[b][5] = hi4.y; v[b][6] = hi4.z; v[b][7] = hi4.w;
     }
 #pragma unroll
     for (int b = 0; b < kBatch; ++b) {
-      if (fb[b] < 0) continue;
-      const long long ia = fb[b] + lo.base_a, ib = fb[b] + lo.base_b;
+      if (fo[b] < 0) continue;
+      float4* p = reinterpret_cast<float4*>(ws + (size_t)(a0 + b - a_begin) * 256);
+      p[0] = make_float4(0.f, 0.f, 0.f, 0.f);
+      p[1] = make_float4(0.f, 0.f, 0.f, 0.f);
       if (g.pool) {
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const int row = k * g.w_out;
-          if (lo.mask >> (2 * k) & 1u) ws[ia + row] = 0.f;
-          if (lo.mask >> (2 * k + 1) & 1u) ws[ib + row] = 0.f;
-        }
         emit_slot_pooled<HALF, RELU>(g, lp, y, (long long)fo[b] * plane_y, bv[b], v[b]);
         continue;
       }
+      const long long fb = (long long)fo[b] * plane;
+      const long long ia = fb + lo.base_a, ib = fb + lo.base_b;
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         const int row = k * g.w_out;
-        if (lo.mask >> (2 * k) & 1u) {
-          ws[ia + row] = 0.f;
-          store_out<HALF, RELU>(y, ia + row, v[b][2 * k] + bv[b]);
-        }
-        if (lo.mask >> (2 * k + 1) & 1u) {
-          ws[ib + row] = 0.f;
-          store_out<HALF, RELU>(y, ib + row, v[b][2 * k + 1] + bv[b]);
-        }
+        if (lo.mask >> (2 * k) & 1u) store_out<HALF, RELU>(y, ia + row, v[b][2 * k] + bv[b]);
+        if (lo.mask >> (2 * k + 1) & 1u) store_out<HALF, RELU>(y, ib + row, v[b][2 * k + 1] + bv[b]);
       }
     }
   }
@@ -1234,7 +1234,10 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
                                                                                    orng, my_o, my_b);
         });
       } else {
-        write_outputs<GENERIC, 1, false, false>(g, lo, lp, y, ws, acc, orng, my_o, my_b);
+        // this lane's floats in the warp's part of the tile's workspace: [tile][warp][slot][lane][8]
+        const int spw = kGroup / (GENERIC ? 1 : g.zs);   // slots a warp writes out
+        float* wsl = ws + ((((size_t)blockIdx.y * gridDim.x + blockIdx.x) * kCW + warp) * spw * 32 + lane) * 8;
+        write_outputs<GENERIC, 1, false, false>(g, lo, lp, y, wsl, acc, orng, my_o, my_b);
         PCONV_MARK(4)
         PCONV_MARK_MAX(10)
         // Every warp owns the same part of the output tile in each of the ks splits, and takes a
@@ -1254,7 +1257,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
         if (t == g.ks - 1) {
           __threadfence();
           with_flags(g, [&](auto half, auto relu) {
-            finalize_outputs<decltype(half)::value, decltype(relu)::value>(g, lo, lp, y, ws, orng.a0,
+            finalize_outputs<decltype(half)::value, decltype(relu)::value>(g, lo, lp, y, wsl, orng.a0,
                                                                           orng.a1, my_o, my_b);
           });
         }
@@ -1493,9 +1496,6 @@ cudaError_t launch_one(const DeviceLayer& L, Geo g, const void* x, const float* 
   return cudaLaunchKernelEx(&cfg, tiled_kernel<S, GENERIC, WIDE>, L, g, x, bias, y, ws, counters);
 }
 
-size_t out_elems(const DeviceLayer& L, int n, int h, int w) {
-  return (size_t)n * L.c_out * ((h - 1) / L.stride + 1) * ((w - 1) / L.stride + 1);
-}
 
 }  // namespace
 
@@ -1506,13 +1506,17 @@ bool tiled_supported(const DeviceLayer& L, int n, int h, int w) {
   return make_geo<true>(L, n, h, w, false, &g) && make_geo<false>(L, n, h, w, false, &g);
 }
 
-// Workspace of the channel-split path: one fp32 partial sum per output element, then one ticket
-// per (pixel tile, filter-group set, consumer warp); 0 if this shape is never split.
+// Workspace of the channel-split path: the partial sums of every (tile, consumer warp, filter slot
+// the warp writes out, lane) as 8 floats -- the layout of the warps that add to it and read it
+// back, not y's --, then one ticket per (tile, consumer warp); 0 if this shape is never split.
+size_t split_sums_bytes(const DeviceLayer& L, const Geo& g) {
+  return (size_t)geo_tiles(L, g) * consumer_warps(false) * (kGroup / g.zs) * 32 * 8 * sizeof(float);
+}
 size_t tiled_workspace_bytes(const DeviceLayer& L, int n, int h, int w) {
   Geo g;
   if (!L.codes_s || !make_geo<false>(L, n, h, w, true, &g) || g.ks <= 1) return 0;
   const size_t ctas = (size_t)geo_tiles(L, g);
-  return ((out_elems(L, n, h, w) * 4 + 255) & ~(size_t)255) +
+  return ((split_sums_bytes(L, g) + 255) & ~(size_t)255) +
          ((ctas * consumer_warps(false) * 4 + 255) & ~(size_t)255);
 }
 
@@ -1560,7 +1564,7 @@ cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias,
   int* counters = nullptr;
   if (g.ks > 1) {
     wsf = (float*)ws;
-    counters = (int*)((char*)ws + ((out_elems(L, n, h, w) * 4 + 255) & ~(size_t)255));
+    counters = (int*)((char*)ws + ((split_sums_bytes(L, g) + 255) & ~(size_t)255));
   }
   const bool wide = L.wide_codes != 0;
   if (L.stride == 1) {
