@@ -50,7 +50,12 @@ extern "C" pconv_status pconv_workspace_bytes(const pconv_handle* h, int n, int 
                                               size_t* bytes) {
   if (!h || !bytes) return PCONV_ERR_NULL;
   if (n < 0 || h_in <= 0 || w_in <= 0) return PCONV_ERR_SHAPE;
-  *bytes = (n == 0) ? 0 : tiled_workspace_bytes(h->d, n, h_in, w_in);
+  // (whichever kernel a forward of this shape may take)
+  *bytes = 0;
+  if (n > 0) {
+    const size_t a = tiled_workspace_bytes(h->d, n, h_in, w_in), b = tensor_workspace_bytes(h->d, n, h_in, w_in);
+    *bytes = a > b ? a : b;
+  }
   return PCONV_OK;
 }
 
@@ -146,9 +151,9 @@ static pconv_status forward_impl(const pconv_handle* h, const void* x, const flo
     return PCONV_ERR_UNSUPPORTED;  // only the tiled kernels fuse the pool
   if (sel == PCONV_KERNEL_TENSOR) {
     if (pool || !tensor_supported(L, n, h_in, w_in)) return PCONV_ERR_UNSUPPORTED;
-    e = launch_tensor(L, x, bias, y, n, h_in, w_in, relu, stream);
+    e = launch_tensor(L, x, bias, y, n, h_in, w_in, relu, repro ? nullptr : ws, ws_bytes, stream);
   } else if (sel == 0 && !pool && tensor_preferred(L, n, h_in, w_in)) {
-    e = launch_tensor(L, x, bias, y, n, h_in, w_in, relu, stream);
+    e = launch_tensor(L, x, bias, y, n, h_in, w_in, relu, repro ? nullptr : ws, ws_bytes, stream);
   } else if (sel == PCONV_KERNEL_SIMPLE) {
     e = launch_simple(L, x, bias, y, n, h_in, w_in, relu, stream);
   } else if (sel == PCONV_KERNEL_TILED || sel == PCONV_KERNEL_GENERIC_TAPS) {
@@ -201,7 +206,8 @@ extern "C" pconv_status pconv_forward_static_ws(const pconv_handle* h, const voi
   if (!h || !x || !y) return PCONV_ERR_NULL;
   if (n < 0 || h_in <= 0 || w_in <= 0) return PCONV_ERR_SHAPE;
   if (n == 0) return PCONV_OK;
-  const size_t need = tiled_workspace_bytes(h->d, n, h_in, w_in);
+  size_t need = 0;
+  if (pconv_workspace_bytes(h, n, h_in, w_in, &need) != PCONV_OK) return PCONV_ERR_SHAPE;
   if (need > (size_t)PCONV_STATIC_WS_BYTES) return PCONV_ERR_WORKSPACE;
   if (need == 0)  // this shape is never split: no scratch involved
     return pconv_forward_ws(h, x, bias, y, n, h_in, w_in, flags, nullptr, 0, stream_v);
@@ -350,8 +356,9 @@ extern "C" pconv_status pconv_stack_create(const pconv_handle* const* layers,
       pconv_stack_free(s);
       return PCONV_ERR_SHAPE;
     }
-    const size_t wsb = tiled_workspace_bytes(L, n, ch, cw);
+    const size_t wsb = tiled_workspace_bytes(L, n, ch, cw), wsd = tensor_workspace_bytes(L, n, ch, cw);
     if (wsb > s->ws_bytes) s->ws_bytes = wsb;
+    if (wsd > s->ws_bytes) s->ws_bytes = wsd;
     ch = (ch - 1) / L.stride + 1;
     cw = (cw - 1) / L.stride + 1;
     cc = L.c_out;

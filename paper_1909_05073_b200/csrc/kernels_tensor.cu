@@ -84,13 +84,14 @@ struct TGeo {
   int tiles_x;       // column tiles of the virtual width cpr * wc
   int strip_rows, tiles_y;   // strip rows of the batch; items along the strip
   int n_t, n_tiles_n, k_steps;
+  int ksplit, kpp;   // parts the channel steps of an item are cut in (1 = none), steps per part
   int a_stages, b_stages;  // ring depths
   int b_resident;          // 1: the layer's whole weight operand fits the ring and is loaded once per CTA
   int a_copy_bytes, a_lbo, row_bytes, a_stage_bytes, a_off;
   int b_bytes, b_sub_bytes, b_off;   // weights of a step (nine taps) / of a sub-stage (three taps)
   int out_off, bias_off;   // the epilogue's staging tile [n_t / 2][128][2] fp16 and the tile's bias [n_t] fp32
   int relu;
-  long long total_items;   // tiles_y * tiles_x * n_tiles_n
+  long long total_items;   // tiles_y * tiles_x * n_tiles_n * ksplit
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -285,10 +286,36 @@ __device__ __forceinline__ void load_task(const TGeo& g, const unsigned short* p
   }
 }
 
+// A work item: pixel tiles (ty, tx), filter tile nt, and -- when the channel steps are cut in
+// `ksplit` parts that different CTAs take -- the first step k0 of its part; mn numbers the
+// (pixel, filter) tile whatever the part.
+struct TItem {
+  int ty, tx, nt, k0;
+  long long mn;
+};
+__device__ __forceinline__ TItem decode_item(const TGeo& g, long long item) {
+  TItem it;
+  const int kp = (int)(item % g.ksplit);
+  it.mn = item / g.ksplit;
+  const int mti = (int)(it.mn / g.n_tiles_n);
+  it.nt = (int)(it.mn - (long long)mti * g.n_tiles_n);
+  it.ty = mti / g.tiles_x;
+  it.tx = mti - it.ty * g.tiles_x;
+  it.k0 = kp * g.kpp;
+  return it;
+}
+
+__device__ __forceinline__ void red_add_v4(float* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("red.global.v4.f32.add [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(__uint_as_float(a)),
+               "f"(__uint_as_float(b)), "f"(__uint_as_float(c)), "f"(__uint_as_float(d))
+               : "memory");
+}
+
 template <int MODE>
 __global__ void __launch_bounds__(kTensorThreads, 1)
 tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
-              const float* __restrict__ bias, __half* __restrict__ y) {
+              const float* __restrict__ bias, __half* __restrict__ y, float* __restrict__ ws,
+              int* __restrict__ tickets) {
   extern __shared__ __align__(128) unsigned char smem[];
   const uint32_t sbase = smem_u32(smem);
   const int tid = threadIdx.x, lane = tid & 31;
@@ -360,7 +387,7 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * acc_cols);
-        for (int ks = 0; ks < g.k_steps && ok; ++ks, ++ita) {
+        for (int ks = 0; ks < g.kpp && ok; ++ks, ++ita) {
           const int sa = (int)(ita % g.a_stages);
           t0 = T_NOW();
           ok = mbar_wait(bar_afull + 8 * sa, (uint32_t)((ita / g.a_stages) & 1), L.err, 21);
@@ -435,11 +462,11 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
     RegSet set0, set1;
     const unsigned short* src[kMaxTasks];   // of the item being loaded: a task's 8 pixels at step 0 (null = padding)
     uint32_t aux[kMaxTasks];
+    int l_k0 = 0;                           // first channel step of the item being loaded
     auto setup_item = [&](int ti) {
-      const long long item = blockIdx.x + (long long)ti * gridDim.x;
-      const int mti = (int)(item / g.n_tiles_n);
-      const int ty = mti / g.tiles_x;
-      const int tx = mti - ty * g.tiles_x;
+      const TItem wi = decode_item(g, blockIdx.x + (long long)ti * gridDim.x);
+      const int ty = wi.ty, tx = wi.tx;
+      l_k0 = wi.k0;
 #pragma unroll
       for (int q = 0; q < kMaxTasks; ++q) {
         const int t = gt + q * kProdThreads;
@@ -476,8 +503,8 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
       }
       if (l_ti >= my_items) return;
       // channels beyond c_in (last step of a layer whose depth is no multiple of 16) are zeros
-      const int ch_limit = g.c_in - l_ks * 16;
-      const size_t chan_off = (size_t)l_ks * step;
+      const int ch_limit = g.c_in - (l_k0 + l_ks) * 16;
+      const size_t chan_off = (size_t)(l_k0 + l_ks) * step;
 #pragma unroll
       for (int q = 0; q < kMaxTasks; ++q) {
         if (src[q] == nullptr) continue;
@@ -487,13 +514,13 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
         }
         load_task<MODE>(g, src[q] + chan_off, aux[q], img, &rs.v[q], &rs.lft[q], &rs.rgt[q]);
       }
-      if (++l_ks == g.k_steps) {
+      if (++l_ks == g.kpp) {
         l_ks = 0;
         if (++l_ti < my_items) setup_item(l_ti);
       }
     };
     const uint32_t copy_b = (uint32_t)g.a_copy_bytes;
-    const long long n_stages = (long long)my_items * g.k_steps;
+    const long long n_stages = (long long)my_items * g.kpp;
     T_DECL;
     auto store_stage = [&](const RegSet& rs, long long it) -> bool {
       const int s = (int)(it % g.a_stages);
@@ -555,10 +582,10 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
       long long itb = 0;
       T_DECL;
       for (int ti = 0; ti < (g.b_resident ? min(my_items, 1) : my_items) && ok; ++ti) {
-        const long long item = blockIdx.x + (long long)ti * gridDim.x;
-        const int nt = (int)(item % g.n_tiles_n);
-        const char* wsrc = reinterpret_cast<const char*>(L.wdense) + (size_t)nt * g.k_steps * g.b_bytes;
-        for (int ks = 0; ks < g.k_steps && ok; ++ks) {
+        const TItem wi = decode_item(g, blockIdx.x + (long long)ti * gridDim.x);
+        const char* wsrc = reinterpret_cast<const char*>(L.wdense) +
+                           ((size_t)wi.nt * g.k_steps + wi.k0) * g.b_bytes;
+        for (int ks = 0; ks < g.kpp && ok; ++ks) {
           for (int u = 0; u < 3; ++u, ++itb) {
             const int sb = (int)(itb % g.b_stages);
             const long long t0 = T_NOW();
@@ -591,11 +618,8 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
     bool ok = true;
     T_DECL;
     for (int ti = 0; ti < my_items && ok; ++ti) {
-      const long long item = blockIdx.x + (long long)ti * gridDim.x;
-      const int mti = (int)(item / g.n_tiles_n);
-      const int nt = (int)(item - (long long)mti * g.n_tiles_n);
-      const int ty = mti / g.tiles_x;
-      const int tx = mti - ty * g.tiles_x;
+      const TItem wi = decode_item(g, blockIdx.x + (long long)ti * gridDim.x);
+      const int nt = wi.nt, ty = wi.ty, tx = wi.tx;
       const int buf = ti % g.n_buf;
       const uint32_t use = (uint32_t)(ti / g.n_buf);
       const int o_base = nt * g.n_t;
@@ -610,7 +634,42 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
       if (!ok) break;
       t0 = T_NOW();
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      for (int j = 0; j < g.mt; ++j) {
+      // Channel steps cut in parts: every part adds its accumulators to the (pixel, filter) tile's
+      // fp32 sums in the workspace ([tile j][filter / 4][pixel][4]: a lane's four consecutive
+      // filters are one 16-byte reduction) and takes a ticket; the part that draws the last one
+      // reads the sums back -- instead of Tensor Memory -- and finishes the tile as usual,
+      // leaving sums and ticket zeroed.
+      float* wsb = nullptr;
+      bool finish = true;
+      if (g.ksplit > 1) {
+        wsb = ws + (size_t)wi.mn * ((size_t)g.mt * g.n_t * 128);
+        for (int j = 0; j < g.mt; ++j) {
+          const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * acc_cols + j * g.n_t);
+          for (int j0 = 0; j0 < n_f; j0 += 32) {
+            uint32_t acc[32];
+            tmem_ld32_issue(acc, taddr + (uint32_t)j0);
+            tmem_ld_wait();
+            float* pw = wsb + (((size_t)j * (g.n_t / 4) + (j0 >> 2)) * 128 + m) * 4;
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              red_add_v4(pw + (size_t)i * 512, acc[4 * i], acc[4 * i + 1], acc[4 * i + 2], acc[4 * i + 3]);
+          }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        mbar_arrive(bar_acce + 8 * buf);                       // the accumulators have been read
+        __threadfence();
+        epi_sync();
+        volatile int* last_s = reinterpret_cast<volatile int*>(smem + 16 * (kMaxAStages + kMaxBStages) + 36);
+        if (et == 0) {
+          const int t = atomicAdd(tickets + wi.mn, 1);
+          if (t == g.ksplit - 1) tickets[wi.mn] = 0;
+          *last_s = (t == g.ksplit - 1) ? 1 : 0;
+        }
+        epi_sync();
+        finish = *last_s != 0;
+        if (finish) __threadfence();
+      }
+      for (int j = 0; finish && j < g.mt; ++j) {
         long long t1 = T_NOW();
         const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * acc_cols + j * g.n_t);
         // Two adjacent filters of a pixel are converted together (the packed fp16 conversion runs
@@ -643,21 +702,38 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
           }
         };
         uint32_t acc0[32], acc1[32];
-        tmem_ld32_issue(acc0, taddr);
-        tmem_ld_wait();
-        for (int j0 = 0; j0 < n_f; j0 += 64) {
-          if (j0 + 32 < n_f) tmem_ld32_issue(acc1, taddr + (uint32_t)(j0 + 32));
-          stage_block(acc0, j0);
-          tmem_ld_wait();
-          if (j0 + 32 < n_f) {
-            if (j0 + 64 < n_f) tmem_ld32_issue(acc0, taddr + (uint32_t)(j0 + 64));
-            stage_block(acc1, j0 + 32);
-            tmem_ld_wait();
+        if (g.ksplit > 1) {
+          for (int j0 = 0; j0 < n_f; j0 += 32) {
+            float4* pw = reinterpret_cast<float4*>(wsb + (((size_t)j * (g.n_t / 4) + (j0 >> 2)) * 128 + m) * 4);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const float4 f4 = __ldcg(pw + (size_t)i * 128);
+              acc0[4 * i] = __float_as_uint(f4.x);
+              acc0[4 * i + 1] = __float_as_uint(f4.y);
+              acc0[4 * i + 2] = __float_as_uint(f4.z);
+              acc0[4 * i + 3] = __float_as_uint(f4.w);
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) pw[(size_t)i * 128] = make_float4(0.f, 0.f, 0.f, 0.f);
+            stage_block(acc0, j0);
           }
-        }
-        if (j == g.mt - 1) {   // the accumulators have been read: the MMA warp may reuse them
-          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-          mbar_arrive(bar_acce + 8 * buf);
+        } else {
+          tmem_ld32_issue(acc0, taddr);
+          tmem_ld_wait();
+          for (int j0 = 0; j0 < n_f; j0 += 64) {
+            if (j0 + 32 < n_f) tmem_ld32_issue(acc1, taddr + (uint32_t)(j0 + 32));
+            stage_block(acc0, j0);
+            tmem_ld_wait();
+            if (j0 + 32 < n_f) {
+              if (j0 + 64 < n_f) tmem_ld32_issue(acc0, taddr + (uint32_t)(j0 + 64));
+              stage_block(acc1, j0 + 32);
+              tmem_ld_wait();
+            }
+          }
+          if (j == g.mt - 1) {   // the accumulators have been read: the MMA warp may reuse them
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            mbar_arrive(bar_acce + 8 * buf);
+          }
         }
         T_ADD(11, t1);
         t1 = T_NOW();
@@ -740,7 +816,7 @@ tensor_kernel(const DeviceLayer L, const TGeo g, const __half* __restrict__ x,
 }
 
 // Geometry of a launch with mt pixel tiles per work item; false if it does not fit.
-bool tensor_geo_mt(const DeviceLayer& L, int n, int h, int w, int mt, TGeo* out) {
+bool tensor_geo_mt(const DeviceLayer& L, int n, int h, int w, int mt, int ksplit, TGeo* out) {
   if (!L.wdense || L.dense_nt <= 0 || L.stride != 1 || L.storage != PCONV_F16) return false;
   TGeo g;
   g.n = n;
@@ -775,6 +851,9 @@ bool tensor_geo_mt(const DeviceLayer& L, int n, int h, int w, int mt, TGeo* out)
   g.tiles_y = (g.strip_rows + mt * g.r - 1) / (mt * g.r);
   g.n_tiles_n = (L.c_out + g.n_t - 1) / g.n_t;
   g.k_steps = (L.c_in + 15) / 16;
+  if (ksplit < 1 || g.k_steps % ksplit != 0) return false;
+  g.ksplit = ksplit;
+  g.kpp = g.k_steps / ksplit;
   g.row_bytes = (g.tw / 8) * 128;
   g.a_lbo = g.rows_a * g.row_bytes;
   g.a_copy_bytes = 2 * g.a_lbo;
@@ -795,7 +874,7 @@ bool tensor_geo_mt(const DeviceLayer& L, int n, int h, int w, int mt, TGeo* out)
   if (g.b_stages < 3) return false;
   // a layer with one filter tile whose weights all fit keeps them: nothing is streamed again
   g.b_resident = 0;
-  if (g.n_tiles_n == 1 && 3 * g.k_steps <= kMaxBStages &&
+  if (ksplit == 1 && g.n_tiles_n == 1 && 3 * g.k_steps <= kMaxBStages &&
       2 * g.a_stage_bytes + 3 * g.k_steps * g.b_sub_bytes <= avail) {
     g.b_resident = 1;
     g.b_stages = 3 * g.k_steps;
@@ -810,7 +889,7 @@ bool tensor_geo_mt(const DeviceLayer& L, int n, int h, int w, int mt, TGeo* out)
   g.bias_off = g.out_off + g.n_t * 256;
   if (g.rows_a * 2 * (g.tw / 8) * 8 > kMaxTasks * kProdThreads) return false;
   g.relu = 0;
-  g.total_items = (long long)g.tiles_y * g.tiles_x * g.n_tiles_n;
+  g.total_items = (long long)g.tiles_y * g.tiles_x * g.n_tiles_n * ksplit;
   *out = g;
   return true;
 }
@@ -821,13 +900,13 @@ bool tensor_geo_mt(const DeviceLayer& L, int n, int h, int w, int mt, TGeo* out)
 // producers, the weight stream and the MMA warp (measured: about eighteen MMAs' time per step when
 // the step itself is shorter: the rings then cover less than the time a stage takes to come back); an item ends with the epilogue of its mt tiles, overlapped with the next item's steps
 // only if two accumulator sets fit.
-bool tensor_geo(const DeviceLayer& L, int n, int h, int w, TGeo* out) {
+bool tensor_geo(const DeviceLayer& L, int n, int h, int w, bool allow_split, TGeo* out) {
   const long long sms = device_sm_count();
   bool found = false;
   double best = 0.0;
   for (int mt = 4; mt >= 1; mt /= 2) {
     TGeo g;
-    if (!tensor_geo_mt(L, n, h, w, mt, &g)) continue;
+    if (!tensor_geo_mt(L, n, h, w, mt, 1, &g)) continue;
     const double waves = (double)((g.total_items + sms - 1) / sms);
     const double step = 9.0 * mt > 18.0 ? 9.0 * mt : 18.0;
     const double epilogue = 6.0 * mt;
@@ -838,14 +917,35 @@ bool tensor_geo(const DeviceLayer& L, int n, int h, int w, TGeo* out) {
       *out = g;
     }
   }
+  // Too few tiles for the device even one by one (small maps, deep layers): cut the channel steps
+  // in parts that different CTAs take; the parts meet in an fp32 workspace (see the epilogue).
+  if (found && allow_split && out->mt == 1 && 2 * out->total_items <= sms) {
+    int ksplit = 1;
+    for (int d = 2; d <= 8; ++d)
+      if (out->k_steps % d == 0 && out->k_steps / d >= 4 && out->total_items * d <= sms) ksplit = d;
+    TGeo g;
+    if (ksplit > 1 && tensor_geo_mt(L, n, h, w, 1, ksplit, &g)) *out = g;
+  }
   return found;
+}
+
+// Workspace of a split launch: fp32 sums of every (pixel, filter) tile, then a ticket per tile.
+size_t tensor_sums_bytes(const TGeo& g) {
+  return (size_t)(g.total_items / g.ksplit) * g.mt * g.n_t * 128 * sizeof(float);
 }
 
 }  // namespace
 
 bool tensor_supported(const DeviceLayer& L, int n, int h, int w) {
   TGeo g;
-  return n > 0 && h > 0 && w > 0 && tensor_geo(L, n, h, w, &g);
+  return n > 0 && h > 0 && w > 0 && tensor_geo(L, n, h, w, false, &g);
+}
+
+size_t tensor_workspace_bytes(const DeviceLayer& L, int n, int h, int w) {
+  TGeo g;
+  if (n <= 0 || h <= 0 || w <= 0 || !tensor_geo(L, n, h, w, true, &g) || g.ksplit <= 1) return 0;
+  return ((tensor_sums_bytes(g) + 255) & ~(size_t)255) +
+         (((size_t)(g.total_items / g.ksplit) * sizeof(int) + 255) & ~(size_t)255);
 }
 
 // Whether the dense tensor-core path is expected to beat the pattern-sparse kernel: it needs
@@ -857,7 +957,7 @@ bool tensor_supported(const DeviceLayer& L, int n, int h, int w) {
 // sparse kernel.)
 bool tensor_preferred(const DeviceLayer& L, int n, int h, int w) {
   TGeo g;
-  if (!tensor_geo(L, n, h, w, &g)) return false;
+  if (!tensor_geo(L, n, h, w, false, &g)) return false;
   if (g.total_items * g.mt < device_sm_count() / 4) return false;
   const double dense = 2.0 * 9.0 * (16.0 * g.k_steps) * ((double)g.n_tiles_n * g.n_t);   // per pixel
   const double sparse = 8.0 * (double)L.n_kept;
@@ -866,7 +966,7 @@ bool tensor_preferred(const DeviceLayer& L, int n, int h, int w) {
 
 template <int MODE>
 cudaError_t launch_tensor_mode(const DeviceLayer& L, const TGeo& g, const void* x, const float* bias, void* y,
-                               cudaStream_t stream) {
+                               float* ws, int* tickets, cudaStream_t stream) {
   const int smem = g.bias_off + g.n_t * 4;
   cudaError_t e = cudaFuncSetAttribute(tensor_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        kTSmemLimit);
@@ -883,19 +983,27 @@ cudaError_t launch_tensor_mode(const DeviceLayer& L, const TGeo& g, const void* 
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, tensor_kernel<MODE>, L, g, (const __half*)x, bias, (__half*)y);
+  return cudaLaunchKernelEx(&cfg, tensor_kernel<MODE>, L, g, (const __half*)x, bias, (__half*)y, ws, tickets);
 }
 
 cudaError_t launch_tensor(const DeviceLayer& L, const void* x, const float* bias, void* y, int n, int h,
-                          int w, bool relu, cudaStream_t stream) {
+                          int w, bool relu, void* ws, size_t ws_bytes, cudaStream_t stream) {
   TGeo g;
-  if (!tensor_geo(L, n, h, w, &g)) return cudaErrorInvalidValue;
+  const size_t need = ws ? tensor_workspace_bytes(L, n, h, w) : 0;
+  const bool split = need > 0 && ws_bytes >= need;
+  if (!tensor_geo(L, n, h, w, split, &g)) return cudaErrorInvalidValue;
   g.relu = relu ? 1 : 0;
-  if (w >= 8 && w % 8 == 0) return launch_tensor_mode<kModeW8>(L, g, x, bias, y, stream);
-  if (w >= 5) return launch_tensor_mode<kModeWX>(L, g, x, bias, y, stream);
-  if (w == 4) return launch_tensor_mode<kModeN4>(L, g, x, bias, y, stream);
-  if (w == 2) return launch_tensor_mode<kModeN2>(L, g, x, bias, y, stream);
-  return launch_tensor_mode<kModeNX>(L, g, x, bias, y, stream);
+  float* sums = nullptr;
+  int* tickets = nullptr;
+  if (g.ksplit > 1) {
+    sums = (float*)ws;
+    tickets = (int*)((char*)ws + ((tensor_sums_bytes(g) + 255) & ~(size_t)255));
+  }
+  if (w >= 8 && w % 8 == 0) return launch_tensor_mode<kModeW8>(L, g, x, bias, y, sums, tickets, stream);
+  if (w >= 5) return launch_tensor_mode<kModeWX>(L, g, x, bias, y, sums, tickets, stream);
+  if (w == 4) return launch_tensor_mode<kModeN4>(L, g, x, bias, y, sums, tickets, stream);
+  if (w == 2) return launch_tensor_mode<kModeN2>(L, g, x, bias, y, sums, tickets, stream);
+  return launch_tensor_mode<kModeNX>(L, g, x, bias, y, sums, tickets, stream);
 }
 
 }  // namespace pconv

@@ -131,7 +131,8 @@ cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias,
                          int h, int w, bool relu, bool pool, bool reproducible, bool generic_taps,
                          void* ws, size_t ws_bytes, cudaStream_t stream);
 cudaError_t launch_tensor(const DeviceLayer& L, const void* x, const float* bias, void* y, int n,
-                          int h, int w, bool relu, cudaStream_t stream);
+                          int h, int w, bool relu, void* ws, size_t ws_bytes, cudaStream_t stream);
+size_t tensor_workspace_bytes(const DeviceLayer& L, int n, int h, int w);
 bool tensor_supported(const DeviceLayer& L, int n, int h, int w);
 bool tensor_preferred(const DeviceLayer& L, int n, int h, int w);
 size_t tiled_workspace_bytes(const DeviceLayer& L, int n, int h, int w);

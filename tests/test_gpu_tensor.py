@@ -65,6 +65,30 @@ def test_tensor_path_matches_the_oracle(case):
     layer.close()
 
 
+@pytest.mark.parametrize("case", [(512, 256, 2, 2, 64, 0.25), (256, 130, 4, 4, 40, 0.3), (192, 64, 8, 8, 12, 0.4)],
+                         ids=lambda c: "x".join(str(v) for v in c))
+def test_tensor_path_with_the_channel_steps_split_across_ctas(case):
+    """Few pixel tiles, deep layer: with a workspace the channel steps of a tile are cut in parts
+    that different CTAs take; the parts meet in fp32 sums in the workspace, which must be zero
+    again afterwards (two forwards in a row use it)."""
+    c_in, c_out, h, w, n, keep = case
+    spec = synth.LayerSpec("t", c_in, c_out, h, w, 1, keep)
+    wt, bias, _ = synth.gen_weights(spec, 555 + c_in)
+    x = synth.gen_input(spec, n, 555 + c_in)
+    layer = B.Layer(wt, synth.PATTERNS8, 1, B.F16, bias)
+    assert B.pconv_workspace_bytes(layer.handle, n, h, w) > 0
+    xt = torch.from_numpy(x).cuda().half()
+    ref = oracle.conv3x3(x, wt, bias, 1, True, "f16")
+    for rep in range(2):
+        got = layer.forward(xt, relu=True, kernel=B.KERNEL_TENSOR, split=True)
+        check_close(got.float().cpu().numpy(), ref, "f16", "%s split, call %d" % (case, rep))
+        assert not layer._ws.any()
+    same = layer.forward(xt, relu=True, kernel=B.KERNEL_TENSOR, split=False)       # no workspace: no split
+    check_close(same.float().cpu().numpy(), ref, "f16", "%s unsplit" % (case,))
+    assert B.pconv_device_status(layer.handle) == (0, 0)
+    layer.close()
+
+
 def test_tensor_path_without_bias_and_with_twelve_patterns():
     spec = synth.LayerSpec("t", 32, 48, 16, 16, 1, 0.4, probs=(1 / 12,) * 12)
     wt, _, _ = synth.gen_weights(spec, 91, synth.PATTERNS12)
