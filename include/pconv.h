@@ -69,6 +69,11 @@ enum {
                               channel range is not split across thread blocks (a workspace, if
                               given, is left untouched).  Without it the grouping of the fp32 partial
                               sums -- not the result beyond rounding -- may vary from run to run. */
+  PCONV_NO_CHAIN = 0x10u,  /* stacks: every layer is a launch of its own.  By default a stack runs
+                              consecutive layers whose launch plans are single waves of CTAs
+                              (batch-1 inference) as one persistent kernel: Tensor Memory, barriers
+                              and the CTA itself stay, a CTA prefetches the next layer's weights
+                              while others finish, and layers are crossed on a grid-wide count. */
   PCONV_KERNEL_SIMPLE = 0x100u, /* one thread per output, walks the per-filter kernel list */
   PCONV_KERNEL_TILED = 0x200u,  /* shared-memory halo tiles, packed FMAs, one straight-line body per
                                    pattern mask (any set of 4-of-9 masks); the default */
@@ -303,6 +308,10 @@ pconv_status pconv_project(const float* w_dev, long long n_kernels, const uint16
 pconv_status pconv_stack_create(const pconv_handle* const* layers, const float* const* bias_dev,
                                 const unsigned char* pool_after, int n_layers, int n, int h, int w,
                                 unsigned flags, pconv_stack** out);
+
+/* Kernel launches one forward of the stack makes: a run of layers executed by one persistent
+ * kernel counts once, a max-pool that is not fused into its layer counts as one more. */
+pconv_status pconv_stack_launches(const pconv_stack* s, int* launches);
 
 /* Shape of the stack's result: [n][c][h][w] (any pointer may be NULL). */
 pconv_status pconv_stack_out_shape(const pconv_stack* s, int* n, int* c, int* h, int* w);

@@ -14,7 +14,7 @@ LIB_PATH = os.path.join(HERE, "libpconv.so")
 
 OK = 0
 F32, F16 = 0, 1
-RELU, STRICT4, POOL2X2, REPRODUCIBLE = 1, 2, 4, 8
+RELU, STRICT4, POOL2X2, REPRODUCIBLE, NO_CHAIN = 1, 2, 4, 8, 0x10
 KERNEL_SIMPLE, KERNEL_TILED, KERNEL_GENERIC_TAPS, KERNEL_TENSOR = 0x100, 0x200, 0x400, 0x800
 MAX_PATTERNS = 16
 
@@ -27,7 +27,7 @@ EXPORTS = ["pconv_pack", "pconv_forward", "pconv_forward_ws", "pconv_forward_sta
            "pconv_free", "pconv_maxpool2x2", "pconv_unpack",
            "pconv_stats", "pconv_filter_order", "pconv_device_status", "pconv_status_str",
            "pconv_stack_create", "pconv_stack_out_shape", "pconv_stack_forward",
-           "pconv_stack_forward_host", "pconv_stack_free", "pconv_stack_capture", "pconv_stack_replay", "pconv_stack_status",
+           "pconv_stack_forward_host", "pconv_stack_free", "pconv_stack_capture", "pconv_stack_replay", "pconv_stack_status", "pconv_stack_launches",
            "pconv_project", "pconv_project_workspace_bytes"]
 
 
@@ -101,6 +101,7 @@ def load(path):
     L.pconv_stack_capture.argtypes = [vp, vp, vp, vp]
     L.pconv_stack_replay.argtypes = [vp, vp]
     L.pconv_stack_status.argtypes = [vp, ip]
+    L.pconv_stack_launches.argtypes = [vp, ip]
     L.pconv_stack_free.argtypes = [vp]
     L.pconv_stack_free.restype = None
     return L
@@ -390,6 +391,12 @@ class Stack:
         yp = y_host.data_ptr() if hasattr(y_host, "data_ptr") else y_host.ctypes.data
         _check(lib().pconv_stack_forward_host(self.ptr, ctypes.c_void_p(xp), ctypes.c_void_p(yp),
                                               _stream_ptr(stream)), "pconv_stack_forward_host")
+
+    def launches(self):
+        """Kernel launches of one forward (a run of layers in one persistent kernel counts once)."""
+        k = ctypes.c_int(0)
+        _check(lib().pconv_stack_launches(self.ptr, ctypes.byref(k)), "pconv_stack_launches")
+        return k.value
 
     def status(self):
         """(status, wait id): PCONV_ERR_DEVICE_TIMEOUT if a kernel of this stack gave up a bounded

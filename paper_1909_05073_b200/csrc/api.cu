@@ -1,7 +1,9 @@
 // C ABI entry points: argument checks, kernel selection, layer stacks.
 #include <cstring>
+#include <cstdlib>
 #include <mutex>
 #include <new>
+#include <vector>
 
 #include "pconv_internal.h"
 #ifdef PCONV_DEV
@@ -119,7 +121,7 @@ static pconv_status forward_impl(const pconv_handle* h, const void* x, const flo
   if (!h || !x || !y) return PCONV_ERR_NULL;
   if (n < 0 || h_in <= 0 || w_in <= 0) return PCONV_ERR_SHAPE;
   const unsigned known =
-      PCONV_RELU | PCONV_POOL2X2 | PCONV_REPRODUCIBLE | PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED |
+      PCONV_RELU | PCONV_POOL2X2 | PCONV_REPRODUCIBLE | PCONV_NO_CHAIN | PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED |
       PCONV_KERNEL_GENERIC_TAPS | PCONV_KERNEL_TENSOR;
   if (flags & ~known) return PCONV_ERR_UNSUPPORTED;
   const unsigned sel = flags & (PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED | PCONV_KERNEL_GENERIC_TAPS |
@@ -300,6 +302,16 @@ struct pconv_stack {
   void* graph_y;
   cudaGraphExec_t host_exec;   // the host entry point's own graph (io[0] -> io[1])
   bool host_graph_failed;      // its capture was tried and is not possible on the stream given
+  // chains: runs of consecutive layers that one persistent kernel executes (batch-1 stacks, where
+  // every layer is a single wave of CTAs and launch, set-up and first-data latencies dominate)
+  struct Chain {
+    int begin, end;            // layers [begin, end)
+    void* table_host;          // the chain kernel's per-layer table, and its device copy
+    void* table_dev;
+    std::vector<void*> mid;    // outputs of the chain's inner layers (never reused inside the launch)
+  };
+  std::vector<Chain>* chains;
+  unsigned int* sync_dev;      // the chain kernel's two counters (zero between launches)
 };
 
 extern "C" void pconv_stack_free(pconv_stack* s) {
@@ -309,6 +321,16 @@ extern "C" void pconv_stack_free(pconv_stack* s) {
     if (s->io[i]) cudaFree(s->io[i]);
   }
   if (s->ws) cudaFree(s->ws);
+  if (s->chains) {
+    for (pconv_stack::Chain& c : *s->chains) {
+      std::free(c.table_host);
+      if (c.table_dev) cudaFree(c.table_dev);
+      for (void* m : c.mid)
+        if (m) cudaFree(m);
+    }
+    delete s->chains;
+  }
+  if (s->sync_dev) cudaFree(s->sync_dev);
   if (s->status_dev) cudaFree(s->status_dev);
   if (s->status_host) cudaFreeHost(s->status_host);
   if (s->graph_exec) cudaGraphExecDestroy(s->graph_exec);
@@ -317,6 +339,84 @@ extern "C" void pconv_stack_free(pconv_stack* s) {
   delete[] s->bias;
   delete[] s->pool;
   delete s;
+}
+
+// Finds the runs of consecutive layers that a chain kernel can execute, builds their tables and
+// inner buffers, and allocates the workspace (the layers' and the chains' largest need).
+static bool build_chains(pconv_stack* s) {
+  s->chains = new (std::nothrow) std::vector<pconv_stack::Chain>();
+  if (!s->chains) return false;
+  const unsigned sel_bits = PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED | PCONV_KERNEL_GENERIC_TAPS | PCONV_KERNEL_TENSOR;
+  const size_t es = (s->storage == PCONV_F16) ? 2 : 4;
+  if (!(s->flags & (sel_bits | PCONV_REPRODUCIBLE | PCONV_NO_CHAIN))) {
+    // shapes of every layer's input and output
+    std::vector<int> hi(s->n_layers), wi(s->n_layers);
+    int ch = s->h, cw = s->w;
+    std::vector<bool> ok(s->n_layers, false);
+    for (int i = 0; i < s->n_layers; ++i) {
+      const pconv::DeviceLayer& L = s->layers[i]->d;
+      hi[i] = ch;
+      wi[i] = cw;
+      ok[i] = pconv::chain_layer_ok(L, s->n, ch, cw, s->pool[i] != 0, nullptr) &&
+              !pconv::tensor_preferred(L, s->n, ch, cw);
+      ch = (ch - 1) / L.stride + 1;
+      cw = (cw - 1) / L.stride + 1;
+      if (s->pool[i]) {
+        ch /= 2;
+        cw /= 2;
+      }
+    }
+    for (int b = 0; b < s->n_layers;) {
+      int e = b;
+      while (e < s->n_layers && ok[e] && e - b < 16) ++e;
+      if (e - b < 2) {
+        b = e > b ? e : b + 1;
+        continue;
+      }
+      pconv_stack::Chain c;
+      c.begin = b;
+      c.end = e;
+      c.table_dev = nullptr;
+      c.table_host = std::malloc(pconv::chain_table_bytes(e - b));
+      if (!c.table_host) return false;
+      s->chains->push_back(c);
+      pconv_stack::Chain& cc = s->chains->back();
+      const void* x = nullptr;     // the chain's input: given at launch
+      for (int i = b; i < e; ++i) {
+        const pconv::DeviceLayer& L = s->layers[i]->d;
+        int ho = hi[i], wo = wi[i];
+        if (s->pool[i]) {
+          ho /= 2;
+          wo /= 2;
+        }
+        void* y = nullptr;         // the chain's output: given at launch
+        if (i + 1 < e) {
+          if (cudaMalloc(&y, (size_t)s->n * L.c_out * ho * wo * es) != cudaSuccess) return false;
+          cc.mid.push_back(y);
+        }
+        if (!pconv::chain_fill(cc.table_host, i - b, L, x, s->bias[i], y, s->n, hi[i], wi[i],
+                               (s->flags & PCONV_RELU) != 0, s->pool[i] != 0, s->status_dev))
+          return false;
+        x = y;
+      }
+      const size_t tb = pconv::chain_table_bytes(e - b);
+      if (cudaMalloc(&cc.table_dev, tb) != cudaSuccess ||
+          cudaMemcpy(cc.table_dev, cc.table_host, tb, cudaMemcpyHostToDevice) != cudaSuccess)
+        return false;
+      const size_t wsb = pconv::chain_workspace_bytes(cc.table_host, e - b);
+      if (wsb > s->ws_bytes) s->ws_bytes = wsb;
+      b = e;
+    }
+  }
+  if (s->ws_bytes) {
+    if (cudaMalloc(&s->ws, s->ws_bytes) != cudaSuccess || cudaMemset(s->ws, 0, s->ws_bytes) != cudaSuccess)
+      return false;
+  }
+  if (!s->chains->empty()) {
+    if (cudaMalloc((void**)&s->sync_dev, 256) != cudaSuccess || cudaMemset(s->sync_dev, 0, 256) != cudaSuccess)
+      return false;
+  }
+  return true;
 }
 
 extern "C" pconv_status pconv_stack_create(const pconv_handle* const* layers,
@@ -382,14 +482,11 @@ extern "C" pconv_status pconv_stack_create(const pconv_handle* const* layers,
   if (e == cudaSuccess) e = cudaMalloc(&s->act[1], max_act);
   if (e == cudaSuccess) e = cudaMalloc(&s->io[0], s->in_bytes);
   if (e == cudaSuccess) e = cudaMalloc(&s->io[1], s->out_bytes);
-  if (e == cudaSuccess && s->ws_bytes) {
-    e = cudaMalloc(&s->ws, s->ws_bytes);
-    if (e == cudaSuccess) e = cudaMemset(s->ws, 0, s->ws_bytes);
-  }
   if (e == cudaSuccess) e = cudaMalloc(&s->status_dev, pconv::kStatusBlockBytes);
   if (e == cudaSuccess) e = cudaMemset(s->status_dev, 0, pconv::kStatusBlockBytes);
   if (e == cudaSuccess) e = cudaMallocHost(&s->status_host, sizeof(int));
   if (e == cudaSuccess) *s->status_host = 0;
+  if (e == cudaSuccess && !build_chains(s)) e = cudaErrorMemoryAllocation;
   if (e != cudaSuccess) {
     cudaGetLastError();
     pconv_stack_free(s);
@@ -409,11 +506,67 @@ extern "C" pconv_status pconv_stack_out_shape(const pconv_stack* s, int* n, int*
   return PCONV_OK;
 }
 
+extern "C" pconv_status pconv_stack_launches(const pconv_stack* s, int* launches) {
+  if (!s || !launches) return PCONV_ERR_NULL;
+  int n = 0, ch = s->h, cw = s->w;
+  for (int i = 0; i < s->n_layers; ++i) {
+    const pconv_stack::Chain* chain = nullptr;
+    if (s->chains)
+      for (const pconv_stack::Chain& c : *s->chains)
+        if (c.begin == i) chain = &c;
+    const int last = chain ? chain->end : i + 1;
+    ++n;
+    for (int k = i; k < last; ++k) {
+      const pconv::DeviceLayer& L = s->layers[k]->d;
+      const unsigned sel_bits = PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED | PCONV_KERNEL_GENERIC_TAPS | PCONV_KERNEL_TENSOR;
+      const bool tensor = (s->flags & PCONV_KERNEL_TENSOR) ||
+                          (!(s->flags & sel_bits) && pconv::tensor_preferred(L, s->n, ch, cw));
+      const bool fuse = s->pool[k] && !(s->flags & PCONV_KERNEL_SIMPLE) && !tensor &&
+                        pconv::tiled_supported(L, s->n, ch, cw);
+      if (!chain && s->pool[k] && !fuse) ++n;      // a max-pool kernel of its own
+      ch = (ch - 1) / L.stride + 1;
+      cw = (cw - 1) / L.stride + 1;
+      if (s->pool[k]) {
+        ch /= 2;
+        cw /= 2;
+      }
+    }
+    i = last - 1;
+  }
+  *launches = n;
+  return PCONV_OK;
+}
+
 extern "C" pconv_status pconv_stack_forward(pconv_stack* s, const void* x, void* y, void* stream) {
   if (!s || !x || !y) return PCONV_ERR_NULL;
   const void* cur = x;
   int ch = s->h, cw = s->w, which = 0;
   for (int i = 0; i < s->n_layers; ++i) {
+    const pconv_stack::Chain* chain = nullptr;
+    if (s->chains)
+      for (const pconv_stack::Chain& c : *s->chains)
+        if (c.begin == i) chain = &c;
+    if (chain) {   // layers [begin, end) in one persistent launch
+      void* dst = (chain->end == s->n_layers) ? y : s->act[which];
+      if (pconv::launch_chain(chain->table_dev, chain->table_host, chain->end - chain->begin, cur, dst, s->ws,
+                              s->ws_bytes, s->sync_dev, (cudaStream_t)stream) != cudaSuccess) {
+        cudaGetLastError();
+        return PCONV_ERR_CUDA;
+      }
+      for (int k = chain->begin; k < chain->end; ++k) {
+        const int st = s->layers[k]->d.stride;
+        ch = (ch - 1) / st + 1;
+        cw = (cw - 1) / st + 1;
+        if (s->pool[k]) {
+          ch /= 2;
+          cw /= 2;
+        }
+      }
+      cur = dst;
+      which ^= 1;
+      i = chain->end - 1;
+      continue;
+    }
     const pconv::DeviceLayer& L = s->layers[i]->d;
     // a pool that follows the layer is fused into the layer's epilogue when a tiled kernel runs it
     // (not when the layer takes the dense tensor-core kernel, which has no pooled epilogue: the
@@ -546,6 +699,7 @@ extern "C" pconv_status pconv_stack_status(pconv_stack* s, int* where) {
   // the abandoned launch may have left partial sums and tickets in the workspace
   if (cudaMemset(s->status_dev, 0, sizeof(int)) != cudaSuccess ||
       (s->ws && cudaMemset(s->ws, 0, s->ws_bytes) != cudaSuccess) ||
+      (s->sync_dev && cudaMemset(s->sync_dev, 0, 256) != cudaSuccess) ||
       cudaDeviceSynchronize() != cudaSuccess) {
     cudaGetLastError();
     return PCONV_ERR_CUDA;

@@ -34,6 +34,7 @@
 // previous kernel finishes, and griddepcontrol.wait precedes the first access to activations.
 #include <cuda_fp16.h>
 
+#include <cstring>
 #include <type_traits>
 #ifdef PCONV_DEV
 #include <cstdlib>
@@ -176,7 +177,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* er
 //   11 / 12 cycles warp 0 of CTA (0,0,0) spent waiting for chunks / working on them, 13 its chunks.
 #ifdef PCONV_DEV
 #define PCONV_MARK(i)                                                         \
-  if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) { \
+  if (threadIdx.x == 0 && bp.x == 0 && bp.y == 0 && bp.z == 0) { \
     unsigned long long t_;                                                    \
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                    \
     trace_words(L)[i] = t_;                                                   \
@@ -944,14 +945,56 @@ __device__ __forceinline__ void finalize_outputs(const Geo& g, const LaneOut& lo
   }
 }
 
+// Where a CTA stands in a layer's grid (a chain kernel gives every layer its own virtual grid).
+struct BlockPos {
+  int x, y, z, gx;
+};
+// A layer inside a chain kernel (several layers of a stack in one persistent launch, one CTA per
+// SM): Tensor Memory is allocated once by the chain kernel and kept across layers; a CTA that has
+// finished its part of a layer counts itself in `sync` and goes on to the next layer's set-up
+// and weight blocks at once, and waits for `target` arrivals -- every CTA's part of the previous
+// layer -- only where a stand-alone kernel waits for the previous kernel of the stream.
+struct ChainCtx {
+  unsigned int* sync;     // nullptr: a stand-alone launch of one layer
+  unsigned int target;    // 0: the chain's first layer (waits for the previous kernel instead)
+  int own_tmem;           // 1: the body allocates and releases Tensor Memory (stand-alone launch)
+  int reinit;             // 1: the CTA's barriers were used by an earlier layer: invalidate them first
+};
+constexpr uint32_t kGridSpinLimit = 1u << 21;
+
+// What a role does before it first touches activations, workspace or tickets: wait for the
+// previous kernel of the stream or, inside a chain, for the previous layer.  Bounded: false (and
+// wait id 9 recorded) if the other CTAs never arrive.
+__device__ __forceinline__ bool dependency_wait(const ChainCtx& cc, int lane, int* err) {
+  if (cc.sync == nullptr || cc.target == 0) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    return true;
+  }
+  uint32_t ok = 1;
+  if (lane == 0) {
+    uint32_t it = 0, seen = 0;
+    for (;;) {
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(cc.sync) : "memory");
+      if (seen >= cc.target) break;
+      if (++it > kGridSpinLimit) {
+        atomicCAS(err, 0, 9);
+        ok = 0;
+        break;
+      }
+      __nanosleep(40);
+    }
+  }
+  ok = __shfl_sync(0xffffffffu, ok, 0);
+  return ok != 0;
+}
+
 template <int S, bool GENERIC, bool WIDE>
-__global__ void __launch_bounds__(cta_threads(GENERIC), 1)
-tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
-             const float* __restrict__ bias, void* __restrict__ y, float* __restrict__ ws,
-             int* __restrict__ counters) {
+__device__ __forceinline__ void tiled_body(const DeviceLayer& L, const Geo& g, const void* __restrict__ x,
+                                           const float* __restrict__ bias, void* __restrict__ y,
+                                           float* __restrict__ ws, int* __restrict__ counters,
+                                           unsigned char* smem, const BlockPos bp, const ChainCtx cc) {
   constexpr int kCW = consumer_warps(GENERIC);
   constexpr int kThreads = cta_threads(GENERIC);
-  extern __shared__ __align__(16) unsigned char smem[];
   const uint32_t sbase = smem_u32(smem);
   const int tid = threadIdx.x, lane = tid & 31;
   // broadcast from lane 0: tells the compiler that everything derived from it is warp-uniform
@@ -964,18 +1007,24 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   PCONV_MARK_MAX(8)
   // The next kernel of the stream may start its own set-up while this one runs (it waits for this
   // grid to finish before it touches activations, see below).
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (cc.own_tmem) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (tid < kCW) unit_ctr[tid] = 0;
   const uint32_t coop_bar = sbase + 8 * 2 * kMaxStages + 16 + 64;   // kMaxCoop barriers
   if (tid == 0) {
+    // every barrier is initialised, used or not, so that a chain's next layer may invalidate
+    // and initialise them all again (its ring may be deeper)
+    if (cc.reinit)
+      for (int j = 0; j < 2 * kMaxStages + 2 + 8 + kMaxCoop; ++j)
+        if (j < 2 * kMaxStages || j >= 2 * kMaxStages + 10)
+          asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(sbase + 8 * j) : "memory");
     for (int j = 0; j < kMaxCoop; ++j) mbar_init(coop_bar + 8 * j, 32 * kCW);
-    for (int s = 0; s < g.stages; ++s) {
+    for (int s = 0; s < kMaxStages; ++s) {
       mbar_init(sbase + 8 * s, 32 * kProducerWarps);
       mbar_init(sbase + 8 * (kMaxStages + s), kCW / (GENERIC ? 1 : g.zs));
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (!GENERIC && warp == 0) {  // the whole TMEM of this SM (one CTA per SM by shared-memory use)
+  if (!GENERIC && warp == 0 && cc.own_tmem) {  // the whole TMEM of this SM (one CTA per SM by shared-memory use)
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                      smem_u32((const void*)tmem_base_s)),
                  "n"(kTmemCols)
@@ -983,7 +1032,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   for (int i = tid; i < 2 * g.pairs; i += kThreads) {
-    const long long q = (long long)blockIdx.x * (2 * g.pairs) + i;
+    const long long q = (long long)bp.x * (2 * g.pairs) + i;
     SubTile t;
     t.valid = q < g.q_total;
     const int qq = t.valid ? (int)q : 0;
@@ -995,14 +1044,14 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
     t.x0 = (rem - tyi * g.tx) * g.tw;
     tab[i] = t;
   }
-  const int k0 = blockIdx.z * g.cps;                       // this CTA's chunk range
+  const int k0 = bp.z * g.cps;                             // this CTA's chunk range
   const int nk = min(L.n_chunks, k0 + g.cps) - k0;
   // Block descriptors of the CTA's groups and chunks, two 16-byte words each:
   // {first kernel record, records, code offset, code bytes}, {-, -, first channel, -}.
   uint4* desc = reinterpret_cast<uint4*>(smem + g.desc_off);
   for (int i = tid; i < g.ng * g.cps; i += kThreads) {
     const int j = i / g.cps, kk = i - j * g.cps;
-    const int gj = blockIdx.y * g.ng + j;
+    const int gj = bp.y * g.ng + j;
     uint4 d0 = make_uint4(0u, 0u, 0u, 0u), d1 = d0;
     if (gj < L.n_groups && kk < nk) {
       const uint4* src = reinterpret_cast<const uint4*>(L.blocks + (size_t)gj * L.n_chunks + k0 + kk);
@@ -1036,7 +1085,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
     z = warp >> 2;
   }
   const int wyi = unit % g.wys, wgi = unit / g.wys;
-  const int gi = blockIdx.y * g.ng + wgi;
+  const int gi = bp.y * g.ng + wgi;
   const bool active = (wyi < g.wy) && (gi < L.n_groups);
   const int slot = wyi * g.sw + lane / g.tw;  // sub-tile pair of this lane
   const int col = lane % g.tw;
@@ -1073,8 +1122,8 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
         pre[i] = raw_elem<S>(g, e < n_elem ? e : 0);
         if (e >= n_elem) pre[i].dst = kSkipElem;
       }
-      asm volatile("griddepcontrol.wait;" ::: "memory");
-      produce_raw_stream<S>(L, g, (const __half*)x, tab, pre, desc, codes, sbase, k0, nk, ptid);
+      if (dependency_wait(cc, lane, L.err))
+        produce_raw_stream<S>(L, g, (const __half*)x, tab, pre, desc, codes, sbase, k0, nk, ptid);
     } else {
       precompute_elems<S>(pre, L, g, tab, ptid);
       // the weight records and codes of the first ring-full of chunks do not depend on the previous
@@ -1088,8 +1137,9 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
         // landed: arrive now, so that the barrier does not also wait for the later chunks' blocks
         if (kk < n_coop && !PCONV_WITHHELD(kk, ptid)) cp_async_arrive(sbase + 8 * kk);
       }
-      asm volatile("griddepcontrol.wait;" ::: "memory");
-      if (g.is_half) {
+      if (!dependency_wait(cc, lane, L.err)) {
+        // the previous layer never completed: nothing more is staged, the consumers give up too
+      } else if (g.is_half) {
         produce_half_stream<S>(L, g, (const __half*)x, tab, pre, desc, codes, sbase, k0, nk, n_early, ptid);
       } else {
         for (int kk = n_coop; kk < nk; ++kk) {
@@ -1114,10 +1164,10 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
       for (int a = 0; a < kGroup; ++a) tmem_st8_zero(tq + a * 8);
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
     }
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    ok = dependency_wait(cc, lane, L.err);
     // (each consumer thread arrives on the chunk's own barrier when its copies for that chunk
     // have landed; a warp waits for that barrier as well as for the producers' before the chunk)
-    for (int kk = 0; kk < n_coop; ++kk) {
+    for (int kk = 0; ok && kk < n_coop; ++kk) {
       fill_chunk_x<S>(L, g, (const float*)x, tab, sbase + g.stage_off + kk * g.stage_bytes, k0 + kk,
                       warp * 32 + lane, 32 * kCW);
       cp_async_arrive(coop_bar + 8 * kk);
@@ -1194,7 +1244,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
 #endif
     }
 #ifdef PCONV_DEV
-    if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {
+    if (threadIdx.x == 0 && bp.x == 0 && bp.y == 0 && bp.z == 0) {
       trace_words(L)[11] = (unsigned long long)t_wait;
       trace_words(L)[12] = (unsigned long long)t_work;
       trace_words(L)[13] = (unsigned long long)nk;
@@ -1236,7 +1286,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
       } else {
         // this lane's floats in the warp's part of the tile's workspace: [tile][warp][slot][lane][8]
         const int spw = kGroup / (GENERIC ? 1 : g.zs);   // slots a warp writes out
-        float* wsl = ws + ((((size_t)blockIdx.y * gridDim.x + blockIdx.x) * kCW + warp) * spw * 32 + lane) * 8;
+        float* wsl = ws + ((((size_t)bp.y * bp.gx + bp.x) * kCW + warp) * spw * 32 + lane) * 8;
         write_outputs<GENERIC, 1, false, false>(g, lo, lp, y, wsl, acc, orng, my_o, my_b);
         PCONV_MARK(4)
         PCONV_MARK_MAX(10)
@@ -1247,7 +1297,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
         // tile spreads over the CTAs that share it.
         __threadfence();
         __syncwarp();
-        int* ticket = counters + ((size_t)blockIdx.y * gridDim.x + blockIdx.x) * kCW + warp;
+        int* ticket = counters + ((size_t)bp.y * bp.gx + bp.x) * kCW + warp;
         int t = 0;
         if (lane == 0) {
           t = atomicAdd(ticket, 1);
@@ -1271,11 +1321,103 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     PCONV_MARK(6)
-    if (warp == 0)
+    if (warp == 0 && cc.own_tmem)
       asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols)
                    : "memory");
   }
   PCONV_MARK_MAX(7)
+}
+
+template <int S, bool GENERIC, bool WIDE>
+__global__ void __launch_bounds__(cta_threads(GENERIC), 1)
+tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
+             const float* __restrict__ bias, void* __restrict__ y, float* __restrict__ ws,
+             int* __restrict__ counters) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  BlockPos bp;
+  bp.x = (int)blockIdx.x;
+  bp.y = (int)blockIdx.y;
+  bp.z = (int)blockIdx.z;
+  bp.gx = (int)gridDim.x;
+  ChainCtx cc;
+  cc.sync = nullptr;
+  cc.target = 0;
+  cc.own_tmem = 1;
+  cc.reinit = 0;
+  tiled_body<S, GENERIC, WIDE>(L, g, x, bias, y, ws, counters, smem, bp, cc);
+}
+
+// One layer of a chain, as the chain kernel reads it from device memory.
+struct ChainLayer {
+  DeviceLayer L;
+  Geo g;
+  const void* x;
+  const float* bias;
+  void* y;
+  int gx, gy, gz;     // the layer's own grid: CTA c works at (c % gx, c / gx % gy, c / (gx * gy)) if c < gx * gy * gz
+  int pad;
+};
+
+// Several consecutive layers of a stack in one persistent launch (canonical pattern sets, stride
+// 1; one CTA per SM, every layer's grid no larger than the launch's).  `sync` = {arrivals,
+// CTAs that have left}: both zero before the launch and zero again after it.
+__global__ void __launch_bounds__(cta_threads(false), 1)
+tiled_chain_kernel(const ChainLayer* __restrict__ layers, int n_layers, const void* __restrict__ x_first,
+                   void* __restrict__ y_last, float* __restrict__ ws, int* __restrict__ counters,
+                   unsigned int* __restrict__ sync) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  const int n_ctas = (int)gridDim.x;
+  const int cta = (int)blockIdx.x;
+  const int warp = __shfl_sync(0xffffffffu, (int)threadIdx.x >> 5, 0);
+  volatile uint32_t* tmem_base_s = reinterpret_cast<volatile uint32_t*>(smem + 8 * 2 * kMaxStages);
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (warp == 0) {   // the whole TMEM of this SM, kept for every layer of the chain
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32((const void*)tmem_base_s)),
+                 "n"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  bool used = false;     // this CTA's barriers have been initialised by an earlier layer
+  for (int li = 0; li < n_layers; ++li) {
+    ChainLayer cl = layers[li];
+    if (li == 0) cl.x = x_first;                 // the chain's input and output are the caller's
+    if (li == n_layers - 1) cl.y = y_last;
+    ChainCtx cc;
+    cc.sync = sync;
+    cc.target = (unsigned int)li * (unsigned int)n_ctas;
+    cc.own_tmem = 0;
+    cc.reinit = used ? 1 : 0;
+    if (cta < cl.gx * cl.gy * cl.gz) {     // (a CTA outside a layer's grid only counts itself in)
+      BlockPos bp;
+      bp.gx = cl.gx;
+      bp.x = cta % cl.gx;
+      bp.y = (cta / cl.gx) % cl.gy;
+      bp.z = cta / (cl.gx * cl.gy);
+      tiled_body<1, false, false>(cl.L, cl.g, cl.x, cl.bias, cl.y, ws, counters, smem, bp, cc);
+      used = true;
+    } else if (warp == 0) {
+      // (in step with the others all the same: its arrival for this layer must not be counted
+      // before the previous layer is complete)
+      dependency_wait(cc, (int)threadIdx.x & 31, cl.L.err);
+    }
+    if (threadIdx.x == 0 && li + 1 < n_layers) {   // this CTA's part of the layer is complete and visible
+      __threadfence();
+      atomicAdd(sync, 1u);
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(*tmem_base_s), "n"(kTmemCols)
+                 : "memory");
+  if (threadIdx.x == 0) {                 // the last CTA to leave puts the counters back to zero
+    __threadfence();
+    if (atomicAdd(sync + 1, 1u) == (unsigned int)n_ctas - 1u) {
+      sync[0] = 0u;
+      sync[1] = 0u;
+    }
+  }
 }
 
 // Places descriptors, the raw ring (if any) and the stages for `cps` chunks per CTA, and picks the
@@ -1575,6 +1717,102 @@ cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias,
   if (generic_taps) return launch_one<2, true, false>(L, g, x, bias, y, wsf, counters, stream);
   return wide ? launch_one<2, false, true>(L, g, x, bias, y, wsf, counters, stream)
               : launch_one<2, false, false>(L, g, x, bias, y, wsf, counters, stream);
+}
+
+// ---- chains ---------------------------------------------------------------------------------------
+// Whether a layer may be part of a chain kernel for this input shape: fp32 or fp16 storage with
+// stride 1 and a canonical pattern set (the chain kernel is one instantiation), and a launch plan
+// of at most one CTA per SM.  *ctas / *ws_bytes (optional) receive the plan's CTA count and
+// workspace need.
+bool chain_layer_ok(const DeviceLayer& L, int n, int h, int w, bool pool, long long* ctas) {
+  if (!L.codes_s || L.wide_codes || L.stride != 1) return false;
+  Geo g;
+  if (!make_geo<false>(L, n, h, w, true, &g)) return false;
+  if (pool && (g.h_out < 2 || g.w_out < 2)) return false;
+  const long long c = geo_tiles(L, g) * g.ks;
+  if (ctas) *ctas = c;
+  return c <= device_sm_count();
+}
+
+size_t chain_table_bytes(int n_layers) { return (size_t)n_layers * sizeof(ChainLayer); }
+
+// Fills entry `index` of a chain's table (HOST memory, `table` has chain_table_bytes(n) bytes):
+// the layer, its geometry for this input shape (with the channel split the workspace allows) and
+// its buffers (x / y of the chain's first / last layer are given at launch).
+bool chain_fill(void* table, int index, const DeviceLayer& L, const void* x, const float* bias, void* y, int n,
+                int h, int w, bool relu, bool pool, int* status_dev) {
+  ChainLayer& cl = reinterpret_cast<ChainLayer*>(table)[index];
+  std::memset(&cl, 0, sizeof(cl));
+  cl.L = L;
+  if (status_dev) cl.L.err = status_dev;
+  if (!make_geo<false>(L, n, h, w, true, &cl.g)) return false;
+  cl.g.relu = relu ? 1 : 0;
+  if (pool) {
+    cl.g.pool = 1;
+    cl.g.h_y = cl.g.h_out / 2;
+    cl.g.w_y = cl.g.w_out / 2;
+  }
+  cl.x = x;
+  cl.bias = bias;
+  cl.y = y;
+  cl.gx = (int)(((long long)cl.g.q_total + 2 * cl.g.pairs - 1) / (2 * cl.g.pairs));
+  cl.gy = (L.n_groups + cl.g.ng - 1) / cl.g.ng;
+  cl.gz = cl.g.ks;
+  return true;
+}
+
+// Workspace a chain needs: the largest split layer's sums, then tickets for one grid of CTAs.
+size_t chain_workspace_bytes(const void* table_host, int n_layers) {
+  const ChainLayer* t = reinterpret_cast<const ChainLayer*>(table_host);
+  size_t sums_max = 0;
+  for (int i = 0; i < n_layers; ++i)
+    if (t[i].g.ks > 1) {
+      const size_t need = split_sums_bytes(t[i].L, t[i].g);
+      if (need > sums_max) sums_max = need;
+    }
+  if (!sums_max) return 0;
+  return ((sums_max + 255) & ~(size_t)255) + (((size_t)device_sm_count() * consumer_warps(false) * 4 + 255) & ~(size_t)255);
+}
+
+// Launches a chain: `table_dev` is the DEVICE copy of a filled table, `table_host` the host one
+// (for the launch geometry); ws = the stack's channel-split workspace (sums, tickets), sync = two
+// zeroed counters.
+cudaError_t launch_chain(const void* table_dev, const void* table_host, int n_layers, const void* x_first,
+                         void* y_last, void* ws, size_t ws_bytes, unsigned int* sync, cudaStream_t stream) {
+  const ChainLayer* t = reinterpret_cast<const ChainLayer*>(table_host);
+  long long ctas = 0;
+  int smem = 0;
+  size_t sums_max = 0;
+  for (int i = 0; i < n_layers; ++i) {
+    const long long c = (long long)t[i].gx * t[i].gy * t[i].gz;
+    if (c > ctas) ctas = c;
+    const int sm = t[i].g.stage_off + t[i].g.stages * t[i].g.stage_bytes;
+    if (sm > smem) smem = sm;
+    if (t[i].g.ks > 1) {
+      const size_t need = split_sums_bytes(t[i].L, t[i].g);
+      if (need > sums_max) sums_max = need;
+    }
+  }
+  if (ctas < 1 || ctas > device_sm_count()) return cudaErrorInvalidValue;
+  // every layer of the chain finds its tickets behind the largest layer's sums
+  const size_t tick_off = (sums_max + 255) & ~(size_t)255;
+  if (sums_max && (!ws || ws_bytes < tick_off + (size_t)device_sm_count() * consumer_warps(false) * 4))
+    return cudaErrorInvalidValue;
+  if (smem < 120 * 1024) smem = 120 * 1024;
+  cudaError_t e = cudaFuncSetAttribute(tiled_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)ctas, 1, 1);
+  cfg.blockDim = dim3(cta_threads(false), 1, 1);
+  cfg.dynamicSmemBytes = (size_t)smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, tiled_chain_kernel, reinterpret_cast<const ChainLayer*>(table_dev), n_layers,
+                            x_first, y_last, (float*)ws, (int*)((char*)ws + tick_off), sync);
 }
 
 #ifdef PCONV_DEV

@@ -142,6 +142,14 @@ bool tiled_plan(const DeviceLayer& L, int n, int h, int w, bool generic_taps, bo
 #ifdef PCONV_DEV
 cudaError_t dev_set_withhold(int chunk, unsigned spin_limit);   // see pconv_dev.h
 #endif
+// chains: several consecutive layers of a stack in one persistent launch (kernels_tiled.cu)
+bool chain_layer_ok(const DeviceLayer& L, int n, int h, int w, bool pool, long long* ctas);
+size_t chain_table_bytes(int n_layers);
+bool chain_fill(void* table_host, int index, const DeviceLayer& L, const void* x, const float* bias, void* y,
+                int n, int h, int w, bool relu, bool pool, int* status_dev);
+size_t chain_workspace_bytes(const void* table_host, int n_layers);
+cudaError_t launch_chain(const void* table_dev, const void* table_host, int n_layers, const void* x_first,
+                         void* y_last, void* ws, size_t ws_bytes, unsigned int* sync, cudaStream_t stream);
 cudaError_t launch_maxpool(const void* x, void* y, int n, int c, int h, int w, int storage,
                            cudaStream_t stream);
 }  // namespace pconv
