@@ -402,6 +402,27 @@ def run_ours(args):
     # (not bit-equal: the grouping of the fp32 partial sums varies from launch to launch)
     graph_same = bool(torch.allclose(y_graph, y, rtol=1e-4, atol=1e-6))
 
+    # ---- the same step as chains: runs of layers in one persistent kernel (PCONV_CHAIN) --------
+    chain_stack = B.Stack(conv_layers, pools, 1, spec0.h, spec0.w, B.RELU | B.CHAIN)
+    y_chain = torch.empty_like(y)
+    for _ in range(args.warmup):
+        chain_stack.forward(x, y_chain)
+    torch.cuda.synchronize()
+    cev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+           for _ in range(args.steps)]
+    for e0, e1 in cev:
+        flush.zero_()
+        e0.record()
+        chain_stack.forward(x, y_chain)
+        e1.record()
+    torch.cuda.synchronize()
+    chain_ms = sum(e0.elapsed_time(e1) for e0, e1 in cev) / args.steps
+    chain_same = bool(torch.allclose(y_chain, y, rtol=1e-4, atol=1e-6))
+    chain_launches = chain_stack.launches()
+    if chain_stack.status()[0]:
+        raise SystemExit("device reported an abandoned wait in the chained stack")
+    chain_stack.close()
+
     # ---- per-kernel pass: the dominant kernel's launches timed one by one ------------------------
     acts = []
     a = x
@@ -487,9 +508,13 @@ def run_ours(args):
                     "ms_per_step": e2e_ms, "h2d_bytes_per_step": int(x_host.numel() * 4),
                     "d2h_bytes_per_step": int(y_host.numel() * 4)},
             # one launch per conv layer: the four max-pools are fused into the epilogue of the layer before
-            "gpu_launches": args.steps * len(conv_layers),
+            "gpu_launches": args.steps * stack.launches(),
             "graph_replay": {"ms_per_step": graph_ms, "value": flops / (graph_ms * 1e-3) / 1e12,
                              "unit": "TFLOP/s", "matches_eager_output": graph_same},
+            # not the default: one persistent kernel per run of single-wave layers
+            "chained": {"ms_per_step": chain_ms, "value": flops / (chain_ms * 1e-3) / 1e12,
+                        "unit": "TFLOP/s", "launches_per_step": chain_launches,
+                        "matches_eager_output": chain_same},
             "roofline": {"bound": "alu", "kernel": "tiled_kernel (13 conv launches per step)",
                          "achieved": achieved, "peak": ALU_PEAK_TFLOPS, "unit": "TFLOP/s",
                          "frac": achieved / ALU_PEAK_TFLOPS,

@@ -14,7 +14,7 @@ LIB_PATH = os.path.join(HERE, "libpconv.so")
 
 OK = 0
 F32, F16 = 0, 1
-RELU, STRICT4, POOL2X2, REPRODUCIBLE, NO_CHAIN = 1, 2, 4, 8, 0x10
+RELU, STRICT4, POOL2X2, REPRODUCIBLE, CHAIN = 1, 2, 4, 8, 0x10
 KERNEL_SIMPLE, KERNEL_TILED, KERNEL_GENERIC_TAPS, KERNEL_TENSOR = 0x100, 0x200, 0x400, 0x800
 MAX_PATTERNS = 16
 

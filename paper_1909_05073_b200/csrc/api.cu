@@ -121,7 +121,7 @@ static pconv_status forward_impl(const pconv_handle* h, const void* x, const flo
   if (!h || !x || !y) return PCONV_ERR_NULL;
   if (n < 0 || h_in <= 0 || w_in <= 0) return PCONV_ERR_SHAPE;
   const unsigned known =
-      PCONV_RELU | PCONV_POOL2X2 | PCONV_REPRODUCIBLE | PCONV_NO_CHAIN | PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED |
+      PCONV_RELU | PCONV_POOL2X2 | PCONV_REPRODUCIBLE | PCONV_CHAIN | PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED |
       PCONV_KERNEL_GENERIC_TAPS | PCONV_KERNEL_TENSOR;
   if (flags & ~known) return PCONV_ERR_UNSUPPORTED;
   const unsigned sel = flags & (PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED | PCONV_KERNEL_GENERIC_TAPS |
@@ -348,7 +348,7 @@ static bool build_chains(pconv_stack* s) {
   if (!s->chains) return false;
   const unsigned sel_bits = PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED | PCONV_KERNEL_GENERIC_TAPS | PCONV_KERNEL_TENSOR;
   const size_t es = (s->storage == PCONV_F16) ? 2 : 4;
-  if (!(s->flags & (sel_bits | PCONV_REPRODUCIBLE | PCONV_NO_CHAIN))) {
+  if ((s->flags & PCONV_CHAIN) && !(s->flags & (sel_bits | PCONV_REPRODUCIBLE))) {
     // shapes of every layer's input and output
     std::vector<int> hi(s->n_layers), wi(s->n_layers);
     int ch = s->h, cw = s->w;

@@ -965,23 +965,46 @@ constexpr uint32_t kGridSpinLimit = 1u << 21;
 // What a role does before it first touches activations, workspace or tickets: wait for the
 // previous kernel of the stream or, inside a chain, for the previous layer.  Bounded: false (and
 // wait id 9 recorded) if the other CTAs never arrive.
-__device__ __forceinline__ bool dependency_wait(const ChainCtx& cc, int lane, int* err) {
+__device__ __forceinline__ bool dependency_wait(const ChainCtx& cc, int lane, int warp, unsigned char* smem,
+                                                int* err) {
   if (cc.sync == nullptr || cc.target == 0) {
     asm volatile("griddepcontrol.wait;" ::: "memory");
     return true;
   }
+  // One warp of the CTA polls the grid's counter (every warp of every CTA polling the same word
+  // kept the arrivals themselves waiting); the others watch a word in shared memory that it sets.
+  volatile uint32_t* seen_s = reinterpret_cast<volatile uint32_t*>(smem + 8 * 2 * kMaxStages + 4);
   uint32_t ok = 1;
   if (lane == 0) {
     uint32_t it = 0, seen = 0;
-    for (;;) {
-      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(cc.sync) : "memory");
-      if (seen >= cc.target) break;
-      if (++it > kGridSpinLimit) {
-        atomicCAS(err, 0, 9);
-        ok = 0;
-        break;
+    if (warp == 0) {
+      for (;;) {
+        asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(cc.sync) : "memory");
+        if (seen >= cc.target) break;
+        if (++it > kGridSpinLimit) {
+          atomicCAS(err, 0, 9);
+          ok = 0;
+          seen = 0xFFFFFFFFu;      // releases the CTA's other warps, which then find the status set
+          break;
+        }
+        __nanosleep(100);
       }
-      __nanosleep(40);
+      // acquire once, after the count has been seen (an acquiring load in the polling loop costs
+      // the SM an L1 invalidation per try), then tell the CTA's other warps
+      asm volatile("fence.acq_rel.gpu;" ::: "memory");
+      *seen_s = seen;
+    } else {
+      for (;;) {
+        seen = *seen_s;
+        if (seen >= cc.target) break;
+        if (++it > (kGridSpinLimit << 2)) {
+          atomicCAS(err, 0, 9);
+          break;
+        }
+        __nanosleep(40);
+      }
+      if (seen == 0xFFFFFFFFu || seen < cc.target) ok = 0;
+      asm volatile("fence.acq_rel.cta;" ::: "memory");   // order this warp's reads after the flag's value
     }
   }
   ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -1122,7 +1145,7 @@ __device__ __forceinline__ void tiled_body(const DeviceLayer& L, const Geo& g, c
         pre[i] = raw_elem<S>(g, e < n_elem ? e : 0);
         if (e >= n_elem) pre[i].dst = kSkipElem;
       }
-      if (dependency_wait(cc, lane, L.err))
+      if (dependency_wait(cc, lane, warp, smem, L.err))
         produce_raw_stream<S>(L, g, (const __half*)x, tab, pre, desc, codes, sbase, k0, nk, ptid);
     } else {
       precompute_elems<S>(pre, L, g, tab, ptid);
@@ -1137,7 +1160,7 @@ __device__ __forceinline__ void tiled_body(const DeviceLayer& L, const Geo& g, c
         // landed: arrive now, so that the barrier does not also wait for the later chunks' blocks
         if (kk < n_coop && !PCONV_WITHHELD(kk, ptid)) cp_async_arrive(sbase + 8 * kk);
       }
-      if (!dependency_wait(cc, lane, L.err)) {
+      if (!dependency_wait(cc, lane, warp, smem, L.err)) {
         // the previous layer never completed: nothing more is staged, the consumers give up too
       } else if (g.is_half) {
         produce_half_stream<S>(L, g, (const __half*)x, tab, pre, desc, codes, sbase, k0, nk, n_early, ptid);
@@ -1164,7 +1187,7 @@ __device__ __forceinline__ void tiled_body(const DeviceLayer& L, const Geo& g, c
       for (int a = 0; a < kGroup; ++a) tmem_st8_zero(tq + a * 8);
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
     }
-    ok = dependency_wait(cc, lane, L.err);
+    ok = dependency_wait(cc, lane, warp, smem, L.err);
     // (each consumer thread arrives on the chunk's own barrier when its copies for that chunk
     // have landed; a warp waits for that barrier as well as for the producers' before the chunk)
     for (int kk = 0; ok && kk < n_coop; ++kk) {
@@ -1378,11 +1401,13 @@ tiled_chain_kernel(const ChainLayer* __restrict__ layers, int n_layers, const vo
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  if (threadIdx.x == 0) *reinterpret_cast<volatile uint32_t*>(smem + 8 * 2 * kMaxStages + 4) = 0u;
   bool used = false;     // this CTA's barriers have been initialised by an earlier layer
   for (int li = 0; li < n_layers; ++li) {
-    ChainLayer cl = layers[li];
-    if (li == 0) cl.x = x_first;                 // the chain's input and output are the caller's
-    if (li == n_layers - 1) cl.y = y_last;
+    // (read in place: a private copy of the layer's 400 bytes cost registers all through the body)
+    const ChainLayer& cl = layers[li];
+    const void* xl = (li == 0) ? x_first : cl.x;              // the chain's input and output are the caller's
+    void* yl = (li == n_layers - 1) ? y_last : cl.y;
     ChainCtx cc;
     cc.sync = sync;
     cc.target = (unsigned int)li * (unsigned int)n_ctas;
@@ -1394,12 +1419,12 @@ tiled_chain_kernel(const ChainLayer* __restrict__ layers, int n_layers, const vo
       bp.x = cta % cl.gx;
       bp.y = (cta / cl.gx) % cl.gy;
       bp.z = cta / (cl.gx * cl.gy);
-      tiled_body<1, false, false>(cl.L, cl.g, cl.x, cl.bias, cl.y, ws, counters, smem, bp, cc);
+      tiled_body<1, false, false>(cl.L, cl.g, xl, cl.bias, yl, ws, counters, smem, bp, cc);
       used = true;
     } else if (warp == 0) {
       // (in step with the others all the same: its arrival for this layer must not be counted
       // before the previous layer is complete)
-      dependency_wait(cc, (int)threadIdx.x & 31, cl.L.err);
+      dependency_wait(cc, (int)threadIdx.x & 31, 0, smem, cl.L.err);
     }
     if (threadIdx.x == 0 && li + 1 < n_layers) {   // this CTA's part of the layer is complete and visible
       __threadfence();

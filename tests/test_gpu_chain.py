@@ -1,7 +1,7 @@
-"""Chains: a stack runs consecutive layers whose launch plans are single waves of CTAs (batch-1
-inference) as ONE persistent kernel -- Tensor Memory and the CTAs stay, layers are crossed on a
-grid-wide count.  The result must be the oracle's, the same as with one launch per layer
-(PCONV_NO_CHAIN), and the counters must be back at zero so that the next forward works."""
+"""Chains: with PCONV_CHAIN a stack runs consecutive layers whose launch plans are single waves of
+CTAs (batch-1 inference) as ONE persistent kernel -- Tensor Memory and the CTAs stay, layers are
+crossed on a grid-wide count.  The result must be the oracle's, the same as with one launch per
+layer (the default), and the counters must be back at zero so that the next forward works."""
 import numpy as np
 import pytest
 import torch
@@ -57,8 +57,8 @@ def test_chain_matches_the_oracle_and_the_layer_by_layer_stack(case):
     pools = [s.pool_after for s in specs]
     dt = torch.float16 if storage == "f16" else torch.float32
     xt = torch.from_numpy(x).cuda().to(dt)
-    chained = B.Stack(layers, pools, n, specs[0].h, specs[0].w, B.RELU)
-    plain = B.Stack(layers, pools, n, specs[0].h, specs[0].w, B.RELU | B.NO_CHAIN)
+    chained = B.Stack(layers, pools, n, specs[0].h, specs[0].w, B.RELU | B.CHAIN)
+    plain = B.Stack(layers, pools, n, specs[0].h, specs[0].w, B.RELU)
     assert plain.launches() == len(specs)
     assert chained.launches() < len(specs), "no chain was formed for a batch-1 stack of small layers"
     for rep in range(3):                      # the counters must come back to zero every time
@@ -78,7 +78,7 @@ def test_chain_matches_the_oracle_and_the_layer_by_layer_stack(case):
 def test_chain_inside_a_captured_graph_and_through_the_host_entry_point():
     specs = [synth.LayerSpec("a", 16, 32, 14, 14, 1, 0.4), synth.LayerSpec("b", 32, 32, 14, 14, 1, 0.4)]
     layers, x, ref = _stack_case(specs, 1, "f32", 77)
-    stack = B.Stack(layers, [False, False], 1, 14, 14, B.RELU)
+    stack = B.Stack(layers, [False, False], 1, 14, 14, B.RELU | B.CHAIN)
     assert stack.launches() == 1
     side = torch.cuda.Stream()
     y = np.empty(stack.out_shape, np.float32)

@@ -86,6 +86,42 @@ def test_abandoned_wait_in_the_channel_split_path_then_cleared_workspace():
     layer.close()
 
 
+def test_chain_kernel_reports_an_abandoned_wait_and_recovers():
+    """The same inside a chain (several layers in one persistent kernel): the layer whose chunk
+    never arrives gives up, the grid-wide crossing still completes (every CTA counts itself in,
+    finished or not), the launch ends, and after pconv_stack_status the stack works again."""
+    specs = [synth.LayerSpec("a", 16, 32, 14, 14, 1, 0.5), synth.LayerSpec("b", 32, 32, 14, 14, 1, 0.5),
+             synth.LayerSpec("c", 32, 16, 14, 14, 1, 0.5)]
+    ws, layers = [], []
+    for i, s in enumerate(specs):
+        w, b, _ = synth.gen_weights(s, 60 + i)
+        ws.append((w, b))
+        layers.append(B.Layer(w, synth.PATTERNS8, 1, B.F32, b))
+    x = synth.gen_input(specs[0], 1, 60)
+    ref = x
+    for w, b in ws:
+        ref = oracle.conv3x3(ref, w, b, 1, True)
+    stack = B.Stack(layers, [False] * 3, 1, 14, 14, B.RELU | B.CHAIN)
+    assert stack.launches() == 1
+    xt = torch.from_numpy(x).cuda()
+    y = torch.empty(stack.out_shape, device="cuda")
+    stack.forward(xt, y)
+    torch.cuda.synchronize()
+    check_close(y.cpu().numpy(), ref, "f32", "chain before")
+    _arm(1)
+    stack.forward(xt, y)
+    torch.cuda.synchronize()
+    _disarm()
+    status, where = stack.status()
+    assert status == TIMEOUT and where in (1, 2, 3, 9)
+    assert stack.status() == (0, 0)
+    y.fill_(float("nan"))
+    stack.forward(xt, y)
+    torch.cuda.synchronize()
+    check_close(y.cpu().numpy(), ref, "f32", "chain after")
+    stack.close()
+
+
 def test_stack_host_entry_point_reports_the_abandoned_wait():
     specs = [synth.LayerSpec("a", 16, 32, 12, 12, 1, 0.5, pool_after=True),
              synth.LayerSpec("b", 32, 32, 6, 6, 1, 0.5)]
