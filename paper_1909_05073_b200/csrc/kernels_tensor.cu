@@ -23,14 +23,15 @@
 //    moved by one row of core matrices.  Nothing is ever im2col'ed in global memory.
 //  * B operand (weights): the packer writes, per (filter tile, 16-channel step), the nine
 //    zero-inserted [n_t x 16] fp16 matrices already in the K-major canonical core-matrix order; a
-//    stage's 9 x n_t x 32 bytes arrive with one bulk copy (cp.async.bulk, no tensor map, no
-//    multicast) that completes on the stage's mbarrier.
+//    step's weights arrive as three bulk copies of three taps each (cp.async.bulk, no tensor map,
+//    no multicast), each completing on the mbarrier of its own sub-stage of the weight ring.
 //  * Warp roles: warps 0-3 epilogue (warp q reads TMEM lanes 32q..32q+31, adds the bias, applies
 //    ReLU, converts to fp16 and stages the tile in shared memory as [filter][pixel]; the 128
 //    threads then copy it out in 16-byte pieces, a filter's 8 consecutive pixels each -- the
 //    first version stored 2 bytes per lane and column straight from the registers and spent more
-//    time in its epilogue than in its MMAs), warp 4 issues the MMAs (one thread) and owns the TMEM allocation,
-//    warps 5-12 are the A producers (each thread keeps the loads of the next two stages in
+//    time in its epilogue than in its MMAs), warp 4 issues the MMAs and owns the TMEM allocation
+//    (the whole warp runs the issue loop and waits, elect.sync picks the lane that issues, so the
+//    loop stays warp-uniform), warps 5-12 are the A producers (each thread keeps the loads of the next two stages in
 //    flight in two register sets while it shifts and stores the current one), warp 13 streams
 //    the weights through a ring of their own (three taps per bulk copy).  Two accumulator buffers
 //    (2 x n_t columns) let the epilogue of a tile overlap the next tile's MMAs.  CTAs are

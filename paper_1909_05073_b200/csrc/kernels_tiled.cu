@@ -117,9 +117,6 @@ __device__ __forceinline__ void sts128f(uint32_t addr, float a, float b, float c
   asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d)
                : "memory");
 }
-__device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
-  asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
-}
 __device__ __forceinline__ void cp_async4(uint32_t dst, const void* src, uint32_t src_bytes) {
   asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(src_bytes)
                : "memory");
@@ -239,13 +236,6 @@ __device__ __forceinline__ void dispatch_chunk_wide(uint32_t cp, uint32_t wp, ui
   }
 }
 
-__device__ __forceinline__ void tmem_ld8(uint32_t (&r)[8], uint32_t taddr) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
-                 "=r"(r[7])
-               : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
 __device__ __forceinline__ void tmem_ld8_nowait(uint32_t (&r)[8], uint32_t taddr) {
   asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
@@ -291,8 +281,6 @@ __device__ __forceinline__ void load_window(u64 (&win)[Win<S>::kRows][3], uint32
     kernel_body_generic<S, G>(acc, win, code & 0x1FFu, wp); \
     break;
 #define PG_CASES8(B) PG_CASE(B + 0) PG_CASE(B + 1) PG_CASE(B + 2) PG_CASE(B + 3) PG_CASE(B + 4) PG_CASE(B + 5) PG_CASE(B + 6) PG_CASE(B + 7)
-
-__device__ __forceinline__ float ldg_f(const __half* p) { return __half2float(__ldg(p)); }
 
 // ---- producer: stage one chunk -----------------------------------------------------------------------
 // Input columns staged for row element i of a sub-tile, relative to its first output column
