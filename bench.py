@@ -4,7 +4,7 @@ the four 2x2 max-pools after conv2/4/7/10, fused into those layers' epilogues) o
 per GPU, fp32.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-configs]
-    python bench.py --layer C_IN,C_OUT,H,N,STRIDE,KEEP[,f32|f16[,4|8|12[,split]]]  [--steps K]
+    python bench.py --layer C_IN,C_OUT,H,N,STRIDE,KEEP[,f32|f16[,4|8|12[,split][,rows4|rows8]]]  [--steps K]
     python bench.py --layer cfg5:0          (layer 0 of benchmark configuration 5, at its batch)
 
 A step is one pass of the whole stack over one image (per rank).  `value` is effective TFLOP/s
@@ -287,7 +287,9 @@ def run_layer(args):
     torch.cuda.set_device(0)
     a = args.layer.split(",")
     split = "split" in a
-    a = [v for v in a if v != "split"]
+    kernel = {"rows4": B.ROWS4, "rows8": B.ROWS8}                       # pin the tiled kernel's rows per lane
+    kflags = sum(f for k, f in kernel.items() if k in a)
+    a = [v for v in a if v != "split" and v not in kernel]
     if a[0].startswith("cfg"):
         cid, li = a[0][3:].split(":")[:2]
         cfg = synth.config(int(cid), int(a[1]) if len(a) > 1 else None)
@@ -309,10 +311,10 @@ def run_layer(args):
     if half:
         x = x.half()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-    y = layer.forward(x, split=split)
+    y = layer.forward(x, split=split, kernel=kflags)
     for _ in range(max(args.warmup - 1, 0)):
-        layer.forward(x, out=y, split=split)
-    us = _time_launch(torch, flush, lambda: layer.forward(x, out=y, split=split), args.steps)
+        layer.forward(x, out=y, split=split, kernel=kflags)
+    us = _time_launch(torch, flush, lambda: layer.forward(x, out=y, split=split, kernel=kflags), args.steps)
     hbm, src = hbm_peak_gbs()
     roof = layer_roof_us(spec, kept, n, 2 if half else 4, hbm)
     assert B.pconv_device_status(layer.handle)[0] == 0
@@ -320,7 +322,7 @@ def run_layer(args):
         "layer": {"c_in": spec.c_in, "c_out": spec.c_out, "h": spec.h, "w": spec.w, "n": n,
                   "stride": spec.stride, "keep": spec.keep, "storage": storage,
                   "patterns": len(patterns), "kept_kernels": kept, "workspace": split},
-        "plan": B.pconv_plan(layer.handle, n, spec.h, spec.w, 0, split),
+        "plan": B.pconv_plan(layer.handle, n, spec.h, spec.w, kflags, split),
         "us": round(us, 2), "tflops": round(layer_flops(spec, kept, n) / us / 1e6, 3),
         "frac_of_alu_peak": round(layer_flops(spec, kept, n) / us / 1e6 / ALU_PEAK_TFLOPS, 4),
         "roof_us": round(roof, 3), "frac": round(roof / us, 4), "hbm_peak": src,

@@ -81,6 +81,13 @@ enum {
                                    pattern mask (any set of 4-of-9 masks); the default */
   PCONV_KERNEL_GENERIC_TAPS = 0x400u, /* tiled path that tests the 9 mask bits at run time; slower,
                                          kept as a cross-check of the per-mask bodies */
+  PCONV_ROWS4 = 0x1000u, /* tiled kernel with one-byte codes (canonical pattern sets): pins the */
+  PCONV_ROWS8 = 0x2000u, /* output rows a lane owns per sub-tile.  4: sixteen consumer warps, a
+                            decoded kernel runs 16 packed FMAs; 8: eight consumer warps with twice
+                            the Tensor Memory columns each, 32 packed FMAs per decoded kernel (less
+                            decoding per multiply-add, for layers with many pixels).  Default: the
+                            planner picks per shape.  PCONV_ROWS8 with another pattern set or with
+                            PCONV_KERNEL_GENERIC_TAPS: PCONV_ERR_UNSUPPORTED. */
   PCONV_KERNEL_TENSOR = 0x800u /* fp16 storage, stride 1 only: the layer as a dense implicit GEMM over
                                   the zero-inserted weights on the tensor cores (tcgen05.mma, fp32
                                   accumulators in Tensor Memory).  It multiplies the pruned zeros too
@@ -223,11 +230,12 @@ pconv_status pconv_unpack(const pconv_handle* h, float* w_oihw_host_out);
  * tile sizes off line; here the library picks them per call from the shape). */
 typedef struct pconv_plan_t {
   int generic_taps;      /* 1 = run-time masks (asked for with PCONV_KERNEL_GENERIC_TAPS) */
+  int rows_per_lane;     /* output rows a lane owns per sub-tile: 4 or 8 (see PCONV_ROWS4 / PCONV_ROWS8) */
   int warps_per_unit;    /* consumer warps that share one (pixels, filter group) and split each chunk's
                             channels among themselves: 1, 2 or 4 */
   int channel_splits;    /* CTAs that share one output tile through the workspace (1 = none) */
   int groups_per_cta;    /* filter groups (of 16) per CTA */
-  int pixel_sets;        /* independent sets of 256 pixels per CTA */
+  int pixel_sets;        /* independent sets of 64 x rows_per_lane pixels per CTA */
   int tile_width;        /* output columns of a sub-tile (2..32) */
   int stages;            /* depth of the staging ring */
   int smem_bytes;        /* dynamic shared memory the geometry needs */
@@ -239,7 +247,7 @@ typedef struct pconv_plan_t {
 
 /* Test / tuning aid: fills *plan with the geometry a tiled forward of this shape would use;
  * with_workspace != 0 asks for the plan of pconv_forward_ws with a large enough workspace.
- * flags: 0 or PCONV_KERNEL_GENERIC_TAPS.  Launches nothing.  PCONV_ERR_UNSUPPORTED if the tiled
+ * flags: 0, PCONV_KERNEL_GENERIC_TAPS, PCONV_ROWS4 or PCONV_ROWS8.  Launches nothing.  PCONV_ERR_UNSUPPORTED if the tiled
  * kernel cannot take the shape. */
 pconv_status pconv_plan(const pconv_handle* h, int n, int h_in, int w_in, unsigned flags,
                         int with_workspace, pconv_plan_t* plan);

@@ -16,6 +16,7 @@ OK = 0
 F32, F16 = 0, 1
 RELU, STRICT4, POOL2X2, REPRODUCIBLE, CHAIN = 1, 2, 4, 8, 0x10
 KERNEL_SIMPLE, KERNEL_TILED, KERNEL_GENERIC_TAPS, KERNEL_TENSOR = 0x100, 0x200, 0x400, 0x800
+ROWS4, ROWS8 = 0x1000, 0x2000
 MAX_PATTERNS = 16
 
 STATUS_NAMES = ["PCONV_OK", "PCONV_ERR_NULL", "PCONV_ERR_SHAPE", "PCONV_ERR_PATTERN_SET",
@@ -52,7 +53,8 @@ class Stats(ctypes.Structure):
 
 
 class Plan(ctypes.Structure):
-    _fields_ = [("generic_taps", ctypes.c_int), ("warps_per_unit", ctypes.c_int),
+    _fields_ = [("generic_taps", ctypes.c_int), ("rows_per_lane", ctypes.c_int),
+                ("warps_per_unit", ctypes.c_int),
                 ("channel_splits", ctypes.c_int), ("groups_per_cta", ctypes.c_int),
                 ("pixel_sets", ctypes.c_int), ("tile_width", ctypes.c_int), ("stages", ctypes.c_int),
                 ("smem_bytes", ctypes.c_int), ("ctas", ctypes.c_longlong),

@@ -48,6 +48,23 @@ extern "C" const char* pconv_status_str(pconv_status s) {
   return "unknown status";
 }
 
+// Rows per lane a caller pinned for the tiled kernel (0 = the planner chooses).
+static int rows_mode(unsigned flags) {
+  return (flags & PCONV_ROWS8) ? 8 : (flags & PCONV_ROWS4) ? 4 : 0;
+}
+
+// Scratch a forward of this shape may use, whichever kernel takes it.  rmode: the rows per lane
+// the caller pins for the tiled kernel (0 = the planner's choice), -1 = whatever it may pin.
+static size_t workspace_need(const pconv::DeviceLayer& L, int n, int h_in, int w_in, int rmode) {
+  size_t need = tensor_workspace_bytes(L, n, h_in, w_in);
+  for (int r = 0; r <= 8; r += 4) {
+    if (rmode >= 0 && r != rmode) continue;
+    const size_t a = tiled_workspace_bytes(L, n, h_in, w_in, r);
+    if (a > need) need = a;
+  }
+  return need;
+}
+
 extern "C" pconv_status pconv_workspace_bytes(const pconv_handle* h, int n, int h_in, int w_in,
                                               size_t* bytes) {
   if (!h || !bytes) return PCONV_ERR_NULL;
@@ -55,8 +72,7 @@ extern "C" pconv_status pconv_workspace_bytes(const pconv_handle* h, int n, int 
   // (whichever kernel a forward of this shape may take)
   *bytes = 0;
   if (n > 0) {
-    const size_t a = tiled_workspace_bytes(h->d, n, h_in, w_in), b = tensor_workspace_bytes(h->d, n, h_in, w_in);
-    *bytes = a > b ? a : b;
+    *bytes = workspace_need(h->d, n, h_in, w_in, -1);
   }
   return PCONV_OK;
 }
@@ -66,7 +82,8 @@ extern "C" pconv_status pconv_plan(const pconv_handle* h, int n, int h_in, int w
   if (!h || !plan) return PCONV_ERR_NULL;
   if (n <= 0 || h_in <= 0 || w_in <= 0) return PCONV_ERR_SHAPE;
   std::memset(plan, 0, sizeof(*plan));
-  if (!tiled_plan(h->d, n, h_in, w_in, (flags & PCONV_KERNEL_GENERIC_TAPS) != 0, with_workspace != 0, plan))
+  if (!tiled_plan(h->d, n, h_in, w_in, (flags & PCONV_KERNEL_GENERIC_TAPS) != 0, with_workspace != 0,
+                  rows_mode(flags), plan))
     return PCONV_ERR_UNSUPPORTED;
   plan->tensor_path = tensor_preferred(h->d, n, h_in, w_in) ? 1 : 0;
   return PCONV_OK;
@@ -91,7 +108,8 @@ extern "C" pconv_status pconv_plan_shape(int c_out, int c_in, long long kept_ker
   L.wide_codes = n_patterns_canonical ? 0 : 1;
   L.codes_s = reinterpret_cast<const uint8_t*>(&L);   // only tested for presence by the planner
   std::memset(plan, 0, sizeof(*plan));
-  if (!tiled_plan(L, n, h_in, w_in, (flags & PCONV_KERNEL_GENERIC_TAPS) != 0, with_workspace != 0, plan))
+  if (!tiled_plan(L, n, h_in, w_in, (flags & PCONV_KERNEL_GENERIC_TAPS) != 0, with_workspace != 0,
+                  rows_mode(flags), plan))
     return PCONV_ERR_UNSUPPORTED;
   return PCONV_OK;
 }
@@ -122,8 +140,10 @@ static pconv_status forward_impl(const pconv_handle* h, const void* x, const flo
   if (n < 0 || h_in <= 0 || w_in <= 0) return PCONV_ERR_SHAPE;
   const unsigned known =
       PCONV_RELU | PCONV_POOL2X2 | PCONV_REPRODUCIBLE | PCONV_CHAIN | PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED |
-      PCONV_KERNEL_GENERIC_TAPS | PCONV_KERNEL_TENSOR;
+      PCONV_KERNEL_GENERIC_TAPS | PCONV_KERNEL_TENSOR | PCONV_ROWS4 | PCONV_ROWS8;
   if (flags & ~known) return PCONV_ERR_UNSUPPORTED;
+  if ((flags & PCONV_ROWS4) && (flags & PCONV_ROWS8)) return PCONV_ERR_UNSUPPORTED;
+  const int rmode = rows_mode(flags);
   const unsigned sel = flags & (PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED | PCONV_KERNEL_GENERIC_TAPS |
                                 PCONV_KERNEL_TENSOR);
   if (sel & (sel - 1)) return PCONV_ERR_UNSUPPORTED;  // at most one selection bit
@@ -161,9 +181,11 @@ static pconv_status forward_impl(const pconv_handle* h, const void* x, const flo
   } else if (sel == PCONV_KERNEL_TILED || sel == PCONV_KERNEL_GENERIC_TAPS) {
     if (!tiled_supported(L, n, h_in, w_in)) return PCONV_ERR_UNSUPPORTED;
     const bool generic = (sel == PCONV_KERNEL_GENERIC_TAPS);
-    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, pool, repro, generic, ws, ws_bytes, stream);
+    if (rmode == 8 && (generic || L.wide_codes || !L.codes_s)) return PCONV_ERR_UNSUPPORTED;
+    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, pool, repro, generic, rmode, ws, ws_bytes, stream);
   } else if (tiled_supported(L, n, h_in, w_in)) {
-    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, pool, repro, false, ws, ws_bytes, stream);
+    if (rmode == 8 && (L.wide_codes || !L.codes_s)) return PCONV_ERR_UNSUPPORTED;
+    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, pool, repro, false, rmode, ws, ws_bytes, stream);
   } else {
     e = launch_simple(L, x, bias, y, n, h_in, w_in, relu, stream);
   }
@@ -208,8 +230,7 @@ extern "C" pconv_status pconv_forward_static_ws(const pconv_handle* h, const voi
   if (!h || !x || !y) return PCONV_ERR_NULL;
   if (n < 0 || h_in <= 0 || w_in <= 0) return PCONV_ERR_SHAPE;
   if (n == 0) return PCONV_OK;
-  size_t need = 0;
-  if (pconv_workspace_bytes(h, n, h_in, w_in, &need) != PCONV_OK) return PCONV_ERR_SHAPE;
+  const size_t need = workspace_need(h->d, n, h_in, w_in, rows_mode(flags));
   if (need > (size_t)PCONV_STATIC_WS_BYTES) return PCONV_ERR_WORKSPACE;
   if (need == 0)  // this shape is never split: no scratch involved
     return pconv_forward_ws(h, x, bias, y, n, h_in, w_in, flags, nullptr, 0, stream_v);
@@ -456,7 +477,7 @@ extern "C" pconv_status pconv_stack_create(const pconv_handle* const* layers,
       pconv_stack_free(s);
       return PCONV_ERR_SHAPE;
     }
-    const size_t wsb = tiled_workspace_bytes(L, n, ch, cw), wsd = tensor_workspace_bytes(L, n, ch, cw);
+    const size_t wsb = tiled_workspace_bytes(L, n, ch, cw, rows_mode(flags)), wsd = tensor_workspace_bytes(L, n, ch, cw);
     if (wsb > s->ws_bytes) s->ws_bytes = wsb;
     if (wsd > s->ws_bytes) s->ws_bytes = wsd;
     ch = (ch - 1) / L.stride + 1;

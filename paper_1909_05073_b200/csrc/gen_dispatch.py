@@ -1,5 +1,6 @@
 """Generates the PTX text of the tiled kernel's per-chunk dispatch loop (dispatch_s<stride>.inc for
-pattern sets inside the canonical eight, dispatch_s<stride>w.inc for any other set), which
+pattern sets inside the canonical eight, dispatch_s<stride>w.inc for any other set,
+dispatch_s<stride>t.inc for the canonical sets with 8 instead of 4 output rows per lane), which
 kernels_tiled.cu includes inside one `asm volatile` statement.
 
 Why PTX text, and why this shape (all measured on B200):
@@ -59,14 +60,16 @@ def taps(mask):
     return [t for t in range(9) if mask >> t & 1]
 
 
-def gen(stride, wide):
-    rows = 6 if stride == 1 else 9
+def gen(stride, wide, R=4):
+    """R = output rows per lane and sub-tile: a body runs 4 * R packed FMAs on 2 * R TMEM columns."""
+    rows = stride * (R - 1) + 3
+    nv = 2 * R                      # TMEM columns (32-bit registers) of one filter slot
     out = []
     emit = out.append
     emit("{")
-    emit(".reg .b32 a<8>;")
-    emit(".reg .b32 s<8>;")
-    emit(".reg .b64 acc<4>;")
+    emit(".reg .b32 a<%d>;" % nv)
+    emit(".reg .b32 s<%d>;" % nv)
+    emit(".reg .b64 acc<%d>;" % R)
     emit(".reg .b64 win<%d>;" % (rows * 3))
     emit(".reg .b64 w0, w1, w2, w3;")
     emit(".reg .b32 r0, r1, r2, r3;")          # raw weights of the next kernel
@@ -89,8 +92,9 @@ def gen(stride, wide):
     emit("tcgen05.wait::st.sync.aligned;")
     emit("bra.uni ADV;")                      # the entry code leads to the block's first channel
 
-    A8 = "{a0, a1, a2, a3, a4, a5, a6, a7}"
-    S8 = "{s0, s1, s2, s3, s4, s5, s6, s7}"
+    A8 = "{" + ", ".join("a%d" % i for i in range(nv)) + "}"
+    S8 = "{" + ", ".join("s%d" % i for i in range(nv)) + "}"
+    slot_shift = 3 if R == 4 else 4
 
     def prep():
         """Shift the next byte code out of the record registers; decode its jump index and the
@@ -111,7 +115,7 @@ def gen(stride, wide):
             emit("shr.u32 c3, c3, 8;")
             emit("and.b32 idx, code, 15;")
             emit("shr.u32 tn, code, 4;")
-        emit("shl.b32 tn, tn, 3;")
+        emit("shl.b32 tn, tn, %d;" % slot_shift)
         emit("add.u32 tn, tn, tq;")
 
     def jump():
@@ -134,16 +138,16 @@ def gen(stride, wide):
         emit("add.u32 wp, wp, 16;")
         prep()
         emit("tcgen05.wait::ld.sync.aligned;")
-        for k in range(4):
+        for k in range(R):
             emit("mov.b64 acc%d, {a%d, a%d};" % (k, 2 * k, 2 * k + 1))
         for s_, t in enumerate(tp):
             u, v = divmod(t, 3)
-            for k in range(4):
+            for k in range(R):
                 emit("fma.rn.f32x2 acc%d, win%d, w%d, acc%d;" % (k, (stride * k + u) * 3 + v, s_, k))
-        for k in range(4):
+        for k in range(R):
             emit("mov.b64 {s%d, s%d}, acc%d;" % (2 * k, 2 * k + 1, k))
-        emit("tcgen05.st.sync.aligned.32x32b.x8.b32 [ta], %s;" % S8)
-        emit("tcgen05.ld.sync.aligned.32x32b.x8.b32 %s, [tn];" % A8)
+        emit("tcgen05.st.sync.aligned.32x32b.x%d.b32 [ta], %s;" % (nv, S8))
+        emit("tcgen05.ld.sync.aligned.32x32b.x%d.b32 %s, [tn];" % (nv, A8))
         jump()
 
     for p in range(len(CANON_MASKS)):
@@ -175,7 +179,7 @@ def gen(stride, wide):
         if rows % 2:
             emit("ld.shared.b64 win%d, [ra+%d];" % ((rows - 1) * 3 + v, (rows - 1) * 8))
     prep()
-    emit("tcgen05.ld.sync.aligned.32x32b.x8.b32 %s, [tn];" % A8)
+    emit("tcgen05.ld.sync.aligned.32x32b.x%d.b32 %s, [tn];" % (nv, A8))
     jump()
     if wide:
         # Continue: the channel has more kernels than a record holds; fetch the next record.
@@ -184,7 +188,7 @@ def gen(stride, wide):
         emit("ld.shared.v4.b32 {c0, c1, c2, c3}, [cp];")
         emit("add.u32 cp, cp, 16;")
         prep()
-        emit("tcgen05.ld.sync.aligned.32x32b.x8.b32 %s, [tn];" % A8)
+        emit("tcgen05.ld.sync.aligned.32x32b.x%d.b32 %s, [tn];" % (nv, A8))
         jump()
     emit("END:")
     emit("tcgen05.wait::ld.sync.aligned;")
@@ -211,6 +215,7 @@ def main(outdir):
     for stride in (1, 2):
         write(os.path.join(outdir, "dispatch_s%d.inc" % stride), gen(stride, False))
         write(os.path.join(outdir, "dispatch_s%dw.inc" % stride), gen(stride, True))
+        write(os.path.join(outdir, "dispatch_s%dt.inc" % stride), gen(stride, False, 8))
 
 
 if __name__ == "__main__":

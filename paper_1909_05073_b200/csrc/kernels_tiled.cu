@@ -21,6 +21,11 @@
 //    channel range from a counter, accumulate in their own columns, and add the column sets up
 //    before the epilogue.  The channel range can also be split across CTAs (grid.z), with fp32
 //    atomics into a workspace and per-warp tickets that elect who finishes each part of a tile.
+//    Template parameter R (canonical masks only): a lane owns R = 4 or 8 output rows per sub-tile.
+//    R = 8: eight consumer warps with 256 TMEM columns each, a unit is 512 pixels and a decoded
+//    kernel runs 32 packed FMAs; measured 3-10 % faster where a warp owns a unit's whole channel
+//    range (large batches) and slower where channels are split (only two warps share a TMEM lane
+//    quadrant), so the planner takes it for unsplit plans only.
 //  * run-time masks (GENERIC = true): 8 consumer warps with register accumulators, a switch on the
 //    filter slot and nine warp-uniform tap tests per kernel (384 threads leave 168 registers each,
 //    which the accumulators fit); a slower cross-check of the generated bodies.
@@ -48,11 +53,14 @@ namespace {
 typedef unsigned long long u64;
 
 constexpr int kProducerWarps = 4;
-__host__ __device__ constexpr int consumer_warps(bool generic) { return generic ? 8 : 16; }
-__host__ __device__ constexpr int cta_threads(bool generic) {
-  return 32 * (consumer_warps(generic) + kProducerWarps);
+// R = output rows per lane and sub-tile: 4 (16 consumer warps with 128 TMEM columns each) or 8
+// (8 consumer warps with 256 columns each: twice the packed FMAs per decoded kernel).
+__host__ __device__ constexpr int consumer_warps(bool generic, int R = 4) { return (generic || R == 8) ? 8 : 16; }
+__host__ __device__ constexpr int cta_threads(bool generic, int R = 4) {
+  return 32 * (consumer_warps(generic, R) + kProducerWarps);
 }
-constexpr int kTmemCols = 512;  // whole TMEM of the SM: 16 warps x 16 slots x 8 columns
+constexpr int kMaxConsumerWarps = 16;
+constexpr int kTmemCols = 512;  // whole TMEM of the SM: 16 warps x 16 slots x 8 columns (8 x 16 x 16)
 constexpr int kMaxStages = 8;
 constexpr int kMaxCoop = 4;   // chunks whose x the consumer warps copy at the start of a launch
 constexpr int kWSlot = kMaxBlockKernels * 16 + 16;  // bytes per (group, stage): 4 fp32 per kernel
@@ -75,6 +83,7 @@ struct Geo {
   int zs;                // consumer warps that share one (pixel set, filter group) and split its channels
   int wys, wy, ng;       // warp grid: unit -> (unit % wys, unit / wys); rows >= wy are idle
   int pairs;             // sub-tile pairs per CTA = wy * sw
+  int rpl;               // output rows per lane and sub-tile (4 or 8)
   int rows, pitch;       // staged rows and columns of one sub-tile
   int colstride;         // bytes between staged columns (rows are contiguous float2)
   int substride, chan_stride;  // bytes per (sub-tile pair, channel) and per channel
@@ -190,26 +199,38 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* er
 #define PCONV_MARK_MAX(i)
 #endif
 
-template <int S>
+template <int S, int R = 4>
 struct Win {
-  static constexpr int kRows = (S == 1) ? 6 : 9;
+  static constexpr int kRows = S * (R - 1) + 3;   // input rows under R output rows
 };
 
 // The specialised dispatch loop of one (warp, chunk): generated PTX (see gen_dispatch.py); the
 // accumulators stay in TMEM at `tq` (+ 8 columns per filter slot).
-template <int S>
+template <int S, int R>
 __device__ __forceinline__ void dispatch_chunk(uint32_t cp, uint32_t wp, uint32_t xptr,
                                                uint32_t chan_b, uint32_t col_b, uint32_t off_mid,
                                                uint32_t tq, uint32_t entry_code) {
-  if (S == 1) {
+  if constexpr (S == 1 && R == 4) {
     asm volatile(
 #include "dispatch_s1.inc"
         :
         : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(col_b), "r"(off_mid), "r"(tq), "r"(entry_code)
         : "memory");
-  } else {
+  } else if constexpr (S == 2 && R == 4) {
     asm volatile(
 #include "dispatch_s2.inc"
+        :
+        : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(col_b), "r"(off_mid), "r"(tq), "r"(entry_code)
+        : "memory");
+  } else if constexpr (S == 1) {
+    asm volatile(
+#include "dispatch_s1t.inc"
+        :
+        : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(col_b), "r"(off_mid), "r"(tq), "r"(entry_code)
+        : "memory");
+  } else {
+    asm volatile(
+#include "dispatch_s2t.inc"
         :
         : "r"(cp), "r"(wp), "r"(xptr), "r"(chan_b), "r"(col_b), "r"(off_mid), "r"(tq), "r"(entry_code)
         : "memory");
@@ -236,11 +257,17 @@ __device__ __forceinline__ void dispatch_chunk_wide(uint32_t cp, uint32_t wp, ui
   }
 }
 
-__device__ __forceinline__ void tmem_ld8_nowait(uint32_t (&r)[8], uint32_t taddr) {
+__device__ __forceinline__ void tmem_ld8_nowait(uint32_t* r, uint32_t taddr) {
   asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
                  "=r"(r[7])
                : "r"(taddr));
+}
+// The NV = 8 or 16 columns of one filter slot.
+template <int NV>
+__device__ __forceinline__ void tmem_ld_slot_nowait(uint32_t (&r)[NV], uint32_t taddr) {
+  tmem_ld8_nowait(r, taddr);
+  if constexpr (NV == 16) tmem_ld8_nowait(r + 8, taddr + 8);
 }
 __device__ __forceinline__ void tmem_st8_zero(uint32_t taddr) {
   const uint32_t z = 0;
@@ -298,10 +325,10 @@ struct StagedElem {
   long long off_a, off_b;   // element offsets into x for channel c0 of the chunk, or -1
   uint32_t dst;             // byte offset inside the channel's staged block
 };
-template <int S>
+template <int S, int R>
 __device__ __forceinline__ StagedElem staged_elem(const DeviceLayer& L, const Geo& g,
                                                   const SubTile* tab, int e, int c0) {
-  constexpr int kRows = (S == 1) ? 6 : 9;
+  constexpr int kRows = Win<S, R>::kRows;
   const int q = e / g.pitch, i = e - q * g.pitch;   // q = pair * rows + row
   const int p = q / kRows, r = q - p * kRows;
   const SubTile A = tab[2 * p], B = tab[2 * p + 1];
@@ -325,7 +352,7 @@ constexpr int kPreElems = 4;
 constexpr uint32_t kSkipElem = 0xFFFFFFFFu;
 constexpr int kProducerThreads = 32 * kProducerWarps;
 
-template <int S>
+template <int S, int R>
 __device__ __forceinline__ void precompute_elems(StagedElem (&pre)[kPreElems], const DeviceLayer& L,
                                                  const Geo& g, const SubTile* tab, int ptid) {
   const int n_elem = g.pairs * g.rows * g.pitch;
@@ -333,7 +360,7 @@ __device__ __forceinline__ void precompute_elems(StagedElem (&pre)[kPreElems], c
   for (int i = 0; i < kPreElems; ++i) {
     const int e = ptid + i * kProducerThreads;
     if (e < n_elem) {
-      pre[i] = staged_elem<S>(L, g, tab, e, 0);
+      pre[i] = staged_elem<S, R>(L, g, tab, e, 0);
     } else {
       pre[i].off_a = pre[i].off_b = -1;
       pre[i].dst = kSkipElem;
@@ -394,7 +421,7 @@ __device__ __forceinline__ void stage_blocks_half(const DeviceLayer& L, const Ge
 // fp32 storage: everything is fetched with cp.async (zero-fill outside the image), so the producer
 // never waits for data and several chunks are in flight; each thread's arrival on the stage's full
 // barrier fires when its own copies have landed.
-template <int S>
+template <int S, int R>
 __device__ __forceinline__ void produce_chunk_async(const DeviceLayer& L, const Geo& g,
                                                     const float* __restrict__ x, const SubTile* tab,
                                                     const StagedElem (&pre)[kPreElems], const uint4* desc,
@@ -433,7 +460,7 @@ __device__ __forceinline__ void produce_chunk_async(const DeviceLayer& L, const 
       if (pre[i].dst != kSkipElem) copy_elem(pre[i], (size_t)c0 * hw);
   }
   for (int e = ptid + kPreElems * kProducerThreads; e < n_elem; e += kProducerThreads)
-    copy_elem(staged_elem<S>(L, g, tab, e, c0), 0);
+    copy_elem(staged_elem<S, R>(L, g, tab, e, c0), 0);
   if (with_blocks) stage_blocks_async(L, g, desc, codes, stage_base, kk, ptid);
 }
 
@@ -441,7 +468,7 @@ __device__ __forceinline__ void produce_chunk_async(const DeviceLayer& L, const 
 // consumer warps, which have nothing else to do yet, for the first chunks of a launch.  A warp can
 // keep only a few cp.async in flight, so twenty warps fill a chunk several times faster than the
 // four producer warps.
-template <int S>
+template <int S, int R>
 __device__ __forceinline__ void fill_chunk_x(const DeviceLayer& L, const Geo& g, const float* __restrict__ x,
                                              const SubTile* tab, uint32_t stage_base, int k, int t,
                                              int n_threads) {
@@ -451,7 +478,7 @@ __device__ __forceinline__ void fill_chunk_x(const DeviceLayer& L, const Geo& g,
   const int n_elem = g.pairs * g.rows * g.pitch;
   const uint32_t chan_b = (uint32_t)g.chan_stride;
   for (int e = t; e < n_elem; e += n_threads) {
-    const StagedElem se = staged_elem<S>(L, g, tab, e, c0);
+    const StagedElem se = staged_elem<S, R>(L, g, tab, e, c0);
     const float* sa = se.off_a >= 0 ? x + se.off_a : x;
     const float* sb = se.off_b >= 0 ? x + se.off_b : x;
     const size_t step_a = se.off_a >= 0 ? hw : 0, step_b = se.off_b >= 0 ? hw : 0;
@@ -476,9 +503,9 @@ __device__ __forceinline__ void fill_chunk_x(const DeviceLayer& L, const Geo& g,
 
 // Byte offsets of a staged element's A and B halves inside a raw slot (channel 0) and of its
 // place in the stage, in the fields of a StagedElem (off_a, off_b, dst).
-template <int S>
+template <int S, int R>
 __device__ __forceinline__ StagedElem raw_elem(const Geo& g, int e) {
-  constexpr int kRows = (S == 1) ? 6 : 9;
+  constexpr int kRows = Win<S, R>::kRows;
   const int q = e / g.pitch, i = e - q * g.pitch;   // q = pair * rows + row
   const int p = q / kRows, r = q - p * kRows;
   const int hidx = staged_dx<S>(i, g.tw) + 2;        // column inside the raw row
@@ -490,11 +517,11 @@ __device__ __forceinline__ StagedElem raw_elem(const Geo& g, int e) {
   return se;
 }
 
-template <int S>
+template <int S, int R>
 __device__ __forceinline__ void issue_raw(const DeviceLayer& L, const Geo& g, const __half* __restrict__ x,
                                           const SubTile* tab, const uint4* desc, const uint8_t* codes,
                                           uint32_t raw_base, int k, int kk, int ptid) {
-  constexpr int kRows = (S == 1) ? 6 : 9;
+  constexpr int kRows = Win<S, R>::kRows;
   const int c0 = k * kChunk;
   const int nc = min(kChunk, L.c_in - c0);
   const size_t hw = (size_t)g.h * g.w;
@@ -528,11 +555,11 @@ __device__ __forceinline__ void issue_raw(const DeviceLayer& L, const Geo& g, co
   }
 }
 
-template <int S>
+template <int S, int R>
 __device__ __forceinline__ void widen_raw(const Geo& g, const StagedElem (&pre)[kPreElems],
                                           const uint4* desc, uint32_t raw_base, uint32_t stage_base,
                                           int kk, int ptid) {
-  constexpr int kRows = (S == 1) ? 6 : 9;
+  constexpr int kRows = Win<S, R>::kRows;
   const int n_elem = g.pairs * g.rows * g.pitch;
   const uint32_t raw_chan = (uint32_t)(kRows * g.raw_pitch * 2);
   auto widen = [&](const StagedElem& se) {
@@ -552,7 +579,7 @@ __device__ __forceinline__ void widen_raw(const Geo& g, const StagedElem (&pre)[
 #pragma unroll
   for (int i = 0; i < kPreElems; ++i)
     if (pre[i].dst != kSkipElem) widen(pre[i]);
-  for (int e = ptid + kPreElems * kProducerThreads; e < n_elem; e += kProducerThreads) widen(raw_elem<S>(g, e));
+  for (int e = ptid + kPreElems * kProducerThreads; e < n_elem; e += kProducerThreads) widen(raw_elem<S, R>(g, e));
   const uint32_t rw = raw_base + g.raw_x_bytes, rc = rw + g.ng * kWRawSlot;
   const uint32_t wbase = stage_base + g.x_stage_bytes, cbase = wbase + g.ng * kWSlot;
   for (int j = 0; j < g.ng; ++j) {
@@ -580,34 +607,34 @@ __device__ __forceinline__ void widen_raw(const Geo& g, const StagedElem (&pre)[
 // The producers' loop of the raw-ring path.  Every producer thread passes through every named
 // barrier of every chunk, also after a bounded wait ran out (it then does no more work), so the
 // barrier counts always match.
-template <int S>
+template <int S, int R>
 __device__ __forceinline__ void produce_raw_stream(const DeviceLayer& L, const Geo& g,
                                                    const __half* __restrict__ x, const SubTile* tab,
                                                    const StagedElem (&pre)[kPreElems], const uint4* desc,
                                                    const uint8_t* codes, uint32_t sbase, int k0, int nk,
                                                    int ptid) {
-  const int R = g.raw_stages;
+  const int RS = g.raw_stages;
   bool ok = true;
-  auto raw_base = [&](int kk) { return sbase + g.raw_off + (kk % R) * g.raw_slot; };
+  auto raw_base = [&](int kk) { return sbase + g.raw_off + (kk % RS) * g.raw_slot; };
   auto producers_sync = [] { asm volatile("bar.sync 2, %0;" ::"n"(kProducerThreads) : "memory"); };
-  // one cp.async group per chunk (empty past the last chunk), R - 1 chunks ahead of the one being
-  // widened, so "all but the newest R - 1 groups" is exactly "chunk kk has landed"
-  for (int j = 0; j < R - 1; ++j) {
-    if (j < nk) issue_raw<S>(L, g, x, tab, desc, codes, raw_base(j), k0 + j, j, ptid);
+  // one cp.async group per chunk (empty past the last chunk), RS - 1 chunks ahead of the one being
+  // widened, so "all but the newest RS - 1 groups" is exactly "chunk kk has landed"
+  for (int j = 0; j < RS - 1; ++j) {
+    if (j < nk) issue_raw<S, R>(L, g, x, tab, desc, codes, raw_base(j), k0 + j, j, ptid);
     asm volatile("cp.async.commit_group;" ::: "memory");
   }
   for (int kk = 0; kk < nk; ++kk) {
-    const int ahead = kk + R - 1;
-    if (ok && ahead < nk) issue_raw<S>(L, g, x, tab, desc, codes, raw_base(ahead), k0 + ahead, ahead, ptid);
+    const int ahead = kk + RS - 1;
+    if (ok && ahead < nk) issue_raw<S, R>(L, g, x, tab, desc, codes, raw_base(ahead), k0 + ahead, ahead, ptid);
     asm volatile("cp.async.commit_group;" ::: "memory");
-    if (R >= 3) asm volatile("cp.async.wait_group 2;" ::: "memory");
-    else if (R == 2) asm volatile("cp.async.wait_group 1;" ::: "memory");
+    if (RS >= 3) asm volatile("cp.async.wait_group 2;" ::: "memory");
+    else if (RS == 2) asm volatile("cp.async.wait_group 1;" ::: "memory");
     else asm volatile("cp.async.wait_group 0;" ::: "memory");
     producers_sync();   // everybody's copies of chunk kk have landed
     const int s = kk % g.stages, it = kk / g.stages;
     if (ok && it > 0) ok = mbar_wait(sbase + 8 * (kMaxStages + s), (it - 1) & 1, L.err, 1);
     if (ok) {
-      widen_raw<S>(g, pre, desc, raw_base(kk), sbase + g.stage_off + s * g.stage_bytes, kk, ptid);
+      widen_raw<S, R>(g, pre, desc, raw_base(kk), sbase + g.stage_off + s * g.stage_bytes, kk, ptid);
       if (!PCONV_WITHHELD(kk, ptid)) mbar_arrive(sbase + 8 * s);
     }
     producers_sync();   // the raw slot may be overwritten
@@ -624,7 +651,7 @@ struct HalfBatch {
   uint32_t dst[2];           // byte offset in the channel's staged block, kSkipElem = none
 };
 
-template <int S>
+template <int S, int R>
 __device__ __forceinline__ bool produce_half_stream(const DeviceLayer& L, const Geo& g,
                                                     const __half* __restrict__ x, const SubTile* tab,
                                                     const StagedElem (&pre)[kPreElems], const uint4* desc,
@@ -650,7 +677,7 @@ __device__ __forceinline__ bool produce_half_stream(const DeviceLayer& L, const 
           for (int j = 0; j < kPreElems; ++j)   // static indices keep `pre` in registers
             if (i == j) se = pre[j];
         } else {
-          se = staged_elem<S>(L, g, tab, e, 0);
+          se = staged_elem<S, R>(L, g, tab, e, 0);
         }
       }
       bt.dst[u] = se.dst;
@@ -694,12 +721,13 @@ __device__ __forceinline__ bool produce_half_stream(const DeviceLayer& L, const 
 
 
 // Where a lane's outputs go: the element offsets (inside filter 0's plane of the A / B image) of
-// row 0 of its two pixels, and which of the 8 outputs lie inside the image and the batch
+// row 0 of its two pixels, and which of the 2 R outputs lie inside the image and the batch
 // (bit 2k = A row k, bit 2k+1 = B row k).  Rows are w_out elements apart.
 struct LaneOut {
   long long base_a, base_b;
   uint32_t mask;
 };
+template <int R>
 __device__ __forceinline__ LaneOut lane_outputs(const DeviceLayer& L, const Geo& g, const SubTile* tab,
                                                 int slot, int col) {
   const SubTile A = tab[2 * slot], B = tab[2 * slot + 1];
@@ -711,7 +739,7 @@ __device__ __forceinline__ LaneOut lane_outputs(const DeviceLayer& L, const Geo&
   r.base_b = (long long)B.n * L.c_out * plane + (long long)B.y0 * g.w_out + ox_b;
   r.mask = 0;
 #pragma unroll
-  for (int k = 0; k < 4; ++k) {
+  for (int k = 0; k < R; ++k) {
     if (col_a && A.y0 + k < g.h_out) r.mask |= 1u << (2 * k);
     if (col_b && B.y0 + k < g.h_out) r.mask |= 2u << (2 * k);
   }
@@ -719,9 +747,10 @@ __device__ __forceinline__ LaneOut lane_outputs(const DeviceLayer& L, const Geo&
 }
 
 // The same for the pooled output: a lane in an even column writes, for each of its two pixels,
-// the two pooled rows that its four conv rows give (bit 0/1 = A/B upper, bit 2/3 = A/B lower);
-// rows are w_y elements apart.  A pooled position inside the pooled map has all four of its
-// sources inside the conv map, so no source needs masking.
+// the R / 2 pooled rows that its R conv rows give (bit 2j / 2j+1 = A / B pooled row j); rows are
+// w_y elements apart.  A pooled position inside the pooled map has all four of its sources inside
+// the conv map, so no source needs masking.
+template <int R>
 __device__ __forceinline__ LaneOut lane_outputs_pooled(const DeviceLayer& L, const Geo& g,
                                                        const SubTile* tab, int slot, int col) {
   const SubTile A = tab[2 * slot], B = tab[2 * slot + 1];
@@ -734,7 +763,7 @@ __device__ __forceinline__ LaneOut lane_outputs_pooled(const DeviceLayer& L, con
   r.base_b = (long long)B.n * L.c_out * plane + (long long)(B.y0 >> 1) * g.w_y + px_b;
   r.mask = 0;
 #pragma unroll
-  for (int k = 0; k < 2; ++k) {
+  for (int k = 0; k < R / 2; ++k) {
     if (col_a && (A.y0 >> 1) + k < g.h_y) r.mask |= 1u << (2 * k);
     if (col_b && (B.y0 >> 1) + k < g.h_y) r.mask |= 2u << (2 * k);
   }
@@ -766,99 +795,109 @@ __device__ __forceinline__ void red_add_v4(float* p, uint32_t a, uint32_t b, uin
                : "memory");
 }
 
-// The 8 outputs of one filter slot.  MODE 0: y = act(v + bias); MODE 1: workspace += v, where
-// `ws` points at this lane's 8 floats of the slot in the warp's part of the workspace (the
+// The 2 R outputs of one filter slot.  MODE 0: y = act(v + bias); MODE 1: workspace += v, where
+// `ws` points at this lane's 2 R floats of the slot in the warp's part of the workspace (the
 // workspace is laid out for the warps that write and read it, not like y: [tile][warp][slot]
-// [lane][8], so that a lane's partial sums go out as two 16-byte reductions and come back as two
+// [lane][2 R], so that a lane's partial sums go out as 16-byte reductions and come back as
 // 16-byte loads; lanes and rows outside the image carry zeros or garbage that nobody uses).
-template <int MODE, bool HALF, bool RELU>
+template <int R, int MODE, bool HALF, bool RELU>
 __device__ __forceinline__ void emit_slot(const Geo& g, const LaneOut& lo, void* __restrict__ y,
                                           float* __restrict__ ws, long long fbase, float bv,
-                                          const uint32_t (&v)[8]) {
+                                          const uint32_t (&v)[2 * R]) {
   if (MODE == 1) {
-    red_add_v4(ws, v[0], v[1], v[2], v[3]);
-    red_add_v4(ws + 4, v[4], v[5], v[6], v[7]);
+#pragma unroll
+    for (int i = 0; i < 2 * R; i += 4) red_add_v4(ws + i, v[i], v[i + 1], v[i + 2], v[i + 3]);
     return;
   }
   const long long ia = fbase + lo.base_a, ib = fbase + lo.base_b;
 #pragma unroll
-  for (int k = 0; k < 4; ++k) {
+  for (int k = 0; k < R; ++k) {
     const int row = k * g.w_out;
     if (lo.mask >> (2 * k) & 1u) store_out<HALF, RELU>(y, ia + row, __uint_as_float(v[2 * k]) + bv);
     if (lo.mask >> (2 * k + 1) & 1u) store_out<HALF, RELU>(y, ib + row, __uint_as_float(v[2 * k + 1]) + bv);
   }
 }
 
-// 2x2 max over a slot's 8 values (rows pairwise inside the lane, columns with the neighbour
+// 2x2 max over a slot's 2 R values (rows pairwise inside the lane, columns with the neighbour
 // lane), bias and activation after the max (both are monotone), stored by the even lane.  Must be
 // called by the whole warp.
-template <bool HALF, bool RELU>
+template <int R, bool HALF, bool RELU>
 __device__ __forceinline__ void emit_slot_pooled(const Geo& g, const LaneOut& lp, void* __restrict__ y,
-                                                 long long fbase, float bv, const float (&v)[8]) {
-  float m[4] = {fmaxf(v[0], v[2]), fmaxf(v[1], v[3]), fmaxf(v[4], v[6]), fmaxf(v[5], v[7])};
+                                                 long long fbase, float bv, const float (&v)[2 * R]) {
+  float m[R];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) m[i] = fmaxf(m[i], __shfl_xor_sync(0xffffffffu, m[i], 1));
+  for (int j = 0; j < R / 2; ++j) {
+    m[2 * j] = fmaxf(v[4 * j], v[4 * j + 2]);
+    m[2 * j + 1] = fmaxf(v[4 * j + 1], v[4 * j + 3]);
+  }
+#pragma unroll
+  for (int i = 0; i < R; ++i) m[i] = fmaxf(m[i], __shfl_xor_sync(0xffffffffu, m[i], 1));
   const long long ia = fbase + lp.base_a, ib = fbase + lp.base_b;
-  if (lp.mask & 1u) store_out<HALF, RELU>(y, ia, m[0] + bv);
-  if (lp.mask & 2u) store_out<HALF, RELU>(y, ib, m[1] + bv);
-  if (lp.mask & 4u) store_out<HALF, RELU>(y, ia + g.w_y, m[2] + bv);
-  if (lp.mask & 8u) store_out<HALF, RELU>(y, ib + g.w_y, m[3] + bv);
+#pragma unroll
+  for (int j = 0; j < R / 2; ++j) {
+    if (lp.mask >> (2 * j) & 1u) store_out<HALF, RELU>(y, ia + j * g.w_y, m[2 * j] + bv);
+    if (lp.mask >> (2 * j + 1) & 1u) store_out<HALF, RELU>(y, ib + j * g.w_y, m[2 * j + 1] + bv);
+  }
 }
 
 // Which accumulators a consumer warp writes out: filter slots [a0, a1) of the `zs` column sets
-// that start at TMEM address `t0` (128 columns apart), summed.  zs = 1: the warp's own 16 slots.
+// that start at TMEM address `t0` (16 slots x 2 R columns apart), summed.  zs = 1: the warp's own 16 slots.
 struct OutRange {
   uint32_t t0;
   int zs, a0, a1;
 };
 
-// Four filter slots of a lane's accumulators, summed over the warps that split the channels.
-__device__ __forceinline__ void tmem_sum4(uint32_t (&v)[4][8], const OutRange& r, int a) {
+// 16 / R filter slots of a lane's accumulators, summed over the warps that split the channels.
+template <int R>
+__device__ __forceinline__ void tmem_sum_slots(uint32_t (&v)[16 / R][2 * R], const OutRange& r, int a) {
+  constexpr int kB = 16 / R, kNV = 2 * R;
 #pragma unroll
-  for (int b = 0; b < 4; ++b) tmem_ld8_nowait(v[b], r.t0 + (a + b) * 8);
+  for (int b = 0; b < kB; ++b) tmem_ld_slot_nowait<kNV>(v[b], r.t0 + (a + b) * kNV);
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll 1
   for (int j = 1; j < r.zs; ++j) {
-    uint32_t t[4][8];
+    uint32_t t[kB][kNV];
 #pragma unroll
-    for (int b = 0; b < 4; ++b) tmem_ld8_nowait(t[b], r.t0 + j * (kGroup * 8) + (a + b) * 8);
+    for (int b = 0; b < kB; ++b) tmem_ld_slot_nowait<kNV>(t[b], r.t0 + j * (kGroup * kNV) + (a + b) * kNV);
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-    for (int b = 0; b < 4; ++b)
+    for (int b = 0; b < kB; ++b)
 #pragma unroll
-      for (int e = 0; e < 8; ++e)
+      for (int e = 0; e < kNV; ++e)
         v[b][e] = __float_as_uint(__uint_as_float(v[b][e]) + __uint_as_float(t[b][e]));
   }
 }
 
-// Outputs of one consumer warp (filter slots x 4 rows x {A,B} per lane).  `my_o` / `my_b` hold, in
+// Outputs of one consumer warp (filter slots x R rows x {A,B} per lane).  `my_o` / `my_b` hold, in
 // lane a < 16, the original filter index and the bias of slot a (loaded at kernel start).
-template <bool GENERIC, int MODE, bool HALF, bool RELU>
+template <int R, bool GENERIC, int MODE, bool HALF, bool RELU>
 __device__ __forceinline__ void write_outputs(const Geo& g, const LaneOut& lo, const LaneOut& lp,
                                               void* __restrict__ y, float* __restrict__ ws,
                                               const u64 (&acc)[GENERIC ? kGroup : 1][4],
                                               const OutRange& r, int my_o, float my_b) {
+  constexpr int kNV = 2 * R;
   const long long plane = (long long)g.h_out * g.w_out;
   const long long plane_y = (long long)g.h_y * g.w_y;
   // one filter slot: plain stores / atomics, or the fused 2x2 max-pool (warp-uniform choice)
-  auto emit = [&](int o, float bv, const uint32_t (&v)[8]) {
+  auto emit = [&](int o, float bv, const uint32_t (&v)[kNV]) {
     if (MODE == 0 && g.pool) {
-      float f[8];
+      float f[kNV];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[e]);
-      emit_slot_pooled<HALF, RELU>(g, lp, y, (long long)o * plane_y, bv, f);
+      for (int e = 0; e < kNV; ++e) f[e] = __uint_as_float(v[e]);
+      emit_slot_pooled<R, HALF, RELU>(g, lp, y, (long long)o * plane_y, bv, f);
     } else {
-      emit_slot<MODE, HALF, RELU>(g, lo, y, ws, (long long)o * plane, bv, v);
+      emit_slot<R, MODE, HALF, RELU>(g, lo, y, ws, (long long)o * plane, bv, v);
     }
   };
-  // MODE 1: `ws` is the lane's first float of the warp's first slot (r.a0); slots are 256 floats apart
-  auto emit_ws = [&](int a, const uint32_t (&v)[8]) {
-    emit_slot<1, false, false>(g, lo, y, ws + (size_t)(a - r.a0) * 256, 0, 0.f, v);
+  // MODE 1: `ws` is the lane's first float of the warp's first slot (r.a0); slots are 32 x 2 R floats apart
+  auto emit_ws = [&](int a, const uint32_t (&v)[kNV]) {
+    emit_slot<R, 1, false, false>(g, lo, y, ws + (size_t)(a - r.a0) * (32 * kNV), 0, 0.f, v);
   };
   if constexpr (GENERIC) {
+    static_assert(!GENERIC || R == 4, "register accumulators hold 4 rows");
 #pragma unroll
     for (int a = 0; a < kGroup; ++a) {
-      uint32_t v[8];
+      uint32_t v[kNV];
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         v[2 * k] = (uint32_t)acc[a][k];
@@ -869,12 +908,13 @@ __device__ __forceinline__ void write_outputs(const Geo& g, const LaneOut& lo, c
       if (o >= 0) emit(o, bv, v);
     }
   } else {
+    constexpr int kB = 16 / R;
 #pragma unroll 1
-    for (int a = r.a0; a < r.a1; a += 4) {  // run-time TMEM addresses: four slots per round trip
-      uint32_t v[4][8];
-      tmem_sum4(v, r, a);
+    for (int a = r.a0; a < r.a1; a += kB) {  // run-time TMEM addresses: several slots per round trip
+      uint32_t v[kB][kNV];
+      tmem_sum_slots<R>(v, r, a);
 #pragma unroll
-      for (int b = 0; b < 4; ++b) {
+      for (int b = 0; b < kB; ++b) {
         const int o = __shfl_sync(0xffffffffu, my_o, a + b);
         const float bv = __shfl_sync(0xffffffffu, my_b, a + b);
         if (o >= 0) {
@@ -887,44 +927,45 @@ __device__ __forceinline__ void write_outputs(const Geo& g, const LaneOut& lo, c
 }
 
 // The last split to finish a warp's part of an output tile: workspace -> y, leaving the workspace
-// zeroed.  `ws` is the lane's first float of the warp's first slot (a_begin); a slot's 8 sums
-// come back as two 16-byte loads, four slots (eight loads per lane) in flight at once.
-template <bool HALF, bool RELU>
+// zeroed.  `ws` is the lane's first float of the warp's first slot (a_begin); a slot's 2 R sums
+// come back as 16-byte loads, 16 / R slots (eight loads per lane) in flight at once.
+template <int R, bool HALF, bool RELU>
 __device__ __forceinline__ void finalize_outputs(const Geo& g, const LaneOut& lo, const LaneOut& lp,
                                                  void* __restrict__ y, float* __restrict__ ws,
                                                  int a_begin, int a_end, int my_o, float my_b) {
   const long long plane = (long long)g.h_out * g.w_out;
   const long long plane_y = (long long)g.h_y * g.w_y;
-  constexpr int kBatch = 4;
+  constexpr int kBatch = 16 / R, kNV = 2 * R;
 #pragma unroll 1
   for (int a0 = a_begin; a0 < a_end; a0 += kBatch) {
-    float v[kBatch][8];
+    float v[kBatch][kNV];
     int fo[kBatch];
     float bv[kBatch];
 #pragma unroll
     for (int b = 0; b < kBatch; ++b) {
       fo[b] = __shfl_sync(0xffffffffu, my_o, a0 + b);
       bv[b] = __shfl_sync(0xffffffffu, my_b, a0 + b);
-      float4* p = reinterpret_cast<float4*>(ws + (size_t)(a0 + b - a_begin) * 256);
-      const float4 lo4 = (fo[b] < 0) ? make_float4(0.f, 0.f, 0.f, 0.f) : __ldcg(p);
-      const float4 hi4 = (fo[b] < 0) ? make_float4(0.f, 0.f, 0.f, 0.f) : __ldcg(p + 1);
-      v[b][0] = lo4.x; v[b][1] = lo4.y; v[b][2] = lo4.z; v[b][3] = lo4.w;
-      v[b][4] = hi4.x; v[b][5] = hi4.y; v[b][6] = hi4.z; v[b][7] = hi4.w;
+      float4* p = reinterpret_cast<float4*>(ws + (size_t)(a0 + b - a_begin) * (32 * kNV));
+#pragma unroll
+      for (int i = 0; i < kNV / 4; ++i) {
+        const float4 q = (fo[b] < 0) ? make_float4(0.f, 0.f, 0.f, 0.f) : __ldcg(p + i);
+        v[b][4 * i] = q.x; v[b][4 * i + 1] = q.y; v[b][4 * i + 2] = q.z; v[b][4 * i + 3] = q.w;
+      }
     }
 #pragma unroll
     for (int b = 0; b < kBatch; ++b) {
       if (fo[b] < 0) continue;
-      float4* p = reinterpret_cast<float4*>(ws + (size_t)(a0 + b - a_begin) * 256);
-      p[0] = make_float4(0.f, 0.f, 0.f, 0.f);
-      p[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+      float4* p = reinterpret_cast<float4*>(ws + (size_t)(a0 + b - a_begin) * (32 * kNV));
+#pragma unroll
+      for (int i = 0; i < kNV / 4; ++i) p[i] = make_float4(0.f, 0.f, 0.f, 0.f);
       if (g.pool) {
-        emit_slot_pooled<HALF, RELU>(g, lp, y, (long long)fo[b] * plane_y, bv[b], v[b]);
+        emit_slot_pooled<R, HALF, RELU>(g, lp, y, (long long)fo[b] * plane_y, bv[b], v[b]);
         continue;
       }
       const long long fb = (long long)fo[b] * plane;
       const long long ia = fb + lo.base_a, ib = fb + lo.base_b;
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
+      for (int k = 0; k < R; ++k) {
         const int row = k * g.w_out;
         if (lo.mask >> (2 * k) & 1u) store_out<HALF, RELU>(y, ia + row, v[b][2 * k] + bv[b]);
         if (lo.mask >> (2 * k + 1) & 1u) store_out<HALF, RELU>(y, ib + row, v[b][2 * k + 1] + bv[b]);
@@ -999,13 +1040,15 @@ __device__ __forceinline__ bool dependency_wait(const ChainCtx& cc, int lane, in
   return ok != 0;
 }
 
-template <int S, bool GENERIC, bool WIDE>
+template <int S, bool GENERIC, bool WIDE, int R>
 __device__ __forceinline__ void tiled_body(const DeviceLayer& L, const Geo& g, const void* __restrict__ x,
                                            const float* __restrict__ bias, void* __restrict__ y,
                                            float* __restrict__ ws, int* __restrict__ counters,
                                            unsigned char* smem, const BlockPos bp, const ChainCtx cc) {
-  constexpr int kCW = consumer_warps(GENERIC);
-  constexpr int kThreads = cta_threads(GENERIC);
+  static_assert(R == 4 || (R == 8 && !GENERIC && !WIDE), "8 rows per lane: canonical TMEM bodies only");
+  constexpr int kCW = consumer_warps(GENERIC, R);
+  constexpr int kThreads = cta_threads(GENERIC, R);
+  constexpr int kNV = 2 * R;              // TMEM columns of one filter slot
   const uint32_t sbase = smem_u32(smem);
   const int tid = threadIdx.x, lane = tid & 31;
   // broadcast from lane 0: tells the compiler that everything derived from it is warp-uniform
@@ -1051,7 +1094,7 @@ __device__ __forceinline__ void tiled_body(const DeviceLayer& L, const Geo& g, c
     t.n = qq / per_img;
     const int rem = qq - t.n * per_img;
     const int tyi = rem / g.tx;
-    t.y0 = tyi * 4;
+    t.y0 = tyi * R;
     t.x0 = (rem - tyi * g.tx) * g.tw;
     tab[i] = t;
   }
@@ -1085,15 +1128,12 @@ __device__ __forceinline__ void tiled_body(const DeviceLayer& L, const Geo& g, c
 
   // Consumer-warp coordinates (meaningless for producer warps).  zs warps of one TMEM lane
   // quadrant form a unit: they work on the same pixels and filter group and take the chunks in
-  // turn, each with accumulators in its own 128 TMEM columns.
+  // turn, each with accumulators in its own 16 x 2 R TMEM columns.
   const int zs = GENERIC ? 1 : g.zs;
   int unit = warp, z = 0;
-  if (zs == 2) {
-    unit = (warp & 3) + 4 * (warp >> 3);
-    z = (warp >> 2) & 1;
-  } else if (zs == 4) {
-    unit = warp & 3;
-    z = warp >> 2;
+  if (zs > 1) {
+    z = (warp >> 2) % zs;
+    unit = (warp & 3) + 4 * ((warp >> 2) / zs);
   }
   const int wyi = unit % g.wys, wgi = unit / g.wys;
   const int gi = bp.y * g.ng + wgi;
@@ -1105,10 +1145,10 @@ __device__ __forceinline__ void tiled_body(const DeviceLayer& L, const Geo& g, c
   const uint32_t off_right = (S == 1) ? 2 * col_b : col_b;                   // window column 2
   const uint32_t chan_b = (uint32_t)g.chan_stride;
   const uint32_t lane_off = (uint32_t)(slot * g.substride) + (uint32_t)col * col_b;
-  // TMEM: a warp reaches the 32 lanes of its quadrant (warp % 4); 4 warps share a quadrant and
-  // take 128 columns each = 16 filter slots x (4 rows x {A,B}).
+  // TMEM: a warp reaches the 32 lanes of its quadrant (warp % 4); the 4 (R = 4) or 2 (R = 8) warps
+  // of a quadrant take 128 or 256 columns each = 16 filter slots x (R rows x {A,B}).
   const uint32_t tquad = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);
-  const uint32_t tq = tquad + (uint32_t)((warp >> 2) * (kGroup * 8));
+  const uint32_t tq = tquad + (uint32_t)((warp >> 2) * (kGroup * kNV));
 
   // lane a < 16 keeps the original filter index and bias of slot a for the epilogue
   int my_o = -1;
@@ -1130,13 +1170,13 @@ __device__ __forceinline__ void tiled_body(const DeviceLayer& L, const Geo& g, c
 #pragma unroll
       for (int i = 0; i < kPreElems; ++i) {
         const int e = ptid + i * kProducerThreads;
-        pre[i] = raw_elem<S>(g, e < n_elem ? e : 0);
+        pre[i] = raw_elem<S, R>(g, e < n_elem ? e : 0);
         if (e >= n_elem) pre[i].dst = kSkipElem;
       }
       if (dependency_wait(cc, lane, warp, smem, L.err))
-        produce_raw_stream<S>(L, g, (const __half*)x, tab, pre, desc, codes, sbase, k0, nk, ptid);
+        produce_raw_stream<S, R>(L, g, (const __half*)x, tab, pre, desc, codes, sbase, k0, nk, ptid);
     } else {
-      precompute_elems<S>(pre, L, g, tab, ptid);
+      precompute_elems<S, R>(pre, L, g, tab, ptid);
       // the weight records and codes of the first ring-full of chunks do not depend on the previous
       // kernel: fetch them while it finishes
       const int n_early = min(g.stages, nk);
@@ -1151,13 +1191,13 @@ __device__ __forceinline__ void tiled_body(const DeviceLayer& L, const Geo& g, c
       if (!dependency_wait(cc, lane, warp, smem, L.err)) {
         // the previous layer never completed: nothing more is staged, the consumers give up too
       } else if (g.is_half) {
-        produce_half_stream<S>(L, g, (const __half*)x, tab, pre, desc, codes, sbase, k0, nk, n_early, ptid);
+        produce_half_stream<S, R>(L, g, (const __half*)x, tab, pre, desc, codes, sbase, k0, nk, n_early, ptid);
       } else {
         for (int kk = n_coop; kk < nk; ++kk) {
           const int s = kk % g.stages, it = kk / g.stages;
           if (it > 0 && !mbar_wait(sbase + 8 * (kMaxStages + s), (it - 1) & 1, L.err, 1)) break;
           const uint32_t stage_base = sbase + g.stage_off + s * g.stage_bytes;
-          produce_chunk_async<S>(L, g, (const float*)x, tab, pre, desc, codes, stage_base, k0 + kk, kk, ptid,
+          produce_chunk_async<S, R>(L, g, (const float*)x, tab, pre, desc, codes, stage_base, k0 + kk, kk, ptid,
                                  true, kk >= n_early);
           if (!PCONV_WITHHELD(kk, ptid)) cp_async_arrive(sbase + 8 * s);
         }
@@ -1172,14 +1212,14 @@ __device__ __forceinline__ void tiled_body(const DeviceLayer& L, const Geo& g, c
 #pragma unroll
         for (int k = 0; k < 4; ++k) acc[a][k] = 0ull;
     } else {
-      for (int a = 0; a < kGroup; ++a) tmem_st8_zero(tq + a * 8);
+      for (int a = 0; a < kGroup * kNV; a += 8) tmem_st8_zero(tq + a);
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
     }
     ok = dependency_wait(cc, lane, warp, smem, L.err);
     // (each consumer thread arrives on the chunk's own barrier when its copies for that chunk
     // have landed; a warp waits for that barrier as well as for the producers' before the chunk)
     for (int kk = 0; ok && kk < n_coop; ++kk) {
-      fill_chunk_x<S>(L, g, (const float*)x, tab, sbase + g.stage_off + kk * g.stage_bytes, k0 + kk,
+      fill_chunk_x<S, R>(L, g, (const float*)x, tab, sbase + g.stage_off + kk * g.stage_bytes, k0 + kk,
                       warp * 32 + lane, 32 * kCW);
       cp_async_arrive(coop_bar + 8 * kk);
     }
@@ -1224,7 +1264,7 @@ __device__ __forceinline__ void tiled_body(const DeviceLayer& L, const Geo& g, c
           const uint4 d0 = desc[2 * (wgi * g.cps + kk)], d1 = desc[2 * (wgi * g.cps + kk) + 1];
           if (d0.y) {  // the block has kernels: enter at its first channel
             if constexpr (WIDE) dispatch_chunk_wide<S>(cp, wp, xptr, chan_b, col_b, off_mid, tq, (d1.z + 1u) << 8);
-            else dispatch_chunk<S>(cp, wp, xptr, chan_b, col_b, off_mid, tq, (d1.z + 1u) << 4);
+            else dispatch_chunk<S, R>(cp, wp, xptr, chan_b, col_b, off_mid, tq, (d1.z + 1u) << 4);
           }
         } else {
           u64 win[Win<S>::kRows][3];
@@ -1278,27 +1318,27 @@ __device__ __forceinline__ void tiled_body(const DeviceLayer& L, const Geo& g, c
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         asm volatile("bar.sync %0, %1;" ::"r"(3 + unit), "r"(32 * zs) : "memory");
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        orng.t0 = tquad + (uint32_t)(((warp >> 2) - z) * (kGroup * 8));
+        orng.t0 = tquad + (uint32_t)(((warp >> 2) - z) * (kGroup * kNV));
         orng.zs = zs;
         orng.a0 = z * (kGroup / zs);
         orng.a1 = orng.a0 + kGroup / zs;
       }
     }
     if (active && ok) {
-      const LaneOut lo = lane_outputs(L, g, tab, slot, col);
-      const LaneOut lp = g.pool ? lane_outputs_pooled(L, g, tab, slot, col) : lo;
+      const LaneOut lo = lane_outputs<R>(L, g, tab, slot, col);
+      const LaneOut lp = g.pool ? lane_outputs_pooled<R>(L, g, tab, slot, col) : lo;
       bool split = false;
       if constexpr (!GENERIC) split = g.ks > 1;
       if (!split) {
         with_flags(g, [&](auto half, auto relu) {
-          write_outputs<GENERIC, 0, decltype(half)::value, decltype(relu)::value>(g, lo, lp, y, ws, acc,
-                                                                                   orng, my_o, my_b);
+          write_outputs<R, GENERIC, 0, decltype(half)::value, decltype(relu)::value>(g, lo, lp, y, ws, acc,
+                                                                                      orng, my_o, my_b);
         });
       } else {
-        // this lane's floats in the warp's part of the tile's workspace: [tile][warp][slot][lane][8]
+        // this lane's floats in the warp's part of the tile's workspace: [tile][warp][slot][lane][2 R]
         const int spw = kGroup / (GENERIC ? 1 : g.zs);   // slots a warp writes out
-        float* wsl = ws + ((((size_t)bp.y * bp.gx + bp.x) * kCW + warp) * spw * 32 + lane) * 8;
-        write_outputs<GENERIC, 1, false, false>(g, lo, lp, y, wsl, acc, orng, my_o, my_b);
+        float* wsl = ws + ((((size_t)bp.y * bp.gx + bp.x) * kCW + warp) * spw * 32 + lane) * kNV;
+        write_outputs<R, GENERIC, 1, false, false>(g, lo, lp, y, wsl, acc, orng, my_o, my_b);
         PCONV_MARK(4)
         PCONV_MARK_MAX(10)
         // Every warp owns the same part of the output tile in each of the ks splits, and takes a
@@ -1318,8 +1358,8 @@ __device__ __forceinline__ void tiled_body(const DeviceLayer& L, const Geo& g, c
         if (t == g.ks - 1) {
           __threadfence();
           with_flags(g, [&](auto half, auto relu) {
-            finalize_outputs<decltype(half)::value, decltype(relu)::value>(g, lo, lp, y, wsl, orng.a0,
-                                                                          orng.a1, my_o, my_b);
+            finalize_outputs<R, decltype(half)::value, decltype(relu)::value>(g, lo, lp, y, wsl, orng.a0,
+                                                                             orng.a1, my_o, my_b);
           });
         }
       }
@@ -1339,8 +1379,8 @@ __device__ __forceinline__ void tiled_body(const DeviceLayer& L, const Geo& g, c
   PCONV_MARK_MAX(7)
 }
 
-template <int S, bool GENERIC, bool WIDE>
-__global__ void __launch_bounds__(cta_threads(GENERIC), 1)
+template <int S, bool GENERIC, bool WIDE, int R>
+__global__ void __launch_bounds__(cta_threads(GENERIC, R), 1)
 tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
              const float* __restrict__ bias, void* __restrict__ y, float* __restrict__ ws,
              int* __restrict__ counters) {
@@ -1355,7 +1395,7 @@ tiled_kernel(const DeviceLayer L, const Geo g, const void* __restrict__ x,
   cc.target = 0;
   cc.own_tmem = 1;
   cc.reinit = 0;
-  tiled_body<S, GENERIC, WIDE>(L, g, x, bias, y, ws, counters, smem, bp, cc);
+  tiled_body<S, GENERIC, WIDE, R>(L, g, x, bias, y, ws, counters, smem, bp, cc);
 }
 
 // One layer of a chain, as the chain kernel reads it from device memory.
@@ -1407,7 +1447,7 @@ tiled_chain_kernel(const ChainLayer* __restrict__ layers, int n_layers, const vo
       bp.x = cta % cl.gx;
       bp.y = (cta / cl.gx) % cl.gy;
       bp.z = cta / (cl.gx * cl.gy);
-      tiled_body<1, false, false>(cl.L, cl.g, xl, cl.bias, yl, ws, counters, smem, bp, cc);
+      tiled_body<1, false, false, 4>(cl.L, cl.g, xl, cl.bias, yl, ws, counters, smem, bp, cc);
       used = true;
     } else if (warp == 0) {
       // (in step with the others all the same: its arrival for this layer must not be counted
@@ -1466,11 +1506,15 @@ int pick_stages(int fit, int zs, int cps) {
   return s >= (zs == 1 ? 2 : zs) ? s : 0;
 }
 
-// Geometry for `zs` consumer warps per unit and no channel split across CTAs.
+// Geometry for `zs` consumer warps per unit, R output rows per lane and no channel split across CTAs.
 template <bool GENERIC>
-bool geo_for(const DeviceLayer& L, int n, int h, int w, int zs, Geo* out) {
-  const int units = consumer_warps(GENERIC) / zs;
+bool geo_for(const DeviceLayer& L, int n, int h, int w, int zs, int R, Geo* out) {
+  // the warps of a unit add up column sets of the same TMEM lanes: they sit in one lane quadrant,
+  // which holds a quarter of the consumer warps
+  if (zs > consumer_warps(GENERIC, R) / 4) return false;
+  const int units = consumer_warps(GENERIC, R) / zs;
   Geo g;
+  g.rpl = R;
   g.n = n;
   g.h = h;
   g.w = w;
@@ -1481,7 +1525,7 @@ bool geo_for(const DeviceLayer& L, int n, int h, int w, int zs, Geo* out) {
   while (g.tw > 2 && g.tw / 2 >= g.w_out) g.tw /= 2;
   g.sw = 32 / g.tw;
   g.tx = (g.w_out + g.tw - 1) / g.tw;
-  g.ty = (g.h_out + 3) / 4;
+  g.ty = (g.h_out + R - 1) / R;
   const long long q = (long long)n * g.tx * g.ty;
   if (q > 0x7FFFFFFF) return false;
   g.q_total = (int)q;
@@ -1502,13 +1546,13 @@ bool geo_for(const DeviceLayer& L, int n, int h, int w, int zs, Geo* out) {
     const long long need = (pairs_needed + g.sw - 1) / g.sw;
     if (need < g.wy) g.wy = need < 1 ? 1 : (int)need;
   }
-  g.rows = (L.stride == 1) ? 6 : 9;
+  g.rows = L.stride * (R - 1) + 3;
   g.pitch = (L.stride == 1) ? (g.tw + 2) : (2 * g.tw + 1);
   // The staged tile is column-major: the rows of a column are contiguous float2, so a lane's
-  // window column comes in 16-byte loads.  48 B (80 B at stride 2) between columns keeps the 8
-  // lanes of a quarter-warp on distinct 16-byte bank groups; narrower sub-tiles are offset so that
-  // the sub-tiles sharing a quarter-warp do not collide.
-  g.colstride = (L.stride == 1) ? 48 : 80;
+  // window column comes in 16-byte loads.  48 B (80 B at stride 2; 80 B and 144 B with 8 rows per
+  // lane) between columns keeps the 8 lanes of a quarter-warp on distinct 16-byte bank groups;
+  // narrower sub-tiles are offset so that the sub-tiles sharing a quarter-warp do not collide.
+  g.colstride = (g.rows * 8 + 15) & ~15;
   g.substride = g.pitch * g.colstride;
   if (g.tw == 4) while (g.substride % 128 != 64) g.substride += 16;
   if (g.tw == 2) while (g.substride % 128 != 32) g.substride += 16;
@@ -1563,11 +1607,16 @@ void set_split(const DeviceLayer& L, Geo* g, int ks) {
 // staged elements (measured 0.5 us + 4 ns per element), zs chunks being consumed at a time; CTAs
 // run in waves of one per SM; a channel split across CTAs adds the atomic traffic of every CTA's
 // tile and its draining.
+constexpr double kTallKernelTime = 0.93;
 double geo_cost(const DeviceLayer& L, const Geo& g) {
   const double k_unit = (double)L.n_kept / (L.n_groups > 0 ? L.n_groups : 1);  // kernels of one group
   const double per_chunk = 1.5;                                                // barrier, entry, exit
   const int turns = (g.cps + g.zs - 1) / g.zs;                                 // chunks per warp
-  const double consume = k_unit / L.n_chunks + per_chunk;
+  // (with 8 rows per lane a warp's kernel covers 512 pixels and its scheduler serves two warps
+  // instead of four: measured per-warp time per kernel relative to the 4-row form, on layers
+  // with one warp per unit)
+  const double k_time = (g.rpl == 8) ? kTallKernelTime : 1.0;
+  const double consume = k_time * k_unit / L.n_chunks + per_chunk;
   const double produce = 3.0 + 0.024 * (g.pairs * g.rows * g.pitch);
   const double chunk = consume > g.zs * produce ? consume : g.zs * produce;
   const double loop = turns * chunk;
@@ -1578,61 +1627,71 @@ double geo_cost(const DeviceLayer& L, const Geo& g) {
   return waves * (fixed + loop) + (g.ks > 1 ? 100.0 / g.zs : 0.0);
 }
 
-// The geometry of a launch.  Canonical pattern sets choose how the 16 consumer warps are used
-// (zs = 1, 2 or 4 warps per unit) and, when a workspace is available, whether the channel range
-// is also split across CTAs, by the estimate above.
+// The geometry of a launch.  Canonical pattern sets choose the rows per lane (`rmode`: 4, 8 or
+// 0 = by the estimate; 8 needs one-byte codes), how the consumer warps are used (zs = 1, 2 or 4
+// warps per unit) and, when a workspace is available, whether the channel range is also split
+// across CTAs, by the estimate above.
 template <bool GENERIC>
-bool make_geo(const DeviceLayer& L, int n, int h, int w, bool allow_split, Geo* out) {
-  if (GENERIC) return geo_for<true>(L, n, h, w, 1, out);
+bool make_geo(const DeviceLayer& L, int n, int h, int w, bool allow_split, int rmode, Geo* out) {
+  if (GENERIC) return geo_for<true>(L, n, h, w, 1, 4, out);
   bool found = false;
   double best = 0.0;
 #ifdef PCONV_DEV
   const char* force_zs = getenv("PCONV_FORCE_ZS");
   const char* force_ks = getenv("PCONV_FORCE_KS");
 #endif
-  for (int zs = 1; zs <= 4; zs *= 2) {
-    Geo g;
+  for (int R = 4; R <= 8; R *= 2) {
+    if (rmode && rmode != R) continue;
+    if (R == 8 && L.wide_codes) continue;
+    // Left to itself the planner takes 8 rows per lane only where the 4-row form already runs one
+    // warp per unit on the whole channel range (large batches): measured 3-10 % faster there, and
+    // slower wherever channels are split (a TMEM lane quadrant then holds two warps, not four).
+    if (R == 8 && !rmode && found && (out->zs != 1 || out->ks != 1)) continue;
+    for (int zs = 1; zs <= 4; zs *= 2) {
+      if (R == 8 && !rmode && zs != 1) continue;
+      Geo g;
 #ifdef PCONV_DEV
-    if (force_zs && atoi(force_zs) != zs) continue;
+      if (force_zs && atoi(force_zs) != zs) continue;
 #endif
-    if (!geo_for<false>(L, n, h, w, zs, &g)) continue;
+      if (!geo_for<false>(L, n, h, w, zs, R, &g)) continue;
 #ifdef PCONV_DEV
-    if (force_ks && allow_split) {
-      set_split(L, &g, atoi(force_ks));
-      if (g.stages < 1) continue;
-      *out = g;
-      return true;
-    }
-#endif
-    for (int pass = 0; pass < 2; ++pass) {
-      Geo c = g;
-      if (pass == 1) {
-        if (!allow_split) break;
-        const long long tiles = geo_tiles(L, g);
-        const long long ks = device_sm_count() / tiles;   // fill one wave
-        if (ks < 2) break;
-        set_split(L, &c, (int)ks);
-        if (c.ks < 2 || c.stages < 1) break;
+      if (force_ks && allow_split) {
+        set_split(L, &g, atoi(force_ks));
+        if (g.stages < 1) continue;
+        *out = g;
+        return true;
       }
-      const double cost = geo_cost(L, c);
-      if (!found || cost < best) {
-        found = true;
-        best = cost;
-        *out = c;
+#endif
+      for (int pass = 0; pass < 2; ++pass) {
+        Geo c = g;
+        if (pass == 1) {
+          if (!allow_split || (R == 8 && !rmode)) break;
+          const long long tiles = geo_tiles(L, g);
+          const long long ks = device_sm_count() / tiles;   // fill one wave
+          if (ks < 2) break;
+          set_split(L, &c, (int)ks);
+          if (c.ks < 2 || c.stages < 1) break;
+        }
+        const double cost = geo_cost(L, c);
+        if (!found || cost < best) {
+          found = true;
+          best = cost;
+          *out = c;
+        }
       }
     }
   }
   return found;
 }
 
-template <int S, bool GENERIC, bool WIDE>
+template <int S, bool GENERIC, bool WIDE, int R>
 cudaError_t launch_one(const DeviceLayer& L, Geo g, const void* x, const float* bias, void* y, float* ws,
                        int* counters, cudaStream_t stream) {
   int smem = g.stage_off + g.stages * g.stage_bytes;
   // the TMEM variant must be alone on its SM (it takes all 512 columns): make sure two CTAs can
   // never be co-resident by asking for more than half of the shared memory
   if (!GENERIC && smem < 120 * 1024) smem = 120 * 1024;
-  cudaError_t e = cudaFuncSetAttribute(tiled_kernel<S, GENERIC, WIDE>,
+  cudaError_t e = cudaFuncSetAttribute(tiled_kernel<S, GENERIC, WIDE, R>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
   if (e != cudaSuccess) return e;
   const long long ctas_x = ((long long)g.q_total + 2 * g.pairs - 1) / (2 * g.pairs);
@@ -1640,7 +1699,7 @@ cudaError_t launch_one(const DeviceLayer& L, Geo g, const void* x, const float* 
   if (ctas_x > 0x7FFFFFFF || ctas_y > 65535 || g.ks > 65535) return cudaErrorInvalidValue;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)ctas_x, (unsigned)ctas_y, (unsigned)g.ks);
-  cfg.blockDim = dim3(cta_threads(GENERIC), 1, 1);
+  cfg.blockDim = dim3(cta_threads(GENERIC, R), 1, 1);
   cfg.dynamicSmemBytes = (size_t)smem;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
@@ -1648,7 +1707,7 @@ cudaError_t launch_one(const DeviceLayer& L, Geo g, const void* x, const float* 
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, tiled_kernel<S, GENERIC, WIDE>, L, g, x, bias, y, ws, counters);
+  return cudaLaunchKernelEx(&cfg, tiled_kernel<S, GENERIC, WIDE, R>, L, g, x, bias, y, ws, counters);
 }
 
 
@@ -1658,31 +1717,34 @@ bool tiled_supported(const DeviceLayer& L, int n, int h, int w) {
   Geo g;
   if (n <= 0 || h <= 0 || w <= 0) return false;
   if (L.n_groups > 65535) return false;
-  return make_geo<true>(L, n, h, w, false, &g) && make_geo<false>(L, n, h, w, false, &g);
+  return make_geo<true>(L, n, h, w, false, 4, &g) && make_geo<false>(L, n, h, w, false, 4, &g);
 }
 
 // Workspace of the channel-split path: the partial sums of every (tile, consumer warp, filter slot
 // the warp writes out, lane) as 8 floats -- the layout of the warps that add to it and read it
 // back, not y's --, then one ticket per (tile, consumer warp); 0 if this shape is never split.
 size_t split_sums_bytes(const DeviceLayer& L, const Geo& g) {
-  return (size_t)geo_tiles(L, g) * consumer_warps(false) * (kGroup / g.zs) * 32 * 8 * sizeof(float);
+  return (size_t)geo_tiles(L, g) * consumer_warps(false, g.rpl) * (kGroup / g.zs) * 32 * (2 * g.rpl) * sizeof(float);
 }
-size_t tiled_workspace_bytes(const DeviceLayer& L, int n, int h, int w) {
+// `rmode`: rows per lane the launch will be asked for (4, 8, 0 = the planner's choice).
+size_t tiled_workspace_bytes(const DeviceLayer& L, int n, int h, int w, int rmode) {
   Geo g;
-  if (!L.codes_s || !make_geo<false>(L, n, h, w, true, &g) || g.ks <= 1) return 0;
+  if (!L.codes_s || !make_geo<false>(L, n, h, w, true, rmode, &g) || g.ks <= 1) return 0;
   const size_t ctas = (size_t)geo_tiles(L, g);
   return ((split_sums_bytes(L, g) + 255) & ~(size_t)255) +
-         ((ctas * consumer_warps(false) * 4 + 255) & ~(size_t)255);
+         ((ctas * kMaxConsumerWarps * 4 + 255) & ~(size_t)255);
 }
 
 // The launch geometry launch_tiled would use (see pconv_plan_t).
 bool tiled_plan(const DeviceLayer& L, int n, int h, int w, bool generic_taps, bool with_workspace,
-                pconv_plan_t* out) {
+                int rmode, pconv_plan_t* out) {
   if (!generic_taps && !L.codes_s) generic_taps = true;
   Geo g;
-  if (!(generic_taps ? make_geo<true>(L, n, h, w, false, &g) : make_geo<false>(L, n, h, w, with_workspace, &g)))
+  if (!(generic_taps ? make_geo<true>(L, n, h, w, false, 4, &g)
+                     : make_geo<false>(L, n, h, w, with_workspace, rmode, &g)))
     return false;
   out->generic_taps = generic_taps ? 1 : 0;
+  out->rows_per_lane = g.rpl;
   out->warps_per_unit = g.zs;
   out->channel_splits = g.ks;
   out->groups_per_cta = g.ng;
@@ -1695,13 +1757,14 @@ bool tiled_plan(const DeviceLayer& L, int n, int h, int w, bool generic_taps, bo
 }
 
 cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias, void* y, int n, int h,
-                         int w, bool relu, bool pool, bool reproducible, bool generic_taps, void* ws,
-                         size_t ws_bytes, cudaStream_t stream) {
+                         int w, bool relu, bool pool, bool reproducible, bool generic_taps, int rmode,
+                         void* ws, size_t ws_bytes, cudaStream_t stream) {
   if (!generic_taps && !L.codes_s) generic_taps = true;
+  if (rmode == 8 && (generic_taps || L.wide_codes)) return cudaErrorInvalidValue;
   Geo g;
-  const size_t need = generic_taps ? 0 : tiled_workspace_bytes(L, n, h, w);
+  const size_t need = generic_taps ? 0 : tiled_workspace_bytes(L, n, h, w, rmode);
   const bool split = !reproducible && need > 0 && ws && ws_bytes >= need;
-  if (!(generic_taps ? make_geo<true>(L, n, h, w, false, &g) : make_geo<false>(L, n, h, w, split, &g)))
+  if (!(generic_taps ? make_geo<true>(L, n, h, w, false, 4, &g) : make_geo<false>(L, n, h, w, split, rmode, &g)))
     return cudaErrorInvalidValue;
   g.relu = relu ? 1 : 0;
   if (reproducible && g.zs > 1) {
@@ -1723,13 +1786,15 @@ cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias,
   }
   const bool wide = L.wide_codes != 0;
   if (L.stride == 1) {
-    if (generic_taps) return launch_one<1, true, false>(L, g, x, bias, y, wsf, counters, stream);
-    return wide ? launch_one<1, false, true>(L, g, x, bias, y, wsf, counters, stream)
-                : launch_one<1, false, false>(L, g, x, bias, y, wsf, counters, stream);
+    if (generic_taps) return launch_one<1, true, false, 4>(L, g, x, bias, y, wsf, counters, stream);
+    if (wide) return launch_one<1, false, true, 4>(L, g, x, bias, y, wsf, counters, stream);
+    return g.rpl == 8 ? launch_one<1, false, false, 8>(L, g, x, bias, y, wsf, counters, stream)
+                      : launch_one<1, false, false, 4>(L, g, x, bias, y, wsf, counters, stream);
   }
-  if (generic_taps) return launch_one<2, true, false>(L, g, x, bias, y, wsf, counters, stream);
-  return wide ? launch_one<2, false, true>(L, g, x, bias, y, wsf, counters, stream)
-              : launch_one<2, false, false>(L, g, x, bias, y, wsf, counters, stream);
+  if (generic_taps) return launch_one<2, true, false, 4>(L, g, x, bias, y, wsf, counters, stream);
+  if (wide) return launch_one<2, false, true, 4>(L, g, x, bias, y, wsf, counters, stream);
+  return g.rpl == 8 ? launch_one<2, false, false, 8>(L, g, x, bias, y, wsf, counters, stream)
+                    : launch_one<2, false, false, 4>(L, g, x, bias, y, wsf, counters, stream);
 }
 
 // ---- chains ---------------------------------------------------------------------------------------
@@ -1740,7 +1805,7 @@ cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias,
 bool chain_layer_ok(const DeviceLayer& L, int n, int h, int w, bool pool, long long* ctas) {
   if (!L.codes_s || L.wide_codes || L.stride != 1) return false;
   Geo g;
-  if (!make_geo<false>(L, n, h, w, true, &g)) return false;
+  if (!make_geo<false>(L, n, h, w, true, 4, &g)) return false;   // (the chain kernel is the 4-row form)
   if (pool && (g.h_out < 2 || g.w_out < 2)) return false;
   const long long c = geo_tiles(L, g) * g.ks;
   if (ctas) *ctas = c;
@@ -1758,7 +1823,7 @@ bool chain_fill(void* table, int index, const DeviceLayer& L, const void* x, con
   std::memset(&cl, 0, sizeof(cl));
   cl.L = L;
   if (status_dev) cl.L.err = status_dev;
-  if (!make_geo<false>(L, n, h, w, true, &cl.g)) return false;
+  if (!make_geo<false>(L, n, h, w, true, 4, &cl.g)) return false;
   cl.g.relu = relu ? 1 : 0;
   if (pool) {
     cl.g.pool = 1;
@@ -1784,7 +1849,7 @@ size_t chain_workspace_bytes(const void* table_host, int n_layers) {
       if (need > sums_max) sums_max = need;
     }
   if (!sums_max) return 0;
-  return ((sums_max + 255) & ~(size_t)255) + (((size_t)device_sm_count() * consumer_warps(false) * 4 + 255) & ~(size_t)255);
+  return ((sums_max + 255) & ~(size_t)255) + (((size_t)device_sm_count() * kMaxConsumerWarps * 4 + 255) & ~(size_t)255);
 }
 
 // Launches a chain: `table_dev` is the DEVICE copy of a filled table, `table_host` the host one
@@ -1809,7 +1874,7 @@ cudaError_t launch_chain(const void* table_dev, const void* table_host, int n_la
   if (ctas < 1 || ctas > device_sm_count()) return cudaErrorInvalidValue;
   // every layer of the chain finds its tickets behind the largest layer's sums
   const size_t tick_off = (sums_max + 255) & ~(size_t)255;
-  if (sums_max && (!ws || ws_bytes < tick_off + (size_t)device_sm_count() * consumer_warps(false) * 4))
+  if (sums_max && (!ws || ws_bytes < tick_off + (size_t)device_sm_count() * kMaxConsumerWarps * 4))
     return cudaErrorInvalidValue;
   if (smem < 120 * 1024) smem = 120 * 1024;
   cudaError_t e = cudaFuncSetAttribute(tiled_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);

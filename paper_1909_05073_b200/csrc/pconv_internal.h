@@ -129,16 +129,17 @@ cudaError_t launch_simple(const DeviceLayer& L, const void* x, const float* bias
                           int h, int w, bool relu, cudaStream_t stream);
 cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias, void* y, int n,
                          int h, int w, bool relu, bool pool, bool reproducible, bool generic_taps,
-                         void* ws, size_t ws_bytes, cudaStream_t stream);
+                         int rmode, void* ws, size_t ws_bytes, cudaStream_t stream);
 cudaError_t launch_tensor(const DeviceLayer& L, const void* x, const float* bias, void* y, int n,
                           int h, int w, bool relu, void* ws, size_t ws_bytes, cudaStream_t stream);
 size_t tensor_workspace_bytes(const DeviceLayer& L, int n, int h, int w);
 bool tensor_supported(const DeviceLayer& L, int n, int h, int w);
 bool tensor_preferred(const DeviceLayer& L, int n, int h, int w);
-size_t tiled_workspace_bytes(const DeviceLayer& L, int n, int h, int w);
+// rmode: output rows per lane of the tiled kernel (4, 8, or 0 = the planner chooses)
+size_t tiled_workspace_bytes(const DeviceLayer& L, int n, int h, int w, int rmode);
 bool tiled_supported(const DeviceLayer& L, int n, int h, int w);
 bool tiled_plan(const DeviceLayer& L, int n, int h, int w, bool generic_taps, bool with_workspace,
-                pconv_plan_t* out);
+                int rmode, pconv_plan_t* out);
 #ifdef PCONV_DEV
 cudaError_t dev_set_withhold(int chunk, unsigned spin_limit);   // see pconv_dev.h
 #endif

@@ -360,7 +360,9 @@ def test_every_warp_sharing_plan_matches_the_oracle():
             plan = B.pconv_plan(layer.handle, n, h, w, 0, with_ws)
             assert plan["generic_taps"] == 0 and plan["warps_per_unit"] in (1, 2, 4)
             assert plan["smem_bytes"] <= 227 * 1024 and plan["stages"] >= 1
-            assert (plan["channel_splits"] > 1) == (with_ws and B.pconv_workspace_bytes(layer.handle, n, h, w) > 0)
+            # (the workspace size covers the pinned forms too, so it may be non-zero where the
+            # planner's own choice does not split)
+            assert plan["channel_splits"] == 1 or (with_ws and B.pconv_workspace_bytes(layer.handle, n, h, w) > 0)
             seen.add((plan["warps_per_unit"], plan["channel_splits"] > 1))
             for _ in range(2):
                 y = layer.forward(xt, relu=True, split=with_ws)

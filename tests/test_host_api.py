@@ -112,8 +112,18 @@ def test_launch_plans_are_well_formed_over_many_shapes(lib):
         ws = bool(rng.random() < 0.5)
         kept = int(keep * c_in * c_out)
         flags = binding.KERNEL_GENERIC_TAPS if generic else 0
+        rows = int(rng.choice([0, 0, 4, 8])) if (canonical and not generic) else 0
+        flags |= {0: 0, 4: binding.ROWS4, 8: binding.ROWS8}[rows]
         p = binding.pconv_plan_shape(c_out, c_in, kept, stride, storage, canonical, n, h, w, flags, ws)
-        what = (c_out, c_in, h, w, n, stride, storage, keep, canonical, generic, ws, p)
+        what = (c_out, c_in, h, w, n, stride, storage, keep, canonical, generic, ws, rows, p)
+        assert p["rows_per_lane"] in (4, 8) and (rows == 0 or p["rows_per_lane"] == rows), what
+        if not canonical or generic:
+            assert p["rows_per_lane"] == 4, what
+        if p["rows_per_lane"] == 8:     # eight consumer warps, two per Tensor-Memory lane quadrant
+            assert p["warps_per_unit"] in (1, 2), what
+            assert p["groups_per_cta"] * p["pixel_sets"] * p["warps_per_unit"] <= 8, what
+            if rows == 0:               # the planner's own choice: unsplit plans only
+                assert p["warps_per_unit"] == 1 and p["channel_splits"] == 1, what
         assert p["smem_bytes"] <= 227 * 1024, what
         assert p["stages"] >= 1 and p["ctas"] >= 1, what
         assert p["warps_per_unit"] in (1, 2, 4) and p["tile_width"] in (2, 4, 8, 16, 32), what
