@@ -140,10 +140,11 @@ static pconv_status forward_impl(const pconv_handle* h, const void* x, const flo
   if (n < 0 || h_in <= 0 || w_in <= 0) return PCONV_ERR_SHAPE;
   const unsigned known =
       PCONV_RELU | PCONV_POOL2X2 | PCONV_REPRODUCIBLE | PCONV_CHAIN | PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED |
-      PCONV_KERNEL_GENERIC_TAPS | PCONV_KERNEL_TENSOR | PCONV_ROWS4 | PCONV_ROWS8;
+      PCONV_KERNEL_GENERIC_TAPS | PCONV_KERNEL_TENSOR | PCONV_ROWS4 | PCONV_ROWS8 | PCONV_CLUSTER;
   if (flags & ~known) return PCONV_ERR_UNSUPPORTED;
   if ((flags & PCONV_ROWS4) && (flags & PCONV_ROWS8)) return PCONV_ERR_UNSUPPORTED;
   const int rmode = rows_mode(flags);
+  const bool cluster = (flags & PCONV_CLUSTER) != 0;
   const unsigned sel = flags & (PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED | PCONV_KERNEL_GENERIC_TAPS |
                                 PCONV_KERNEL_TENSOR);
   if (sel & (sel - 1)) return PCONV_ERR_UNSUPPORTED;  // at most one selection bit
@@ -182,10 +183,10 @@ static pconv_status forward_impl(const pconv_handle* h, const void* x, const flo
     if (!tiled_supported(L, n, h_in, w_in)) return PCONV_ERR_UNSUPPORTED;
     const bool generic = (sel == PCONV_KERNEL_GENERIC_TAPS);
     if (rmode == 8 && (generic || L.wide_codes || !L.codes_s)) return PCONV_ERR_UNSUPPORTED;
-    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, pool, repro, generic, rmode, ws, ws_bytes, stream);
+    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, pool, repro, generic, rmode, cluster, ws, ws_bytes, stream);
   } else if (tiled_supported(L, n, h_in, w_in)) {
     if (rmode == 8 && (L.wide_codes || !L.codes_s)) return PCONV_ERR_UNSUPPORTED;
-    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, pool, repro, false, rmode, ws, ws_bytes, stream);
+    e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, pool, repro, false, rmode, cluster, ws, ws_bytes, stream);
   } else {
     e = launch_simple(L, x, bias, y, n, h_in, w_in, relu, stream);
   }

@@ -40,6 +40,9 @@
 #include <cuda_fp16.h>
 
 #include <cstring>
+#include <map>
+#include <mutex>
+#include <tuple>
 #include <type_traits>
 #ifdef PCONV_DEV
 #include <cstdlib>
@@ -95,6 +98,8 @@ struct Geo {
   int relu, is_half;
   int pool, h_y, w_y;     // fused 2x2 max-pool: y holds [h_y][w_y] = [h_out/2][w_out/2] maps
   int fixed_turns;        // 1 = the warps of a unit take the chunks in a fixed order (reproducible sums)
+  int cluster;            // 1 = the ks CTAs of a tile form a thread-block cluster and add their partial
+                          // sums up through distributed shared memory (no workspace, no tickets)
 };
 
 // ---- PTX helpers ----------------------------------------------------------------------------------
@@ -177,7 +182,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* er
 
 // Built with -DPCONV_DEV (build.py: build(dev=True) -> libpconv_dev.so) the kernel leaves
 // timestamps in the trace words of the handle's status block (pconv_trace_read):
-//   0 start, 1 set-up done, 2 warp 0's first chunk landed, 3 loop end, 4 partial sums issued (split only),
+//   0 start, 1 set-up done, 2 warp 0's first chunk landed, 3 loop end, 4 partial sums issued (split only;
+//   cluster form: partial sums in shared memory, before the cluster's first barrier),
 //   5 epilogue end, 6 after the CTA's last barrier -- thread 0 of CTA (0,0,0), globaltimer ns;
 //   7 end, 8 start, 9 loop end, 10 partial sums issued -- latest over all CTAs;
 //   11 / 12 cycles warp 0 of CTA (0,0,0) spent waiting for chunks / working on them, 13 its chunks.
@@ -795,6 +801,25 @@ __device__ __forceinline__ void red_add_v4(float* p, uint32_t a, uint32_t b, uin
                : "memory");
 }
 
+// ---- thread-block clusters: the CTAs that share an output tile ---------------------------------------
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// The address, in the cluster's shared-memory window, of `addr` (a shared::cta address) in CTA `rank`.
+__device__ __forceinline__ uint32_t cluster_map(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float4 ld_cluster_v4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+               : "r"(addr));
+  return v;
+}
+
 // The 2 R outputs of one filter slot.  MODE 0: y = act(v + bias); MODE 1: workspace += v, where
 // `ws` points at this lane's 2 R floats of the slot in the warp's part of the workspace (the
 // workspace is laid out for the warps that write and read it, not like y: [tile][warp][slot]
@@ -807,6 +832,12 @@ __device__ __forceinline__ void emit_slot(const Geo& g, const LaneOut& lo, void*
   if (MODE == 1) {
 #pragma unroll
     for (int i = 0; i < 2 * R; i += 4) red_add_v4(ws + i, v[i], v[i + 1], v[i + 2], v[i + 3]);
+    return;
+  }
+  if (MODE == 2) {   // `ws` is a generic pointer into this CTA's shared memory (same layout)
+#pragma unroll
+    for (int i = 0; i < 2 * R; i += 4)
+      *reinterpret_cast<uint4*>(ws + i) = make_uint4(v[i], v[i + 1], v[i + 2], v[i + 3]);
     return;
   }
   const long long ia = fbase + lo.base_a, ib = fbase + lo.base_b;
@@ -889,9 +920,9 @@ __device__ __forceinline__ void write_outputs(const Geo& g, const LaneOut& lo, c
       emit_slot<R, MODE, HALF, RELU>(g, lo, y, ws, (long long)o * plane, bv, v);
     }
   };
-  // MODE 1: `ws` is the lane's first float of the warp's first slot (r.a0); slots are 32 x 2 R floats apart
+  // MODE 1 / 2: `ws` is the lane's first float of the warp's first slot (r.a0); slots are 32 x 2 R floats apart
   auto emit_ws = [&](int a, const uint32_t (&v)[kNV]) {
-    emit_slot<R, 1, false, false>(g, lo, y, ws + (size_t)(a - r.a0) * (32 * kNV), 0, 0.f, v);
+    emit_slot<R, MODE, false, false>(g, lo, y, ws + (size_t)(a - r.a0) * (32 * kNV), 0, 0.f, v);
   };
   if constexpr (GENERIC) {
     static_assert(!GENERIC || R == 4, "register accumulators hold 4 rows");
@@ -918,7 +949,7 @@ __device__ __forceinline__ void write_outputs(const Geo& g, const LaneOut& lo, c
         const int o = __shfl_sync(0xffffffffu, my_o, a + b);
         const float bv = __shfl_sync(0xffffffffu, my_b, a + b);
         if (o >= 0) {
-          if (MODE == 1) emit_ws(a + b, v[b]);
+          if (MODE != 0) emit_ws(a + b, v[b]);
           else emit(o, bv, v[b]);
         }
       }
@@ -970,6 +1001,86 @@ __device__ __forceinline__ void finalize_outputs(const Geo& g, const LaneOut& lo
         if (lo.mask >> (2 * k) & 1u) store_out<HALF, RELU>(y, ia + row, v[b][2 * k] + bv[b]);
         if (lo.mask >> (2 * k + 1) & 1u) store_out<HALF, RELU>(y, ib + row, v[b][2 * k + 1] + bv[b]);
       }
+    }
+  }
+}
+
+// Cluster form of the channel split: every CTA of a tile's cluster leaves the partial sums of its
+// warps in its own shared memory at `part` ([warp][slot][lane][2 R], the workspace layout); the
+// slot parts of the tile are dealt to the cluster's warps (part sp -> rank sp % ks, warp
+// sp / ks % CW), and a warp adds a part up over the ranks in rank order -- so the sums do not
+// depend on timing -- through distributed shared memory, applies bias / ReLU (pools) and writes y.
+constexpr int kMaxClusterParts = 4;   // slot parts a warp may be dealt: CW * 16 / zs parts over ks * CW warps, ks >= 2, zs >= 2
+struct ClusterPart {
+  int sp, o;       // slot part (-1 = none) and the original filter index of its slot (-1 = padding)
+  float bv;        // the filter's bias
+  int slot2;       // sub-tile pair of this lane in the part's pixel set
+};
+// What a warp will add up, worked out (and its filter indices and biases fetched) before the
+// CTAs meet, while the slower warps still compute.
+template <int R, int CW>
+__device__ __forceinline__ void cluster_parts(ClusterPart (&cp)[kMaxClusterParts], const DeviceLayer& L,
+                                              const Geo& g, const float* __restrict__ bias, int group0,
+                                              int rank, int warp, int lane) {
+  const int zs = g.zs, spw = kGroup / zs, n_sp = CW * spw;
+#pragma unroll
+  for (int i = 0; i < kMaxClusterParts; ++i) {
+    const int sp = rank + g.ks * (warp + CW * i);
+    cp[i].sp = -1;
+    cp[i].o = -1;
+    cp[i].bv = 0.f;
+    cp[i].slot2 = 0;
+    if (sp >= n_sp) continue;
+    const int w2 = sp / spw, j = sp - w2 * spw;        // the warp that holds this part in every rank
+    int unit2 = w2, z2 = 0;
+    if (zs > 1) {
+      z2 = (w2 >> 2) % zs;
+      unit2 = (w2 & 3) + 4 * ((w2 >> 2) / zs);
+    }
+    const int wyi2 = unit2 % g.wys, gi2 = group0 + unit2 / g.wys;
+    if (wyi2 >= g.wy || gi2 >= L.n_groups) continue;
+    cp[i].sp = sp;
+    cp[i].o = __ldg(L.perm + gi2 * kGroup + z2 * spw + j);
+    cp[i].slot2 = wyi2 * g.sw + lane / g.tw;
+  }
+#pragma unroll
+  for (int i = 0; i < kMaxClusterParts; ++i)
+    if (cp[i].o >= 0 && bias) cp[i].bv = __ldg(bias + cp[i].o);
+}
+
+template <int R, bool HALF, bool RELU>
+__device__ __forceinline__ void cluster_reduce_emit(const DeviceLayer& L, const Geo& g, const SubTile* tab,
+                                                    void* __restrict__ y, uint32_t part,
+                                                    const ClusterPart (&cp)[kMaxClusterParts], int lane) {
+  constexpr int kNV = 2 * R;
+  const long long plane = (long long)g.h_out * g.w_out;
+  const long long plane_y = (long long)g.h_y * g.w_y;
+#pragma unroll
+  for (int i = 0; i < kMaxClusterParts; ++i) {
+    if (cp[i].o < 0) continue;
+    const uint32_t off = part + (uint32_t)((cp[i].sp * 32 + lane) * kNV * 4);
+    float v[kNV];
+#pragma unroll
+    for (int e = 0; e < kNV; ++e) v[e] = 0.f;
+#pragma unroll 4
+    for (int q = 0; q < g.ks; ++q) {
+      const uint32_t ra = cluster_map(off, (uint32_t)q);
+#pragma unroll
+      for (int k = 0; k < kNV; k += 4) {
+        const float4 t = ld_cluster_v4(ra + k * 4);
+        v[k] += t.x; v[k + 1] += t.y; v[k + 2] += t.z; v[k + 3] += t.w;
+      }
+    }
+    const int col = lane % g.tw;
+    if (g.pool) {
+      const LaneOut lp = lane_outputs_pooled<R>(L, g, tab, cp[i].slot2, col);
+      emit_slot_pooled<R, HALF, RELU>(g, lp, y, (long long)cp[i].o * plane_y, cp[i].bv, v);
+    } else {
+      const LaneOut lo = lane_outputs<R>(L, g, tab, cp[i].slot2, col);
+      uint32_t u[kNV];
+#pragma unroll
+      for (int e = 0; e < kNV; ++e) u[e] = __float_as_uint(v[e]);
+      emit_slot<R, 0, HALF, RELU>(g, lo, y, nullptr, (long long)cp[i].o * plane, cp[i].bv, u);
     }
   }
 }
@@ -1324,6 +1435,11 @@ __device__ __forceinline__ void tiled_body(const DeviceLayer& L, const Geo& g, c
         orng.a1 = orng.a0 + kGroup / zs;
       }
     }
+    if (!GENERIC && g.cluster) {
+      // the partial sums overwrite the staging ring: wait until every consumer warp of the CTA has
+      // left its loop (all chunks consumed, so the producers' copies have all landed too)
+      asm volatile("bar.sync 1, %0;" ::"n"(32 * kCW) : "memory");
+    }
     if (active && ok) {
       const LaneOut lo = lane_outputs<R>(L, g, tab, slot, col);
       const LaneOut lp = g.pool ? lane_outputs_pooled<R>(L, g, tab, slot, col) : lo;
@@ -1334,6 +1450,12 @@ __device__ __forceinline__ void tiled_body(const DeviceLayer& L, const Geo& g, c
           write_outputs<R, GENERIC, 0, decltype(half)::value, decltype(relu)::value>(g, lo, lp, y, ws, acc,
                                                                                       orng, my_o, my_b);
         });
+      } else if (g.cluster) {
+        // cluster form: the warp's partial sums go to this CTA's shared memory (the staging ring is
+        // free: every consumer warp has passed the barrier above), in the workspace layout
+        const int spw = kGroup / (GENERIC ? 1 : g.zs);
+        float* part = reinterpret_cast<float*>(smem + g.stage_off) + ((size_t)(warp * spw) * 32 + lane) * kNV;
+        write_outputs<R, GENERIC, 2, false, false>(g, lo, lp, y, part, acc, orng, my_o, my_b);
       } else {
         // this lane's floats in the warp's part of the tile's workspace: [tile][warp][slot][lane][2 R]
         const int spw = kGroup / (GENERIC ? 1 : g.zs);   // slots a warp writes out
@@ -1365,6 +1487,25 @@ __device__ __forceinline__ void tiled_body(const DeviceLayer& L, const Geo& g, c
       }
     }
     PCONV_MARK(5)
+  }
+
+  // ---- cluster form of the channel split: all warps of all CTAs of the tile meet twice ------------
+  if constexpr (!GENERIC) {
+    if (g.cluster) {
+      ClusterPart cparts[kMaxClusterParts];
+      if (warp < kCW) cluster_parts<R, kCW>(cparts, L, g, bias, bp.y * g.ng, bp.z, warp, lane);
+      PCONV_MARK(4)
+      PCONV_MARK_MAX(10)
+      cluster_sync_all();          // every CTA's partial sums are in its shared memory
+      if (warp < kCW) {
+        with_flags(g, [&](auto half, auto relu) {
+          cluster_reduce_emit<R, decltype(half)::value, decltype(relu)::value>(
+              L, g, tab, y, sbase + (uint32_t)g.stage_off, cparts, lane);
+        });
+      }
+      PCONV_MARK(5)
+      cluster_sync_all();          // nobody leaves while a peer may still read its shared memory
+    }
   }
 
   // ---- common exit: every warp arrives here, then the TMEM columns are handed back ---------------
@@ -1579,6 +1720,7 @@ bool geo_for(const DeviceLayer& L, int n, int h, int w, int zs, int R, Geo* out)
   if (g.stages < 1) return false;
   g.relu = 0;
   g.fixed_turns = 0;
+  g.cluster = 0;
   g.pool = 0;
   g.h_y = g.h_out;
   g.w_y = g.w_out;
@@ -1702,11 +1844,52 @@ cudaError_t launch_one(const DeviceLayer& L, Geo g, const void* x, const float* 
   cfg.blockDim = dim3(cta_threads(GENERIC, R), 1, 1);
   cfg.dynamicSmemBytes = (size_t)smem;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (g.cluster) {
+    // The ks CTAs of a tile as one thread-block cluster.  More than 8 CTAs per cluster is beyond
+    // the portable size: allowed per kernel, and taken only if all the launch's clusters can be
+    // resident at once (a cluster needs its SMs inside one GPC); otherwise, and on any error here,
+    // the launch falls back to the workspace form.
+    bool ok = true;
+    if (g.ks > 8)
+      ok = cudaFuncSetAttribute(tiled_kernel<S, GENERIC, WIDE, R>, cudaFuncAttributeNonPortableClusterSizeAllowed,
+                                1) == cudaSuccess;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 1;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = (unsigned)g.ks;
+    cfg.numAttrs = 2;
+    int n_clusters = 0;
+    if (ok) {
+      // (asked once per kernel, shared-memory size, cluster size and device: the answer does not change)
+      static std::mutex mu;
+      static std::map<std::tuple<int, int, int>, int> known;
+      int dev = 0;
+      ok = cudaGetDevice(&dev) == cudaSuccess;
+      if (ok) {
+        std::lock_guard<std::mutex> lock(mu);
+        const auto key = std::make_tuple(dev, smem, g.ks);
+        const auto it = known.find(key);
+        if (it != known.end()) {
+          n_clusters = it->second;
+        } else {
+          ok = cudaOccupancyMaxActiveClusters(&n_clusters, tiled_kernel<S, GENERIC, WIDE, R>, &cfg) == cudaSuccess;
+          if (ok) known[key] = n_clusters;
+        }
+      }
+    }
+    if (ok) ok = (long long)n_clusters >= ctas_x * ctas_y;
+    if (!ok) {
+      (void)cudaGetLastError();
+      if (!ws) return cudaErrorInvalidValue;   // (launch_tiled only asks for a cluster with a workspace to fall back on)
+      g.cluster = 0;
+      cfg.numAttrs = 1;
+    }
+  }
   return cudaLaunchKernelEx(&cfg, tiled_kernel<S, GENERIC, WIDE, R>, L, g, x, bias, y, ws, counters);
 }
 
@@ -1758,7 +1941,7 @@ bool tiled_plan(const DeviceLayer& L, int n, int h, int w, bool generic_taps, bo
 
 cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias, void* y, int n, int h,
                          int w, bool relu, bool pool, bool reproducible, bool generic_taps, int rmode,
-                         void* ws, size_t ws_bytes, cudaStream_t stream) {
+                         bool allow_cluster, void* ws, size_t ws_bytes, cudaStream_t stream) {
   if (!generic_taps && !L.codes_s) generic_taps = true;
   if (rmode == 8 && (generic_taps || L.wide_codes)) return cudaErrorInvalidValue;
   Geo g;
@@ -1783,6 +1966,13 @@ cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias,
   if (g.ks > 1) {
     wsf = (float*)ws;
     counters = (int*)((char*)ws + ((split_sums_bytes(L, g) + 255) & ~(size_t)255));
+    // The CTAs that share a tile add their partial sums up through distributed shared memory when
+    // they can form one cluster (at most 16 CTAs) and a CTA's partial sums fit the staging ring;
+    // the workspace stays untouched then.
+    const size_t part_bytes = (size_t)consumer_warps(false, g.rpl) * (kGroup / g.zs) * 32 * (2 * g.rpl) * sizeof(float);
+    const int parts_per_warp = (kGroup / g.zs + g.ks - 1) / g.ks;
+    g.cluster = (allow_cluster && g.ks <= 16 && parts_per_warp <= kMaxClusterParts &&
+                 part_bytes <= (size_t)g.stages * g.stage_bytes) ? 1 : 0;
   }
   const bool wide = L.wide_codes != 0;
   if (L.stride == 1) {

@@ -129,7 +129,7 @@ cudaError_t launch_simple(const DeviceLayer& L, const void* x, const float* bias
                           int h, int w, bool relu, cudaStream_t stream);
 cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias, void* y, int n,
                          int h, int w, bool relu, bool pool, bool reproducible, bool generic_taps,
-                         int rmode, void* ws, size_t ws_bytes, cudaStream_t stream);
+                         int rmode, bool allow_cluster, void* ws, size_t ws_bytes, cudaStream_t stream);
 cudaError_t launch_tensor(const DeviceLayer& L, const void* x, const float* bias, void* y, int n,
                           int h, int w, bool relu, void* ws, size_t ws_bytes, cudaStream_t stream);
 size_t tensor_workspace_bytes(const DeviceLayer& L, int n, int h, int w);
