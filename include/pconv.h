@@ -98,6 +98,17 @@ enum {
                               (49 us on the 512-filter 28x28 layer either way) and 3 % slower on
                               the VGG stack at batch 1 (0.396 against 0.384 ms), where a cluster
                               must find its SMs free inside one GPC while the previous layer drains. */
+  PCONV_STAGE_BULK = 0x8000u, /* tiled kernel, fp32 storage: input chunks are fetched by the copy engine
+                                 (cp.async.bulk: a sub-tile's rows where the image is wider than a
+                                 sub-tile and its width a multiple of 4, one span of the plane per
+                                 channel where the sub-tile is as wide as the image and the plane a
+                                 multiple of 4 elements; other shapes are unaffected) into a raw ring
+                                 that the producer warps rebuild into the kernel's tile layout,
+                                 instead of by 4-byte cp.async straight into that layout.  Off by
+                                 default: measured slower on every VGG layer at batch 1 (a bulk copy
+                                 takes ~2 us to land here and the raw ring is two deep: the first
+                                 chunk is ready after 8.7-15 us against 4.3-5.6 us; 0.57 against
+                                 0.38 ms for the stack). */
   PCONV_KERNEL_TENSOR = 0x800u /* fp16 storage, stride 1 only: the layer as a dense implicit GEMM over
                                   the zero-inserted weights on the tensor cores (tcgen05.mma, fp32
                                   accumulators in Tensor Memory).  It multiplies the pruned zeros too
@@ -250,6 +261,10 @@ typedef struct pconv_plan_t {
   int stages;            /* depth of the staging ring */
   int smem_bytes;        /* dynamic shared memory the geometry needs */
   long long ctas;        /* CTAs launched */
+  int staging;           /* how input chunks reach shared memory: 0 = element-wise (cp.async for fp32,
+                            loads for fp16), 1 = fp16 pairs by cp.async into a raw ring, 2 / 3 = fp32 rows /
+                            plane spans by bulk copies (cp.async.bulk) into a raw ring; the raw ring is
+                            rebuilt into the kernel's tile layout by the producer warps */
   int tensor_path;       /* 1 = a default forward of this shape (no kernel-selection flag, no fused
                             pool) runs the dense tensor-core kernel instead of the tiled one; the
                             fields above still describe the tiled kernel */

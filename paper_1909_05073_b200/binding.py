@@ -16,7 +16,7 @@ OK = 0
 F32, F16 = 0, 1
 RELU, STRICT4, POOL2X2, REPRODUCIBLE, CHAIN = 1, 2, 4, 8, 0x10
 KERNEL_SIMPLE, KERNEL_TILED, KERNEL_GENERIC_TAPS, KERNEL_TENSOR = 0x100, 0x200, 0x400, 0x800
-ROWS4, ROWS8, CLUSTER = 0x1000, 0x2000, 0x4000
+ROWS4, ROWS8, CLUSTER, STAGE_BULK = 0x1000, 0x2000, 0x4000, 0x8000
 MAX_PATTERNS = 16
 
 STATUS_NAMES = ["PCONV_OK", "PCONV_ERR_NULL", "PCONV_ERR_SHAPE", "PCONV_ERR_PATTERN_SET",
@@ -58,7 +58,7 @@ class Plan(ctypes.Structure):
                 ("channel_splits", ctypes.c_int), ("groups_per_cta", ctypes.c_int),
                 ("pixel_sets", ctypes.c_int), ("tile_width", ctypes.c_int), ("stages", ctypes.c_int),
                 ("smem_bytes", ctypes.c_int), ("ctas", ctypes.c_longlong),
-                ("tensor_path", ctypes.c_int)]
+                ("staging", ctypes.c_int), ("tensor_path", ctypes.c_int)]
 
 
 _lib = None

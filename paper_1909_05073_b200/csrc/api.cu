@@ -48,20 +48,22 @@ extern "C" const char* pconv_status_str(pconv_status s) {
   return "unknown status";
 }
 
-// Rows per lane a caller pinned for the tiled kernel (0 = the planner chooses).
+// What a caller pinned for the tiled kernel: rows per lane (0 = the planner chooses) and the
+// bulk-copy staging.
 static int rows_mode(unsigned flags) {
-  return (flags & PCONV_ROWS8) ? 8 : (flags & PCONV_ROWS4) ? 4 : 0;
+  return ((flags & PCONV_ROWS8) ? 8 : (flags & PCONV_ROWS4) ? 4 : 0) | ((flags & PCONV_STAGE_BULK) ? pconv::kPinBulk : 0);
 }
 
 // Scratch a forward of this shape may use, whichever kernel takes it.  rmode: the rows per lane
 // the caller pins for the tiled kernel (0 = the planner's choice), -1 = whatever it may pin.
 static size_t workspace_need(const pconv::DeviceLayer& L, int n, int h_in, int w_in, int rmode) {
   size_t need = tensor_workspace_bytes(L, n, h_in, w_in);
-  for (int r = 0; r <= 8; r += 4) {
-    if (rmode >= 0 && r != rmode) continue;
-    const size_t a = tiled_workspace_bytes(L, n, h_in, w_in, r);
-    if (a > need) need = a;
-  }
+  for (int r = 0; r <= 8; r += 4)
+    for (int bulk = 0; bulk <= pconv::kPinBulk; bulk += pconv::kPinBulk) {
+      if (rmode >= 0 && (r | bulk) != rmode) continue;
+      const size_t a = tiled_workspace_bytes(L, n, h_in, w_in, r | bulk);
+      if (a > need) need = a;
+    }
   return need;
 }
 
@@ -140,7 +142,8 @@ static pconv_status forward_impl(const pconv_handle* h, const void* x, const flo
   if (n < 0 || h_in <= 0 || w_in <= 0) return PCONV_ERR_SHAPE;
   const unsigned known =
       PCONV_RELU | PCONV_POOL2X2 | PCONV_REPRODUCIBLE | PCONV_CHAIN | PCONV_KERNEL_SIMPLE | PCONV_KERNEL_TILED |
-      PCONV_KERNEL_GENERIC_TAPS | PCONV_KERNEL_TENSOR | PCONV_ROWS4 | PCONV_ROWS8 | PCONV_CLUSTER;
+      PCONV_KERNEL_GENERIC_TAPS | PCONV_KERNEL_TENSOR | PCONV_ROWS4 | PCONV_ROWS8 | PCONV_CLUSTER |
+      PCONV_STAGE_BULK;
   if (flags & ~known) return PCONV_ERR_UNSUPPORTED;
   if ((flags & PCONV_ROWS4) && (flags & PCONV_ROWS8)) return PCONV_ERR_UNSUPPORTED;
   const int rmode = rows_mode(flags);
@@ -182,10 +185,10 @@ static pconv_status forward_impl(const pconv_handle* h, const void* x, const flo
   } else if (sel == PCONV_KERNEL_TILED || sel == PCONV_KERNEL_GENERIC_TAPS) {
     if (!tiled_supported(L, n, h_in, w_in)) return PCONV_ERR_UNSUPPORTED;
     const bool generic = (sel == PCONV_KERNEL_GENERIC_TAPS);
-    if (rmode == 8 && (generic || L.wide_codes || !L.codes_s)) return PCONV_ERR_UNSUPPORTED;
+    if ((rmode & pconv::kPinRowsMask) == 8 && (generic || L.wide_codes || !L.codes_s)) return PCONV_ERR_UNSUPPORTED;
     e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, pool, repro, generic, rmode, cluster, ws, ws_bytes, stream);
   } else if (tiled_supported(L, n, h_in, w_in)) {
-    if (rmode == 8 && (L.wide_codes || !L.codes_s)) return PCONV_ERR_UNSUPPORTED;
+    if ((rmode & pconv::kPinRowsMask) == 8 && (L.wide_codes || !L.codes_s)) return PCONV_ERR_UNSUPPORTED;
     e = launch_tiled(L, x, bias, y, n, h_in, w_in, relu, pool, repro, false, rmode, cluster, ws, ws_bytes, stream);
   } else {
     e = launch_simple(L, x, bias, y, n, h_in, w_in, relu, stream);

@@ -94,6 +94,10 @@ struct Geo {
   // fp16 storage with an even image width: raw copies of the chunk (fp16, row-major, fetched with
   // cp.async) wait in a ring of raw_stages slots until the producers widen them into a stage
   int raw_stages, raw_off, raw_slot, raw_pitch, raw_x_bytes;
+  // how a chunk reaches the raw ring: 0 = no raw ring (element-wise cp.async or loads straight into
+  // the stage), 1 = fp16 element pairs by cp.async, 2 / 3 = fp32 rows / plane spans by bulk copies
+  // (raw_sub = bytes per (sub-tile, channel) of a raw slot); raw_want = the mode the shape allows
+  int raw_mode, raw_want, raw_sub;
   int ks, cps;           // channel splits (grid.z) and chunks per split
   int relu, is_half;
   int pool, h_y, w_y;     // fused 2x2 max-pool: y holds [h_y][w_y] = [h_out/2][w_out/2] maps
@@ -647,6 +651,189 @@ __device__ __forceinline__ void produce_raw_stream(const DeviceLayer& L, const G
   }
 }
 
+// ---- fp32 storage: bulk copies into the raw ring -----------------------------------------------------
+// Where the rows (or whole planes) of the input start on 16-byte boundaries, a chunk is fetched by
+// the copy engine instead of by element-wise cp.async: cp.async.bulk (no tensor map, this CTA's own
+// shared memory, no multicast) brings, per sub-tile and channel, either its rows (raw_mode 2:
+// image wider than a sub-tile, width a multiple of 4; a raw row starts 4 columns left of the
+// sub-tile so that every copy is aligned) or one contiguous span of the plane (raw_mode 3:
+// sub-tile as wide as the image, plane size a multiple of 4 elements), and the chunk's weight
+// records and codes, all completing on the raw slot's mbarrier.  The producer warps then build the
+// stage from the raw slot (shared memory to shared memory): the {A,B}-interleaved column-major
+// tile, with zeros for everything outside the image -- the copies carry no padding.
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void sts64u(uint32_t addr, uint32_t a, uint32_t b) {
+  asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(addr), "r"(a), "r"(b) : "memory");
+}
+// First element of the plane that a sub-tile's span holds (raw_mode 3): its first input row,
+// rounded down to a multiple of 4 elements.
+template <int S>
+__device__ __forceinline__ int span_origin(const Geo& g, const SubTile& T) {
+  const int iy0 = T.y0 * S - 1;
+  return (iy0 > 0 ? iy0 * g.w : 0) & ~3;
+}
+
+// Byte offsets of a staged element's A and B sources inside a raw slot (channel 0 of the chunk),
+// or -1 where the element lies outside the image or the batch (the stage gets a zero there).
+template <int S, int R>
+__device__ __forceinline__ StagedElem bulk_elem(const Geo& g, const SubTile* tab, int e) {
+  constexpr int kRows = Win<S, R>::kRows;
+  const int q = e / g.pitch, i = e - q * g.pitch;   // q = pair * rows + row
+  const int p = q / kRows, r = q - p * kRows;
+  const int dx = staged_dx<S>(i, g.tw);
+  auto src = [&](int sub) -> long long {
+    const SubTile T = tab[sub];
+    const int iy = T.y0 * S - 1 + r, ix = T.x0 * S + dx;
+    if (!T.valid || iy < 0 || iy >= g.h || ix < 0 || ix >= g.w) return -1;
+    const int idx = (g.raw_mode == 2) ? r * g.raw_pitch + dx + 4 : iy * g.w + ix - span_origin<S>(g, T);
+    return (long long)sub * kChunk * g.raw_sub + (long long)idx * 4;
+  };
+  StagedElem se;
+  se.off_a = src(2 * p);
+  se.off_b = src(2 * p + 1);
+  se.dst = (uint32_t)(p * g.substride + i * g.colstride + r * 8);
+  return se;
+}
+
+// This thread's share of the copies of chunk k (kk-th of the CTA) into the raw slot at raw_base;
+// it then arrives on the slot's barrier with the bytes it asked for.
+template <int S, int R>
+__device__ __forceinline__ void issue_bulk(const DeviceLayer& L, const Geo& g, const float* __restrict__ x,
+                                           const SubTile* tab, const uint4* desc, const uint8_t* codes,
+                                           uint32_t raw_base, uint32_t bar, int k, int kk, int ptid) {
+  constexpr int kRows = Win<S, R>::kRows;
+  const int c0 = k * kChunk;
+  const int nc = min(kChunk, L.c_in - c0);
+  const size_t hw = (size_t)g.h * g.w;
+  uint32_t bytes = 0;
+  if (g.raw_mode == 2) {
+    const int n_copy = g.pairs * 2 * kChunk * kRows;
+    for (int v = ptid; v < n_copy; v += kProducerThreads) {
+      const int t = v / kRows, r = v - t * kRows;
+      const int sub = t / kChunk, cc = t - sub * kChunk;
+      const SubTile T = tab[sub];
+      const int iy = T.y0 * S - 1 + r;
+      if (!T.valid || cc >= nc || iy < 0 || iy >= g.h) continue;
+      const int xo = T.x0 * S - 4;                       // column of the raw row's first element
+      const int xs = xo > 0 ? xo : 0;
+      const int xe = min(g.w, xo + g.raw_pitch);
+      if (xe <= xs) continue;
+      const uint32_t nb = (uint32_t)(xe - xs) * 4u;
+      bulk_copy_g2s(raw_base + (uint32_t)((sub * kChunk + cc) * g.raw_sub + (r * g.raw_pitch + xs - xo) * 4),
+                    x + ((size_t)T.n * L.c_in + c0 + cc) * hw + (size_t)iy * g.w + xs, nb, bar);
+      bytes += nb;
+    }
+  } else {
+    const int n_copy = g.pairs * 2 * kChunk;
+    for (int v = ptid; v < n_copy; v += kProducerThreads) {
+      const int sub = v / kChunk, cc = v - sub * kChunk;
+      const SubTile T = tab[sub];
+      if (!T.valid || cc >= nc) continue;
+      const int fo = span_origin<S>(g, T);
+      const int last_row = min(g.h, T.y0 * S - 1 + kRows);
+      const int fe = min((int)hw, (last_row * g.w + 3) & ~3);
+      if (fe <= fo) continue;
+      const uint32_t nb = (uint32_t)(fe - fo) * 4u;
+      bulk_copy_g2s(raw_base + (uint32_t)((sub * kChunk + cc) * g.raw_sub),
+                    x + ((size_t)T.n * L.c_in + c0 + cc) * hw + fo, nb, bar);
+      bytes += nb;
+    }
+  }
+  // the chunk's weight records and codes, one copy each per filter group
+  const uint32_t wbase = raw_base + g.raw_x_bytes;
+  const uint32_t cbase = wbase + g.ng * kWSlot;
+  for (int v = ptid; v < 2 * g.ng; v += kProducerThreads) {
+    const int j = v >> 1;
+    const uint4 d = desc[2 * (j * g.cps + kk)];   // {w_off, n_k, code_off, code_len}
+    if (v & 1) {
+      const uint32_t nb = (d.w + 15u) & ~15u;
+      if (nb) {
+        bulk_copy_g2s(cbase + j * kCodeSlot, codes + d.z, nb, bar);
+        bytes += nb;
+      }
+    } else if (d.y) {
+      bulk_copy_g2s(wbase + j * kWSlot, reinterpret_cast<const float*>(L.wvals) + (size_t)d.x * 4, d.y * 16u, bar);
+      bytes += d.y * 16u;
+    }
+  }
+  mbar_arrive_expect_tx(bar, bytes);
+}
+
+// Raw slot -> stage: the interleaved tile (zeros outside the image), the weight records, the codes.
+template <int S, int R>
+__device__ __forceinline__ void widen_bulk(const Geo& g, const SubTile* tab, const StagedElem (&pre)[kPreElems],
+                                           const uint4* desc, uint32_t raw_base, uint32_t stage_base,
+                                           int kk, int ptid) {
+  const int n_elem = g.pairs * g.rows * g.pitch;
+  const uint32_t raw_chan = (uint32_t)g.raw_sub;
+  auto widen = [&](const StagedElem& se) {
+    uint32_t va[kChunk], vb[kChunk];
+#pragma unroll
+    for (int cc = 0; cc < kChunk; ++cc) {
+      va[cc] = se.off_a >= 0 ? lds32(raw_base + (uint32_t)se.off_a + cc * raw_chan) : 0u;
+      vb[cc] = se.off_b >= 0 ? lds32(raw_base + (uint32_t)se.off_b + cc * raw_chan) : 0u;
+    }
+#pragma unroll
+    for (int cc = 0; cc < kChunk; ++cc)
+      sts64u(stage_base + se.dst + (uint32_t)(cc * g.chan_stride), va[cc], vb[cc]);
+  };
+#pragma unroll
+  for (int i = 0; i < kPreElems; ++i)
+    if (pre[i].dst != kSkipElem) widen(pre[i]);
+  for (int e = ptid + kPreElems * kProducerThreads; e < n_elem; e += kProducerThreads)
+    widen(bulk_elem<S, R>(g, tab, e));
+  const uint32_t rw = raw_base + g.raw_x_bytes, rc = rw + g.ng * kWSlot;
+  const uint32_t wbase = stage_base + g.x_stage_bytes, cbase = wbase + g.ng * kWSlot;
+  auto copy16 = [](uint32_t dst, uint32_t src) {
+    uint32_t c0, c1, c2, c3;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(c0), "=r"(c1), "=r"(c2), "=r"(c3) : "r"(src));
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+  };
+  for (int j = 0; j < g.ng; ++j) {
+    const uint4 d = desc[2 * (j * g.cps + kk)];
+    if ((uint32_t)ptid < d.y) copy16(wbase + j * kWSlot + ptid * 16, rw + j * kWSlot + ptid * 16);
+    if ((uint32_t)ptid * 16 < d.w) copy16(cbase + j * kCodeSlot + ptid * 16, rc + j * kCodeSlot + ptid * 16);
+  }
+}
+
+// The producers' loop of the bulk-copy path: the copies of a chunk are issued raw_stages - 1 chunks
+// ahead of the chunk being turned into a stage.  Every wait is bounded (id 4: a raw slot's copies).
+template <int S, int R>
+__device__ __forceinline__ void produce_bulk_stream(const DeviceLayer& L, const Geo& g,
+                                                    const float* __restrict__ x, const SubTile* tab,
+                                                    const StagedElem (&pre)[kPreElems], const uint4* desc,
+                                                    const uint8_t* codes, uint32_t sbase, uint32_t raw_bar0,
+                                                    int k0, int nk, int ptid) {
+  const int RS = g.raw_stages;
+  bool ok = true;
+  auto raw_base = [&](int kk) { return sbase + g.raw_off + (kk % RS) * g.raw_slot; };
+  auto raw_bar = [&](int kk) { return raw_bar0 + 8u * (uint32_t)(kk % RS); };
+  auto producers_sync = [] { asm volatile("bar.sync 2, %0;" ::"n"(kProducerThreads) : "memory"); };
+  for (int j = 0; j < RS - 1; ++j)
+    if (j < nk) issue_bulk<S, R>(L, g, x, tab, desc, codes, raw_base(j), raw_bar(j), k0 + j, j, ptid);
+  for (int kk = 0; kk < nk; ++kk) {
+    const int ahead = kk + RS - 1;
+    if (ok && ahead < nk)
+      issue_bulk<S, R>(L, g, x, tab, desc, codes, raw_base(ahead), raw_bar(ahead), k0 + ahead, ahead, ptid);
+    if (ok) ok = mbar_wait(raw_bar(kk), (kk / RS) & 1, L.err, 4);
+    const int s = kk % g.stages, it = kk / g.stages;
+    if (ok && it > 0) ok = mbar_wait(sbase + 8 * (kMaxStages + s), (it - 1) & 1, L.err, 1);
+    if (ok) {
+      widen_bulk<S, R>(g, tab, pre, desc, raw_base(kk), sbase + g.stage_off + s * g.stage_bytes, kk, ptid);
+      if (!PCONV_WITHHELD(kk, ptid)) mbar_arrive(sbase + 8 * s);
+    }
+    producers_sync();   // everybody has read the raw slot: the copy engine may overwrite it
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+}
+
 // fp16 storage: loads, converts to fp32 and stores (the interleaved fp32 layout cannot be produced
 // by an asynchronous copy of 2-byte elements).  The loads of a batch (two staged elements x 8
 // channels x {A,B}) are issued before the previous batch is converted and stored, across chunk
@@ -1175,14 +1362,16 @@ __device__ __forceinline__ void tiled_body(const DeviceLayer& L, const Geo& g, c
   if (cc.own_tmem) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (tid < kCW) unit_ctr[tid] = 0;
   const uint32_t coop_bar = sbase + 8 * 2 * kMaxStages + 16 + 64;   // kMaxCoop barriers
+  const uint32_t raw_bar0 = coop_bar + 8 * kMaxCoop;                // kRawStages barriers (bulk copies of a raw slot)
   if (tid == 0) {
     // every barrier is initialised, used or not, so that a chain's next layer may invalidate
     // and initialise them all again (its ring may be deeper)
     if (cc.reinit)
-      for (int j = 0; j < 2 * kMaxStages + 2 + 8 + kMaxCoop; ++j)
+      for (int j = 0; j < 2 * kMaxStages + 2 + 8 + kMaxCoop + kRawStages; ++j)
         if (j < 2 * kMaxStages || j >= 2 * kMaxStages + 10)
           asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(sbase + 8 * j) : "memory");
     for (int j = 0; j < kMaxCoop; ++j) mbar_init(coop_bar + 8 * j, 32 * kCW);
+    for (int j = 0; j < kRawStages; ++j) mbar_init(raw_bar0 + 8 * j, kProducerThreads);
     for (int s = 0; s < kMaxStages; ++s) {
       mbar_init(sbase + 8 * s, 32 * kProducerWarps);
       mbar_init(sbase + 8 * (kMaxStages + s), kCW / (GENERIC ? 1 : g.zs));
@@ -1276,7 +1465,17 @@ __device__ __forceinline__ void tiled_body(const DeviceLayer& L, const Geo& g, c
     const int ptid = (warp - kCW) * 32 + lane;
     const uint8_t* codes = GENERIC ? L.codes_g : L.codes_s;
     StagedElem pre[kPreElems];
-    if (g.raw_stages > 0) {
+    if (g.raw_mode >= 2) {
+      const int n_elem = g.pairs * g.rows * g.pitch;
+#pragma unroll
+      for (int i = 0; i < kPreElems; ++i) {
+        const int e = ptid + i * kProducerThreads;
+        pre[i] = bulk_elem<S, R>(g, tab, e < n_elem ? e : 0);
+        if (e >= n_elem) pre[i].dst = kSkipElem;
+      }
+      if (dependency_wait(cc, lane, warp, smem, L.err))
+        produce_bulk_stream<S, R>(L, g, (const float*)x, tab, pre, desc, codes, sbase, raw_bar0, k0, nk, ptid);
+    } else if (g.raw_stages > 0) {
       const int n_elem = g.pairs * g.rows * g.pitch;
 #pragma unroll
       for (int i = 0; i < kPreElems; ++i) {
@@ -1617,21 +1816,35 @@ tiled_chain_kernel(const ChainLayer* __restrict__ layers, int n_layers, const vo
 // Places descriptors, the raw ring (if any) and the stages for `cps` chunks per CTA, and picks the
 // ring depth; false if nothing fits.
 int pick_stages(int fit, int zs, int cps);
-bool place_stages(Geo* g, int n_chunks_total, int cps, bool want_raw, int stride) {
+bool place_stages(Geo* g, int n_chunks_total, int cps, int raw_mode, int stride) {
   g->stage_off = g->desc_off + g->ng * cps * 32;
   g->raw_stages = 0;
+  g->raw_mode = 0;
   g->raw_off = g->stage_off;
-  g->raw_slot = g->raw_pitch = g->raw_x_bytes = 0;
-  if (want_raw) {
+  g->raw_slot = g->raw_pitch = g->raw_x_bytes = g->raw_sub = 0;
+  if (raw_mode == 1) {
     g->raw_pitch = (stride == 1) ? g->tw + 4 : 2 * g->tw + 2;   // halves per raw row (even)
     g->raw_x_bytes = g->pairs * 2 * kChunk * g->rows * g->raw_pitch * 2;
     g->raw_slot = (g->raw_x_bytes + g->ng * (kWRawSlot + kCodeSlot) + 15) & ~15;
+  } else if (raw_mode == 2) {
+    g->raw_pitch = (stride == 1) ? g->tw + 8 : 2 * g->tw + 8;   // floats per raw row: from 4 columns left of the sub-tile
+    g->raw_sub = g->rows * g->raw_pitch * 4;
+  } else if (raw_mode == 3) {
+    g->raw_sub = ((g->rows * g->w + 8 + 3) & ~3) * 4;           // the rows' span of the plane and its alignment slack
+  }
+  if (raw_mode >= 2) {
+    g->raw_x_bytes = g->pairs * 2 * kChunk * g->raw_sub;
+    g->raw_slot = (g->raw_x_bytes + g->ng * (kWSlot + kCodeSlot) + 15) & ~15;
+  }
+  if (raw_mode) {
+    g->raw_mode = raw_mode;
     g->raw_stages = kRawStages < cps ? kRawStages : cps;
+    if (raw_mode >= 2 && g->raw_stages > 2) g->raw_stages = 2;   // (fp32 slots are twice the size)
     g->stage_off += g->raw_stages * g->raw_slot;
   }
   (void)n_chunks_total;
   g->stages = pick_stages((kSmemLimit - g->stage_off) / g->stage_bytes, g->zs, cps);
-  if (g->stages < 1 && want_raw) return place_stages(g, n_chunks_total, cps, false, stride);
+  if (g->stages < 1 && raw_mode) return place_stages(g, n_chunks_total, cps, 0, stride);
   return g->stages >= 1;
 }
 
@@ -1649,7 +1862,7 @@ int pick_stages(int fit, int zs, int cps) {
 
 // Geometry for `zs` consumer warps per unit, R output rows per lane and no channel split across CTAs.
 template <bool GENERIC>
-bool geo_for(const DeviceLayer& L, int n, int h, int w, int zs, int R, Geo* out) {
+bool geo_for(const DeviceLayer& L, int n, int h, int w, int zs, int R, bool bulk, Geo* out) {
   // the warps of a unit add up column sets of the same TMEM lanes: they sit in one lane quadrant,
   // which holds a quarter of the consumer warps
   if (zs > consumer_warps(GENERIC, R) / 4) return false;
@@ -1697,17 +1910,29 @@ bool geo_for(const DeviceLayer& L, int n, int h, int w, int zs, int R, Geo* out)
   g.substride = g.pitch * g.colstride;
   if (g.tw == 4) while (g.substride % 128 != 64) g.substride += 16;
   if (g.tw == 2) while (g.substride % 128 != 32) g.substride += 16;
-  g.tab_off = 8 * 2 * kMaxStages + 16 + 64 + 8 * kMaxCoop;  // barriers, TMEM base word, unit counters, first-chunk barriers
+  // barriers, TMEM base word, unit counters, first-chunk barriers, raw-slot barriers
+  g.tab_off = 8 * 2 * kMaxStages + 16 + 64 + 8 * kMaxCoop + 8 * (kRawStages + 1);
   if (L.n_chunks > 512) return false;   // descriptor table budget (c_in <= 4096)
   g.ks = 1;
   g.cps = L.n_chunks;
+  // how chunks are fetched: fp16 pairs by cp.async where rows start on 4-byte boundaries; fp32, when
+  // asked for, by bulk copies where plane spans (sub-tile as wide as the image) or rows start on
+  // 16-byte boundaries (measured slower than element-wise cp.async: see PCONV_STAGE_BULK)
+  g.raw_want = 0;
+  if (L.storage == PCONV_F16) {
+    if (w % 2 == 0) g.raw_want = 1;
+  } else if (bulk && g.tx == 1 && ((long long)h * w) % 4 == 0) {
+    g.raw_want = 3;
+  } else if (bulk && g.tx > 1 && w % 4 == 0) {
+    g.raw_want = 2;
+  }
   for (;;) {
     g.pairs = g.wy * g.sw;
     g.chan_stride = g.pairs * g.substride;
     g.x_stage_bytes = kChunk * g.chan_stride;
     g.stage_bytes = (g.x_stage_bytes + g.ng * (kWSlot + kCodeSlot) + 15) & ~15;
     g.desc_off = (g.tab_off + 2 * g.pairs * (int)sizeof(SubTile) + 15) & ~15;
-    if (place_stages(&g, L.n_chunks, g.cps, L.storage == PCONV_F16 && (w % 2) == 0, L.stride)) break;
+    if (place_stages(&g, L.n_chunks, g.cps, g.raw_want, L.stride)) break;
     if (g.wy > 1) {
       g.wy /= 2;          // fewer pixel sets (the other warp rows idle)
     } else if (g.ng > 1) {
@@ -1739,7 +1964,7 @@ void set_split(const DeviceLayer& L, Geo* g, int ks) {
   if (ks > L.n_chunks) ks = L.n_chunks;
   g->cps = (L.n_chunks + ks - 1) / ks;
   g->ks = (L.n_chunks + g->cps - 1) / g->cps;
-  if (!place_stages(g, L.n_chunks, g->cps, g->raw_stages > 0, L.stride)) g->stages = 0;
+  if (!place_stages(g, L.n_chunks, g->cps, g->raw_want, L.stride)) g->stages = 0;
 }
 
 // Estimated duration of a launch in units of one kernel (4 taps on a warp's 256 pixels, about
@@ -1769,13 +1994,16 @@ double geo_cost(const DeviceLayer& L, const Geo& g) {
   return waves * (fixed + loop) + (g.ks > 1 ? 100.0 / g.zs : 0.0);
 }
 
-// The geometry of a launch.  Canonical pattern sets choose the rows per lane (`rmode`: 4, 8 or
-// 0 = by the estimate; 8 needs one-byte codes), how the consumer warps are used (zs = 1, 2 or 4
+// The geometry of a launch.  `pin` = what the caller pinned: the rows per lane (4, 8 or 0 = by the
+// estimate; 8 needs one-byte codes), | kPinBulk = fp32 chunks by bulk copies.  Canonical pattern
+// sets choose the rows per lane, how the consumer warps are used (zs = 1, 2 or 4
 // warps per unit) and, when a workspace is available, whether the channel range is also split
 // across CTAs, by the estimate above.
 template <bool GENERIC>
-bool make_geo(const DeviceLayer& L, int n, int h, int w, bool allow_split, int rmode, Geo* out) {
-  if (GENERIC) return geo_for<true>(L, n, h, w, 1, 4, out);
+bool make_geo(const DeviceLayer& L, int n, int h, int w, bool allow_split, int pin, Geo* out) {
+  const int rmode = pin & kPinRowsMask;
+  const bool bulk = (pin & kPinBulk) != 0;
+  if (GENERIC) return geo_for<true>(L, n, h, w, 1, 4, bulk, out);
   bool found = false;
   double best = 0.0;
 #ifdef PCONV_DEV
@@ -1795,7 +2023,7 @@ bool make_geo(const DeviceLayer& L, int n, int h, int w, bool allow_split, int r
 #ifdef PCONV_DEV
       if (force_zs && atoi(force_zs) != zs) continue;
 #endif
-      if (!geo_for<false>(L, n, h, w, zs, R, &g)) continue;
+      if (!geo_for<false>(L, n, h, w, zs, R, bulk, &g)) continue;
 #ifdef PCONV_DEV
       if (force_ks && allow_split) {
         set_split(L, &g, atoi(force_ks));
@@ -1928,6 +2156,7 @@ bool tiled_plan(const DeviceLayer& L, int n, int h, int w, bool generic_taps, bo
     return false;
   out->generic_taps = generic_taps ? 1 : 0;
   out->rows_per_lane = g.rpl;
+  out->staging = g.raw_mode;
   out->warps_per_unit = g.zs;
   out->channel_splits = g.ks;
   out->groups_per_cta = g.ng;
@@ -1943,11 +2172,12 @@ cudaError_t launch_tiled(const DeviceLayer& L, const void* x, const float* bias,
                          int w, bool relu, bool pool, bool reproducible, bool generic_taps, int rmode,
                          bool allow_cluster, void* ws, size_t ws_bytes, cudaStream_t stream) {
   if (!generic_taps && !L.codes_s) generic_taps = true;
-  if (rmode == 8 && (generic_taps || L.wide_codes)) return cudaErrorInvalidValue;
+  if ((rmode & kPinRowsMask) == 8 && (generic_taps || L.wide_codes)) return cudaErrorInvalidValue;
   Geo g;
   const size_t need = generic_taps ? 0 : tiled_workspace_bytes(L, n, h, w, rmode);
   const bool split = !reproducible && need > 0 && ws && ws_bytes >= need;
-  if (!(generic_taps ? make_geo<true>(L, n, h, w, false, 4, &g) : make_geo<false>(L, n, h, w, split, rmode, &g)))
+  if (!(generic_taps ? make_geo<true>(L, n, h, w, false, 4 | (rmode & kPinBulk), &g)
+                     : make_geo<false>(L, n, h, w, split, rmode, &g)))
     return cudaErrorInvalidValue;
   g.relu = relu ? 1 : 0;
   if (reproducible && g.zs > 1) {

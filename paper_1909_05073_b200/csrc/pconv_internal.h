@@ -135,7 +135,10 @@ cudaError_t launch_tensor(const DeviceLayer& L, const void* x, const float* bias
 size_t tensor_workspace_bytes(const DeviceLayer& L, int n, int h, int w);
 bool tensor_supported(const DeviceLayer& L, int n, int h, int w);
 bool tensor_preferred(const DeviceLayer& L, int n, int h, int w);
-// rmode: output rows per lane of the tiled kernel (4, 8, or 0 = the planner chooses)
+// rmode: what the caller pinned for the tiled kernel: output rows per lane (4, 8, or 0 = the planner
+// chooses) | kPinBulk (fp32 chunks fetched by bulk copies into a raw ring)
+constexpr int kPinRowsMask = 0xff;
+constexpr int kPinBulk = 0x100;
 size_t tiled_workspace_bytes(const DeviceLayer& L, int n, int h, int w, int rmode);
 bool tiled_supported(const DeviceLayer& L, int n, int h, int w);
 bool tiled_plan(const DeviceLayer& L, int n, int h, int w, bool generic_taps, bool with_workspace,

@@ -203,7 +203,7 @@ def test_forward_argument_errors():
     x = torch.zeros(1, 4, 8, 8, device="cuda")
     y = torch.zeros(1, 4, 8, 8, device="cuda")
     with pytest.raises(B.PconvError) as e:
-        B.pconv_forward(layer.handle, x, None, y, flags=0x8000)
+        B.pconv_forward(layer.handle, x, None, y, flags=0x40000)   # an unknown bit
     assert e.value.status == 6
     with pytest.raises(B.PconvError) as e:
         B.pconv_forward(layer.handle, x, None, y, flags=B.KERNEL_SIMPLE | B.KERNEL_TILED)
