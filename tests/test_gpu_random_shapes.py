@@ -59,3 +59,35 @@ def test_random_shape_matches_the_oracle(seed):
         assert not ws.any()
     assert B.pconv_device_status(layer.handle)[0] == 0
     layer.close()
+
+
+@pytest.mark.parametrize("seed", range(32))
+def test_random_shape_with_the_pinned_forms_matches_the_oracle(seed):
+    """The same shapes through the forms a caller can pin: 8 rows per lane, the cluster reduction
+    of the channel split and the bulk-copy staging, alone and together (canonical pattern sets;
+    a form a shape cannot take must leave the result unchanged)."""
+    rng = np.random.default_rng(9500 + seed)
+    c_in, c_out, h, w, n, stride, keep, storage, _ = random_case(rng)
+    if seed % 4 == 0:          # shapes whose rows or planes start on 16-byte boundaries
+        h, w = int(rng.choice([4, 8, 14, 16, 28])), int(rng.choice([4, 8, 14, 16, 28, 36, 64]))
+    spec = synth.LayerSpec("r", c_in, c_out, h, w, stride, keep)
+    wt, bias, _ = synth.gen_weights(spec, 9500 + seed)
+    x = synth.gen_input(spec, n, 9500 + seed)
+    layer = B.Layer(wt, synth.PATTERNS8, stride, B.F16 if storage == "f16" else B.F32, bias)
+    xt = torch.from_numpy(x).cuda()
+    if storage == "f16":
+        xt = xt.half()
+    ref = oracle.conv3x3(x, wt, bias, stride, True, storage)
+    pooled = oracle.maxpool2x2(ref) if ref.shape[2] >= 2 and ref.shape[3] >= 2 else None
+    what = "seed %d: %s" % (seed, (c_in, c_out, h, w, n, stride, keep, storage))
+    for flags in (B.ROWS8, B.CLUSTER, B.STAGE_BULK, B.ROWS8 | B.CLUSTER | B.STAGE_BULK):
+        for split in (False, True):
+            y = layer.forward(xt, relu=True, kernel=B.KERNEL_TILED | flags, split=split)
+            check_close(y.float().cpu().numpy(), ref, storage, what + " flags %x split=%s" % (flags, split))
+            if pooled is not None:
+                yp = layer.forward(xt, relu=True, kernel=B.KERNEL_TILED | flags, split=split, pool=True)
+                check_close(yp.float().cpu().numpy(), pooled, storage, what + " flags %x pooled split=%s" % (flags, split))
+    ws = getattr(layer, "_ws", None)
+    if ws is not None:
+        assert not ws.any()
+    assert B.pconv_device_status(layer.handle)[0] == 0
