@@ -1667,17 +1667,19 @@ __device__ __forceinline__ void tiled_body(const DeviceLayer& L, const Geo& g, c
         // ticket turns the summed partials into the layer's output and leaves workspace and
         // ticket zeroed for the next launch; nobody waits for anybody, and the finishing work of a
         // tile spreads over the CTAs that share it.
-        __threadfence();
+        // (one release-acquire atomic by lane 0 after the warp has synchronised: the release covers
+        // the whole warp's partial sums, the acquire orders the last arriver's reads after every
+        // other split's release)
         __syncwarp();
         int* ticket = counters + ((size_t)bp.y * bp.gx + bp.x) * kCW + warp;
         int t = 0;
         if (lane == 0) {
-          t = atomicAdd(ticket, 1);
+          asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(t) : "l"(ticket) : "memory");
           if (t == g.ks - 1) *ticket = 0;
         }
         t = __shfl_sync(0xffffffffu, t, 0);
+        __syncwarp();
         if (t == g.ks - 1) {
-          __threadfence();
           with_flags(g, [&](auto half, auto relu) {
             finalize_outputs<R, decltype(half)::value, decltype(relu)::value>(g, lo, lp, y, wsl, orng.a0,
                                                                              orng.a1, my_o, my_b);
